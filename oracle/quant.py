@@ -1,0 +1,86 @@
+"""Uniform quantizer of the paper's Background section (Eq. 1-3).  Test infrastructure.
+
+Q(X|b) = clip(round(X / s) + z, 0, 2^b - 1)                                  (Eq. 1)
+l = min X, u = max X                                                        (Eq. 2)
+s = (u - l) / (2^b - 1),  z = clip(round(-l / s), 0, 2^b - 1)                (Eq. 3)
+
+Readings taken where the paper is silent or garbled:
+  * Eq. 3 prints z on both sides; the inner "+z" is dropped.
+  * round() is round-half-to-even.
+  * X / s is evaluated as one float32 product X * (1/s) with 1/s rounded to
+    float32 once; the rounding decision is taken in float32.
+  * Besides the unsigned range of Eq. 1 a symmetric signed range [-127, 127]
+    with z = 0 is supported (s = max|X| / 127); weights use it per output channel
+    and activations per tensor ("channel-wise ... weights, tensor-wise ...
+    activations", Comparison on Performance).
+  * A degenerate range (u == l, or max|X| == 0) takes s = 1.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import numpy as np
+
+F32 = np.float32
+
+
+@dataclass(frozen=True)
+class QParams:
+    scale: float       # s, representable in float32
+    zero_point: int    # z
+    qmin: int
+    qmax: int
+
+    @property
+    def inv_scale(self) -> np.float32:
+        return F32(1.0) / F32(self.scale)
+
+
+def qparams_minmax(X: np.ndarray, bits: int = 8) -> QParams:
+    """Eq. 2-3: asymmetric parameters from the range of X; codes in [0, 2^b - 1]."""
+    levels = (1 << bits) - 1
+    l = F32(np.min(X))
+    u = F32(np.max(X))
+    s = F32(u - l) / F32(levels)
+    if not s > 0:
+        s = F32(1.0)
+    z = int(np.clip(np.rint(np.float64(-l) / np.float64(s)), 0, levels))
+    return QParams(float(s), z, 0, levels)
+
+
+def qparams_symmetric(absmax: float, bits: int = 8) -> QParams:
+    """Signed symmetric parameters: s = absmax / (2^(b-1) - 1), z = 0."""
+    top = (1 << (bits - 1)) - 1
+    s = F32(absmax) / F32(top)
+    if not s > 0:
+        s = F32(1.0)
+    return QParams(float(s), 0, -top, top)
+
+
+def quantize(X: np.ndarray, qp: QParams) -> np.ndarray:
+    """Eq. 1.  X is rounded to float32 first; returns int32 codes in [qmin, qmax]."""
+    x32 = np.asarray(X).astype(F32)
+    r = np.rint(x32 * qp.inv_scale)          # float32 product, half-to-even
+    r = r.astype(np.float64) + qp.zero_point
+    return np.clip(r, qp.qmin, qp.qmax).astype(np.int32)
+
+
+def dequantize(q: np.ndarray, qp: QParams) -> np.ndarray:
+    """Inverse map of Eq. 1 inside the clip range: s * (q - z), float64."""
+    return np.float64(F32(qp.scale)) * (np.asarray(q, dtype=np.float64) - qp.zero_point)
+
+
+def quantize_weight_per_channel(W: np.ndarray, bits: int = 8):
+    """Channel-wise symmetric weights: one scale per output row of W[N, K].
+
+    Returns (q int32 [N,K], scale float32 [N], colsum int64 [N]) where
+    colsum[n] = sum_k q[n,k] (needed to undo an activation zero-point).
+    """
+    W = np.asarray(W, dtype=F32)
+    top = (1 << (bits - 1)) - 1
+    absmax = np.max(np.abs(W), axis=1)
+    s = (absmax / F32(top)).astype(F32)
+    s[~(s > 0)] = F32(1.0)
+    inv = (F32(1.0) / s).astype(F32)
+    q = np.clip(np.rint(W * inv[:, None]), -top, top).astype(np.int32)
+    return q, s, q.sum(axis=1, dtype=np.int64)

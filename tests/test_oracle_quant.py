@@ -1,0 +1,129 @@
+"""Pins for oracle.quant (Eq. 1-3): hand-worked values, round-trip bound, grid points, ties, saturation."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import quant
+from oracle.quant import QParams
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "quantizer_eq1.txt")
+
+
+def _golden_rows():
+    rows = []
+    with open(GOLDEN) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                a, b = line.split()
+                rows.append((float(a), int(b)))
+    return rows
+
+
+def test_hand_worked_example_eq1_eq3():
+    # b = 4, l = -1.5, u = 6 -> s = 0.5, z = 3 (worked in the fixture's header)
+    X = np.array([-1.5, 6.0, 0.1], dtype=np.float32)
+    qp = quant.qparams_minmax(X, bits=4)
+    assert qp.scale == 0.5 and qp.zero_point == 3 and (qp.qmin, qp.qmax) == (0, 15)
+    xs = np.array([r[0] for r in _golden_rows()])
+    want = np.array([r[1] for r in _golden_rows()])
+    np.testing.assert_array_equal(quant.quantize(xs, qp), want)
+
+
+def test_eq2_eq3_8bit_range_ends():
+    X = np.array([-1.0, 3.0, 0.5, 2.0], dtype=np.float32)
+    qp = quant.qparams_minmax(X)
+    assert qp.scale == pytest.approx(4.0 / 255.0, rel=1e-7)
+    assert qp.zero_point == 64                    # round(63.75)
+    q = quant.quantize(X, qp)
+    assert q[0] == 0 and q[1] == 255              # l -> 0, u -> 2^b - 1
+
+
+@pytest.mark.parametrize("mode", ["sym", "minmax"])
+def test_round_trip_bound_inside_clip_range(mode):
+    rng = np.random.default_rng(7)
+    X = (rng.standard_normal(20000) * 3).astype(np.float32)
+    qp = quant.qparams_symmetric(float(np.abs(X).max())) if mode == "sym" else quant.qparams_minmax(X)
+    lo, hi = qp.scale * (qp.qmin - qp.zero_point), qp.scale * (qp.qmax - qp.zero_point)
+    inside = (X >= lo) & (X <= hi)
+    assert inside.mean() > 0.99
+    err = np.abs(X.astype(np.float64) - quant.dequantize(quant.quantize(X, qp), qp))
+    # s/2 plus float32 slack of the single product x * (1/s)
+    assert err[inside].max() <= qp.scale / 2 * (1 + 1e-5)
+    # and the bound is attained to within 2 % somewhere (a truncating quantizer would give ~s)
+    assert err[inside].max() >= 0.49 * qp.scale
+
+
+def test_grid_points_map_to_their_index():
+    for qp in (QParams(0.037, 0, -127, 127), QParams(0.11, 17, 0, 255)):
+        k = np.arange(qp.qmin - qp.zero_point, qp.qmax - qp.zero_point + 1)
+        x = (np.float32(qp.scale) * k.astype(np.float32)).astype(np.float32)
+        np.testing.assert_array_equal(quant.quantize(x, qp), k + qp.zero_point)
+
+
+def test_ties_go_to_even():
+    qp = QParams(0.25, 5, 0, 255)        # power-of-two scale: x/s exact
+    x = np.array([0.5, 1.5, 2.5, 3.5, -0.5, -1.5, -2.5]) * 0.25
+    np.testing.assert_array_equal(quant.quantize(x, qp), np.array([0, 2, 2, 4, 0, -2, -2]) + 5)
+
+
+def test_saturation_both_ends():
+    qp = QParams(0.1, 0, -127, 127)
+    with np.errstate(over="ignore"):
+        q = quant.quantize(np.array([-1e9, -12.75, 12.75, 1e9, np.float32(3e38)]), qp)
+    np.testing.assert_array_equal(q, [-127, -127, 127, 127, 127])
+    qp = QParams(0.1, 10, 0, 255)
+    np.testing.assert_array_equal(quant.quantize(np.array([-5.0, 50.0]), qp), [0, 255])
+
+
+def test_rounding_decision_is_taken_in_float32():
+    # find float32 (x, s) whose float32 product x*(1/s) is an exact tie k+0.5 while the float64
+    # product of the same operands falls on the side that rounds AWAY from the even neighbour
+    rng = np.random.default_rng(99)
+    cases = []
+    for _ in range(20000):
+        s = np.float32(rng.uniform(0.01, 0.2))
+        inv = np.float32(1.0) / s
+        k = int(rng.integers(-100, 100))
+        x = np.float32((k + 0.5) * float(s))
+        p32 = np.float32(x * inv)
+        p64 = np.float64(x) * np.float64(inv)
+        if p32 == np.float32(k + 0.5) and p64 != k + 0.5:
+            even = k if k % 2 == 0 else k + 1
+            if int(np.rint(p64)) != even:
+                cases.append((x, s, even))
+        if len(cases) >= 5:
+            break
+    assert len(cases) >= 5
+    for x, s, even in cases:
+        assert quant.quantize(np.array([x]), QParams(float(s), 0, -127, 127))[0] == even
+
+
+def test_degenerate_range_takes_unit_scale():
+    assert quant.qparams_symmetric(0.0).scale == 1.0
+    assert quant.qparams_minmax(np.full(5, 2.0, dtype=np.float32)).scale == 1.0
+
+
+def test_weight_per_channel():
+    rng = np.random.default_rng(3)
+    W = (rng.standard_normal((9, 40)) * 0.02).astype(np.float32)
+    W[4] = 0
+    q, s, cs = quant.quantize_weight_per_channel(W)
+    assert q.shape == W.shape and s.dtype == np.float32
+    for n in range(9):
+        if n == 4:
+            assert s[n] == 1.0 and not q[n].any()
+            continue
+        j = np.argmax(np.abs(W[n]))
+        assert abs(q[n, j]) == 127 and np.sign(q[n, j]) == np.sign(W[n, j])
+        assert np.abs(q[n]).max() == 127
+        assert s[n] == np.float32(np.abs(W[n]).max()) / np.float32(127)
+        assert np.abs(W[n] - s[n] * q[n]).max() <= s[n] / 2 * (1 + 1e-5)
+        assert cs[n] == int(q[n].sum())
+    # channel-wise: scaling one row changes only that row's scale, never its codes
+    W2 = W.copy()
+    W2[2] *= 4
+    q2, s2, _ = quant.quantize_weight_per_channel(W2)
+    np.testing.assert_array_equal(q2, q)
+    assert s2[2] == pytest.approx(4 * s[2]) and s2[3] == s[3]

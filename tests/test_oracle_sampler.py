@@ -1,0 +1,182 @@
+"""Pins for oracle.sampler and oracle.vc: cache schedule, DDIM identities, VC identities and fit."""
+import numpy as np
+import pytest
+
+import synth
+from oracle import calib, dit, sampler, vc
+
+
+def test_cache_schedule():
+    assert all(sampler.should_refresh(i, 1) for i in range(10))
+    assert [sampler.should_refresh(i, 2) for i in range(5)] == [True, False, True, False, True]
+    assert [i for i in range(50) if sampler.should_refresh(i, 100)] == [0]
+    assert sum(sampler.should_refresh(i, 2) for i in range(50)) == 25
+    assert sum(sampler.should_refresh(i, 3) for i in range(100)) == 34
+    with pytest.raises(ValueError):
+        sampler.should_refresh(0, 0)
+
+
+def test_ddim_table_and_identities():
+    tab = sampler.ddim_table(50)
+    assert [r[0] for r in tab[:3]] == [980, 960, 940] and tab[-1][0] == 0
+    for r in tab:
+        assert abs(r[1] ** 2 + r[2] ** 2 - 1) < 1e-12 and abs(r[3] ** 2 + r[4] ** 2 - 1) < 1e-12
+    assert abs(tab[-1][1] ** 2 - (1 - 1e-4)) < 1e-15          # alpha_bar_0 = 1 - beta_0
+    assert tab[-1][3] == 1.0 and tab[-1][4] == 0.0            # after the last step alpha_bar_prev = 1
+    for a, b in zip(tab[:-1], tab[1:]):
+        assert a[3] == b[1] and a[1] < b[1]                    # prev of step i is t of step i+1; alpha_bar grows
+    # closed form of alpha_bar at t = 980: prod_{j<=980} (1 - beta_j)
+    betas = [1e-4 + (2e-2 - 1e-4) * j / 999 for j in range(1000)]
+    ab = 1.0
+    for j in range(981):
+        ab *= 1 - betas[j]
+    assert abs(tab[0][1] - np.sqrt(ab)) < 1e-12
+    # if eps is the true noise, the update lands exactly on the same (x0, eps) at the previous level
+    rng = np.random.default_rng(0)
+    x0, eps = rng.standard_normal((2, 4, 8, 8)), rng.standard_normal((2, 4, 8, 8))
+    for row in (tab[0], tab[17], tab[-1]):
+        xt = row[1] * x0 + row[2] * eps
+        np.testing.assert_allclose(sampler.ddim_update(xt, eps, row), row[3] * x0 + row[4] * eps, atol=1e-12)
+    np.testing.assert_allclose(sampler.ddim_update(tab[-1][1] * x0 + tab[-1][2] * eps, eps, tab[-1]), x0, atol=1e-12)
+    # equivalent textbook form: x_prev = sqrt(ab_p/ab_t) x + (sqrt(1-ab_p) - sqrt(ab_p (1-ab_t)/ab_t)) eps
+    row = tab[5]
+    xt = rng.standard_normal((2, 4, 8, 8))
+    alt = row[3] / row[1] * xt + (row[4] - row[3] * row[2] / row[1]) * eps
+    np.testing.assert_allclose(sampler.ddim_update(xt, eps, row), alt, atol=1e-12)
+
+
+def test_cfg_combine():
+    rng = np.random.default_rng(1)
+    e = rng.standard_normal((6, 4, 2, 2))
+    np.testing.assert_array_equal(sampler.cfg_combine(e, 1.0), e[3:] + 1.0 * (e[:3] - e[3:]))
+    np.testing.assert_allclose(sampler.cfg_combine(e, 1.0), e[:3], atol=1e-15)      # g = 1: conditional
+    np.testing.assert_allclose(sampler.cfg_combine(e, 0.0), e[3:], atol=0)          # g = 0: unconditional
+    np.testing.assert_allclose(sampler.cfg_combine(e, 1.5), 1.5 * e[:3] - 0.5 * e[3:], atol=1e-15)
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    cfg = synth.DIT_TINY
+    model = dit.make_qmodel(cfg, synth.model_weights(21, cfg))
+    latent = synth.normal(21, "latent", (2, cfg.channels, cfg.latent_side, cfg.latent_side))
+    labels = np.array([3, 77])
+    scales = calib.calibrate_model(model, [(latent, np.array([500.0, 500.0]), labels)])
+    return cfg, model, latent, labels, scales
+
+
+def test_interval_one_equals_uncached_bit_for_bit(tiny):
+    cfg, model, latent, labels, scales = tiny
+    ctx = dit.Context(quant="static", scales=scales)
+    a = sampler.sample(model, ctx, sampler.SamplerConfig(6, cache_interval=1, guidance=1.5), latent, labels)
+    b = sampler.sample(model, ctx, sampler.SamplerConfig(6, use_cache=False, guidance=1.5), latent, labels)
+    np.testing.assert_array_equal(a, b)
+    c = sampler.sample(model, ctx, sampler.SamplerConfig(6, cache_interval=2, guidance=1.5), latent, labels)
+    assert not np.array_equal(a, c)           # the cache changes the trajectory ...
+    assert np.linalg.norm(a - c) / np.linalg.norm(a) < 0.2     # ... but only mildly
+
+
+def test_large_interval_computes_only_step_zero(tiny):
+    cfg, model, latent, labels, scales = tiny
+    ctx = dit.Context(quant="static", scales=scales)
+    flags = []
+    sampler.sample(model, ctx, sampler.SamplerConfig(5, cache_interval=9), latent, labels,
+                   on_step=lambda i, x, reuse: flags.append(reuse))
+    assert flags == [False, True, True, True, True]
+
+
+def test_reuse_step_closed_form_and_state_error(tiny):
+    cfg, model, latent, labels, scales = tiny
+    ctx = dit.Context(quant="static", scales=scales, storage=dit.Storage.exact())
+    t0, t1 = np.full(2, 900.0), np.full(2, 800.0)
+    with pytest.raises(KeyError):
+        dit.forward(model, ctx, latent, t1, labels, cache={}, reuse=True)
+    cache = {}
+    dit.forward(model, ctx, latent, t0, labels, cache=cache)
+    assert sorted(cache) == sorted((i, b) for i in range(cfg.depth) for b in ("attn", "mlp"))
+    taps = {}
+    ctx2 = dit.Context(quant="static", scales=scales, storage=dit.Storage.exact(),
+                       tap=lambda n, a: taps.__setitem__(n, np.array(a)))
+    lat1 = latent * 0.9 + 0.05
+    dit.forward(model, ctx2, lat1, t1, labels, cache=cache, reuse=True)
+    # x_final = x_embed + sum_b (gate_msa_b * A_b + gate_mlp_b * Mo_b) with gates of the CURRENT step
+    rows = np.arange(2 * cfg.tokens) // cfg.tokens
+    want = taps["x_embed"].copy()
+    D = cfg.hidden
+    for i in range(cfg.depth):
+        mod = taps[f"blk{i}.mod"]
+        want += mod[rows, 2 * D:3 * D] * cache[(i, "attn")] + mod[rows, 5 * D:6 * D] * cache[(i, "mlp")]
+    np.testing.assert_allclose(taps["x_final"], want, rtol=1e-13, atol=1e-13)
+    # no attention / MLP linear ran on the reuse step
+    assert not any(k.endswith((".qkv.in", ".fc1.in", ".proj.in", ".fc2.in")) for k in taps)
+    # the cached tensors are the pre-gate branch outputs of the refresh step
+    taps0 = {}
+    ctx3 = dit.Context(quant="static", scales=scales, storage=dit.Storage.exact(),
+                       tap=lambda n, a: taps0.__setitem__(n, np.array(a)))
+    dit.forward(model, ctx3, latent, t0, labels, cache={})
+    np.testing.assert_array_equal(cache[(1, "attn")], taps0["blk1.attn_branch"])
+    np.testing.assert_array_equal(cache[(1, "mlp")], taps0["blk1.mlp_branch"])
+
+
+# ----------------------------------------------------------------------------- VC
+def test_vc_apply_identities():
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((3, 4, 8, 8)) * np.array([0.5, 1, 2, 3]).reshape(1, 4, 1, 1) + 0.7
+    np.testing.assert_allclose(vc.apply(x, np.ones(4)), x, atol=1e-15)
+    K = np.array([0.9, 1.0, 1.1, 1.3])
+    y = vc.apply(x, K)
+    np.testing.assert_allclose(y.mean(axis=(2, 3)), x.mean(axis=(2, 3)), atol=1e-14)      # mean preserved
+    np.testing.assert_allclose(y.var(axis=(2, 3)), x.var(axis=(2, 3)) * K ** 2, rtol=1e-12)  # variance scaled by K^2
+    # rescaling identity: var_ratio mode reaches the target variance; factor 1 when variances already match
+    tgt = np.array([0.3, 1.0, 2.5, 4.0])
+    z = vc.apply(x, tgt, mode="var_ratio", eps=0.0)
+    np.testing.assert_allclose(z.var(axis=(2, 3)), np.broadcast_to(tgt, (3, 4)), rtol=1e-12)
+    same = vc.apply(x[:1], x[0].var(axis=(1, 2)), mode="var_ratio", eps=0.0)
+    np.testing.assert_allclose(same, x[:1], atol=1e-13)
+    z6 = vc.apply(x, tgt, mode="var_ratio", eps=1e-6)
+    np.testing.assert_allclose(z6.var(axis=(2, 3)), np.broadcast_to(tgt, (3, 4)), rtol=1e-5)
+
+
+def _objective(K, xh, xt, eps):
+    mu = xh.mean(axis=(2, 3), keepdims=True)
+    xtil = mu + K.reshape(1, -1, 1, 1) * (xh - mu)
+    d = xtil - xt
+    return (d ** 2 / (xt ** 2 + eps)).sum(axis=(0, 2, 3)) + (d ** 2).sum(axis=(0, 2, 3))
+
+
+def test_vc_fit_closed_form():
+    rng = np.random.default_rng(4)
+    xt = rng.standard_normal((5, 4, 6, 6)) + 0.3
+    # x^ = mu + r (x' - mu)  =>  K = 1/r ;  x^ = x'  =>  K = 1
+    np.testing.assert_allclose(vc.fit(xt, xt), np.ones(4), atol=1e-13)
+    r = np.array([0.8, 0.9, 1.25, 2.0]).reshape(1, 4, 1, 1)
+    mu = xt.mean(axis=(2, 3), keepdims=True)
+    xh = mu + r * (xt - mu)
+    np.testing.assert_allclose(vc.fit(xh, xt), 1 / r.ravel(), rtol=1e-12)
+    # general case: the closed form is the minimiser of rQNSR^2 + MSE (checked by bracketing)
+    xh = xt * 0.9 + 0.2 * rng.standard_normal(xt.shape)
+    K = vc.fit(xh, xt, eps=1e-6)
+    f0 = _objective(K, xh, xt, 1e-6)
+    for d in (1e-3, -1e-3, 0.05, -0.05):
+        assert (_objective(K + d, xh, xt, 1e-6) > f0).all()
+    # the form as printed coincides with the derived one when mu = 0 and eps = 0
+    xh0 = xh - xh.mean(axis=(2, 3), keepdims=True)
+    np.testing.assert_allclose(vc.fit(xh0, xt, eps=0.0, form="printed"), vc.fit(xh0, xt, eps=0.0), rtol=1e-10)
+
+
+def test_sampler_applies_vc_every_step(tiny):
+    cfg, model, latent, labels, scales = tiny
+    ctx = dit.Context(quant="static", scales=scales)
+    S = 4
+    base = sampler.sample(model, ctx, sampler.SamplerConfig(S, cache_interval=2), latent, labels)
+    ones = sampler.sample(model, ctx, sampler.SamplerConfig(S, cache_interval=2, vc_table=np.ones((S, 4))), latent, labels)
+    np.testing.assert_allclose(ones, base, atol=1e-6)         # K = 1 is the identity (up to float32 storage)
+    K = np.full((S, 4), 1.05)
+    seen = []
+    out = sampler.sample(model, ctx, sampler.SamplerConfig(S, cache_interval=2, vc_table=K), latent, labels,
+                         on_step=lambda i, x, r: seen.append(x.copy()))
+    assert len(seen) == S and not np.allclose(out, base)
+    # first step by hand: DDIM update of the un-corrected run, then mu + K (x - mu)
+    first = []
+    sampler.sample(model, ctx, sampler.SamplerConfig(1 * S, cache_interval=2), latent, labels,
+                   on_step=lambda i, x, r: first.append(x.copy()))
+    np.testing.assert_allclose(seen[0], vc.apply(first[0], K[0]), atol=1e-6)
