@@ -1,0 +1,290 @@
+/*
+ * qdit.h - C ABI of libqdit: the quantized-and-cached DiT denoising step of
+ * Q&C ("When Quantization Meets Cache in Efficient Image Generation") as
+ * hand-written CUDA kernels for NVIDIA B200 (sm_100a).
+ *
+ * Conventions
+ *   - Every call returns an int32 status: QDIT_OK (0) or a negative QDIT_ERR_*.
+ *     qdit_status_string() names a code; qdit_last_error() gives the detail of
+ *     the last failing call on a context.  No call throws, traps or aborts.
+ *   - Unless a parameter says "host", every tensor pointer is DEVICE memory owned
+ *     by the caller, 16-byte aligned, row-major with the stated leading
+ *     dimension in ELEMENTS.  The library allocates only inside *_create calls
+ *     and frees in the matching *_destroy.
+ *   - Work is enqueued on the context's CUDA stream and is asynchronous.
+ *     Argument errors are reported before anything is launched.  Every wait
+ *     inside a kernel is bounded; a wait that runs out sets a device status word
+ *     that the next qdit_sync() returns as QDIT_ERR_TIMEOUT.
+ *   - Rows of a token matrix are ordered sample-major: row m belongs to sample
+ *     m / tokens_per_sample.
+ *   - There is no CPU fallback: on a machine without an sm_100 device
+ *     qdit_create fails with QDIT_ERR_CUDA.
+ */
+#ifndef QDIT_H_
+#define QDIT_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  QDIT_OK = 0,
+  QDIT_ERR_INVALID_ARG = -1, /* null pointer, bad enum, bad flag combination */
+  QDIT_ERR_SHAPE = -2,       /* size not supported (e.g. K not a multiple of 16) */
+  QDIT_ERR_ALIGN = -3,       /* pointer or leading dimension not 16-byte aligned */
+  QDIT_ERR_UNSUPPORTED = -4,
+  QDIT_ERR_CUDA = -5,        /* a CUDA runtime/driver call failed; see qdit_last_error */
+  QDIT_ERR_STATE = -6,       /* e.g. cache reuse before any store, step out of order */
+  QDIT_ERR_TIMEOUT = -7,     /* a bounded device-side wait ran out */
+  QDIT_ERR_NOMEM = -8
+};
+
+enum { QDIT_BF16 = 0, QDIT_F32 = 1, QDIT_I8 = 2, QDIT_I32 = 3 };
+
+typedef struct qdit_ctx qdit_ctx;
+
+/* Context = device + borrowed stream + tensor-map cache + device status word.
+ * cuda_stream is a cudaStream_t (NULL = the legacy default stream). */
+int32_t qdit_create(qdit_ctx** out, int device, void* cuda_stream);
+int32_t qdit_destroy(qdit_ctx* ctx);
+/* Waits for the stream; returns QDIT_ERR_TIMEOUT / QDIT_ERR_CUDA if work since the last sync failed. */
+int32_t qdit_sync(qdit_ctx* ctx);
+const char* qdit_status_string(int32_t status);
+const char* qdit_last_error(const qdit_ctx* ctx);
+/* Number of kernels this context has launched since creation (for launch accounting). */
+int64_t qdit_launch_count(const qdit_ctx* ctx);
+
+/* ------------------------------------------------------------------------------------------------
+ * Uniform quantizer, Eq. 1:  Q(X|b) = clip(round(X/s) + z, qmin, qmax).
+ * round = nearest, ties to even; X/s is evaluated as the float32 product X * (1/s).
+ * Eq. 1's range is [0, 2^b-1] (codes stored as unsigned bytes when qmin >= 0); the symmetric
+ * signed range [-127,127] with z = 0 is the default of the DiT path.  Activations are quantized
+ * tensor-wise, weights channel-wise (Comparison on Performance). */
+typedef struct {
+  float scale;        /* s > 0 */
+  int32_t zero_point; /* z */
+  int32_t qmin, qmax; /* clip range; either within [-128,127] or within [0,255] */
+} qdit_qparams;
+
+enum { QDIT_QUANT_STATIC = 0, QDIT_QUANT_DYNAMIC = 1 };
+
+/* q[m,k] = Q(x[m,k]).  x: [M,K] bf16 or f32 (x_dtype), ldx elements per row; q: [M,K] bytes, ldq
+ * (8-byte alignment of q and ldq suffices).
+ * STATIC : *qp (host) gives s, z and the range.
+ * DYNAMIC: symmetric range [-127,127]; s = max|x| / 127 is reduced on the device first (s = 1 if the
+ *          tensor is all zero) and left in dyn_scale (device, 1 float, required); qp is ignored.
+ * K must be a multiple of 8; M or K of 0 is a no-op. */
+int32_t qdit_quantize_act(qdit_ctx* ctx, const void* x, int x_dtype, int64_t M, int64_t K, int64_t ldx,
+                          int mode, const qdit_qparams* qp, float* dyn_scale, void* q, int64_t ldq);
+
+/* ------------------------------------------------------------------------------------------------
+ * W8A8 linear layer (8-bit weights and activations, Table 1) on quantized activations:
+ *   acc[m,n] = sum_k A[m,k] * W[n,k]                       exact int32 (tcgen05 kind::i8, TMEM)
+ *   f        = (acc - z_a * w_colsum[n]) * (s_a * w_scale[n])
+ *   f       += bias[n]                 QDIT_EPI_BIAS
+ *   f        = GELU_tanh(f)            QDIT_EPI_GELU
+ *   cache_out[m,n] = bf16(f)           QDIT_EPI_CACHE_STORE  (the block-output cache of the cache
+ *                                      mechanism: the branch output BEFORE the adaLN gate)
+ *   f       *= gate[m / tokens, n]     QDIT_EPI_GATE
+ *   f       += residual[m,n]           QDIT_EPI_RESIDUAL
+ *   out[m,n] = f as bf16 / f32, or Q(f | out_qp) as bytes with QDIT_EPI_QUANT_OUT (Eq. 1 again,
+ *              fusing the next layer's activation quantizer), or acc itself with QDIT_EPI_OUT_I32.
+ * Exactly one of OUT_BF16, OUT_F32, OUT_I32, QUANT_OUT must be set.
+ * A: [M,K] bytes (signed, or unsigned when a_qp.qmin >= 0 and a_qp.qmax > 127), W: [N,K] signed bytes,
+ * both K-contiguous with leading dimension K.  K % 16 == 0 and N % 8 == 0 are required; M, N, K are
+ * otherwise free (ragged tiles are handled).  a_scale_dev, if non-NULL, is a device float that
+ * overrides a_qp.scale at run time (used when the scale was just reduced on the device). */
+enum {
+  QDIT_EPI_BIAS = 1u << 0,
+  QDIT_EPI_GELU = 1u << 1,
+  QDIT_EPI_GATE = 1u << 2,
+  QDIT_EPI_RESIDUAL = 1u << 3,
+  QDIT_EPI_CACHE_STORE = 1u << 4,
+  QDIT_EPI_QUANT_OUT = 1u << 5,
+  QDIT_EPI_OUT_BF16 = 1u << 6,
+  QDIT_EPI_OUT_F32 = 1u << 7,
+  QDIT_EPI_OUT_I32 = 1u << 8
+};
+
+typedef struct {
+  const float* w_scale;       /* [N] channel-wise weight scales */
+  const int32_t* w_colsum;    /* [N] sum_k W[n,k]; may be NULL when a_qp.zero_point == 0 */
+  const float* bias;          /* [N] f32 */
+  const float* gate;          /* f32, row b at gate + b*ld_gate, [n] within the row */
+  int64_t ld_gate;
+  int64_t tokens_per_sample;  /* T in b = m / T */
+  const void* residual;       /* [M,N] bf16, leading dimension ldo; may alias out */
+  void* cache_out;            /* [M,N] bf16, leading dimension N */
+  qdit_qparams out_qp;        /* for QDIT_EPI_QUANT_OUT */
+  const float* out_scale_dev; /* optional device override of out_qp.scale */
+} qdit_epilogue;
+
+int32_t qdit_w8a8_linear(qdit_ctx* ctx, const void* A, const void* W, int64_t M, int64_t N, int64_t K,
+                         qdit_qparams a_qp, const float* a_scale_dev, uint32_t flags,
+                         const qdit_epilogue* epi, void* out, int64_t ldo);
+
+/* Channel-wise symmetric weight quantizer (the weight side of Eq. 1): for each output row n of
+ * w[N,K] (f32, device), s[n] = max_k|w| / 127 (1 if the row is zero), q = clip(round(w * (1/s)),-127,127),
+ * colsum[n] = sum_k q[n,k].  q: [N,K] bytes, w_scale: [N] f32, w_colsum: [N] int32.  K % 4 == 0. */
+int32_t qdit_quantize_weight(qdit_ctx* ctx, const float* w, int64_t N, int64_t K, void* q, float* w_scale,
+                             int32_t* w_colsum);
+
+/* ------------------------------------------------------------------------------------------------
+ * Self-attention between the quantized linears (kept in bf16, not quantized):
+ *   out[b,t,h,:] = softmax_s(q[b,t,h,:] . k[b,s,h,:] * softmax_scale) v[b,s,h,:]     (non-causal)
+ * q, k, v: bf16, token-major; element (b,t,h,d) at ptr[(b*T + t)*ld + h*dh + d] (so the three may
+ * point into one packed [B*T, 3*H*dh] QKV matrix).  dh in {64, 72}; T a multiple of 64.
+ * out: [B*T, H*dh] with leading dimension H*dh, as bf16, f32, or bytes Q(. | out_qp) when
+ * out_dtype == QDIT_I8 (fused quantizer of the projection's input).  Softmax statistics in f32. */
+int32_t qdit_attention(qdit_ctx* ctx, const void* q, const void* k, const void* v, int64_t ld, int B, int H,
+                       int T, int dh, float softmax_scale, void* out, int out_dtype,
+                       const qdit_qparams* out_qp, const float* out_scale_dev);
+
+/* LayerNorm (no affine, biased variance, eps) followed by the adaLN modulation of the DiT block:
+ *   y[m,:] = (x[m,:] - mean) / sqrt(var + eps) * (1 + scale[b,:]) + shift[b,:],   b = m / T
+ * x: [M,D] bf16 (leading dimension D).  shift/scale: f32, row b at ptr + b*ld_mod.
+ * out: [M,D] bf16, f32, or bytes Q(y | out_qp) when out_dtype == QDIT_I8 (fused activation quantizer
+ * of the following linear).  D a multiple of 8, D <= 2048. */
+int32_t qdit_adaln_modulate(qdit_ctx* ctx, const void* x, int64_t M, int64_t D, int64_t T, float eps,
+                            const float* shift, const float* scale, int64_t ld_mod, void* out,
+                            int out_dtype, const qdit_qparams* out_qp, const float* out_scale_dev);
+
+/* ------------------------------------------------------------------------------------------------
+ * Block-output cache (Background, "Quantization and Cache"): with cache interval N the model
+ * recomputes and refreshes the cache at sampling steps i with i mod N == 0 (i = 0 is the first step,
+ * which fills it) and reuses it for the following N-1 steps.  Cached per block: the outputs of the
+ * self-attention branch and of the MLP branch, before the adaLN gate, as bf16 [M,D]. */
+typedef struct qdit_cache qdit_cache;
+enum { QDIT_BRANCH_ATTN = 0, QDIT_BRANCH_MLP = 1 };
+
+int32_t qdit_cache_create(qdit_ctx* ctx, int blocks, int64_t M, int64_t D, qdit_cache** out);
+int32_t qdit_cache_destroy(qdit_cache* cache);
+/* Pure host function: 1 if step_index refreshes the cache, 0 if it reuses, <0 on bad arguments. */
+int32_t qdit_cache_should_refresh(int step_index, int interval);
+/* Marks every slot empty (start of a new trajectory). */
+int32_t qdit_cache_invalidate(qdit_cache* cache);
+/* Copies y [M,D] bf16 into slot (block, branch) and marks it filled. */
+int32_t qdit_cache_store(qdit_ctx* ctx, qdit_cache* cache, int block, int branch, const void* y);
+/* Device address of a slot, for a producer that writes it directly (QDIT_EPI_CACHE_STORE);
+ * mark_filled != 0 records the slot as filled.  NULL on bad arguments. */
+void* qdit_cache_slot(qdit_cache* cache, int block, int branch, int mark_filled);
+/* x[m,:] = bf16(x[m,:] + gate[b,:] * slot[m,:]).  QDIT_ERR_STATE if the slot was never stored. */
+int32_t qdit_cache_reuse(qdit_ctx* ctx, qdit_cache* cache, int block, int branch, const float* gate,
+                         int64_t ld_gate, int64_t T, void* x);
+/* A fully skipped step in one pass over the cache:
+ *   x = bf16(x + sum_blocks gate_msa_b * A_b + gate_mlp_b * Mo_b)   (f32 accumulation, one rounding)
+ * mod_all: f32 [B, blocks*6*D]; block b's gate_msa at column b*6D + 2D, gate_mlp at b*6D + 5D. */
+int32_t qdit_cache_reuse_all(qdit_ctx* ctx, qdit_cache* cache, const float* mod_all, int64_t ld_mod,
+                             int64_t T, void* x);
+
+/* ------------------------------------------------------------------------------------------------
+ * Variance compensation (section "Variance Align for Exposure Bias"):
+ *   x~ = mu + K[step,c] * (x^ - mu),  mu = spatial mean of x^ per (sample, channel).
+ * QDIT_VC_K_TABLE  : table[step*C + c] is K.
+ * QDIT_VC_VAR_RATIO: table[step*C + c] is a target variance; K = sqrt(target / (var(x^) + eps))
+ *                    with var the spatial variance per (sample, channel) (the rescaling identity
+ *                    Y = mu + (sigma_new/sigma)(f - mu)).
+ * latent: f32 [B,C,HW] updated in place; table: device f32 [steps, C]; HW % 4 == 0. */
+enum { QDIT_VC_NONE = 0, QDIT_VC_K_TABLE = 1, QDIT_VC_VAR_RATIO = 2 };
+int32_t qdit_vc_correct(qdit_ctx* ctx, float* latent, int B, int C, int HW, int step_index, int mode,
+                        const float* table, float eps);
+
+/* ------------------------------------------------------------------------------------------------
+ * Whole model and sampler.  The DiT architecture (adaLN-Zero blocks, patch 2, learned-sigma output)
+ * is the one the paper evaluates (Experimental Settings); quantized layers are each block's
+ * modulation linear, QKV, projection, fc1 and fc2; embedders and the final layer stay in f32. */
+typedef struct {
+  int32_t hidden, heads, mlp, depth, grid, patch, channels, num_classes, freq_dim;
+} qdit_model_shape;
+
+typedef struct { /* HOST f32 arrays, each linear [out_features, in_features] row-major */
+  const float *w_ada, *b_ada;   /* [6D, D], [6D]: shift_msa, scale_msa, gate_msa, shift_mlp, scale_mlp, gate_mlp */
+  const float *w_qkv, *b_qkv;   /* [3D, D]: output laid out [3, heads, head_dim] */
+  const float *w_proj, *b_proj; /* [D, D] */
+  const float *w_fc1, *b_fc1;   /* [mlp, D] */
+  const float *w_fc2, *b_fc2;   /* [D, mlp] */
+} qdit_block_weights;
+
+typedef struct { /* HOST pointers */
+  qdit_model_shape shape;
+  const float *w_patch, *b_patch; /* [D, C*p*p] (patch vector ordered c, py, px), [D] */
+  const float* pos;               /* [tokens, D] position table */
+  const float *w_t1, *b_t1;       /* [D, freq_dim] */
+  const float *w_t2, *b_t2;       /* [D, D] */
+  const float* y_table;           /* [num_classes + 1, D]; last row = "no class" */
+  const float *w_ada_f, *b_ada_f; /* [2D, D]: shift, scale of the final layer */
+  const float *w_out, *b_out;     /* [p*p*2C, D] (output vector ordered py, px, c) */
+  const qdit_block_weights* blocks; /* [depth] */
+} qdit_model_desc;
+
+typedef struct qdit_model qdit_model;
+/* Uploads the weights and quantizes the five linears of every block on the device
+ * (qdit_quantize_weight).  Activation scales start unset. */
+int32_t qdit_model_create(qdit_ctx* ctx, const qdit_model_desc* desc, qdit_model** out);
+int32_t qdit_model_destroy(qdit_model* model);
+/* Static tensor-wise activation scales (symmetric, z = 0, range [-127,127]), HOST arrays:
+ * ada_scale: 1 float (input SiLU(c) shared by all modulation linears);
+ * block_scales: [depth*4] = per block the inputs of qkv, proj, fc1, fc2. */
+int32_t qdit_model_set_act_scales(qdit_ctx* ctx, qdit_model* model, const float* ada_scale,
+                                  const float* block_scales);
+int32_t qdit_model_get_act_scales(qdit_ctx* ctx, qdit_model* model, float* ada_scale, float* block_scales);
+/* Device views of a quantized linear, for tests and for driving the primitives by hand.
+ * which: 0 ada (of `block`; all blocks are stacked block-major in one [depth*6D, D] matrix),
+ * 1 qkv, 2 proj, 3 fc1, 4 fc2.  Any out pointer may be NULL. */
+int32_t qdit_model_linear(qdit_model* model, int block, int which, const void** w_q, const float** w_scale,
+                          const int32_t** w_colsum, const float** bias, int64_t* N, int64_t* K);
+
+typedef struct {
+  int32_t batch;          /* images per trajectory batch */
+  int32_t num_steps;      /* S: DDIM steps, evenly spaced over 1000 training steps, eta = 0 */
+  int32_t cache_interval; /* N of the cache rule; 1 = recompute every step */
+  int32_t use_cfg;        /* classifier-free guidance: network batch = 2*batch ([cond; uncond]) */
+  float guidance;         /* eps = eps_u + guidance * (eps_c - eps_u) */
+  int32_t vc_mode;        /* QDIT_VC_* */
+  const float* vc_table;  /* HOST f32 [num_steps, channels] (copied) or NULL */
+  float vc_eps;
+} qdit_sampler_desc;
+
+typedef struct qdit_sampler qdit_sampler;
+/* Allocates the activation workspace, the modulation table, the cache and the latent state. */
+int32_t qdit_sampler_create(qdit_ctx* ctx, qdit_model* model, const qdit_sampler_desc* desc, qdit_sampler** out);
+int32_t qdit_sampler_destroy(qdit_sampler* s);
+/* Starts a trajectory: copies latent [batch,C,Hl,Wl] f32 and labels [batch] int32 (DEVICE pointers)
+ * into the sampler, empties the cache. */
+int32_t qdit_sampler_reset(qdit_ctx* ctx, qdit_sampler* s, const float* latent, const int32_t* labels);
+/* Device pointer to the current latent [batch,C,Hl,Wl] f32 (owned by the sampler). */
+float* qdit_sampler_latent(qdit_sampler* s);
+/* One denoising step i (0-based; must be called in order 0..S-1 after a reset):
+ * embed -> modulation for all blocks -> blocks computed (i mod N == 0, cache refreshed) or served
+ * from the cache -> final layer -> guidance -> DDIM update -> VC. */
+int32_t qdit_sample_step(qdit_ctx* ctx, qdit_sampler* s, int step_index);
+/* Whole trajectory from HOST buffers: copies latent_host/labels_host in, runs steps 0..S-1, copies the
+ * final latent to out_host, and synchronises. */
+int32_t qdit_sample(qdit_ctx* ctx, qdit_sampler* s, const float* latent_host, const int32_t* labels_host,
+                    float* out_host);
+
+/* One network evaluation on B <= (use_cfg ? 2 : 1) * batch samples, no sampler update:
+ * latent [B,C,Hl,Wl] f32, t [B] f32 timesteps, y [B] int32 labels, out [B,2C,Hl,Wl] f32 (all DEVICE).
+ * flags: QDIT_FWD_STORE_CACHE writes the cache, QDIT_FWD_REUSE serves all blocks from it,
+ * QDIT_FWD_CALIBRATE runs every activation quantizer in dynamic mode and widens the model's
+ * recorded activation ranges (then call qdit_model_finish_calibration). */
+enum { QDIT_FWD_STORE_CACHE = 1, QDIT_FWD_REUSE = 2, QDIT_FWD_CALIBRATE = 4 };
+int32_t qdit_forward(qdit_ctx* ctx, qdit_sampler* s, const float* latent, const float* t, const int32_t* y,
+                     int B, float* out, uint32_t flags);
+/* Activation-range calibration (text after Eq. 3): begin clears the recorded ranges, forwards with
+ * QDIT_FWD_CALIBRATE widen them, finish turns them into the static scales (s = absmax / 127). */
+int32_t qdit_model_begin_calibration(qdit_ctx* ctx, qdit_model* model);
+int32_t qdit_model_finish_calibration(qdit_ctx* ctx, qdit_model* model);
+
+/* Device buffers of the sampler's last network evaluation, for layer-level tests.
+ * name: "x" residual stream bf16 [M,D]; "mod" f32 [B, depth*6D]; "c" f32 [B,D]; "qkv" bf16 [M,3D];
+ * "h" bytes [M,D]; "a" bytes [M,D]; "u" bytes [M,mlp].  Returns NULL for an unknown name. */
+void* qdit_sampler_buffer(qdit_sampler* s, const char* name);
+qdit_cache* qdit_sampler_cache(qdit_sampler* s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QDIT_H_ */

@@ -1,0 +1,153 @@
+// Context, status reporting and tensor-map creation.
+#include <cstdarg>
+#include <cstdio>
+#include <new>
+
+#include "internal.h"
+
+int32_t qdit_fail(qdit_ctx* ctx, int32_t code, const char* fmt, ...) {
+  if (ctx) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof(buf), fmt, ap);
+    va_end(ap);
+    ctx->last_error = buf;
+  }
+  return code;
+}
+
+int32_t qdit_after_launch(qdit_ctx* ctx, const char* what) {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return qdit_fail(ctx, QDIT_ERR_CUDA, "launch of %s failed: %s", what, cudaGetErrorString(e));
+  ctx->launches += 1;
+  return QDIT_OK;
+}
+
+int32_t qdit_check_qparams(qdit_ctx* ctx, const qdit_qparams* qp, bool scale_from_device) {
+  if (!qp) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "quantizer parameters are NULL");
+  if (!scale_from_device && !(qp->scale > 0.0f)) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "scale must be > 0");
+  const bool is_signed = qp->qmin >= -128 && qp->qmax <= 127;
+  const bool is_unsigned = qp->qmin >= 0 && qp->qmax <= 255;
+  if (qp->qmin > qp->qmax || !(is_signed || is_unsigned))
+    return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "clip range [%d,%d] fits neither int8 nor uint8", qp->qmin, qp->qmax);
+  if (qp->zero_point < -255 || qp->zero_point > 255)
+    return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "zero point %d out of range", qp->zero_point);
+  return QDIT_OK;
+}
+
+extern "C" {
+
+int32_t qdit_create(qdit_ctx** out, int device, void* cuda_stream) {
+  if (!out) return QDIT_ERR_INVALID_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) {
+    cudaGetLastError();
+    return QDIT_ERR_CUDA;
+  }
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return QDIT_ERR_CUDA;
+  if (prop.major != 10) return QDIT_ERR_CUDA;  // kernels are built for sm_100a only
+  if (cudaSetDevice(device) != cudaSuccess) return QDIT_ERR_CUDA;
+  qdit_ctx* ctx = new (std::nothrow) qdit_ctx();
+  if (!ctx) return QDIT_ERR_NOMEM;
+  ctx->device = device;
+  ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+  ctx->num_sms = prop.multiProcessorCount;
+  if (cudaMalloc(&ctx->d_status, sizeof(int)) != cudaSuccess ||
+      cudaMemset(ctx->d_status, 0, sizeof(int)) != cudaSuccess ||
+      cudaMallocHost(&ctx->h_status, sizeof(int)) != cudaSuccess) {
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    delete ctx;
+    return QDIT_ERR_CUDA;
+  }
+  *ctx->h_status = 0;
+  cudaDriverEntryPointQueryResult qres;
+  void* fn = nullptr;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || !fn) {
+    cudaFree(ctx->d_status);
+    cudaFreeHost(ctx->h_status);
+    delete ctx;
+    return QDIT_ERR_CUDA;
+  }
+  ctx->encode_fn = fn;
+  *out = ctx;
+  return QDIT_OK;
+}
+
+int32_t qdit_destroy(qdit_ctx* ctx) {
+  if (!ctx) return QDIT_ERR_INVALID_ARG;
+  cudaSetDevice(ctx->device);
+  if (ctx->d_status) cudaFree(ctx->d_status);
+  if (ctx->h_status) cudaFreeHost(ctx->h_status);
+  delete ctx;
+  return QDIT_OK;
+}
+
+int32_t qdit_sync(qdit_ctx* ctx) {
+  if (!ctx) return QDIT_ERR_INVALID_ARG;
+  QDIT_CUDA_CHECK(ctx, cudaMemcpyAsync(ctx->h_status, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+  QDIT_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));
+  if (*ctx->h_status != QDIT_DEV_OK) {
+    *ctx->h_status = 0;
+    cudaMemsetAsync(ctx->d_status, 0, sizeof(int), ctx->stream);
+    cudaStreamSynchronize(ctx->stream);
+    return qdit_fail(ctx, QDIT_ERR_TIMEOUT, "a bounded device-side wait ran out since the last sync");
+  }
+  return QDIT_OK;
+}
+
+const char* qdit_status_string(int32_t s) {
+  switch (s) {
+    case QDIT_OK: return "ok";
+    case QDIT_ERR_INVALID_ARG: return "invalid argument";
+    case QDIT_ERR_SHAPE: return "unsupported shape";
+    case QDIT_ERR_ALIGN: return "misaligned pointer or leading dimension";
+    case QDIT_ERR_UNSUPPORTED: return "unsupported";
+    case QDIT_ERR_CUDA: return "CUDA error";
+    case QDIT_ERR_STATE: return "invalid state";
+    case QDIT_ERR_TIMEOUT: return "device-side wait timed out";
+    case QDIT_ERR_NOMEM: return "out of memory";
+    default: return "unknown status";
+  }
+}
+
+const char* qdit_last_error(const qdit_ctx* ctx) { return ctx ? ctx->last_error.c_str() : "no context"; }
+int64_t qdit_launch_count(const qdit_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"
+
+int32_t qdit_get_tmap(qdit_ctx* ctx, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows,
+                      uint32_t box_cols, uint32_t swizzle, uint32_t esize, CUtensorMap* out) {
+  TmapKey key{ptr, rows, cols, ld, box_rows, box_cols, swizzle, esize};
+  auto it = ctx->tmaps.find(key);
+  if (it != ctx->tmaps.end()) {
+    *out = it->second;
+    return QDIT_OK;
+  }
+  if (!aligned16(ptr) || (ld * esize) % 16 != 0 || (static_cast<uint64_t>(box_cols) * esize) % 16 != 0)
+    return qdit_fail(ctx, QDIT_ERR_ALIGN, "tensor map needs a 16-byte aligned base, row pitch and box width");
+  if (box_rows > 256 || box_cols > 256) return qdit_fail(ctx, QDIT_ERR_SHAPE, "tensor map box too large");
+  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                               CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  EncodeFn encode = reinterpret_cast<EncodeFn>(ctx->encode_fn);
+  cuuint64_t gdim[2] = {cols, rows};
+  cuuint64_t gstride[1] = {ld * esize};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUtensorMapDataType dt = esize == 1   ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                           : esize == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16
+                                        : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+  CUtensorMap tm;
+  CUresult r = encode(&tm, dt, 2, const_cast<void*>(ptr), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                      swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return qdit_fail(ctx, QDIT_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", static_cast<int>(r));
+  if (ctx->tmaps.size() > 4096) ctx->tmaps.clear();
+  ctx->tmaps.emplace(key, tm);
+  *out = tm;
+  return QDIT_OK;
+}

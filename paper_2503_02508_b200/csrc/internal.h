@@ -1,0 +1,89 @@
+// Internal declarations shared by the translation units of libqdit (not part of the C ABI).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <unordered_map>
+#include <vector>
+
+#include "qdit.h"
+
+// Device status word values (written by kernels, read by qdit_sync).
+enum : int { QDIT_DEV_OK = 0, QDIT_DEV_TIMEOUT = 1 };
+
+struct TmapKey {
+  const void* ptr;
+  uint64_t rows, cols, ld;
+  uint32_t box_rows, box_cols, swizzle, esize;
+  bool operator==(const TmapKey& o) const {
+    return ptr == o.ptr && rows == o.rows && cols == o.cols && ld == o.ld && box_rows == o.box_rows &&
+           box_cols == o.box_cols && swizzle == o.swizzle && esize == o.esize;
+  }
+};
+struct TmapKeyHash {
+  size_t operator()(const TmapKey& k) const {
+    uint64_t h = reinterpret_cast<uint64_t>(k.ptr);
+    auto mix = [&](uint64_t v) { h ^= v + 0x9E3779B97F4A7C15ull + (h << 6) + (h >> 2); };
+    mix(k.rows); mix(k.cols); mix(k.ld); mix(k.box_rows); mix(k.box_cols); mix(k.swizzle); mix(k.esize);
+    return static_cast<size_t>(h);
+  }
+};
+
+struct qdit_ctx {
+  int device = 0;
+  cudaStream_t stream = nullptr;
+  int* d_status = nullptr;  // device status word
+  int* h_status = nullptr;  // pinned host mirror
+  int num_sms = 0;
+  int64_t launches = 0;
+  std::string last_error;
+  void* encode_fn = nullptr;  // cuTensorMapEncodeTiled
+  std::unordered_map<TmapKey, CUtensorMap, TmapKeyHash> tmaps;
+};
+
+// Records a formatted message on the context and returns `code`.
+int32_t qdit_fail(qdit_ctx* ctx, int32_t code, const char* fmt, ...);
+// Checks the last launch; counts it.
+int32_t qdit_after_launch(qdit_ctx* ctx, const char* what);
+
+#define QDIT_CUDA_CHECK(ctx, expr)                                                                             \
+  do {                                                                                                         \
+    cudaError_t e__ = (expr);                                                                                  \
+    if (e__ != cudaSuccess) return qdit_fail((ctx), QDIT_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e__)); \
+  } while (0)
+#define QDIT_TRY(expr)                 \
+  do {                                 \
+    int32_t st__ = (expr);             \
+    if (st__ != QDIT_OK) return st__;  \
+  } while (0)
+
+// 2-D tensor map over a row-major matrix [rows, cols] of `esize`-byte elements with row pitch `ld`
+// elements; box = box_rows x box_cols elements; swizzle: 0 none, 1 = 128-byte.  Cached per context.
+int32_t qdit_get_tmap(qdit_ctx* ctx, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows,
+                      uint32_t box_cols, uint32_t swizzle, uint32_t esize, CUtensorMap* out);
+
+// Quantizer parameters as the kernels take them.
+struct QuantArgs {
+  float scale;             // s (by value)
+  const float* scale_dev;  // if non-null, overrides `scale`
+  float zp, qmin, qmax;    // as floats (exact small integers)
+};
+inline QuantArgs make_quant_args(const qdit_qparams& qp, const float* scale_dev) {
+  QuantArgs a;
+  a.scale = qp.scale;
+  a.scale_dev = scale_dev;
+  a.zp = static_cast<float>(qp.zero_point);
+  a.qmin = static_cast<float>(qp.qmin);
+  a.qmax = static_cast<float>(qp.qmax);
+  return a;
+}
+int32_t qdit_check_qparams(qdit_ctx* ctx, const qdit_qparams* qp, bool scale_from_device);
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ---- internal launchers used by the model/sampler orchestration (all enqueue on ctx->stream) ----
+int32_t launch_absmax(qdit_ctx* ctx, const void* x, int x_dtype, int64_t M, int64_t K, int64_t ldx, float* absmax_dev);
+int32_t launch_absmax_to_scale(qdit_ctx* ctx, const float* absmax_dev, float* scale_dev, float* running_absmax, int n);

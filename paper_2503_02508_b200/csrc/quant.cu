@@ -1,0 +1,316 @@
+// HBM-bound quantizer kernels: activation quantizer (Eq. 1), abs-max reduction for dynamic ranges,
+// channel-wise weight quantizer, and LayerNorm + adaLN modulation with the fused activation quantizer.
+#include "common.cuh"
+#include "internal.h"
+
+namespace {
+
+using namespace qd;
+
+// ----------------------------------------------------------------------------- activation quantizer
+// One thread per 16 consecutive elements of a row (two 8-element halves); K % 8 == 0.
+template <typename T>
+__global__ void __launch_bounds__(256) act_quant_kernel(const T* __restrict__ x, int64_t M, int64_t K, int64_t ldx,
+                                                        QuantArgs qa, uint8_t* __restrict__ q, int64_t ldq) {
+  const int64_t chunks_per_row = (K + 15) / 16;
+  const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (idx >= M * chunks_per_row) return;
+  const int64_t row = idx / chunks_per_row;
+  const int64_t col = (idx - row * chunks_per_row) * 16;
+  const float scale = qa.scale_dev ? __ldg(qa.scale_dev) : qa.scale;
+  const float inv = __fdiv_rn(1.0f, scale);
+  const T* src = x + row * ldx + col;
+  uint8_t* dst = q + row * ldq + col;
+  const bool second = col + 8 < K;
+  float a[8], b[8];
+  Load8<T>::load(src, a);
+  if (second) Load8<T>::load(src + 8, b);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) a[i] = quantize_code(a[i], inv, qa.zp, qa.qmin, qa.qmax);
+  const uint2 lo = pack_codes8(a);
+  if (second) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) b[i] = quantize_code(b[i], inv, qa.zp, qa.qmin, qa.qmax);
+    const uint2 hi = pack_codes8(b);
+    if ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+      *reinterpret_cast<uint4*>(dst) = make_uint4(lo.x, lo.y, hi.x, hi.y);
+    } else {
+      *reinterpret_cast<uint2*>(dst) = lo;
+      *reinterpret_cast<uint2*>(dst + 8) = hi;
+    }
+  } else {
+    *reinterpret_cast<uint2*>(dst) = lo;
+  }
+}
+
+// ----------------------------------------------------------------------------- abs-max reduction
+// Non-negative floats order like their bit patterns, so the global maximum is an atomicMax on uint32.
+template <typename T>
+__global__ void __launch_bounds__(256) absmax_kernel(const T* __restrict__ x, int64_t M, int64_t K, int64_t ldx,
+                                                     float* __restrict__ absmax) {
+  const int64_t vec_per_row = K / 8;
+  const int64_t total = M * vec_per_row;
+  float m = 0.0f;
+  for (int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; idx < total;
+       idx += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+    const int64_t row = idx / vec_per_row;
+    const int64_t col = (idx - row * vec_per_row) * 8;
+    float v[8];
+    Load8<T>::load(x + row * ldx + col, v);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) m = fmaxf(m, fabsf(v[i]));
+  }
+  m = warp_max(m);
+  __shared__ float smax[8];
+  if ((threadIdx.x & 31) == 0) smax[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    m = threadIdx.x < (blockDim.x >> 5) ? smax[threadIdx.x] : 0.0f;
+    m = warp_max(m);
+    if (threadIdx.x == 0) atomicMax(reinterpret_cast<unsigned int*>(absmax), __float_as_uint(m));
+  }
+}
+
+// scale[i] = absmax[i] / 127 (1 if the range is empty); optionally widens a running maximum.
+__global__ void absmax_to_scale_kernel(const float* __restrict__ absmax, float* __restrict__ scale,
+                                       float* __restrict__ running, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const float a = absmax[i];
+  if (running) running[i] = fmaxf(running[i], a);
+  if (scale) {
+    const float s = __fdiv_rn(a, 127.0f);
+    scale[i] = s > 0.0f ? s : 1.0f;
+  }
+}
+
+// ----------------------------------------------------------------------------- channel-wise weight quantizer
+// One CTA per output row: abs-max over K, then codes and their sum.
+__global__ void __launch_bounds__(256) weight_quant_kernel(const float* __restrict__ w, int64_t K,
+                                                           int8_t* __restrict__ q, float* __restrict__ w_scale,
+                                                           int32_t* __restrict__ w_colsum) {
+  const int64_t n = blockIdx.x;
+  const float* row = w + n * K;
+  __shared__ float sm[8];
+  __shared__ int si[8];
+  float m = 0.0f;
+  for (int64_t k = threadIdx.x * 4; k < K; k += blockDim.x * 4) {
+    const float4 v = *reinterpret_cast<const float4*>(row + k);
+    m = fmaxf(fmaxf(m, fmaxf(fabsf(v.x), fabsf(v.y))), fmaxf(fabsf(v.z), fabsf(v.w)));
+  }
+  m = warp_max(m);
+  if ((threadIdx.x & 31) == 0) sm[threadIdx.x >> 5] = m;
+  __syncthreads();
+  m = 0.0f;
+  for (int i = 0; i < (blockDim.x >> 5); ++i) m = fmaxf(m, sm[i]);
+  float s = __fdiv_rn(m, 127.0f);
+  if (!(s > 0.0f)) s = 1.0f;
+  const float inv = __fdiv_rn(1.0f, s);
+  int sum = 0;
+  for (int64_t k = threadIdx.x * 4; k < K; k += blockDim.x * 4) {
+    const float4 v = *reinterpret_cast<const float4*>(row + k);
+    const int c0 = __float2int_rn(quantize_code(v.x, inv, 0.0f, -127.0f, 127.0f));
+    const int c1 = __float2int_rn(quantize_code(v.y, inv, 0.0f, -127.0f, 127.0f));
+    const int c2 = __float2int_rn(quantize_code(v.z, inv, 0.0f, -127.0f, 127.0f));
+    const int c3 = __float2int_rn(quantize_code(v.w, inv, 0.0f, -127.0f, 127.0f));
+    sum += c0 + c1 + c2 + c3;
+    const uint32_t packed = (c0 & 0xFF) | ((c1 & 0xFF) << 8) | ((c2 & 0xFF) << 16) | (static_cast<uint32_t>(c3 & 0xFF) << 24);
+    *reinterpret_cast<uint32_t*>(q + n * K + k) = packed;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  if ((threadIdx.x & 31) == 0) si[threadIdx.x >> 5] = sum;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int t = 0;
+    for (int i = 0; i < (blockDim.x >> 5); ++i) t += si[i];
+    w_scale[n] = s;
+    w_colsum[n] = t;
+  }
+}
+
+// ----------------------------------------------------------------------------- LayerNorm + modulate (+ quantize)
+// One warp per row; the row lives in registers (NV vectors of 8 per lane).  Two-pass statistics in f32.
+template <int NV>
+__global__ void __launch_bounds__(256) ln_modulate_kernel(const __nv_bfloat16* __restrict__ x, int64_t M, int D,
+                                                          int64_t T, float eps, const float* __restrict__ shift,
+                                                          const float* __restrict__ scale, int64_t ld_mod,
+                                                          void* __restrict__ out, int out_dtype, QuantArgs qa) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= M) return;
+  const int nvec = D >> 3;
+  const __nv_bfloat16* xr = x + row * D;
+  float v[NV][8];
+  float sum = 0.0f;
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    const int vi = lane + 32 * j;
+    if (vi < nvec) {
+      Load8<__nv_bfloat16>::load(xr + vi * 8, v[j]);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) sum += v[j][i];
+    }
+  }
+  const float mean = warp_sum(sum) / static_cast<float>(D);
+  float ss = 0.0f;
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    const int vi = lane + 32 * j;
+    if (vi < nvec) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float d = v[j][i] - mean;
+        ss += d * d;
+      }
+    }
+  }
+  const float var = warp_sum(ss) / static_cast<float>(D);
+  const float rstd = 1.0f / sqrtf(var + eps);
+  const int64_t b = row / T;
+  const float* sh = shift + b * ld_mod;
+  const float* sc = scale + b * ld_mod;
+  float inv = 0.0f;
+  if (out_dtype == QDIT_I8) {
+    const float s = qa.scale_dev ? __ldg(qa.scale_dev) : qa.scale;
+    inv = __fdiv_rn(1.0f, s);
+  }
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    const int vi = lane + 32 * j;
+    if (vi < nvec) {
+      float shv[8], scv[8], y[8];
+      Load8<float>::load(sh + vi * 8, shv);
+      Load8<float>::load(sc + vi * 8, scv);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) y[i] = (v[j][i] - mean) * rstd * (1.0f + scv[i]) + shv[i];
+      const int64_t o = row * D + vi * 8;
+      if (out_dtype == QDIT_I8) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) y[i] = quantize_code(y[i], inv, qa.zp, qa.qmin, qa.qmax);
+        *reinterpret_cast<uint2*>(static_cast<uint8_t*>(out) + o) = pack_codes8(y);
+      } else if (out_dtype == QDIT_BF16) {
+        *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(out) + o) = pack_bf16x8(y);
+      } else {
+        float* of = static_cast<float*>(out) + o;
+        *reinterpret_cast<float4*>(of) = make_float4(y[0], y[1], y[2], y[3]);
+        *reinterpret_cast<float4*>(of + 4) = make_float4(y[4], y[5], y[6], y[7]);
+      }
+    }
+  }
+}
+
+template <int NV>
+void launch_ln(qdit_ctx* ctx, const void* x, int64_t M, int D, int64_t T, float eps, const float* shift,
+               const float* scale, int64_t ld_mod, void* out, int out_dtype, QuantArgs qa) {
+  const int warps = 8;
+  const unsigned grid = static_cast<unsigned>((M + warps - 1) / warps);
+  ln_modulate_kernel<NV><<<grid, warps * 32, 0, ctx->stream>>>(static_cast<const __nv_bfloat16*>(x), M, D, T, eps, shift,
+                                                               scale, ld_mod, out, out_dtype, qa);
+}
+
+}  // namespace
+
+int32_t launch_absmax(qdit_ctx* ctx, const void* x, int x_dtype, int64_t M, int64_t K, int64_t ldx, float* absmax_dev) {
+  const int64_t total = M * (K / 8);
+  if (total == 0) return QDIT_OK;
+  const int64_t want = (total + 255) / 256;
+  const unsigned grid = static_cast<unsigned>(want < ctx->num_sms * 16 ? want : ctx->num_sms * 16);
+  if (x_dtype == QDIT_BF16)
+    absmax_kernel<__nv_bfloat16><<<grid, 256, 0, ctx->stream>>>(static_cast<const __nv_bfloat16*>(x), M, K, ldx, absmax_dev);
+  else
+    absmax_kernel<float><<<grid, 256, 0, ctx->stream>>>(static_cast<const float*>(x), M, K, ldx, absmax_dev);
+  return qdit_after_launch(ctx, "absmax_kernel");
+}
+
+int32_t launch_absmax_to_scale(qdit_ctx* ctx, const float* absmax_dev, float* scale_dev, float* running_absmax, int n) {
+  if (n <= 0) return QDIT_OK;
+  absmax_to_scale_kernel<<<(n + 127) / 128, 128, 0, ctx->stream>>>(absmax_dev, scale_dev, running_absmax, n);
+  return qdit_after_launch(ctx, "absmax_to_scale_kernel");
+}
+
+extern "C" {
+
+int32_t qdit_quantize_act(qdit_ctx* ctx, const void* x, int x_dtype, int64_t M, int64_t K, int64_t ldx, int mode,
+                          const qdit_qparams* qp, float* dyn_scale, void* q, int64_t ldq) {
+  if (!ctx) return QDIT_ERR_INVALID_ARG;
+  if (M < 0 || K < 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "negative size");
+  if (M == 0 || K == 0) return QDIT_OK;
+  if (!x || !q) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "x or q is NULL");
+  if (x_dtype != QDIT_BF16 && x_dtype != QDIT_F32) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "x_dtype must be bf16 or f32");
+  if (K % 8 != 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "K = %lld must be a multiple of 8", static_cast<long long>(K));
+  if (ldx < K || ldq < K) return qdit_fail(ctx, QDIT_ERR_SHAPE, "leading dimension smaller than K");
+  const int64_t esz = x_dtype == QDIT_BF16 ? 2 : 4;
+  if (!aligned16(x) || (ldx * esz) % 16 != 0) return qdit_fail(ctx, QDIT_ERR_ALIGN, "x must be 16-byte aligned (base and row pitch)");
+  if ((reinterpret_cast<uintptr_t>(q) & 7u) || ldq % 8 != 0) return qdit_fail(ctx, QDIT_ERR_ALIGN, "q must be 8-byte aligned (base and row pitch)");
+  QuantArgs qa;
+  if (mode == QDIT_QUANT_STATIC) {
+    QDIT_TRY(qdit_check_qparams(ctx, qp, false));
+    qa = make_quant_args(*qp, nullptr);
+  } else if (mode == QDIT_QUANT_DYNAMIC) {
+    if (!dyn_scale) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "dynamic mode needs dyn_scale");
+    // dyn_scale doubles as the abs-max accumulator before it is turned into the scale in place
+    QDIT_CUDA_CHECK(ctx, cudaMemsetAsync(dyn_scale, 0, sizeof(float), ctx->stream));
+    QDIT_TRY(launch_absmax(ctx, x, x_dtype, M, K, ldx, dyn_scale));
+    QDIT_TRY(launch_absmax_to_scale(ctx, dyn_scale, dyn_scale, nullptr, 1));
+    qdit_qparams sym{1.0f, 0, -127, 127};
+    qa = make_quant_args(sym, dyn_scale);
+  } else {
+    return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "unknown quantizer mode %d", mode);
+  }
+  const int64_t threads = M * ((K + 15) / 16);
+  const unsigned grid = static_cast<unsigned>((threads + 255) / 256);
+  if (x_dtype == QDIT_BF16)
+    act_quant_kernel<__nv_bfloat16><<<grid, 256, 0, ctx->stream>>>(static_cast<const __nv_bfloat16*>(x), M, K, ldx, qa,
+                                                                   static_cast<uint8_t*>(q), ldq);
+  else
+    act_quant_kernel<float><<<grid, 256, 0, ctx->stream>>>(static_cast<const float*>(x), M, K, ldx, qa,
+                                                           static_cast<uint8_t*>(q), ldq);
+  return qdit_after_launch(ctx, "act_quant_kernel");
+}
+
+int32_t qdit_quantize_weight(qdit_ctx* ctx, const float* w, int64_t N, int64_t K, void* q, float* w_scale,
+                             int32_t* w_colsum) {
+  if (!ctx) return QDIT_ERR_INVALID_ARG;
+  if (N < 0 || K < 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "negative size");
+  if (N == 0 || K == 0) return QDIT_OK;
+  if (!w || !q || !w_scale || !w_colsum) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "NULL argument");
+  if (K % 4 != 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "K must be a multiple of 4");
+  if (!aligned16(w) || (reinterpret_cast<uintptr_t>(q) & 3u)) return qdit_fail(ctx, QDIT_ERR_ALIGN, "w must be 16-byte, q 4-byte aligned");
+  weight_quant_kernel<<<static_cast<unsigned>(N), 256, 0, ctx->stream>>>(w, K, static_cast<int8_t*>(q), w_scale, w_colsum);
+  return qdit_after_launch(ctx, "weight_quant_kernel");
+}
+
+int32_t qdit_adaln_modulate(qdit_ctx* ctx, const void* x, int64_t M, int64_t D, int64_t T, float eps,
+                            const float* shift, const float* scale, int64_t ld_mod, void* out, int out_dtype,
+                            const qdit_qparams* out_qp, const float* out_scale_dev) {
+  if (!ctx) return QDIT_ERR_INVALID_ARG;
+  if (M < 0 || D <= 0 || T <= 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "bad sizes");
+  if (M == 0) return QDIT_OK;
+  if (!x || !shift || !scale || !out) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "NULL argument");
+  if (D % 8 != 0 || D > 2048) return qdit_fail(ctx, QDIT_ERR_SHAPE, "D must be a multiple of 8 and <= 2048");
+  if (ld_mod % 4 != 0 || !aligned16(shift) || !aligned16(scale) || !aligned16(x) || !aligned16(out))
+    return qdit_fail(ctx, QDIT_ERR_ALIGN, "pointers must be 16-byte aligned and ld_mod a multiple of 4");
+  if (out_dtype != QDIT_I8 && out_dtype != QDIT_BF16 && out_dtype != QDIT_F32)
+    return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "bad out_dtype");
+  QuantArgs qa{};
+  if (out_dtype == QDIT_I8) {
+    QDIT_TRY(qdit_check_qparams(ctx, out_qp, out_scale_dev != nullptr));
+    qa = make_quant_args(*out_qp, out_scale_dev);
+  }
+  const int nv = static_cast<int>((D / 8 + 31) / 32);
+  const int d = static_cast<int>(D);
+  switch (nv) {
+    case 1: launch_ln<1>(ctx, x, M, d, T, eps, shift, scale, ld_mod, out, out_dtype, qa); break;
+    case 2: launch_ln<2>(ctx, x, M, d, T, eps, shift, scale, ld_mod, out, out_dtype, qa); break;
+    case 3: launch_ln<3>(ctx, x, M, d, T, eps, shift, scale, ld_mod, out, out_dtype, qa); break;
+    case 4: launch_ln<4>(ctx, x, M, d, T, eps, shift, scale, ld_mod, out, out_dtype, qa); break;
+    case 5: launch_ln<5>(ctx, x, M, d, T, eps, shift, scale, ld_mod, out, out_dtype, qa); break;
+    case 6: launch_ln<6>(ctx, x, M, d, T, eps, shift, scale, ld_mod, out, out_dtype, qa); break;
+    case 7: launch_ln<7>(ctx, x, M, d, T, eps, shift, scale, ld_mod, out, out_dtype, qa); break;
+    default: launch_ln<8>(ctx, x, M, d, T, eps, shift, scale, ld_mod, out, out_dtype, qa); break;
+  }
+  return qdit_after_launch(ctx, "ln_modulate_kernel");
+}
+
+}  // extern "C"
