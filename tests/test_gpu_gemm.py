@@ -1,0 +1,204 @@
+"""GPU parity: W8A8 linear (tcgen05 int8 GEMM + de-quantising epilogue) vs the oracle."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import dit, linear, quant
+from oracle.quant import QParams
+
+from gpu_util import bf16_to_f64, code_mismatch_report, dev, dev_i8, host_codes, max_rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def q():
+    import paper_2503_02508_b200 as q
+    return q
+
+
+@pytest.fixture(scope="module")
+def ctx(q):
+    c = q.qdit_create(0, None)
+    yield c
+    q.qdit_destroy(c)
+
+
+def _codes(seed, name, shape, lo, hi):
+    return synth.uniform_int(seed, name, shape, lo, hi + 1)
+
+
+def _run_i32(q, ctx, qa, qw, a_unsigned=False):
+    M, K = qa.shape
+    N = qw.shape[0]
+    A, W = dev_i8(qa), dev_i8(qw)
+    out = torch.full((M, N), -7, dtype=torch.int32, device="cuda")
+    qp = q.qparams(1.0, 0, 0, 255) if a_unsigned else q.qparams(1.0)
+    q.qdit_w8a8_linear(ctx, A, W, M, N, K, qp, None, q.QDIT_EPI_OUT_I32, None, out, N)
+    q.qdit_sync(ctx)
+    return out.cpu().numpy().astype(np.int64)
+
+
+SHAPES = [(1, 8, 16), (128, 192, 128), (130, 200, 272), (256, 384, 1152), (517, 1152, 4608), (512, 1152, 384),
+          (1000, 3456, 1152), (64, 6912, 1152), (2048, 64, 64), (129, 1536, 384)]
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+@pytest.mark.parametrize("bn", ["auto", "64", "128", "192"])
+def test_accumulators_bit_exact(q, ctx, M, N, K, bn):
+    if bn == "auto":
+        os.environ.pop("QDIT_GEMM_BN", None)
+    else:
+        os.environ["QDIT_GEMM_BN"] = bn
+    try:
+        qa = _codes(31, f"a{M}.{K}", (M, K), -128, 127)
+        qw = _codes(31, f"w{N}.{K}", (N, K), -127, 127)
+        got = _run_i32(q, ctx, qa, qw)
+    finally:
+        os.environ.pop("QDIT_GEMM_BN", None)
+    np.testing.assert_array_equal(got, linear.gemm_i8(qa, qw))
+
+
+def test_accumulators_extremes_and_structure(q, ctx):
+    K = 4608
+    lo = np.full((130, K), -128)
+    hi = np.full((200, K), 127)
+    assert (_run_i32(q, ctx, lo, hi) == -128 * 127 * K).all()
+    u8 = np.full((130, K), 255)
+    assert (_run_i32(q, ctx, u8, hi, a_unsigned=True) == 255 * 127 * K).all()
+    # identity weights return the activations; catches any K-offset / swizzle / transposition slip
+    A = _codes(32, "aid", (300, 256), -128, 127)
+    np.testing.assert_array_equal(_run_i32(q, ctx, A, np.eye(256, dtype=np.int64)), A)
+    # one-hot rows pick single weights
+    W = _codes(32, "wsel", (200, 1152), -127, 127)
+    onehot = np.zeros((128, 1152), dtype=np.int64)
+    ks = synth.uniform_int(32, "ks", (128,), 0, 1152)
+    onehot[np.arange(128), ks] = 1
+    np.testing.assert_array_equal(_run_i32(q, ctx, onehot, W), W[:, ks].T)
+
+
+def test_unsigned_activations_bit_exact(q, ctx):
+    qa = _codes(33, "au", (260, 1152), 0, 255)
+    qw = _codes(33, "wu", (392, 1152), -127, 127)
+    np.testing.assert_array_equal(_run_i32(q, ctx, qa, qw, a_unsigned=True), linear.gemm_i8(qa, qw))
+
+
+def test_repeatable(q, ctx):
+    qa = _codes(34, "ar", (1024, 1152), -128, 127)
+    qw = _codes(34, "wr", (1152, 1152), -127, 127)
+    a = _run_i32(q, ctx, qa, qw)
+    b = _run_i32(q, ctx, qa, qw)
+    np.testing.assert_array_equal(a, b)
+
+
+def _layer(seed, M, N, K, T, a_qp):
+    x = synth.outlier_activations(seed, "x", M, K, gain=6.0)
+    Wf = synth.normal(seed, "W", (N, K), 0.02)
+    bias = synth.normal(seed, "b", (N,), 0.02)
+    gate = synth.normal(seed, "g", (M // T, N), 0.35)
+    resid = synth.normal(seed, "r", (M, N), 1.0)
+    qw, s_w, cs = quant.quantize_weight_per_channel(Wf)
+    qa = quant.quantize(x, a_qp)
+    return dict(qa=qa, qw=qw, s_w=s_w, cs=cs, bias=bias, gate=gate, resid=resid)
+
+
+@pytest.mark.parametrize("M,N,K,T", [(512, 384, 384, 256), (300, 200, 1152, 100), (1024, 1152, 4608, 256)])
+@pytest.mark.parametrize("a_qp", [QParams(0.05, 0, -127, 127), QParams(0.047, 131, 0, 255)])
+def test_dequant_bias_f32(q, ctx, M, N, K, T, a_qp):
+    L = _layer(41, M, N, K, T, a_qp)
+    A, W = dev_i8(L["qa"]), dev_i8(L["qw"])
+    epi = q.epilogue(w_scale=dev(L["s_w"]), w_colsum=dev(L["cs"].astype(np.int32)), bias=dev(L["bias"]))
+    keep = [epi]
+    ws, wc, bi = dev(L["s_w"]), dev(L["cs"].astype(np.int32)), dev(L["bias"])
+    epi = q.epilogue(w_scale=ws, w_colsum=wc, bias=bi)
+    out = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    q.qdit_w8a8_linear(ctx, A, W, M, N, K, q.qparams(a_qp.scale, a_qp.zero_point, a_qp.qmin, a_qp.qmax), None,
+                       q.QDIT_EPI_BIAS | q.QDIT_EPI_OUT_F32, epi, out, N)
+    q.qdit_sync(ctx)
+    ref = linear.w8a8_linear(L["qa"], a_qp, L["qw"], L["s_w"], L["cs"], L["bias"])
+    assert max_rel_err(out.cpu().numpy(), ref) < 1e-3      # the stated layer tolerance ...
+    assert max_rel_err(out.cpu().numpy(), ref) < 1e-5      # ... and what f32 arithmetic actually gives
+
+
+def test_gate_residual_cache_epilogue(q, ctx):
+    M, N, K, T = 512, 1152, 1152, 256
+    a_qp = QParams(0.05, 0, -127, 127)
+    L = _layer(42, M, N, K, T, a_qp)
+    A, W = dev_i8(L["qa"]), dev_i8(L["qw"])
+    ws, bi, g = dev(L["s_w"]), dev(L["bias"]), dev(L["gate"])
+    x = dev(L["resid"]).to(torch.bfloat16)
+    xh = bf16_to_f64(x)
+    cache = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    epi = q.epilogue(w_scale=ws, bias=bi, gate=g, ld_gate=N, tokens_per_sample=T, residual=x, cache_out=cache)
+    flags = q.QDIT_EPI_BIAS | q.QDIT_EPI_GATE | q.QDIT_EPI_RESIDUAL | q.QDIT_EPI_CACHE_STORE | q.QDIT_EPI_OUT_BF16
+    q.qdit_w8a8_linear(ctx, A, W, M, N, K, q.qparams(a_qp.scale), None, flags, epi, x, N)    # in place on x
+    q.qdit_sync(ctx)
+    f = linear.w8a8_linear(L["qa"], a_qp, L["qw"], L["s_w"], L["cs"], L["bias"])
+    rows = np.arange(M) // T
+    want_x = xh + L["gate"].astype(np.float64)[rows] * f
+    # bf16 outputs: equal to the rounded oracle value up to one bf16 step where f32 and f64 straddle a tie
+    got_c, got_x = bf16_to_f64(cache), bf16_to_f64(x)
+    assert np.abs(got_c - dit.round_bf16(f)).max() <= 2.0 ** -8 * np.abs(f).max()
+    assert (got_c != dit.round_bf16(f)).mean() < 1e-3
+    assert (got_x != dit.round_bf16(want_x)).mean() < 1e-3
+    assert max_rel_err(got_x, want_x) < 2.0 ** -8
+
+
+def test_gelu_requant_epilogue(q, ctx):
+    M, N, K, T = 384, 1536, 384, 128
+    a_qp = QParams(0.04, 0, -127, 127)
+    L = _layer(43, M, N, K, T, a_qp)
+    A, W = dev_i8(L["qa"]), dev_i8(L["qw"])
+    ws, bi = dev(L["s_w"]), dev(L["bias"])
+    u = dit.gelu_tanh(linear.w8a8_linear(L["qa"], a_qp, L["qw"], L["s_w"], L["cs"], L["bias"]))
+    o_qp = quant.qparams_symmetric(float(np.abs(u).max()) * 0.9)
+    epi = q.epilogue(w_scale=ws, bias=bi, out_qp=q.qparams(o_qp.scale))
+    out = torch.empty((M, N), dtype=torch.uint8, device="cuda")
+    q.qdit_w8a8_linear(ctx, A, W, M, N, K, q.qparams(a_qp.scale), None,
+                       q.QDIT_EPI_BIAS | q.QDIT_EPI_GELU | q.QDIT_EPI_QUANT_OUT, epi, out, N)
+    outf = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    q.qdit_w8a8_linear(ctx, A, W, M, N, K, q.qparams(a_qp.scale), None,
+                       q.QDIT_EPI_BIAS | q.QDIT_EPI_GELU | q.QDIT_EPI_OUT_F32, epi, outf, N)
+    q.qdit_sync(ctx)
+    assert max_rel_err(outf.cpu().numpy(), u) < 1e-3
+    assert max_rel_err(outf.cpu().numpy(), u) < 2e-5
+    got, want = host_codes(out), quant.quantize(u, o_qp)
+    pre = u.astype(np.float32).astype(np.float64) * float(o_qp.inv_scale)
+    n_bad, ok = code_mismatch_report(got, want, pre, 2e-5 * np.abs(pre).max() + 1e-6)
+    assert ok and n_bad <= 1e-3 * got.size, (n_bad, got.size)
+    # the fused codes are exactly the quantizer applied to the kernel's own f32 values
+    np.testing.assert_array_equal(got, quant.quantize(outf.cpu().numpy(), o_qp))
+
+
+def test_device_scale_override(q, ctx):
+    M, N, K = 256, 192, 256
+    a_qp = QParams(0.05, 0, -127, 127)
+    L = _layer(44, M, N, K, 256, a_qp)
+    A, W, ws = dev_i8(L["qa"]), dev_i8(L["qw"]), dev(L["s_w"])
+    sd = dev(np.array([a_qp.scale], dtype=np.float32))
+    out = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    q.qdit_w8a8_linear(ctx, A, W, M, N, K, q.qparams(123.0), sd, q.QDIT_EPI_OUT_F32, q.epilogue(w_scale=ws), out, N)
+    q.qdit_sync(ctx)
+    ref = linear.w8a8_linear(L["qa"], a_qp, L["qw"], L["s_w"], L["cs"], None)
+    assert max_rel_err(out.cpu().numpy(), ref) < 1e-5
+
+
+def test_rejects_bad_arguments(q, ctx):
+    import ctypes as C
+    A = torch.zeros((128, 64), dtype=torch.int8, device="cuda")
+    W = torch.zeros((64, 64), dtype=torch.int8, device="cuda")
+    o = torch.zeros((128, 64), dtype=torch.int32, device="cuda")
+    L, qp = q.lib, q.qparams(1.0)
+    f = L.qdit_w8a8_linear
+    assert f(ctx, A.data_ptr(), W.data_ptr(), 128, 64, 24, qp, None, q.QDIT_EPI_OUT_I32, None, o.data_ptr(), 64) == q.QDIT_ERR_SHAPE
+    assert f(ctx, A.data_ptr(), W.data_ptr(), 128, 60, 64, qp, None, q.QDIT_EPI_OUT_I32, None, o.data_ptr(), 64) == q.QDIT_ERR_SHAPE
+    assert f(ctx, None, W.data_ptr(), 128, 64, 64, qp, None, q.QDIT_EPI_OUT_I32, None, o.data_ptr(), 64) == q.QDIT_ERR_INVALID_ARG
+    assert f(ctx, A.data_ptr() + 1, W.data_ptr(), 128, 64, 64, qp, None, q.QDIT_EPI_OUT_I32, None, o.data_ptr(), 64) == q.QDIT_ERR_ALIGN
+    assert f(ctx, A.data_ptr(), W.data_ptr(), 128, 64, 64, qp, None, 0, None, o.data_ptr(), 64) == q.QDIT_ERR_INVALID_ARG
+    assert f(ctx, A.data_ptr(), W.data_ptr(), 128, 64, 64, qp, None, q.QDIT_EPI_OUT_F32 | q.QDIT_EPI_OUT_BF16, None, o.data_ptr(), 64) == q.QDIT_ERR_INVALID_ARG
+    assert f(ctx, A.data_ptr(), W.data_ptr(), 128, 64, 64, qp, None, q.QDIT_EPI_OUT_F32, None, o.data_ptr(), 64) == q.QDIT_ERR_INVALID_ARG
+    assert f(ctx, A.data_ptr(), W.data_ptr(), 0, 64, 64, qp, None, q.QDIT_EPI_OUT_I32, None, o.data_ptr(), 64) == q.QDIT_OK
+    q.qdit_sync(ctx)
