@@ -99,7 +99,7 @@ def attention(q, k, v, scale: Optional[float] = None):
 # ----------------------------------------------------------------------------- quantized model
 @dataclass
 class QLinear:
-    q: np.ndarray        # int32 codes [N,K]
+    q: np.ndarray        # int8 codes [N,K]
     scale: np.ndarray    # float32 [N]
     colsum: np.ndarray   # int64 [N]
     bias: np.ndarray     # float32 [N]
@@ -108,7 +108,7 @@ class QLinear:
 
 def make_qlinear(w, b) -> QLinear:
     q, s, cs = quantize_weight_per_channel(w)
-    return QLinear(q, s, cs, np.asarray(b, dtype=F32), np.asarray(w, dtype=F32))
+    return QLinear(q.astype(np.int8), s, cs, np.asarray(b, dtype=F32), np.asarray(w, dtype=F32))
 
 
 @dataclass

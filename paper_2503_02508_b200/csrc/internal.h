@@ -87,3 +87,6 @@ static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t
 // ---- internal launchers used by the model/sampler orchestration (all enqueue on ctx->stream) ----
 int32_t launch_absmax(qdit_ctx* ctx, const void* x, int x_dtype, int64_t M, int64_t K, int64_t ldx, float* absmax_dev);
 int32_t launch_absmax_to_scale(qdit_ctx* ctx, const float* absmax_dev, float* scale_dev, float* running_absmax, int n);
+// Quantizes an f32 tensor [M,K] (contiguous) with the scale held in device memory.
+int32_t qdit_quantize_act_dev(qdit_ctx* ctx, const float* x, int64_t M, int64_t K, qdit_qparams qp,
+                              const float* scale_dev, uint8_t* q);

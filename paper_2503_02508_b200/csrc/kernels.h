@@ -1,0 +1,22 @@
+// Launchers of the glue kernels (embedders, final layer, sampler update), used by the model/sampler code.
+#pragma once
+#include "internal.h"
+
+struct DdimCoef {
+  float sqrt_ab_t, sqrt_1mab_t, sqrt_ab_prev, sqrt_1mab_prev;
+};
+
+// x[m,:] = bf16(W_patch . patch(m) + b + pos); sample b reads latent[b % latent_batch].
+int32_t launch_embed(qdit_ctx* ctx, const float* latent, int latent_batch, const float* w, const float* bias,
+                     const float* pos, void* x, int64_t M, int D, int grid, int patch, int C);
+// h[b,:] = SiLU(W1 . sinusoid(t_b) + b1)
+int32_t launch_cond1(qdit_ctx* ctx, const float* t, const float* w1, const float* b1, float* h, int B, int D, int F);
+// out[b,n] = W[n,:] . f(in[b,:]) + bias[n] (+ table[y[b],n]); f = SiLU if silu_input; out_silu (optional) = SiLU(out)
+int32_t launch_small_linear(qdit_ctx* ctx, const float* in, const float* w, const float* bias, const float* table,
+                            const int32_t* y, float* out, float* out_silu, int B, int N, int K, int silu_input);
+// LayerNorm + modulate + linear D->OUT + un-patchify into net [B, OUT/p^2, side, side]
+int32_t launch_final(qdit_ctx* ctx, const void* x, int64_t M, int D, int T, float eps, const float* modf,
+                     const float* w, const float* bias, float* net, int grid, int patch, int OUT);
+// guidance combine + DDIM (eta = 0) update of latent [B,C,HW] from net [Beff,2C,HW]
+int32_t launch_cfg_ddim(qdit_ctx* ctx, float* latent, const float* net, int B, int C, int HW, int use_cfg,
+                        float guidance, const DdimCoef& k);

@@ -229,6 +229,15 @@ int32_t launch_absmax_to_scale(qdit_ctx* ctx, const float* absmax_dev, float* sc
   return qdit_after_launch(ctx, "absmax_to_scale_kernel");
 }
 
+int32_t qdit_quantize_act_dev(qdit_ctx* ctx, const float* x, int64_t M, int64_t K, qdit_qparams qp,
+                              const float* scale_dev, uint8_t* q) {
+  if (M == 0 || K == 0) return QDIT_OK;
+  const QuantArgs qa = make_quant_args(qp, scale_dev);
+  const int64_t threads = M * ((K + 15) / 16);
+  act_quant_kernel<float><<<static_cast<unsigned>((threads + 255) / 256), 256, 0, ctx->stream>>>(x, M, K, K, qa, q, K);
+  return qdit_after_launch(ctx, "act_quant_kernel");
+}
+
 extern "C" {
 
 int32_t qdit_quantize_act(qdit_ctx* ctx, const void* x, int x_dtype, int64_t M, int64_t K, int64_t ldx, int mode,

@@ -1,0 +1,108 @@
+"""GPU parity: block-output cache kernels and the variance-compensation kernel vs the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import dit, vc
+
+from gpu_util import bf16_to_f64, dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def q():
+    import paper_2503_02508_b200 as q
+    return q
+
+
+@pytest.fixture(scope="module")
+def ctx(q):
+    c = q.qdit_create(0, None)
+    yield c
+    q.qdit_destroy(c)
+
+
+def test_cache_schedule_host():
+    import paper_2503_02508_b200 as q
+    from oracle import sampler
+    for interval in (1, 2, 3, 7):
+        for i in range(20):
+            assert q.qdit_cache_should_refresh(i, interval) == int(sampler.should_refresh(i, interval))
+    assert q.qdit_cache_should_refresh(0, 0) == q.QDIT_ERR_INVALID_ARG
+    assert q.qdit_cache_should_refresh(-1, 2) == q.QDIT_ERR_INVALID_ARG
+
+
+def test_cache_store_reuse_and_state(q, ctx):
+    blocks, B, T, D = 3, 2, 64, 144
+    M = B * T
+    cache = q.qdit_cache_create(ctx, blocks, M, D)
+    try:
+        x0 = synth.normal(61, "x", (M, D))
+        xd = dev(x0).to(torch.bfloat16)
+        mod = synth.normal(61, "mod", (B, blocks * 6 * D), 0.35)
+        md = dev(mod)
+        # reuse before any store is a state error, not a read of uninitialised memory
+        assert q.lib.qdit_cache_reuse(ctx, cache, 0, 0, md.data_ptr(), blocks * 6 * D, T, xd.data_ptr()) == q.QDIT_ERR_STATE
+        assert q.lib.qdit_cache_reuse_all(ctx, cache, md.data_ptr(), blocks * 6 * D, T, xd.data_ptr()) == q.QDIT_ERR_STATE
+        ys = {}
+        for b in range(blocks):
+            for br in (0, 1):
+                y = dev(synth.normal(61, f"y{b}.{br}", (M, D))).to(torch.bfloat16)
+                ys[(b, br)] = bf16_to_f64(y)
+                q.qdit_cache_store(ctx, cache, b, br, y)
+        rows = np.arange(M) // T
+        # one fused pass == the closed form of a fully skipped step
+        x1 = xd.clone()
+        q.qdit_cache_reuse_all(ctx, cache, md, blocks * 6 * D, T, x1)
+        q.qdit_sync(ctx)
+        want = bf16_to_f64(xd).copy()
+        for b in range(blocks):
+            want += mod[rows, b * 6 * D + 2 * D:b * 6 * D + 3 * D].astype(np.float64) * ys[(b, 0)]
+            want += mod[rows, b * 6 * D + 5 * D:b * 6 * D + 6 * D].astype(np.float64) * ys[(b, 1)]
+        got = bf16_to_f64(x1)
+        assert (got != dit.round_bf16(want)).mean() < 2e-3                     # f32 vs f64 sums straddling a bf16 tie
+        assert np.abs(got - want).max() <= 2.0 ** -8 * np.abs(want).max()
+        # single-slot reuse: x + gate * slot
+        x2 = xd.clone()
+        g = md[:, 2 * D:3 * D]
+        q.qdit_cache_reuse(ctx, cache, 0, q.QDIT_BRANCH_ATTN, g, blocks * 6 * D, T, x2)
+        q.qdit_sync(ctx)
+        want2 = bf16_to_f64(xd) + mod[rows, 2 * D:3 * D].astype(np.float64) * ys[(0, 0)]
+        assert (bf16_to_f64(x2) != dit.round_bf16(want2)).mean() < 2e-3
+        # invalidation empties the cache again
+        q.qdit_cache_invalidate(cache)
+        assert q.lib.qdit_cache_reuse(ctx, cache, 0, 0, md.data_ptr(), blocks * 6 * D, T, xd.data_ptr()) == q.QDIT_ERR_STATE
+        assert q.qdit_cache_slot(cache, blocks, 0) is None and q.qdit_cache_slot(cache, 0, 2) is None
+    finally:
+        q.qdit_cache_destroy(cache)
+
+
+@pytest.mark.parametrize("B,C,HW", [(3, 4, 1024), (2, 4, 4096), (1, 3, 64)])
+def test_vc_correct(q, ctx, B, C, HW):
+    S = 5
+    x = synth.normal(62, f"lat{HW}", (B, C, HW)) * np.array([0.5, 1.0, 2.0, 3.0][:C], dtype=np.float32).reshape(1, C, 1) + 0.4
+    K = (1.0 + 0.1 * synth.normal(62, "K", (S, C))).astype(np.float32)
+    kd = dev(K)
+    side = int(np.sqrt(HW))
+    for step in (0, 3):
+        xd = dev(x)
+        q.qdit_vc_correct(ctx, xd, B, C, HW, step, q.QDIT_VC_K_TABLE, kd, 1e-6)
+        q.qdit_sync(ctx)
+        want = vc.apply(x.reshape(B, C, side, side), K[step]).reshape(B, C, HW)
+        np.testing.assert_allclose(xd.cpu().numpy(), want, rtol=2e-6, atol=2e-6)
+    tgt = np.abs(synth.normal(62, "tgt", (S, C))).astype(np.float32) + 0.2
+    xd = dev(x)
+    q.qdit_vc_correct(ctx, xd, B, C, HW, 2, q.QDIT_VC_VAR_RATIO, dev(tgt), 1e-6)
+    q.qdit_sync(ctx)
+    got = xd.cpu().numpy().astype(np.float64)
+    want = vc.apply(x.reshape(B, C, side, side), tgt[2], mode="var_ratio", eps=1e-6).reshape(B, C, HW)
+    np.testing.assert_allclose(got, want, rtol=5e-6, atol=5e-6)
+    np.testing.assert_allclose(got.var(axis=2), np.broadcast_to(tgt[2], (B, C)), rtol=1e-4)   # reaches the target variance
+    np.testing.assert_allclose(got.mean(axis=2), x.astype(np.float64).mean(axis=2), atol=1e-5)  # mean preserved
+    # K = 1 leaves the latent unchanged up to f32 rounding of mu + (x - mu)
+    xd = dev(x)
+    q.qdit_vc_correct(ctx, xd, B, C, HW, 0, q.QDIT_VC_K_TABLE, dev(np.ones((S, C), dtype=np.float32)), 1e-6)
+    q.qdit_sync(ctx)
+    np.testing.assert_allclose(xd.cpu().numpy(), x, rtol=0, atol=1e-6)
