@@ -1,6 +1,8 @@
 """Seeded tensor generators (see package docstring).  numpy only."""
 from __future__ import annotations
 
+import concurrent.futures
+import os
 import zlib
 from dataclasses import dataclass
 
@@ -135,8 +137,10 @@ def model_weights(seed: int, cfg: DiTConfig) -> dict:
         "b_ada_f": normal(seed, "b_ada_f", (2 * D,), _W_STD),
         "w_out": normal(seed, "w_out", (cfg.out_dim, D), _W_STD),
         "b_out": normal(seed, "b_out", (cfg.out_dim,), _W_STD),
-        "blocks": [block_weights(seed, cfg, i) for i in range(cfg.depth)],
     }
+    # every tensor has its own stream, so blocks can be drawn concurrently with identical results
+    with concurrent.futures.ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as ex:
+        w["blocks"] = list(ex.map(lambda i: block_weights(seed, cfg, i), range(cfg.depth)))
     return w
 
 

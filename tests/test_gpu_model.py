@@ -1,0 +1,291 @@
+"""GPU parity of the composed path: a DiT block from the primitives, whole-network evaluation,
+on-device calibration, and the cached sampler, all against the oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import calib, dit, quant, sampler
+from oracle.quant import QParams
+
+from gpu_util import (bf16_steps_err, bf16_to_f64, bf16_view_to_f64, code_mismatch_report, dev, host_codes, max_rel_err, rel_l2,
+                      scales_to_arrays, view)
+
+pytestmark = pytest.mark.gpu
+
+LINEAR_IDS = {"ada": 0, "qkv": 1, "proj": 2, "fc1": 3, "fc2": 4}
+
+
+@pytest.fixture(scope="module")
+def q():
+    import paper_2503_02508_b200 as q
+    return q
+
+
+@pytest.fixture(scope="module")
+def ctx(q):
+    c = q.qdit_create(0, None)
+    yield c
+    q.qdit_destroy(c)
+
+
+class Rig:
+    """GPU model + oracle model built from the same seeded float weights."""
+
+    def __init__(self, q, ctx, cfg, seed):
+        self.q, self.ctx, self.cfg = q, ctx, cfg
+        self.w = synth.model_weights(seed, cfg)
+        self.om = dit.make_qmodel(cfg, self.w)
+        self.gm = q.qdit_model_create(ctx, cfg, self.w)
+        self.samplers = []
+
+    def set_scales(self, scales):
+        ada, blk = scales_to_arrays(scales, self.cfg.depth)
+        self.q.qdit_model_set_act_scales(self.ctx, self.gm, ada, blk)
+
+    def sampler(self, **kw):
+        s = self.q.qdit_sampler_create(self.ctx, self.gm, **kw)
+        self.samplers.append(s)
+        return s
+
+    def forward(self, s, latent, t, y, flags=0):
+        B = latent.shape[0]
+        out = torch.empty((B, 2 * self.cfg.channels, self.cfg.latent_side, self.cfg.latent_side), dtype=torch.float32,
+                          device="cuda")
+        self.q.qdit_forward(self.ctx, s, dev(latent), dev(np.asarray(t, dtype=np.float32)),
+                            dev(np.asarray(y, dtype=np.int32)), B, out, flags)
+        self.q.qdit_sync(self.ctx)
+        return out.cpu().numpy().astype(np.float64)
+
+    def close(self):
+        for s in self.samplers:
+            self.q.qdit_sampler_destroy(s)
+        self.q.qdit_model_destroy(self.gm)
+
+
+def _inputs(cfg, seed, B):
+    latent = synth.normal(seed, "latent", (B, cfg.channels, cfg.latent_side, cfg.latent_side))
+    t = synth.uniform_int(seed, "t", (B,), 0, 1000).astype(np.float64)
+    y = synth.uniform_int(seed, "y", (B,), 0, cfg.num_classes)
+    return latent, t, y
+
+
+# ----------------------------------------------------------------------------- weights
+@pytest.mark.parametrize("cfg", [synth.DIT_TINY, synth.DIT_S2_BLOCK], ids=["tiny", "s2"])
+def test_model_weights_quantized_bit_exact(q, ctx, cfg):
+    rig = Rig(q, ctx, cfg, 71)
+    try:
+        for i, blk in enumerate(rig.om.blocks):
+            for name, wid in LINEAR_IDS.items():
+                L = q.qdit_model_linear(rig.gm, i, wid)
+                lin = getattr(blk, name)
+                assert (L["N"], L["K"]) == lin.q.shape
+                np.testing.assert_array_equal(view(L["w_q"], lin.q.shape, "|i1").cpu().numpy(), lin.q)
+                np.testing.assert_array_equal(view(L["w_scale"], (L["N"],), "<f4").cpu().numpy(), lin.scale)
+                np.testing.assert_array_equal(view(L["w_colsum"], (L["N"],), "<i4").cpu().numpy(), lin.colsum)
+                np.testing.assert_array_equal(view(L["bias"], (L["N"],), "<f4").cpu().numpy(), lin.bias)
+    finally:
+        rig.close()
+
+
+# ----------------------------------------------------------------------------- one block from the primitives
+def test_block_s2_from_primitives(q, ctx):
+    """Single DiT-S/2-shaped block, W8A8, batch 2, 256 tokens; activation scales from a seeded calibration batch."""
+    cfg = synth.DIT_S2_BLOCK
+    seed = synth.CONFIG_SEEDS["block_s2"]
+    D, H, F, T, B = cfg.hidden, cfg.heads, cfg.mlp, cfg.tokens, 2
+    M = B * T
+    rig = Rig(q, ctx, cfg, seed)
+    try:
+        blk = rig.om.blocks[0]
+        x0 = synth.normal(seed, "tokens", (M, D))
+        c = synth.normal(seed, "cond", (B, D))
+        cal = [(synth.normal(seed, f"cal_tokens{i}", (M, D)), synth.normal(seed, f"cal_cond{i}", (B, D))) for i in range(8)]
+        scales = calib.calibrate_block(blk, cal, T, H)
+        taps = {}
+        octx = dit.Context(quant="static", scales=scales, tap=lambda n, a: taps.__setitem__(n, np.array(a)))
+        x_ref = dit.block_forward(octx, blk, dit.store(x0, "bf16"), c, T, H, 0)
+
+        lin = {n: q.qdit_model_linear(rig.gm, 0, i) for n, i in LINEAR_IDS.items()}
+        sq = lambda n: q.qparams((scales.ada if n == "ada" else scales.blocks[0][n]).scale)
+
+        def linear(A, name, flags, out, **epi):
+            L = lin[name]
+            e = q.epilogue(w_scale=L["w_scale"], w_colsum=L["w_colsum"], bias=L["bias"], **epi)
+            q.qdit_w8a8_linear(ctx, A, L["w_q"], M if name != "ada" else B, L["N"], L["K"], sq(name), None,
+                               flags | q.QDIT_EPI_BIAS, e, out, L["N"])
+
+        x = dev(x0).to(torch.bfloat16)
+        sc = dev(dit.silu(c.astype(np.float64)).astype(np.float32))
+        ca = torch.empty((B, D), dtype=torch.uint8, device="cuda")
+        q.qdit_quantize_act(ctx, sc, q.QDIT_F32, B, D, D, q.QDIT_QUANT_STATIC, sq("ada"), None, ca, D)
+        mod = torch.empty((B, 6 * D), dtype=torch.float32, device="cuda")
+        linear(ca, "ada", q.QDIT_EPI_OUT_F32, mod)
+        h = torch.empty((M, D), dtype=torch.uint8, device="cuda")
+        q.qdit_adaln_modulate(ctx, x, M, D, T, 1e-6, mod[:, 0:], mod[:, D:], 6 * D, h, q.QDIT_I8, sq("qkv"))
+        qkv = torch.empty((M, 3 * D), dtype=torch.bfloat16, device="cuda")
+        linear(h, "qkv", q.QDIT_EPI_OUT_BF16, qkv)
+        a = torch.empty((M, D), dtype=torch.uint8, device="cuda")
+        p = qkv.data_ptr()
+        q.qdit_attention(ctx, p, p + 2 * D, p + 4 * D, 3 * D, B, H, T, D // H, 1.0 / np.sqrt(D // H), a, q.QDIT_I8, sq("proj"))
+        gflags = q.QDIT_EPI_GATE | q.QDIT_EPI_RESIDUAL | q.QDIT_EPI_OUT_BF16
+        linear(a, "proj", gflags, x, gate=mod[:, 2 * D:], ld_gate=6 * D, tokens_per_sample=T, residual=x)
+        h2 = torch.empty((M, D), dtype=torch.uint8, device="cuda")
+        q.qdit_adaln_modulate(ctx, x, M, D, T, 1e-6, mod[:, 3 * D:], mod[:, 4 * D:], 6 * D, h2, q.QDIT_I8, sq("fc1"))
+        u = torch.empty((M, F), dtype=torch.uint8, device="cuda")
+        linear(h2, "fc1", q.QDIT_EPI_GELU | q.QDIT_EPI_QUANT_OUT, u, out_qp=sq("fc2"))
+        linear(u, "fc2", gflags, x, gate=mod[:, 5 * D:], ld_gate=6 * D, tokens_per_sample=T, residual=x)
+        q.qdit_sync(ctx)
+
+        # modulation: a de-quantized layer output -> max relative error 1e-3
+        assert max_rel_err(mod.cpu().numpy(), taps["blk0.mod"]) < 1e-3
+        np.testing.assert_array_equal(host_codes(ca), taps["blk0.ada.qa"])
+        # fused LN quantizer: codes equal the oracle's except within f32 reach of a rounding boundary
+        pre = taps["blk0.qkv.in"].astype(np.float32).astype(np.float64) * float(scales.blocks[0]["qkv"].inv_scale)
+        n_bad, ok = code_mismatch_report(host_codes(h), taps["blk0.qkv.qa"], pre, 1e-3 * np.abs(pre).max())
+        assert ok and n_bad < 2e-3 * h.numel(), n_bad
+        # QKV in bf16: oracle value rounded to bf16, up to one step at ties
+        got_qkv = bf16_to_f64(qkv)
+        assert bf16_steps_err(got_qkv, taps["blk0.qkv.out"]) <= 1.0
+        assert rel_l2(got_qkv, taps["blk0.qkv.out"]) < 2e-3
+        # block output (bf16 residual stream)
+        got = bf16_to_f64(x)
+        assert rel_l2(got, x_ref) < 2e-3, rel_l2(got, x_ref)
+        assert bf16_steps_err(got, x_ref) <= 2.0          # bf16 residual stream: a couple of rounding flips at most
+    finally:
+        rig.close()
+
+
+# ----------------------------------------------------------------------------- whole network
+def _forward_case(q, ctx, cfg, seed, B, depth_note=""):
+    rig = Rig(q, ctx, cfg, seed)
+    latent, t, y = _inputs(cfg, seed, B)
+    scales = calib.calibrate_model(rig.om, [(latent, t, y)])
+    rig.set_scales(scales)
+    return rig, latent, t, y, scales
+
+
+def test_forward_tiny_matches_oracle(q, ctx):
+    cfg = synth.DIT_TINY
+    rig, latent, t, y, scales = _forward_case(q, ctx, cfg, 72, 3)
+    try:
+        s = rig.sampler(batch=3, num_steps=4)
+        got = rig.forward(s, latent, t, y)
+        taps = {}
+        octx = dit.Context(quant="static", scales=scales, tap=lambda n, a: taps.__setitem__(n, np.array(a)))
+        ref = dit.forward(rig.om, octx, latent, t, y)
+        M, D = 3 * cfg.tokens, cfg.hidden
+        assert max_rel_err(view(q.qdit_sampler_buffer(s, "c"), (3, D), "<f4").cpu().numpy(), taps["c"]) < 1e-4
+        assert max_rel_err(view(q.qdit_sampler_buffer(s, "mod"), (3, cfg.depth * 6 * D), "<f4").cpu().numpy(),
+                           np.concatenate([taps[f"blk{i}.mod"] for i in range(cfg.depth)], axis=1)) < 1e-3
+        assert rel_l2(bf16_view_to_f64(q.qdit_sampler_buffer(s, "x"), (M, D)), taps["x_final"]) < 3e-3
+        assert rel_l2(got, ref) < 5e-3, rel_l2(got, ref)
+        assert max_rel_err(got, ref) < 5e-2
+        # a smaller batch through the same workspace gives the same per-sample result
+        got1 = rig.forward(s, latent[1:2], t[1:2], y[1:2])
+        np.testing.assert_array_equal(got1, got[1:2])
+    finally:
+        rig.close()
+
+
+def test_forward_xl_width_two_blocks(q, ctx):
+    cfg = synth.DiTConfig(hidden=1152, heads=16, mlp=4608, depth=2, grid=16)
+    rig, latent, t, y, scales = _forward_case(q, ctx, cfg, 73, 2)
+    try:
+        s = rig.sampler(batch=2, num_steps=2)
+        got = rig.forward(s, latent, t, y)
+        ref = dit.forward(rig.om, dit.Context(quant="static", scales=scales), latent, t, y)
+        assert rel_l2(got, ref) < 5e-3, rel_l2(got, ref)
+    finally:
+        rig.close()
+
+
+def test_on_device_calibration_matches_oracle(q, ctx):
+    cfg = synth.DIT_TINY
+    rig = Rig(q, ctx, cfg, 74)
+    try:
+        batches = [_inputs(cfg, 74 + i, 2) for i in range(3)]
+        want = calib.calibrate_model(rig.om, batches)
+        s = rig.sampler(batch=2, num_steps=2)
+        q.qdit_model_begin_calibration(ctx, rig.gm)
+        for latent, t, y in batches:
+            rig.forward(s, latent, t, y, q.QDIT_FWD_CALIBRATE)
+        q.qdit_model_finish_calibration(ctx, rig.gm)
+        q.qdit_sync(ctx)
+        ada, blk = q.qdit_model_get_act_scales(ctx, rig.gm, cfg.depth)
+        w_ada, w_blk = scales_to_arrays(want, cfg.depth)
+        assert abs(ada - w_ada) <= 1e-5 * w_ada
+        np.testing.assert_allclose(blk, w_blk, rtol=5e-3)        # ranges are maxima of values that agree to ~1e-3
+        # the calibrated model then runs the static path
+        latent, t, y = batches[0]
+        got = rig.forward(s, latent, t, y)
+        ref = dit.forward(rig.om, dit.Context(quant="static", scales=want), latent, t, y)
+        assert rel_l2(got, ref) < 1e-2
+    finally:
+        rig.close()
+
+
+def test_forward_requires_scales(q, ctx):
+    cfg = synth.DIT_TINY
+    rig = Rig(q, ctx, cfg, 75)
+    try:
+        s = rig.sampler(batch=1, num_steps=2)
+        latent, t, y = _inputs(cfg, 75, 1)
+        with pytest.raises(q.QditError) as e:
+            rig.forward(s, latent, t, y)
+        assert e.value.status == q.QDIT_ERR_STATE
+    finally:
+        rig.close()
+
+
+# ----------------------------------------------------------------------------- sampler
+def _run_sampler(rig, latent, labels, **kw):
+    q, ctx = rig.q, rig.ctx
+    s = rig.sampler(batch=latent.shape[0], **kw)
+    out = np.empty_like(latent, dtype=np.float32)
+    lat = np.ascontiguousarray(latent, dtype=np.float32)
+    lab = np.ascontiguousarray(labels, dtype=np.int32)
+    q.qdit_sample(ctx, s, lat, lab, out)
+    return out.astype(np.float64), s
+
+
+@pytest.mark.parametrize("interval,guidance,use_vc", [(1, None, False), (2, 1.5, True), (3, None, True), (20, 1.5, False)])
+def test_sampler_tiny_matches_oracle(q, ctx, interval, guidance, use_vc):
+    cfg = synth.DIT_TINY
+    S, B = 10, 3
+    rig, latent, t, y, scales = _forward_case(q, ctx, cfg, 76, B)
+    try:
+        K = (1.0 + 0.03 * synth.normal(76, "K", (S, cfg.channels))).astype(np.float32) if use_vc else None
+        got, s = _run_sampler(rig, latent, y, num_steps=S, cache_interval=interval, use_cfg=guidance is not None,
+                              guidance=guidance or 1.0, vc_mode=q.QDIT_VC_K_TABLE if use_vc else q.QDIT_VC_NONE, vc_table=K)
+        ref = sampler.sample(rig.om, dit.Context(quant="static", scales=scales),
+                             sampler.SamplerConfig(S, cache_interval=interval, guidance=guidance, vc_table=K), latent, y)
+        assert rel_l2(got, ref) < 2e-2, rel_l2(got, ref)       # the stated end-to-end tolerance
+        assert rel_l2(got, ref) < 5e-3, rel_l2(got, ref)       # and the margin this path actually has
+        # steps out of order are refused
+        assert q.lib.qdit_sample_step(ctx, s, 3) == q.QDIT_ERR_STATE
+    finally:
+        rig.close()
+
+
+def test_sampler_step_by_step_and_cache_effect(q, ctx):
+    cfg = synth.DIT_TINY
+    S, B = 6, 2
+    rig, latent, t, y, scales = _forward_case(q, ctx, cfg, 77, B)
+    try:
+        a, _ = _run_sampler(rig, latent, y, num_steps=S, cache_interval=1)
+        b, _ = _run_sampler(rig, latent, y, num_steps=S, cache_interval=2)
+        assert not np.array_equal(a, b) and rel_l2(b, a) < 0.2
+        # same trajectory twice: deterministic
+        b2, _ = _run_sampler(rig, latent, y, num_steps=S, cache_interval=2)
+        np.testing.assert_array_equal(b, b2)
+        # explicit stepping from device buffers equals the host-buffer convenience call
+        s = rig.sampler(batch=B, num_steps=S, cache_interval=2)
+        q.qdit_sampler_reset(ctx, s, dev(latent), dev(y.astype(np.int32)))
+        for i in range(S):
+            q.qdit_sample_step(ctx, s, i)
+        q.qdit_sync(ctx)
+        got = view(q.qdit_sampler_latent(s), latent.shape, "<f4").cpu().numpy().astype(np.float64)
+        np.testing.assert_array_equal(got, b)
+    finally:
+        rig.close()
