@@ -56,6 +56,19 @@ const char* qdit_last_error(const qdit_ctx* ctx);
 /* Number of kernels this context has launched since creation (for launch accounting). */
 int64_t qdit_launch_count(const qdit_ctx* ctx);
 
+/* Per-kernel timing for measurement (the paper has no counterpart): while enabled, every kernel launch of
+ * this context is bracketed by CUDA events on the context's stream.  qdit_profile_read synchronises the
+ * stream and returns, for one kernel kind, the launches since profiling was enabled, their summed device
+ * time in ms and their summed algorithmic work (integer ops for QDIT_PROF_GEMM, flops for
+ * QDIT_PROF_ATTENTION, bytes that must cross HBM for the others).  Enabling resets the counters.
+ * The events cost a few microseconds per launch: leave profiling off when timing end to end. */
+enum {
+  QDIT_PROF_GEMM = 0, QDIT_PROF_ATTENTION = 1, QDIT_PROF_LN_MODULATE = 2, QDIT_PROF_ACT_QUANT = 3,
+  QDIT_PROF_CACHE_REUSE = 4, QDIT_PROF_OTHER = 5, QDIT_PROF_KINDS = 6
+};
+int32_t qdit_profile_enable(qdit_ctx* ctx, int enable);
+int32_t qdit_profile_read(qdit_ctx* ctx, int kind, int64_t* launches, double* ms, double* work);
+
 /* ------------------------------------------------------------------------------------------------
  * Uniform quantizer, Eq. 1:  Q(X|b) = clip(round(X/s) + z, qmin, qmax).
  * round = nearest, ties to even; X/s is evaluated as the float32 product X * (1/s).

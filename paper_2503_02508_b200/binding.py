@@ -67,6 +67,8 @@ _SIGNATURES = {
     "qdit_status_string": (C.c_char_p, [_i32]),
     "qdit_last_error": (C.c_char_p, [_vp]),
     "qdit_launch_count": (_i64, [_vp]),
+    "qdit_profile_enable": (_i32, [_vp, _int]),
+    "qdit_profile_read": (_i32, [_vp, _int, C.POINTER(_i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]),
     "qdit_quantize_act": (_i32, [_vp, _vp, _int, _i64, _i64, _i64, _int, C.POINTER(qdit_qparams), _vp, _vp, _i64]),
     "qdit_w8a8_linear": (_i32, [_vp, _vp, _vp, _i64, _i64, _i64, qdit_qparams, _vp, _u32, C.POINTER(qdit_epilogue),
                                 _vp, _i64]),
@@ -161,6 +163,21 @@ def qdit_sync(ctx):
 
 def qdit_launch_count(ctx):
     return lib.qdit_launch_count(ctx)
+
+
+QDIT_PROF_GEMM, QDIT_PROF_ATTENTION, QDIT_PROF_LN_MODULATE, QDIT_PROF_ACT_QUANT = 0, 1, 2, 3
+QDIT_PROF_CACHE_REUSE, QDIT_PROF_OTHER, QDIT_PROF_KINDS = 4, 5, 6
+
+
+def qdit_profile_enable(ctx, enable):
+    return check(ctx, lib.qdit_profile_enable(ctx, int(enable)))
+
+
+def qdit_profile_read(ctx, kind):
+    """-> (launches, ms, work)"""
+    n, ms, w = _i64(), C.c_double(), C.c_double()
+    check(ctx, lib.qdit_profile_read(ctx, kind, C.byref(n), C.byref(ms), C.byref(w)))
+    return n.value, ms.value, w.value
 
 
 def qdit_quantize_act(ctx, x, x_dtype, M, K, ldx, mode, qp, dyn_scale, q, ldq):

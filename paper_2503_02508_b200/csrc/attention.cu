@@ -273,6 +273,7 @@ int32_t launch_attention(qdit_ctx* ctx, const void* q, const void* k, const void
   QDIT_TRY(qdit_get_tmap(ctx, k, rows, cols, ld, 64, DH, C::SWZ ? 1 : 0, 2, &tk));
   QDIT_TRY(qdit_get_tmap(ctx, v, rows, cols, ld, 64, DH, C::SWZ ? 1 : 0, 2, &tv));
   dim3 grid(T / BQ, H, B);
+  ProfScope prof(ctx, QDIT_PROF_ATTENTION, 4.0 * B * H * static_cast<double>(T) * T * DH);
   attention_kernel<DH><<<grid, ATT_THREADS, C::SMEM_BYTES, ctx->stream>>>(tq, tk, tv, p);
   return qdit_after_launch(ctx, "attention_kernel");
 }

@@ -36,7 +36,67 @@ int32_t qdit_check_qparams(qdit_ctx* ctx, const qdit_qparams* qp, bool scale_fro
   return QDIT_OK;
 }
 
+static cudaEvent_t take_event(qdit_ctx* ctx) {
+  cudaEvent_t e = nullptr;
+  if (!ctx->event_pool.empty()) {
+    e = ctx->event_pool.back();
+    ctx->event_pool.pop_back();
+  } else if (cudaEventCreate(&e) != cudaSuccess) {
+    cudaGetLastError();
+    e = nullptr;
+  }
+  return e;
+}
+
+ProfScope::ProfScope(qdit_ctx* c, int kind, double work) : ctx(c), on(false), stop(nullptr) {
+  if (!c || !c->profiling) return;
+  cudaEvent_t start = take_event(c);
+  stop = take_event(c);
+  if (!start || !stop) return;
+  cudaEventRecord(start, c->stream);
+  c->prof.push_back(qdit_ctx::ProfRec{kind, work, start, stop});
+  on = true;
+}
+ProfScope::~ProfScope() {
+  if (on) cudaEventRecord(stop, ctx->stream);
+}
+
 extern "C" {
+
+int32_t qdit_profile_enable(qdit_ctx* ctx, int enable) {
+  if (!ctx) return QDIT_ERR_INVALID_ARG;
+  QDIT_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));
+  for (auto& r : ctx->prof) {
+    ctx->event_pool.push_back(r.start);
+    ctx->event_pool.push_back(r.stop);
+  }
+  ctx->prof.clear();
+  ctx->profiling = enable != 0;
+  return QDIT_OK;
+}
+
+int32_t qdit_profile_read(qdit_ctx* ctx, int kind, int64_t* launches, double* ms, double* work) {
+  if (!ctx) return QDIT_ERR_INVALID_ARG;
+  if (kind < 0 || kind >= QDIT_PROF_KINDS) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "unknown kernel kind %d", kind);
+  QDIT_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));
+  int64_t n = 0;
+  double t = 0.0, w = 0.0;
+  for (auto& r : ctx->prof) {
+    if (r.kind != kind) continue;
+    float e = 0.0f;
+    if (cudaEventElapsedTime(&e, r.start, r.stop) != cudaSuccess) {
+      cudaGetLastError();
+      continue;
+    }
+    n += 1;
+    t += e;
+    w += r.work;
+  }
+  if (launches) *launches = n;
+  if (ms) *ms = t;
+  if (work) *work = w;
+  return QDIT_OK;
+}
 
 int32_t qdit_create(qdit_ctx** out, int device, void* cuda_stream) {
   if (!out) return QDIT_ERR_INVALID_ARG;
@@ -82,6 +142,11 @@ int32_t qdit_destroy(qdit_ctx* ctx) {
   cudaSetDevice(ctx->device);
   if (ctx->d_status) cudaFree(ctx->d_status);
   if (ctx->h_status) cudaFreeHost(ctx->h_status);
+  for (auto& r : ctx->prof) {
+    cudaEventDestroy(r.start);
+    cudaEventDestroy(r.stop);
+  }
+  for (cudaEvent_t e : ctx->event_pool) cudaEventDestroy(e);
   delete ctx;
   return QDIT_OK;
 }

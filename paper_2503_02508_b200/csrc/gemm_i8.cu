@@ -274,6 +274,7 @@ int32_t launch_gemm(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p, 
   const int total = p.num_m_tiles * p.num_n_tiles;
   const int grid = total < ctx->num_sms ? total : ctx->num_sms;
   const uint32_t idesc = umma_idesc_i8(BM, BN, a_unsigned);
+  ProfScope prof(ctx, QDIT_PROF_GEMM, 2.0 * p.M * static_cast<double>(p.N) * p.K);
   gemm_i8_kernel<BN><<<grid, NUM_THREADS, C::SMEM_BYTES, ctx->stream>>>(ta, tw, p, idesc);
   return qdit_after_launch(ctx, "gemm_i8_kernel");
 }

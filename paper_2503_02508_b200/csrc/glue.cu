@@ -416,6 +416,7 @@ int32_t qdit_cache_reuse_all(qdit_ctx* ctx, qdit_cache* c, const float* mod_all,
     if (!c->filled[i]) return qdit_fail(ctx, QDIT_ERR_STATE, "cache slot (block %zu, branch %zu) reused before any store", i / 2, i % 2);
   if (!aligned16(mod_all) || !aligned16(x) || ld_mod % 4 != 0) return qdit_fail(ctx, QDIT_ERR_ALIGN, "mod_all and x must be 16-byte aligned, ld_mod a multiple of 4");
   const int64_t n = c->M * (c->D / 8);
+  ProfScope prof(ctx, QDIT_PROF_CACHE_REUSE, static_cast<double>(c->M) * c->D * 2.0 * (2.0 * c->blocks + 2.0));
   cache_reuse_all_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, ctx->stream>>>(
       static_cast<__nv_bfloat16*>(x), c->data, mod_all, ld_mod, c->M, static_cast<int>(c->D), T, c->blocks);
   return qdit_after_launch(ctx, "cache_reuse_all_kernel");

@@ -42,6 +42,20 @@ struct qdit_ctx {
   std::string last_error;
   void* encode_fn = nullptr;  // cuTensorMapEncodeTiled
   std::unordered_map<TmapKey, CUtensorMap, TmapKeyHash> tmaps;
+  // per-kernel event timing (qdit_profile_*)
+  bool profiling = false;
+  struct ProfRec { int kind; double work; cudaEvent_t start, stop; };
+  std::vector<ProfRec> prof;
+  std::vector<cudaEvent_t> event_pool;
+};
+
+// Brackets one kernel launch with events while profiling is enabled.
+struct ProfScope {
+  qdit_ctx* ctx;
+  bool on;
+  cudaEvent_t stop;
+  ProfScope(qdit_ctx* c, int kind, double work);
+  ~ProfScope();
 };
 
 // Records a formatted message on the context and returns `code`.

@@ -269,6 +269,7 @@ int32_t qdit_quantize_act(qdit_ctx* ctx, const void* x, int x_dtype, int64_t M, 
   }
   const int64_t threads = M * ((K + 15) / 16);
   const unsigned grid = static_cast<unsigned>((threads + 255) / 256);
+  ProfScope prof(ctx, QDIT_PROF_ACT_QUANT, static_cast<double>(M) * K * (esz + 1.0));
   if (x_dtype == QDIT_BF16)
     act_quant_kernel<__nv_bfloat16><<<grid, 256, 0, ctx->stream>>>(static_cast<const __nv_bfloat16*>(x), M, K, ldx, qa,
                                                                    static_cast<uint8_t*>(q), ldq);
@@ -309,6 +310,8 @@ int32_t qdit_adaln_modulate(qdit_ctx* ctx, const void* x, int64_t M, int64_t D, 
   }
   const int nv = static_cast<int>((D / 8 + 31) / 32);
   const int d = static_cast<int>(D);
+  const double out_bytes = out_dtype == QDIT_I8 ? 1.0 : out_dtype == QDIT_BF16 ? 2.0 : 4.0;
+  ProfScope prof(ctx, QDIT_PROF_LN_MODULATE, static_cast<double>(M) * D * (2.0 + out_bytes));
   switch (nv) {
     case 1: launch_ln<1>(ctx, x, M, d, T, eps, shift, scale, ld_mod, out, out_dtype, qa); break;
     case 2: launch_ln<2>(ctx, x, M, d, T, eps, shift, scale, ld_mod, out, out_dtype, qa); break;
