@@ -1,11 +1,18 @@
 // W8A8 linear layer: persistent tcgen05 kind::i8 GEMM with TMEM int32 accumulators and a fused
 // de-quantising epilogue (bias / GELU / cache store / adaLN gate / residual / re-quantisation).
 //
-// CTA = 6 warps:  warp 0 lane 0  TMA producer  (A and W tiles -> 128B-swizzled smem ring, mbarrier tx)
+// CTA = 10 warps: warp 0 lane 0  TMA producer  (A and W tiles -> 128B-swizzled smem ring, mbarrier tx)
 //                 warp 1 lane 0  MMA issuer    (tcgen05.mma into one of two TMEM accumulator stages)
-//                 warps 2..5     epilogue      (tcgen05.ld -> registers -> math -> global stores)
+//                 warps 2..9     epilogue      (two warps per TMEM lane quadrant, alternating 32-column chunks)
 // The two accumulator stages let the epilogue of tile i overlap the main loop of tile i+1.
 // Tiles are 128 x BN, K is consumed in blocks of 128 bytes (4 MMAs of K = 32 each).
+//
+// Epilogue data flow per 32x32 chunk: tcgen05.ld gives each thread one ROW of the chunk, which is the
+// wrong shape for global memory (32 lanes -> 32 different lines).  The raw accumulators are therefore
+// transposed through a 4 KB XOR-swizzled shared-memory patch per warp; afterwards lane (r, g) owns 8
+// consecutive columns g of rows r, r+8, r+16, r+24, so that every global load/store instruction of the
+// warp covers 8 rows x 64..128 contiguous bytes, and the per-column parameters (scales, bias, gate) sit
+// in registers for the whole chunk.
 #include "common.cuh"
 #include "internal.h"
 
@@ -16,7 +23,9 @@ using namespace qd;
 constexpr int BM = 128;        // tile rows = TMEM lanes
 constexpr int BK = 128;        // K bytes per stage = one swizzle row
 constexpr int UMMA_K = 32;     // K per kind::i8 instruction
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_EPI_WARPS = 8;
+constexpr int NUM_THREADS = 64 + NUM_EPI_WARPS * 32;
+constexpr int STAGING_BYTES = NUM_EPI_WARPS * 32 * 128;  // one 32 x 32 x int32 patch per epilogue warp
 
 struct GemmParams {
   int M, N, K;
@@ -46,57 +55,78 @@ struct Cfg {
   static constexpr int A_BYTES = BM * BK;
   static constexpr int B_BYTES = BN * BK;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = (200 * 1024) / STAGE_BYTES > 8 ? 8 : (200 * 1024) / STAGE_BYTES;
-  static constexpr int TMEM_COLS = 2 * BN <= 128 ? 128 : (2 * BN <= 256 ? 256 : 512);
   static constexpr int BAR_BYTES = 256;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;  // + alignment slack
+  static constexpr int SMEM_LIMIT = 232448;  // 227 KB per CTA
+  static constexpr int STAGES_FIT = (SMEM_LIMIT - 1024 - BAR_BYTES - STAGING_BYTES) / STAGE_BYTES;
+  static constexpr int STAGES = STAGES_FIT > 8 ? 8 : STAGES_FIT;
+  static constexpr int TMEM_COLS = 2 * BN <= 128 ? 128 : (2 * BN <= 256 ? 256 : 512);
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + BAR_BYTES + 1024;  // + alignment slack
 };
 
-// Epilogue for 8 consecutive columns of one row.
-__device__ __forceinline__ void epilogue8(const GemmParams& p, const uint32_t* acc, int row, int n, int b,
-                                          float a_scale, float o_inv) {
-  if (p.flags & QDIT_EPI_OUT_I32) {
-    int32_t* o = static_cast<int32_t*>(p.out) + static_cast<int64_t>(row) * p.ldo + n;
-    *reinterpret_cast<uint4*>(o) = make_uint4(acc[0], acc[1], acc[2], acc[3]);
-    *reinterpret_cast<uint4*>(o + 4) = make_uint4(acc[4], acc[5], acc[6], acc[7]);
-    return;
-  }
-  float f[8], t[8];
+// Per-column parameters of the 8 columns a lane owns within a chunk.
+struct ColParams {
+  float sc[8];  // s_a * s_w[n]
+  float bi[8];
+  float gt[8];
+  int cs[8];    // z_a * colsum[n]
+};
+
+__device__ __forceinline__ void load_col_params(const GemmParams& p, int n, int b, float a_scale, ColParams& cp) {
+  float t[8];
   Load8<float>::load(p.w_scale + n, t);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) cp.sc[i] = __fmul_rn(a_scale, t[i]);
   if (p.a_zp != 0) {
     const int4 c0 = *reinterpret_cast<const int4*>(p.w_colsum + n);
     const int4 c1 = *reinterpret_cast<const int4*>(p.w_colsum + n + 4);
-    const int cs[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-      f[i] = static_cast<float>(static_cast<int>(acc[i]) - p.a_zp * cs[i]) * __fmul_rn(a_scale, t[i]);
+    cp.cs[0] = p.a_zp * c0.x; cp.cs[1] = p.a_zp * c0.y; cp.cs[2] = p.a_zp * c0.z; cp.cs[3] = p.a_zp * c0.w;
+    cp.cs[4] = p.a_zp * c1.x; cp.cs[5] = p.a_zp * c1.y; cp.cs[6] = p.a_zp * c1.z; cp.cs[7] = p.a_zp * c1.w;
   } else {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) f[i] = static_cast<float>(static_cast<int>(acc[i])) * __fmul_rn(a_scale, t[i]);
+    for (int i = 0; i < 8; ++i) cp.cs[i] = 0;
   }
-  if (p.flags & QDIT_EPI_BIAS) {
-    Load8<float>::load(p.bias + n, t);
+  if (p.flags & QDIT_EPI_BIAS) Load8<float>::load(p.bias + n, cp.bi);
+  if (p.flags & QDIT_EPI_GATE) Load8<float>::load(p.gate + static_cast<int64_t>(b) * p.ld_gate + n, cp.gt);
+}
+
+// Epilogue for 8 consecutive columns of one row; `res` holds the residual's 8 bf16 values (if used).
+__device__ __forceinline__ void epilogue8(const GemmParams& p, const uint4 lo, const uint4 hi, const ColParams& cp,
+                                          const uint4 res, int row, int n, float o_inv) {
+  const int acc[8] = {static_cast<int>(lo.x), static_cast<int>(lo.y), static_cast<int>(lo.z), static_cast<int>(lo.w),
+                      static_cast<int>(hi.x), static_cast<int>(hi.y), static_cast<int>(hi.z), static_cast<int>(hi.w)};
+  const int64_t o = static_cast<int64_t>(row) * p.ldo + n;
+  if (p.flags & QDIT_EPI_OUT_I32) {
+    int32_t* op = static_cast<int32_t*>(p.out) + o;
+    *reinterpret_cast<uint4*>(op) = lo;
+    *reinterpret_cast<uint4*>(op + 4) = hi;
+    return;
+  }
+  float f[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) f[i] += t[i];
+  for (int i = 0; i < 8; ++i) f[i] = static_cast<float>(acc[i] - cp.cs[i]) * cp.sc[i];
+  if (p.flags & QDIT_EPI_BIAS) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) f[i] += cp.bi[i];
   }
   if (p.flags & QDIT_EPI_GELU) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) f[i] = gelu_tanh_f(f[i]);
   }
-  if (p.flags & QDIT_EPI_CACHE_STORE) {
+  if (p.flags & QDIT_EPI_CACHE_STORE)
     *reinterpret_cast<uint4*>(p.cache_out + static_cast<int64_t>(row) * p.N + n) = pack_bf16x8(f);
-  }
   if (p.flags & QDIT_EPI_GATE) {
-    Load8<float>::load(p.gate + static_cast<int64_t>(b) * p.ld_gate + n, t);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) f[i] *= t[i];
+    for (int i = 0; i < 8; ++i) f[i] *= cp.gt[i];
   }
   if (p.flags & QDIT_EPI_RESIDUAL) {
-    Load8<__nv_bfloat16>::load(p.residual + static_cast<int64_t>(row) * p.ldo + n, t);
+    float r[8];
+    unpack_bf16x2(res.x, r[0], r[1]);
+    unpack_bf16x2(res.y, r[2], r[3]);
+    unpack_bf16x2(res.z, r[4], r[5]);
+    unpack_bf16x2(res.w, r[6], r[7]);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) f[i] += t[i];
+    for (int i = 0; i < 8; ++i) f[i] += r[i];
   }
-  const int64_t o = static_cast<int64_t>(row) * p.ldo + n;
   if (p.flags & QDIT_EPI_QUANT_OUT) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) f[i] = quantize_code(f[i], o_inv, p.o_zp, p.o_qmin, p.o_qmax);
@@ -120,7 +150,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sA = smem;
   uint8_t* sB = smem + STAGES * C::A_BYTES;
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * C::STAGE_BYTES);
+  uint8_t* staging = smem + STAGES * C::STAGE_BYTES;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(staging + STAGING_BYTES);
   uint64_t* empty_bar = full_bar + STAGES;
   uint64_t* tfull_bar = empty_bar + STAGES;
   uint64_t* tempty_bar = tfull_bar + 2;
@@ -137,7 +168,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&tfull_bar[s], 1);
-      mbar_init(&tempty_bar[s], 128);
+      mbar_init(&tempty_bar[s], NUM_EPI_WARPS);
     }
     *abort_flag = 0;
     mbar_fence_init();
@@ -210,11 +241,19 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     }
   } else {
     // -------------------------------------------------------------------- epilogue warps
-    const int quad = warp & 3;  // TMEM lane quadrant this warp may access
-    const int row_in_tile = quad * 32 + lane;
+    const int e = warp - 2;
+    const int quad = warp & 3;   // TMEM lane quadrant this warp may access
+    const int half = e >> 2;     // this warp takes chunks half, half + 2, ...
+    const uint32_t stg = smem_u32(staging + e * (32 * 128));  // [32 rows][8 x 16 B], 16-byte index XOR (row & 7)
+    const int cg = lane & 3;     // after the transpose: column group (8 columns) ...
+    const int rsub = lane >> 2;  // ... of rows rsub, rsub + 8, rsub + 16, rsub + 24
     const float a_scale = p.a_scale_dev ? __ldg(p.a_scale_dev) : p.a_scale;
     float o_inv = 0.0f;
     if (p.flags & QDIT_EPI_QUANT_OUT) o_inv = __fdiv_rn(1.0f, p.o_scale_dev ? __ldg(p.o_scale_dev) : p.o_scale);
+    const bool gate_uniform = (p.tokens % 32) == 0;  // the warp's 32 rows then belong to one sample
+    constexpr int CHUNKS = BN / 32;
+    constexpr int LAST_EVEN = ((CHUNKS - 1) / 2) * 2, LAST_ODD = ((CHUNKS - 2) / 2) * 2 + 1;
+    const int c_last = half ? LAST_ODD : LAST_EVEN;
     int it = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
       const int as = it & 1;
@@ -224,26 +263,58 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       if (!mbar_wait(&tfull_bar[as], aphase, abort_flag, p.status)) break;
       __syncwarp();
       tc_fence_after();
-      const int row = m0 + row_in_tile;
-      const int b = (p.flags & QDIT_EPI_GATE) ? row / p.tokens : 0;
+      const int row_base = m0 + quad * 32;
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(as * BN);
-      constexpr int CHUNKS = BN / 32;
 #pragma unroll 1
-      for (int c = 0; c < CHUNKS; ++c) {
+      for (int c = half; c < CHUNKS; c += 2) {
+        const int n = n0 + c * 32 + cg * 8;
+        const bool col_ok = n < p.N;
+        // ---- global loads first: column parameters and the residual rows, in flight during the transpose
+        ColParams cp;
+        uint4 res[4];
+        if (col_ok && !(p.flags & QDIT_EPI_OUT_I32)) {
+          load_col_params(p, n, row_base / p.tokens, a_scale, cp);
+          if (p.flags & QDIT_EPI_RESIDUAL) {
+#pragma unroll
+            for (int sidx = 0; sidx < 4; ++sidx) {
+              const int row = row_base + sidx * 8 + rsub;
+              if (row < p.M) res[sidx] = *reinterpret_cast<const uint4*>(p.residual + static_cast<int64_t>(row) * p.ldo + n);
+            }
+          }
+        }
+        // ---- TMEM -> registers (one row per thread) -> swizzled staging patch
         uint32_t v[32];
-        __syncwarp();
+        __syncwarp();  // the previous chunk's reads of the patch are complete
         tmem_ld_32x32(taddr + static_cast<uint32_t>(c * 32), v);
         tmem_ld_wait();
-        if (c == CHUNKS - 1) {
-          // accumulator stage fully read: hand it back to the MMA warp
+        if (c == c_last) {
+          // this warp has read all of its share of the accumulator stage: hand it back to the MMA warp
           tc_fence_before();
-          mbar_arrive(&tempty_bar[as]);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&tempty_bar[as]);
         }
-        if (row < p.M) {
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            const int n = n0 + c * 32 + g * 8;
-            if (n < p.N) epilogue8(p, v + g * 8, row, n, b, a_scale, o_inv);
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t addr = stg + static_cast<uint32_t>(lane * 128 + ((j ^ (lane & 7)) << 4));
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v[4 * j]), "r"(v[4 * j + 1]),
+                       "r"(v[4 * j + 2]), "r"(v[4 * j + 3])
+                       : "memory");
+        }
+        __syncwarp();
+        // ---- transposed ownership: 8 columns of 4 rows per lane
+#pragma unroll
+        for (int sidx = 0; sidx < 4; ++sidx) {
+          const int r = sidx * 8 + rsub;
+          const int row = row_base + r;
+          uint4 lo, hi;
+          const uint32_t a_lo = stg + static_cast<uint32_t>(r * 128 + (((2 * cg) ^ (r & 7)) << 4));
+          const uint32_t a_hi = stg + static_cast<uint32_t>(r * 128 + (((2 * cg + 1) ^ (r & 7)) << 4));
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(lo.x), "=r"(lo.y), "=r"(lo.z), "=r"(lo.w) : "r"(a_lo));
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(hi.x), "=r"(hi.y), "=r"(hi.z), "=r"(hi.w) : "r"(a_hi));
+          if (row < p.M && col_ok) {
+            if (!gate_uniform && (p.flags & QDIT_EPI_GATE))
+              Load8<float>::load(p.gate + static_cast<int64_t>(row / p.tokens) * p.ld_gate + n, cp.gt);
+            epilogue8(p, lo, hi, cp, res[sidx], row, n, o_inv);
           }
         }
       }
