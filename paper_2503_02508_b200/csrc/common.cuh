@@ -137,6 +137,22 @@ __device__ __forceinline__ float quantize_code(float x, float inv_scale, float z
   float r = rintf(__fmul_rn(x, inv_scale));
   return fminf(fmaxf(r + zp, qmin), qmax);
 }
+// Same decision as quantize_code, as an integer and without conversion instructions: adding 1.5 * 2^23
+// rounds a float of magnitude < 2^22 to the nearest integer (ties to even) and leaves that integer in the
+// low mantissa bits.  The product is clamped to +-1024 first, which cannot change the clipped code.
+__device__ __forceinline__ int quantize_code_i(float x, float inv_scale, int zp, int qmin, int qmax) {
+  const float t = fminf(fmaxf(__fmul_rn(x, inv_scale), -1024.0f), 1024.0f);
+  const int r = __float_as_int(__fadd_rn(t, 12582912.0f)) - 0x4B400000;
+  return min(max(r + zp, qmin), qmax);
+}
+// Exact int32 -> float32 conversion (round to nearest even, as cvt.rn.f32.s32) on the FMA pipe:
+// split into a multiple of 4096 and a 12-bit remainder, both exactly representable, and join with one fma.
+__device__ __forceinline__ float int_to_float_rn(int v) {
+  const int hi = v >> 12, lo = v & 0xFFF;
+  const float fhi = __int_as_float(0x4B400000 + hi) - 12582912.0f;
+  const float flo = __int_as_float(0x4B400000 + lo) - 12582912.0f;
+  return fmaf(fhi, 4096.0f, flo);
+}
 __device__ __forceinline__ float gelu_tanh_f(float x) {
   // 0.5 x (1 + tanh(u)) = x / (1 + exp(-2u)),  u = sqrt(2/pi) (x + 0.044715 x^3)
   const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
@@ -194,6 +210,16 @@ __device__ __forceinline__ uint2 pack_codes8(const float (&c)[8]) {
   for (int i = 0; i < 4; ++i) {
     lo |= (static_cast<uint32_t>(__float2int_rn(c[i])) & 0xFFu) << (8 * i);
     hi |= (static_cast<uint32_t>(__float2int_rn(c[4 + i])) & 0xFFu) << (8 * i);
+  }
+  return make_uint2(lo, hi);
+}
+// 8 integer codes in [-128, 255] -> 8 stored bytes.
+__device__ __forceinline__ uint2 pack_codes8_i(const int (&c)[8]) {
+  uint32_t lo = 0, hi = 0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    lo |= (static_cast<uint32_t>(c[i]) & 0xFFu) << (8 * i);
+    hi |= (static_cast<uint32_t>(c[4 + i]) & 0xFFu) << (8 * i);
   }
   return make_uint2(lo, hi);
 }

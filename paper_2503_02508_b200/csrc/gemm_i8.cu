@@ -103,7 +103,7 @@ __device__ __forceinline__ void epilogue8(const GemmParams& p, const uint4 lo, c
   }
   float f[8];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) f[i] = static_cast<float>(acc[i] - cp.cs[i]) * cp.sc[i];
+  for (int i = 0; i < 8; ++i) f[i] = int_to_float_rn(acc[i] - cp.cs[i]) * cp.sc[i];
   if (p.flags & QDIT_EPI_BIAS) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) f[i] += cp.bi[i];
@@ -128,9 +128,11 @@ __device__ __forceinline__ void epilogue8(const GemmParams& p, const uint4 lo, c
     for (int i = 0; i < 8; ++i) f[i] += r[i];
   }
   if (p.flags & QDIT_EPI_QUANT_OUT) {
+    int code[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) f[i] = quantize_code(f[i], o_inv, p.o_zp, p.o_qmin, p.o_qmax);
-    *reinterpret_cast<uint2*>(static_cast<uint8_t*>(p.out) + o) = pack_codes8(f);
+    for (int i = 0; i < 8; ++i)
+      code[i] = quantize_code_i(f[i], o_inv, static_cast<int>(p.o_zp), static_cast<int>(p.o_qmin), static_cast<int>(p.o_qmax));
+    *reinterpret_cast<uint2*>(static_cast<uint8_t*>(p.out) + o) = pack_codes8_i(code);
   } else if (p.flags & QDIT_EPI_OUT_BF16) {
     *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + o) = pack_bf16x8(f);
   } else {
