@@ -253,7 +253,8 @@ def run_ours(args):
             ms = float(t.item())
         return ms
 
-    for _ in range(max(args.warmup, 3)):
+    n_warm = args.warmup if args.short_warmup else max(args.warmup, 3)
+    for _ in range(n_warm):
         trajectory_device()
     q.qdit_sync(ctx)
     clocks = ClockSampler(local)
@@ -305,7 +306,7 @@ def run_ours(args):
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": "images/s", "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "warmup": n_warm, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int8", "data": "synthetic",
             "config": {"workload": args.workload, "model": "DiT-XL/2", "batch_per_gpu": batch, "network_batch": beff,
                        "sampling_steps": steps, "cache_interval": interval, "guidance": guidance,
@@ -328,16 +329,97 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------ GEMM sweep
+GEMM_SHAPES = [(1152, 3456, "qkv"), (1152, 1152, "proj"), (1152, 4608, "fc1"), (4608, 1152, "fc2")]
+
+
+def run_gemm_sweep(args):
+    """int8 GEMM + fused activation-quantizer sweep over the DiT-XL/2 linear shapes (K -> N) and M.
+    Activations: bf16 N(0,1) with 1 % of the channels scaled x20; weights: int8 with channel-wise scales.
+    Reports TOP/s of the GEMM alone (epilogue of that layer in the model) and of act-quant + GEMM."""
+    import torch
+    import paper_2503_02508_b200 as q
+    seed = synth.CONFIG_SEEDS["gemm_sweep"]
+    peaks = measured_peaks()
+    ctx = q.qdit_create(0, None)
+    rows = []
+    for M in args.m:
+        for K, N, name in GEMM_SHAPES:
+            x = torch.from_numpy(synth.outlier_activations(seed, f"x{M}.{K}", M, K)).cuda().to(torch.bfloat16)
+            wq = torch.from_numpy(synth.uniform_int(seed, f"w{N}.{K}", (N, K), -127, 128).astype(np.int8)).cuda()
+            ws = torch.from_numpy(np.abs(synth.normal(seed, f"ws{N}", (N,), 1e-3)) + 1e-4).cuda()
+            bias = torch.from_numpy(synth.normal(seed, f"b{N}", (N,), 0.02)).cuda()
+            gate = torch.from_numpy(synth.normal(seed, f"g{N}", ((M + 255) // 256, N), 0.3)).cuda()
+            resid = torch.from_numpy(synth.normal(seed, f"r{M}.{N}", (M, N))).cuda().to(torch.bfloat16)
+            cache = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+            a8 = torch.empty((M, K), dtype=torch.uint8, device="cuda")
+            a_qp = q.qparams(float(x.abs().max()) / 127.0)
+            if name == "qkv":
+                flags, out = q.QDIT_EPI_BIAS | q.QDIT_EPI_OUT_BF16, torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+            elif name == "fc1":
+                flags, out = q.QDIT_EPI_BIAS | q.QDIT_EPI_GELU | q.QDIT_EPI_QUANT_OUT, torch.empty((M, N), dtype=torch.uint8, device="cuda")
+            else:
+                flags = q.QDIT_EPI_BIAS | q.QDIT_EPI_GATE | q.QDIT_EPI_RESIDUAL | q.QDIT_EPI_CACHE_STORE | q.QDIT_EPI_OUT_BF16
+                out = resid
+            epi = q.epilogue(w_scale=ws, bias=bias, gate=gate, ld_gate=N, tokens_per_sample=256, residual=resid,
+                             cache_out=cache, out_qp=q.qparams(0.05))
+
+            def quant():
+                q.qdit_quantize_act(ctx, x, q.QDIT_BF16, M, K, K, q.QDIT_QUANT_STATIC, a_qp, None, a8, K)
+
+            def gemm():
+                q.qdit_w8a8_linear(ctx, a8, wq, M, N, K, a_qp, None, flags, epi, out, N)
+
+            def both():
+                quant()
+                gemm()
+
+            def t(fn):
+                for _ in range(3):
+                    fn()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(args.steps):
+                    fn()
+                e1.record()
+                torch.cuda.synchronize()
+                return e0.elapsed_time(e1) / args.steps
+
+            quant()
+            ops = 2.0 * M * N * K
+            ms_g, ms_b, ms_q = t(gemm), t(both), t(quant)
+            rows.append({"layer": name, "M": M, "K": K, "N": N, "gemm_tops": ops / ms_g / 1e9, "quant_gemm_tops": ops / ms_b / 1e9,
+                         "gemm_us": ms_g * 1e3, "act_quant_gbs": 3.0 * M * K / ms_q / 1e6,
+                         "frac_of_2x_bf16_burst": ops / ms_g / 1e9 / (2 * peaks["bf16_burst"]),
+                         "frac_of_nominal_4500": ops / ms_g / 1e9 / 4500.0})
+    q.qdit_sync(ctx)
+    q.qdit_destroy(ctx)
+    best = max(r["gemm_tops"] for r in rows)
+    print(json.dumps({"metric": "int8 GEMM TOP/s (DiT-XL/2 linear shapes)", "value": best, "unit": "TOP/s", "n_gpus": 1,
+                      "steps": args.steps, "warmup": 3, "higher_is_better": True, "dtype": "int8", "data": "synthetic",
+                      "config": {"workload": "gemm_sweep", "l2": "repeated launches on the same operands (L2-warm)"},
+                      "peaks": {"int8_2x_bf16_burst": 2 * peaks["bf16_burst"], "int8_nominal": 4500.0,
+                                "hbm_gbs": peaks["hbm_gbs"], "source": peaks["source"]},
+                      "rows": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="ddim50", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="ddim50", choices=sorted(WORKLOADS) + ["gemm_sweep"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--m", type=lambda v: [int(x) for x in v.split(",")], default=[256, 1024, 4096, 8192, 16384, 65536],
+                    help="row counts of the GEMM sweep")
+    ap.add_argument("--short-warmup", action="store_true",
+                    help="profiling runs only: honour --warmup below 3 (such a run is not a valid measurement)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.workload == "gemm_sweep":
+        run_gemm_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
