@@ -92,6 +92,24 @@ enum { QDIT_QUANT_STATIC = 0, QDIT_QUANT_DYNAMIC = 1 };
 int32_t qdit_quantize_act(qdit_ctx* ctx, const void* x, int x_dtype, int64_t M, int64_t K, int64_t ldx,
                           int mode, const qdit_qparams* qp, float* dyn_scale, void* q, int64_t ldq);
 
+/* Dynamic quantizer for callers that cannot allocate device memory (the paper has no counterpart; this
+ * is a deployment convenience).  Same result as qdit_quantize_act in QDIT_QUANT_DYNAMIC mode: symmetric
+ * codes in q and s = max|x| / 127 (1 for an all-zero tensor) in dyn_scale.  The difference is where the
+ * reduction's intermediate values live: in a fixed 256 KB array inside the library's device image instead
+ * of memory somebody had to cudaMalloc, so the call (and everything it calls) allocates nothing.  Use it
+ * from code that is handed only its tensors and must not touch the allocator: a plug-in inside another
+ * framework's memory plan, a process with a fixed memory budget, a region being recorded for replay.
+ *  - Limit: M*K <= 134,217,728 elements per call (65536 partial maxima of 2048 elements each); larger
+ *    inputs are refused with QDIT_ERR_SHAPE before anything is launched.
+ *  - The first call on a device looks up the array's device address (cudaGetSymbolAddress) with that
+ *    device current; make that first call outside any stream capture.
+ *  - The array is shared by every call on the device and keeps the last call's values.  Each call
+ *    overwrites all slots it later reads, so nothing needs clearing; two calls that overlap on the GPU
+ *    (different streams, no ordering) race on it and must be serialised by the caller.
+ * x, q, ldx, ldq, K % 8 == 0 and alignment as for qdit_quantize_act; dyn_scale: device, 1 float, required. */
+int32_t qdit_quantize_act_dynamic_static(qdit_ctx* ctx, const void* x, int x_dtype, int64_t M, int64_t K,
+                                         int64_t ldx, float* dyn_scale, void* q, int64_t ldq);
+
 /* ------------------------------------------------------------------------------------------------
  * W8A8 linear layer (8-bit weights and activations, Table 1) on quantized activations:
  *   acc[m,n] = sum_k A[m,k] * W[n,k]                       exact int32 (tcgen05 kind::i8, TMEM)

@@ -70,6 +70,7 @@ _SIGNATURES = {
     "qdit_profile_enable": (_i32, [_vp, _int]),
     "qdit_profile_read": (_i32, [_vp, _int, C.POINTER(_i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]),
     "qdit_quantize_act": (_i32, [_vp, _vp, _int, _i64, _i64, _i64, _int, C.POINTER(qdit_qparams), _vp, _vp, _i64]),
+    "qdit_quantize_act_dynamic_static": (_i32, [_vp, _vp, _int, _i64, _i64, _i64, _vp, _vp, _i64]),
     "qdit_w8a8_linear": (_i32, [_vp, _vp, _vp, _i64, _i64, _i64, qdit_qparams, _vp, _u32, C.POINTER(qdit_epilogue),
                                 _vp, _i64]),
     "qdit_quantize_weight": (_i32, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
@@ -183,6 +184,10 @@ def qdit_profile_read(ctx, kind):
 def qdit_quantize_act(ctx, x, x_dtype, M, K, ldx, mode, qp, dyn_scale, q, ldq):
     return check(ctx, lib.qdit_quantize_act(ctx, ptr(x), x_dtype, M, K, ldx, mode,
                                             C.byref(qp) if qp is not None else None, ptr(dyn_scale), ptr(q), ldq))
+
+
+def qdit_quantize_act_dynamic_static(ctx, x, x_dtype, M, K, ldx, dyn_scale, q, ldq):
+    return check(ctx, lib.qdit_quantize_act_dynamic_static(ctx, ptr(x), x_dtype, M, K, ldx, ptr(dyn_scale), ptr(q), ldq))
 
 
 def epilogue(w_scale=None, w_colsum=None, bias=None, gate=None, ld_gate=0, tokens_per_sample=0, residual=None,
