@@ -13,42 +13,11 @@
 // consecutive columns g of rows r, r+8, r+16, r+24, so that every global load/store instruction of the
 // warp covers 8 rows x 64..128 contiguous bytes, and the per-column parameters (scales, bias, gate) sit
 // in registers for the whole chunk.
-#include "common.cuh"
-#include "internal.h"
+#include "gemm_common.cuh"
 
 namespace {
 
-using namespace qd;
-
-constexpr int BM = 128;        // tile rows = TMEM lanes
-constexpr int BK = 128;        // K bytes per stage = one swizzle row
-constexpr int UMMA_K = 32;     // K per kind::i8 instruction
-constexpr int NUM_EPI_WARPS = 8;
-constexpr int NUM_THREADS = 64 + NUM_EPI_WARPS * 32;
-constexpr int STAGING_BYTES = NUM_EPI_WARPS * 32 * 128;  // one 32 x 32 x int32 patch per epilogue warp
-
-struct GemmParams {
-  int M, N, K;
-  uint32_t flags;
-  float a_scale;
-  const float* a_scale_dev;
-  int a_zp;
-  const float* w_scale;
-  const int32_t* w_colsum;
-  const float* bias;
-  const float* gate;
-  int64_t ld_gate;
-  int tokens;
-  const __nv_bfloat16* residual;
-  __nv_bfloat16* cache_out;
-  float o_scale;
-  const float* o_scale_dev;
-  float o_zp, o_qmin, o_qmax;
-  void* out;
-  int64_t ldo;
-  int* status;
-  int num_m_tiles, num_n_tiles;
-};
+using namespace qgemm;
 
 template <int BN>
 struct Cfg {
@@ -62,85 +31,6 @@ struct Cfg {
   static constexpr int TMEM_COLS = 2 * BN <= 128 ? 128 : (2 * BN <= 256 ? 256 : 512);
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + BAR_BYTES + 1024;  // + alignment slack
 };
-
-// Per-column parameters of the 8 columns a lane owns within a chunk.
-struct ColParams {
-  float sc[8];  // s_a * s_w[n]
-  float bi[8];
-  float gt[8];
-  int cs[8];    // z_a * colsum[n]
-};
-
-__device__ __forceinline__ void load_col_params(const GemmParams& p, int n, int b, float a_scale, ColParams& cp) {
-  float t[8];
-  Load8<float>::load(p.w_scale + n, t);
-#pragma unroll
-  for (int i = 0; i < 8; ++i) cp.sc[i] = __fmul_rn(a_scale, t[i]);
-  if (p.a_zp != 0) {
-    const int4 c0 = *reinterpret_cast<const int4*>(p.w_colsum + n);
-    const int4 c1 = *reinterpret_cast<const int4*>(p.w_colsum + n + 4);
-    cp.cs[0] = p.a_zp * c0.x; cp.cs[1] = p.a_zp * c0.y; cp.cs[2] = p.a_zp * c0.z; cp.cs[3] = p.a_zp * c0.w;
-    cp.cs[4] = p.a_zp * c1.x; cp.cs[5] = p.a_zp * c1.y; cp.cs[6] = p.a_zp * c1.z; cp.cs[7] = p.a_zp * c1.w;
-  } else {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) cp.cs[i] = 0;
-  }
-  if (p.flags & QDIT_EPI_BIAS) Load8<float>::load(p.bias + n, cp.bi);
-  if (p.flags & QDIT_EPI_GATE) Load8<float>::load(p.gate + static_cast<int64_t>(b) * p.ld_gate + n, cp.gt);
-}
-
-// Epilogue for 8 consecutive columns of one row; `res` holds the residual's 8 bf16 values (if used).
-__device__ __forceinline__ void epilogue8(const GemmParams& p, const uint4 lo, const uint4 hi, const ColParams& cp,
-                                          const uint4 res, int row, int n, float o_inv) {
-  const int acc[8] = {static_cast<int>(lo.x), static_cast<int>(lo.y), static_cast<int>(lo.z), static_cast<int>(lo.w),
-                      static_cast<int>(hi.x), static_cast<int>(hi.y), static_cast<int>(hi.z), static_cast<int>(hi.w)};
-  const int64_t o = static_cast<int64_t>(row) * p.ldo + n;
-  if (p.flags & QDIT_EPI_OUT_I32) {
-    int32_t* op = static_cast<int32_t*>(p.out) + o;
-    *reinterpret_cast<uint4*>(op) = lo;
-    *reinterpret_cast<uint4*>(op + 4) = hi;
-    return;
-  }
-  float f[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) f[i] = int_to_float_rn(acc[i] - cp.cs[i]) * cp.sc[i];
-  if (p.flags & QDIT_EPI_BIAS) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) f[i] += cp.bi[i];
-  }
-  if (p.flags & QDIT_EPI_GELU) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) f[i] = gelu_tanh_f(f[i]);
-  }
-  if (p.flags & QDIT_EPI_CACHE_STORE)
-    *reinterpret_cast<uint4*>(p.cache_out + static_cast<int64_t>(row) * p.N + n) = pack_bf16x8(f);
-  if (p.flags & QDIT_EPI_GATE) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) f[i] *= cp.gt[i];
-  }
-  if (p.flags & QDIT_EPI_RESIDUAL) {
-    float r[8];
-    unpack_bf16x2(res.x, r[0], r[1]);
-    unpack_bf16x2(res.y, r[2], r[3]);
-    unpack_bf16x2(res.z, r[4], r[5]);
-    unpack_bf16x2(res.w, r[6], r[7]);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) f[i] += r[i];
-  }
-  if (p.flags & QDIT_EPI_QUANT_OUT) {
-    int code[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-      code[i] = quantize_code_i(f[i], o_inv, static_cast<int>(p.o_zp), static_cast<int>(p.o_qmin), static_cast<int>(p.o_qmax));
-    *reinterpret_cast<uint2*>(static_cast<uint8_t*>(p.out) + o) = pack_codes8_i(code);
-  } else if (p.flags & QDIT_EPI_OUT_BF16) {
-    *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + o) = pack_bf16x8(f);
-  } else {
-    float* of = static_cast<float*>(p.out) + o;
-    *reinterpret_cast<float4*>(of) = make_float4(f[0], f[1], f[2], f[3]);
-    *reinterpret_cast<float4*>(of + 4) = make_float4(f[4], f[5], f[6], f[7]);
-  }
-}
 
 template <int BN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
@@ -246,16 +136,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     const int e = warp - 2;
     const int quad = warp & 3;   // TMEM lane quadrant this warp may access
     const int half = e >> 2;     // this warp takes chunks half, half + 2, ...
-    const uint32_t stg = smem_u32(staging + e * (32 * 128));  // [32 rows][8 x 16 B], 16-byte index XOR (row & 7)
-    const int cg = lane & 3;     // after the transpose: column group (8 columns) ...
-    const int rsub = lane >> 2;  // ... of rows rsub, rsub + 8, rsub + 16, rsub + 24
+    const uint32_t stg = smem_u32(staging + e * (2 * 32 * 128));  // [32 rows][8 x 16 B], 16-byte index XOR (row & 7)
     const float a_scale = p.a_scale_dev ? __ldg(p.a_scale_dev) : p.a_scale;
     float o_inv = 0.0f;
     if (p.flags & QDIT_EPI_QUANT_OUT) o_inv = __fdiv_rn(1.0f, p.o_scale_dev ? __ldg(p.o_scale_dev) : p.o_scale);
-    const bool gate_uniform = (p.tokens % 32) == 0;  // the warp's 32 rows then belong to one sample
-    constexpr int CHUNKS = BN / 32;
-    constexpr int LAST_EVEN = ((CHUNKS - 1) / 2) * 2, LAST_ODD = ((CHUNKS - 2) / 2) * 2 + 1;
-    const int c_last = half ? LAST_ODD : LAST_EVEN;
     int it = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
       const int as = it & 1;
@@ -265,61 +149,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       if (!mbar_wait(&tfull_bar[as], aphase, abort_flag, p.status)) break;
       __syncwarp();
       tc_fence_after();
-      const int row_base = m0 + quad * 32;
-      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(as * BN);
-#pragma unroll 1
-      for (int c = half; c < CHUNKS; c += 2) {
-        const int n = n0 + c * 32 + cg * 8;
-        const bool col_ok = n < p.N;
-        // ---- global loads first: column parameters and the residual rows, in flight during the transpose
-        ColParams cp;
-        uint4 res[4];
-        if (col_ok && !(p.flags & QDIT_EPI_OUT_I32)) {
-          load_col_params(p, n, row_base / p.tokens, a_scale, cp);
-          if (p.flags & QDIT_EPI_RESIDUAL) {
-#pragma unroll
-            for (int sidx = 0; sidx < 4; ++sidx) {
-              const int row = row_base + sidx * 8 + rsub;
-              if (row < p.M) res[sidx] = *reinterpret_cast<const uint4*>(p.residual + static_cast<int64_t>(row) * p.ldo + n);
-            }
-          }
-        }
-        // ---- TMEM -> registers (one row per thread) -> swizzled staging patch
-        uint32_t v[32];
-        __syncwarp();  // the previous chunk's reads of the patch are complete
-        tmem_ld_32x32(taddr + static_cast<uint32_t>(c * 32), v);
-        tmem_ld_wait();
-        if (c == c_last) {
-          // this warp has read all of its share of the accumulator stage: hand it back to the MMA warp
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&tempty_bar[as]);
-        }
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const uint32_t addr = stg + static_cast<uint32_t>(lane * 128 + ((j ^ (lane & 7)) << 4));
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v[4 * j]), "r"(v[4 * j + 1]),
-                       "r"(v[4 * j + 2]), "r"(v[4 * j + 3])
-                       : "memory");
-        }
-        __syncwarp();
-        // ---- transposed ownership: 8 columns of 4 rows per lane
-#pragma unroll
-        for (int sidx = 0; sidx < 4; ++sidx) {
-          const int r = sidx * 8 + rsub;
-          const int row = row_base + r;
-          uint4 lo, hi;
-          const uint32_t a_lo = stg + static_cast<uint32_t>(r * 128 + (((2 * cg) ^ (r & 7)) << 4));
-          const uint32_t a_hi = stg + static_cast<uint32_t>(r * 128 + (((2 * cg + 1) ^ (r & 7)) << 4));
-          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(lo.x), "=r"(lo.y), "=r"(lo.z), "=r"(lo.w) : "r"(a_lo));
-          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(hi.x), "=r"(hi.y), "=r"(hi.z), "=r"(hi.w) : "r"(a_hi));
-          if (row < p.M && col_ok) {
-            if (!gate_uniform && (p.flags & QDIT_EPI_GATE))
-              Load8<float>::load(p.gate + static_cast<int64_t>(row / p.tokens) * p.ld_gate + n, cp.gt);
-            epilogue8(p, lo, hi, cp, res[sidx], row, n, o_inv);
-          }
-        }
-      }
+      uint64_t* release_bar = &tempty_bar[as];
+      epilogue_tile<BN>(p, tmem_base + static_cast<uint32_t>(as * BN), m0, n0, quad, half, stg, lane, a_scale, o_inv,
+                        [release_bar]() { mbar_arrive_relaxed(release_bar); });
     }
   }
 
@@ -452,6 +284,11 @@ extern "C" int32_t qdit_w8a8_linear(qdit_ctx* ctx, const void* A, const void* W,
       p.o_qmin = static_cast<float>(epi->out_qp.qmin);
       p.o_qmax = static_cast<float>(epi->out_qp.qmax);
     }
+  }
+  // QDIT_GEMM_PAIR=<bn> selects the CTA-pair kernel with 256 x bn tiles (experimental switch while tuning)
+  if (const char* env = getenv("QDIT_GEMM_PAIR")) {
+    const int bn = atoi(env);
+    if (bn == 128 || bn == 192 || bn == 256) return qdit_launch_gemm_pair(ctx, A, W, p, a_unsigned, bn);
   }
   switch (pick_bn(p.M, p.N, ctx->num_sms)) {
     case 64: return launch_gemm<64>(ctx, A, W, p, a_unsigned);

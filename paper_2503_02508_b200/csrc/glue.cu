@@ -125,83 +125,126 @@ __global__ void __launch_bounds__(256) cfg_ddim_kernel(float* __restrict__ laten
 }
 
 // ----------------------------------------------------------------------------- patch embedding
-// One CTA per token row: x[m,:] = bf16(W_patch . patch(m) + b_patch + pos[t,:]); patch vector (c,py,px).
-__global__ void __launch_bounds__(128) embed_kernel(const float* __restrict__ latent, int latent_batch,
+// x[m,:] = bf16(W_patch . patch(m) + b_patch + pos[t,:]); patch vector ordered (c, py, px).
+// CTA = 32 token rows x 512 columns; a thread keeps the weights of its two columns in registers and walks
+// the rows, so weights are read once per CTA and the bf16 stores of a warp are 128 contiguous bytes.
+constexpr int EMB_ROWS = 32;
+constexpr int EMB_MAX_PD = 64;  // patch vector length limit (C * p * p)
+__global__ void __launch_bounds__(256) embed_kernel(const float* __restrict__ latent, int latent_batch,
                                                     const float* __restrict__ w, const float* __restrict__ bias,
                                                     const float* __restrict__ pos, __nv_bfloat16* __restrict__ x,
-                                                    int D, int grid, int patch, int C) {
-  extern __shared__ float sp[];  // patch vector, C*patch*patch
-  const int T = grid * grid;
-  const int64_t m = blockIdx.x;
-  const int b = static_cast<int>(m / T) % latent_batch;
-  const int t = static_cast<int>(m % T);
-  const int gy = t / grid, gx = t % grid;
-  const int side = grid * patch;
-  const int pd = C * patch * patch;
-  for (int j = threadIdx.x; j < pd; j += blockDim.x) {
-    const int c = j / (patch * patch), py = (j / patch) % patch, px = j % patch;
-    sp[j] = latent[((static_cast<int64_t>(b) * C + c) * side + gy * patch + py) * side + gx * patch + px];
+                                                    int64_t M, int D, int grid, int patch, int C) {
+  __shared__ float sp[EMB_ROWS][EMB_MAX_PD];
+  const int T = grid * grid, side = grid * patch, pd = C * patch * patch;
+  const int64_t m0 = static_cast<int64_t>(blockIdx.x) * EMB_ROWS;
+  for (int i = threadIdx.x; i < EMB_ROWS * pd; i += blockDim.x) {
+    const int r = i / pd, j = i % pd;
+    const int64_t m = m0 + r;
+    float v = 0.0f;
+    if (m < M) {
+      const int b = static_cast<int>(m / T) % latent_batch, t = static_cast<int>(m % T);
+      const int gy = t / grid, gx = t % grid;
+      const int c = j / (patch * patch), py = (j / patch) % patch, px = j % patch;
+      v = latent[((static_cast<int64_t>(b) * C + c) * side + gy * patch + py) * side + gx * patch + px];
+    }
+    sp[r][j] = v;
   }
   __syncthreads();
-  for (int d = threadIdx.x; d < D; d += blockDim.x) {
-    float acc = 0.0f;
-    const float* wr = w + static_cast<int64_t>(d) * pd;
-    for (int j = 0; j < pd; ++j) acc = fmaf(wr[j], sp[j], acc);
-    x[m * D + d] = __float2bfloat16_rn(acc + bias[d] + pos[static_cast<int64_t>(t) * D + d]);
+  const int d = (blockIdx.y * blockDim.x + threadIdx.x) * 2;
+  if (d >= D) return;
+  float w0[EMB_MAX_PD], w1[EMB_MAX_PD];
+#pragma unroll
+  for (int j = 0; j < EMB_MAX_PD; ++j) {
+    if (j < pd) {
+      w0[j] = w[static_cast<int64_t>(d) * pd + j];
+      w1[j] = w[static_cast<int64_t>(d + 1) * pd + j];
+    }
+  }
+  const float b0 = bias[d], b1 = bias[d + 1];
+  for (int r = 0; r < EMB_ROWS; ++r) {
+    const int64_t m = m0 + r;
+    if (m >= M) break;
+    float a0 = 0.0f, a1 = 0.0f;
+#pragma unroll
+    for (int j = 0; j < EMB_MAX_PD; ++j) {
+      if (j < pd) {
+        a0 = fmaf(w0[j], sp[r][j], a0);
+        a1 = fmaf(w1[j], sp[r][j], a1);
+      }
+    }
+    const float2 pv = *reinterpret_cast<const float2*>(pos + static_cast<int64_t>(m % T) * D + d);
+    *reinterpret_cast<uint32_t*>(x + m * D + d) = pack_bf16x2(a0 + b0 + pv.x, a1 + b1 + pv.y);
   }
 }
 
 // ----------------------------------------------------------------------------- conditioning
-// Warp per output.  h[b,d] = SiLU(W1[d,:] . feat(t_b) + b1[d]); features [cos(t f_j), sin(t f_j)],
-// f_j = 10000^(-j/half), evaluated in double so that large arguments keep their phase.
-__global__ void __launch_bounds__(256) cond1_kernel(const float* __restrict__ t, const float* __restrict__ w1,
-                                                    const float* __restrict__ b1, float* __restrict__ h, int B, int D,
-                                                    int F) {
-  const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (gw >= B * D) return;
-  const int b = gw / D, d = gw % D;
-  const int half = F / 2;
-  const double tv = static_cast<double>(t[b]);
-  float acc = 0.0f;
-  for (int j = lane; j < F; j += 32) {
-    const int jj = j < half ? j : j - half;
-    const double arg = tv * exp(-9.210340371976184 * static_cast<double>(jj) / static_cast<double>(half));
-    const float f = static_cast<float>(j < half ? cos(arg) : sin(arg));
-    acc = fmaf(w1[static_cast<int64_t>(d) * F + j], f, acc);
-  }
-  acc = warp_sum(acc);
-  if (lane == 0) h[gw] = silu_f(acc + b1[d]);
+// Sinusoidal timestep features feat[b, :] = [cos(t f_j), sin(t f_j)], f_j = 10000^(-j/half), evaluated in
+// double so that arguments of hundreds of radians keep their phase.
+__global__ void timestep_features_kernel(const float* __restrict__ t, float* __restrict__ feat, int B, int F) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= B * F) return;
+  const int b = i / F, j = i % F, half = F / 2;
+  const int jj = j < half ? j : j - half;
+  const double arg = static_cast<double>(t[b]) * exp(-9.210340371976184 * static_cast<double>(jj) / static_cast<double>(half));
+  feat[i] = static_cast<float>(j < half ? cos(arg) : sin(arg));
 }
 
-// out[b,n] = W[n,:] . in[b,:] + bias[n] (+ table[y[b], n]); optionally also SiLU(out) to out_silu.
+// out[b,n] = W[n,:] . f(in[b,:]) + bias[n] (+ table[y[b],n]), optionally passed through SiLU, and optionally
+// SiLU(out) as a second output.  The inputs of up to `bc` samples sit in shared memory; a warp owns one
+// output feature, keeps its weight row in registers and walks the samples.
+constexpr int SL_MAXV = 16;  // float4 per lane: K <= 2048
 __global__ void __launch_bounds__(256) small_linear_kernel(const float* __restrict__ in, const float* __restrict__ w,
                                                            const float* __restrict__ bias,
                                                            const float* __restrict__ table, const int32_t* __restrict__ y,
                                                            float* __restrict__ out, float* __restrict__ out_silu, int B,
-                                                           int N, int K, int silu_input) {
-  const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (gw >= B * N) return;
-  const int b = gw / N, n = gw % N;
-  float acc = 0.0f;
-  const float* wr = w + static_cast<int64_t>(n) * K;
-  const float* xr = in + static_cast<int64_t>(b) * K;
-  for (int k = lane * 4; k < K; k += 128) {
-    const float4 wv = *reinterpret_cast<const float4*>(wr + k);
-    float4 xv = *reinterpret_cast<const float4*>(xr + k);
-    if (silu_input) {
-      xv.x = silu_f(xv.x); xv.y = silu_f(xv.y); xv.z = silu_f(xv.z); xv.w = silu_f(xv.w);
+                                                           int N, int K, int bc, int silu_input, int silu_output) {
+  extern __shared__ float s_in[];  // [bc][K]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n = blockIdx.x * (blockDim.x >> 5) + warp;
+  float4 wv[SL_MAXV];
+  if (n < N) {
+#pragma unroll
+    for (int j = 0; j < SL_MAXV; ++j) {
+      const int k = lane * 4 + 128 * j;
+      wv[j] = k < K ? *reinterpret_cast<const float4*>(w + static_cast<int64_t>(n) * K + k) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    acc = fmaf(wv.x, xv.x, acc);
-    acc = fmaf(wv.y, xv.y, acc);
-    acc = fmaf(wv.z, xv.z, acc);
-    acc = fmaf(wv.w, xv.w, acc);
   }
-  acc = warp_sum(acc);
-  if (lane == 0) {
-    float v = acc + bias[n];
-    if (table) v += table[static_cast<int64_t>(y[b]) * N + n];
-    out[gw] = v;
-    if (out_silu) out_silu[gw] = silu_f(v);
+  for (int b0 = 0; b0 < B; b0 += bc) {
+    const int nb = B - b0 < bc ? B - b0 : bc;
+    __syncthreads();
+    for (int i = threadIdx.x * 4; i < nb * K; i += blockDim.x * 4) {
+      float4 v = *reinterpret_cast<const float4*>(in + static_cast<int64_t>(b0) * K + i);
+      if (silu_input) {
+        v.x = silu_f(v.x); v.y = silu_f(v.y); v.z = silu_f(v.z); v.w = silu_f(v.w);
+      }
+      *reinterpret_cast<float4*>(s_in + i) = v;
+    }
+    __syncthreads();
+    if (n < N) {
+      for (int b = 0; b < nb; ++b) {
+        float acc = 0.0f;
+#pragma unroll
+        for (int j = 0; j < SL_MAXV; ++j) {
+          const int k = lane * 4 + 128 * j;
+          if (k < K) {
+            const float4 xv = *reinterpret_cast<const float4*>(s_in + b * K + k);
+            acc = fmaf(wv[j].x, xv.x, acc);
+            acc = fmaf(wv[j].y, xv.y, acc);
+            acc = fmaf(wv[j].z, xv.z, acc);
+            acc = fmaf(wv[j].w, xv.w, acc);
+          }
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) {
+          const int64_t o = static_cast<int64_t>(b0 + b) * N + n;
+          float v = acc + bias[n];
+          if (table) v += table[static_cast<int64_t>(y[b0 + b]) * N + n];
+          if (silu_output) v = silu_f(v);
+          out[o] = v;
+          if (out_silu) out_silu[o] = silu_f(v);
+        }
+      }
+    }
   }
 }
 
@@ -284,23 +327,38 @@ __global__ void __launch_bounds__(256) final_kernel(const __nv_bfloat16* __restr
 // ================================================================================ launchers
 int32_t launch_embed(qdit_ctx* ctx, const float* latent, int latent_batch, const float* w, const float* bias,
                      const float* pos, void* x, int64_t M, int D, int grid, int patch, int C) {
-  embed_kernel<<<static_cast<unsigned>(M), 128, C * patch * patch * sizeof(float), ctx->stream>>>(
-      latent, latent_batch, w, bias, pos, static_cast<__nv_bfloat16*>(x), D, grid, patch, C);
+  if (C * patch * patch > EMB_MAX_PD) return qdit_fail(ctx, QDIT_ERR_SHAPE, "patch vector longer than %d", EMB_MAX_PD);
+  dim3 g(static_cast<unsigned>((M + EMB_ROWS - 1) / EMB_ROWS), static_cast<unsigned>((D / 2 + 255) / 256));
+  embed_kernel<<<g, 256, 0, ctx->stream>>>(latent, latent_batch, w, bias, pos, static_cast<__nv_bfloat16*>(x), M, D, grid,
+                                           patch, C);
   return qdit_after_launch(ctx, "embed_kernel");
 }
 
-int32_t launch_cond1(qdit_ctx* ctx, const float* t, const float* w1, const float* b1, float* h, int B, int D, int F) {
-  const int64_t threads = static_cast<int64_t>(B) * D * 32;
-  cond1_kernel<<<static_cast<unsigned>((threads + 255) / 256), 256, 0, ctx->stream>>>(t, w1, b1, h, B, D, F);
-  return qdit_after_launch(ctx, "cond1_kernel");
+int32_t launch_small_linear(qdit_ctx* ctx, const float* in, const float* w, const float* bias, const float* table,
+                            const int32_t* y, float* out, float* out_silu, int B, int N, int K, int silu_input,
+                            int silu_output) {
+  if (K % 4 != 0 || K > 128 * SL_MAXV) return qdit_fail(ctx, QDIT_ERR_SHAPE, "small linear needs K %% 4 == 0 and K <= %d", 128 * SL_MAXV);
+  const int smem_budget = 160 * 1024;
+  int bc = smem_budget / (K * static_cast<int>(sizeof(float)));
+  if (bc > B) bc = B;
+  if (bc < 1) bc = 1;
+  const size_t smem = static_cast<size_t>(bc) * K * sizeof(float);
+  static bool attr_set[64] = {};
+  if (!attr_set[ctx->device & 63]) {
+    QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(small_linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_budget));
+    attr_set[ctx->device & 63] = true;
+  }
+  small_linear_kernel<<<static_cast<unsigned>((N + 7) / 8), 256, smem, ctx->stream>>>(in, w, bias, table, y, out, out_silu, B, N,
+                                                                                    K, bc, silu_input, silu_output);
+  return qdit_after_launch(ctx, "small_linear_kernel");
 }
 
-int32_t launch_small_linear(qdit_ctx* ctx, const float* in, const float* w, const float* bias, const float* table,
-                            const int32_t* y, float* out, float* out_silu, int B, int N, int K, int silu_input) {
-  const int64_t threads = static_cast<int64_t>(B) * N * 32;
-  small_linear_kernel<<<static_cast<unsigned>((threads + 255) / 256), 256, 0, ctx->stream>>>(
-      in, w, bias, table, y, out, out_silu, B, N, K, silu_input);
-  return qdit_after_launch(ctx, "small_linear_kernel");
+// h[b,:] = SiLU(W1 . sinusoid(t_b) + b1); feat: scratch [B, F]
+int32_t launch_cond1(qdit_ctx* ctx, const float* t, const float* w1, const float* b1, float* feat, float* h, int B, int D,
+                     int F) {
+  timestep_features_kernel<<<(B * F + 255) / 256, 256, 0, ctx->stream>>>(t, feat, B, F);
+  QDIT_TRY(qdit_after_launch(ctx, "timestep_features_kernel"));
+  return launch_small_linear(ctx, feat, w1, b1, nullptr, nullptr, h, nullptr, B, D, F, 0, 1);
 }
 
 int32_t launch_final(qdit_ctx* ctx, const void* x, int64_t M, int D, int T, float eps, const float* modf,

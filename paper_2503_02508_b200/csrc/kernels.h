@@ -9,11 +9,14 @@ struct DdimCoef {
 // x[m,:] = bf16(W_patch . patch(m) + b + pos); sample b reads latent[b % latent_batch].
 int32_t launch_embed(qdit_ctx* ctx, const float* latent, int latent_batch, const float* w, const float* bias,
                      const float* pos, void* x, int64_t M, int D, int grid, int patch, int C);
-// h[b,:] = SiLU(W1 . sinusoid(t_b) + b1)
-int32_t launch_cond1(qdit_ctx* ctx, const float* t, const float* w1, const float* b1, float* h, int B, int D, int F);
-// out[b,n] = W[n,:] . f(in[b,:]) + bias[n] (+ table[y[b],n]); f = SiLU if silu_input; out_silu (optional) = SiLU(out)
+// h[b,:] = SiLU(W1 . sinusoid(t_b) + b1); feat is scratch [B, F]
+int32_t launch_cond1(qdit_ctx* ctx, const float* t, const float* w1, const float* b1, float* feat, float* h, int B, int D,
+                     int F);
+// out[b,n] = g(W[n,:] . f(in[b,:]) + bias[n] (+ table[y[b],n])); f = SiLU if silu_input, g = SiLU if silu_output;
+// out_silu (optional) = SiLU(out)
 int32_t launch_small_linear(qdit_ctx* ctx, const float* in, const float* w, const float* bias, const float* table,
-                            const int32_t* y, float* out, float* out_silu, int B, int N, int K, int silu_input);
+                            const int32_t* y, float* out, float* out_silu, int B, int N, int K, int silu_input,
+                            int silu_output);
 // LayerNorm + modulate + linear D->OUT + un-patchify into net [B, OUT/p^2, side, side]
 int32_t launch_final(qdit_ctx* ctx, const void* x, int64_t M, int D, int T, float eps, const float* modf,
                      const float* w, const float* bias, float* net, int grid, int patch, int OUT);

@@ -61,7 +61,7 @@ struct qdit_sampler {
   int64_t M;
   void *x, *qkv;                 // bf16
   uint8_t *h, *a, *u, *ca;       // activation codes
-  float *c, *sc, *hidden, *mod, *modf, *net, *latent, *t_all, *tmpf;   // t_all: [S, Beff] timestep of every step
+  float *c, *sc, *hidden, *feat, *mod, *modf, *net, *latent, *t_all, *tmpf;   // t_all: [S, Beff] timestep of every step
   int32_t *y, *labels;
   float* dyn_absmax;             // [1 + 4*depth] this pass's ranges (calibration)
   float* dyn_scale;              // [1 + 4*depth] and the scales derived from them
@@ -196,8 +196,8 @@ static int32_t forward_impl(qdit_ctx* ctx, qdit_sampler* s, const float* latent,
   const float* scales = calib ? s->dyn_scale : m->d_scales;
 
   QDIT_TRY(launch_embed(ctx, latent, latent_batch, m->w_patch, m->b_patch, m->pos, s->x, M, D, sh.grid, sh.patch, sh.channels));
-  QDIT_TRY(launch_cond1(ctx, t, m->w_t1, m->b_t1, s->hidden, B, D, sh.freq_dim));
-  QDIT_TRY(launch_small_linear(ctx, s->hidden, m->w_t2, m->b_t2, m->y_table, y, s->c, s->sc, B, D, D, 0));
+  QDIT_TRY(launch_cond1(ctx, t, m->w_t1, m->b_t1, s->feat, s->hidden, B, D, sh.freq_dim));
+  QDIT_TRY(launch_small_linear(ctx, s->hidden, m->w_t2, m->b_t2, m->y_table, y, s->c, s->sc, B, D, D, 0, 0));
   // modulation of every block in one stacked GEMM (the conditioning does not depend on the tokens)
   if (calib) {
     QDIT_TRY(dyn_quant(ctx, s, 0, s->sc, B, D, s->ca));
@@ -270,7 +270,7 @@ static int32_t forward_impl(qdit_ctx* ctx, qdit_sampler* s, const float* latent,
     }
   }
   // final layer (f32): modulation from SiLU(c), LayerNorm, linear, un-patchify
-  QDIT_TRY(launch_small_linear(ctx, s->c, m->w_ada_f, m->b_ada_f, nullptr, nullptr, s->modf, nullptr, B, 2 * D, D, 1));
+  QDIT_TRY(launch_small_linear(ctx, s->c, m->w_ada_f, m->b_ada_f, nullptr, nullptr, s->modf, nullptr, B, 2 * D, D, 1, 0));
   QDIT_TRY(launch_final(ctx, s->x, M, D, T, 1e-6f, s->modf, m->w_out, m->b_out, out, sh.grid, sh.patch,
                         2 * sh.channels * sh.patch * sh.patch));
   return QDIT_OK;
@@ -411,6 +411,7 @@ int32_t qdit_sampler_create(qdit_ctx* ctx, qdit_model* m, const qdit_sampler_des
   s->c = a.alloc<float>(B * D);
   s->sc = a.alloc<float>(B * D);
   s->hidden = a.alloc<float>(B * D);
+  s->feat = a.alloc<float>(B * sh.freq_dim);
   s->mod = a.alloc<float>(B * sh.depth * 6 * D);
   s->modf = a.alloc<float>(B * 2 * D);
   s->net = a.alloc<float>(B * 2 * C * HW);
@@ -421,7 +422,7 @@ int32_t qdit_sampler_create(qdit_ctx* ctx, qdit_model* m, const qdit_sampler_des
   s->tmpf = a.alloc<float>(M * F);
   s->dyn_absmax = a.alloc<float>(m->n_scales());
   s->dyn_scale = a.alloc<float>(m->n_scales());
-  bool ok = s->x && s->qkv && s->h && s->a && s->u && s->ca && s->c && s->sc && s->hidden && s->mod && s->modf && s->net &&
+  bool ok = s->x && s->qkv && s->h && s->a && s->u && s->ca && s->c && s->sc && s->hidden && s->feat && s->mod && s->modf && s->net &&
             s->latent && s->t_all && s->y && s->labels && s->tmpf && s->dyn_absmax && s->dyn_scale;
   if (ok && d->vc_mode != QDIT_VC_NONE) {
     s->vc_table = a.alloc<float>(static_cast<int64_t>(d->num_steps) * C);

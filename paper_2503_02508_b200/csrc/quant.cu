@@ -130,46 +130,70 @@ __global__ void __launch_bounds__(256) weight_quant_kernel(const float* __restri
 }
 
 // ----------------------------------------------------------------------------- LayerNorm + modulate (+ quantize)
-// One warp per row; the row lives in registers (NV vectors of 8 per lane).  Two-pass statistics in f32.
+// One warp per row, 8 rows per CTA; the row lives in registers (NV vectors of 8 per lane), statistics are
+// two-pass in f32.  The CTA first copies shift and scale of its first row's sample into shared memory
+// (all its rows share them when T is a multiple of 8; a row of another sample falls back to global reads),
+// while every warp's row is already in flight, so the modulation parameters cost one pass over L2 per CTA
+// instead of one per row and no dependent round trip after the statistics.
 template <int NV>
 __global__ void __launch_bounds__(256) ln_modulate_kernel(const __nv_bfloat16* __restrict__ x, int64_t M, int D,
                                                           int64_t T, float eps, const float* __restrict__ shift,
                                                           const float* __restrict__ scale, int64_t ld_mod,
                                                           void* __restrict__ out, int out_dtype, QuantArgs qa) {
+  extern __shared__ float s_mod[];  // [2][D]: shift, scale of sample b0
   const int lane = threadIdx.x & 31;
-  const int64_t row = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (row >= M) return;
+  const int64_t row0 = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5);
+  const int64_t row = row0 + (threadIdx.x >> 5);
+  const bool active = row < M;
   const int nvec = D >> 3;
-  const __nv_bfloat16* xr = x + row * D;
   float v[NV][8];
+  if (active) {
+    const __nv_bfloat16* xr = x + row * D;
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+      const int vi = lane + 32 * j;
+      if (vi < nvec) Load8<__nv_bfloat16>::load(xr + vi * 8, v[j]);
+    }
+  }
+  const int64_t b0 = row0 / T;
+  {
+    const float4* gs = reinterpret_cast<const float4*>(shift + b0 * ld_mod);
+    const float4* gc = reinterpret_cast<const float4*>(scale + b0 * ld_mod);
+    float4* ss = reinterpret_cast<float4*>(s_mod);
+    float4* sc4 = reinterpret_cast<float4*>(s_mod + D);
+    for (int i = threadIdx.x; i < D / 4; i += blockDim.x) {
+      ss[i] = gs[i];
+      sc4[i] = gc[i];
+    }
+  }
+  __syncthreads();
+  if (!active) return;
   float sum = 0.0f;
 #pragma unroll
   for (int j = 0; j < NV; ++j) {
-    const int vi = lane + 32 * j;
-    if (vi < nvec) {
-      Load8<__nv_bfloat16>::load(xr + vi * 8, v[j]);
+    if (lane + 32 * j < nvec) {
 #pragma unroll
       for (int i = 0; i < 8; ++i) sum += v[j][i];
     }
   }
   const float mean = warp_sum(sum) / static_cast<float>(D);
-  float ss = 0.0f;
+  float ssq = 0.0f;
 #pragma unroll
   for (int j = 0; j < NV; ++j) {
-    const int vi = lane + 32 * j;
-    if (vi < nvec) {
+    if (lane + 32 * j < nvec) {
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const float d = v[j][i] - mean;
-        ss += d * d;
+        ssq += d * d;
       }
     }
   }
-  const float var = warp_sum(ss) / static_cast<float>(D);
+  const float var = warp_sum(ssq) / static_cast<float>(D);
   const float rstd = 1.0f / sqrtf(var + eps);
   const int64_t b = row / T;
-  const float* sh = shift + b * ld_mod;
-  const float* sc = scale + b * ld_mod;
+  const bool staged = b == b0;
+  const float* sh = staged ? s_mod : shift + b * ld_mod;
+  const float* sc = staged ? s_mod + D : scale + b * ld_mod;
   float inv = 0.0f;
   if (out_dtype == QDIT_I8) {
     const float s = qa.scale_dev ? __ldg(qa.scale_dev) : qa.scale;
@@ -205,8 +229,8 @@ void launch_ln(qdit_ctx* ctx, const void* x, int64_t M, int D, int64_t T, float 
                const float* scale, int64_t ld_mod, void* out, int out_dtype, QuantArgs qa) {
   const int warps = 8;
   const unsigned grid = static_cast<unsigned>((M + warps - 1) / warps);
-  ln_modulate_kernel<NV><<<grid, warps * 32, 0, ctx->stream>>>(static_cast<const __nv_bfloat16*>(x), M, D, T, eps, shift,
-                                                               scale, ld_mod, out, out_dtype, qa);
+  ln_modulate_kernel<NV><<<grid, warps * 32, 2 * D * sizeof(float), ctx->stream>>>(
+      static_cast<const __nv_bfloat16*>(x), M, D, T, eps, shift, scale, ld_mod, out, out_dtype, qa);
 }
 
 }  // namespace

@@ -47,11 +47,14 @@ SHAPES = [(1, 8, 16), (128, 192, 128), (130, 200, 272), (256, 384, 1152), (517, 
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)
-@pytest.mark.parametrize("bn", ["auto", "64", "128", "192"])
+@pytest.mark.parametrize("bn", ["auto", "64", "128", "192", "pair128", "pair192", "pair256"])
 def test_accumulators_bit_exact(q, ctx, M, N, K, bn):
-    if bn == "auto":
-        os.environ.pop("QDIT_GEMM_BN", None)
-    else:
+    # "pairNNN": the CTA-pair kernel (256 x NNN tiles); plain numbers: the single-CTA kernel (128 x NNN)
+    os.environ.pop("QDIT_GEMM_BN", None)
+    os.environ.pop("QDIT_GEMM_PAIR", None)
+    if bn.startswith("pair"):
+        os.environ["QDIT_GEMM_PAIR"] = bn[4:]
+    elif bn != "auto":
         os.environ["QDIT_GEMM_BN"] = bn
     try:
         qa = _codes(31, f"a{M}.{K}", (M, K), -128, 127)
@@ -59,6 +62,7 @@ def test_accumulators_bit_exact(q, ctx, M, N, K, bn):
         got = _run_i32(q, ctx, qa, qw)
     finally:
         os.environ.pop("QDIT_GEMM_BN", None)
+        os.environ.pop("QDIT_GEMM_PAIR", None)
     np.testing.assert_array_equal(got, linear.gemm_i8(qa, qw))
 
 
@@ -123,7 +127,16 @@ def test_dequant_bias_f32(q, ctx, M, N, K, T, a_qp):
     assert max_rel_err(out.cpu().numpy(), ref) < 1e-5      # ... and what f32 arithmetic actually gives
 
 
-def test_gate_residual_cache_epilogue(q, ctx):
+@pytest.fixture(params=["single", "pair192", "pair256"])
+def kernel_variant(request):
+    os.environ.pop("QDIT_GEMM_PAIR", None)
+    if request.param.startswith("pair"):
+        os.environ["QDIT_GEMM_PAIR"] = request.param[4:]
+    yield request.param
+    os.environ.pop("QDIT_GEMM_PAIR", None)
+
+
+def test_gate_residual_cache_epilogue(q, ctx, kernel_variant):
     M, N, K, T = 512, 1152, 1152, 256
     a_qp = QParams(0.05, 0, -127, 127)
     L = _layer(42, M, N, K, T, a_qp)
@@ -147,7 +160,7 @@ def test_gate_residual_cache_epilogue(q, ctx):
     assert max_rel_err(got_x, want_x) < 2.0 ** -8
 
 
-def test_gelu_requant_epilogue(q, ctx):
+def test_gelu_requant_epilogue(q, ctx, kernel_variant):
     M, N, K, T = 384, 1536, 384, 128
     a_qp = QParams(0.04, 0, -127, 127)
     L = _layer(43, M, N, K, T, a_qp)
