@@ -12,9 +12,13 @@ using namespace qd;
 constexpr int BM = 128;        // tile rows = TMEM lanes
 constexpr int BK = 128;        // K bytes per stage = one swizzle row
 constexpr int UMMA_K = 32;     // K per kind::i8 instruction
-constexpr int NUM_EPI_WARPS = 8;
+#ifndef QDIT_EPI_WARPS
+#define QDIT_EPI_WARPS 12
+#endif
+constexpr int NUM_EPI_WARPS = QDIT_EPI_WARPS;  // a multiple of 4: EPI_SPLIT warps share each TMEM lane quadrant
+constexpr int EPI_SPLIT = NUM_EPI_WARPS / 4;
 constexpr int NUM_THREADS = 64 + NUM_EPI_WARPS * 32;
-constexpr int STAGING_BYTES = NUM_EPI_WARPS * 2 * 32 * 128;  // two 32 x 32 x int32 patches per epilogue warp
+constexpr int STAGING_BYTES = NUM_EPI_WARPS * 32 * 128;  // one 32 x 32 x int32 patch per epilogue warp
 
 struct GemmParams {
   int M, N, K;
@@ -152,9 +156,9 @@ __device__ __forceinline__ void prefetch_chunk(const GemmParams& p, int n, int r
 
 // Epilogue of one 128 x BN accumulator tile for one epilogue warp (see the data-flow note in gemm_i8.cu).
 // `tacc` = TMEM address of the accumulator stage (lane 0 of the CTA, first column); `release()` hands the
-// stage back to the MMA issuer once this warp has read its share.  `stg` = this warp's two 4 KB staging
-// patches.  The loop is software-pipelined: while chunk k is transposed and written out, the TMEM load and
-// the global loads of chunk k+1 are already in flight.
+// stage back to the MMA issuer once this warp has read its share.  `stg` = this warp's 4 KB staging patch.
+// The epilogue is bound by the latency chain of one chunk (global loads, TMEM load, transpose, stores), so
+// the tile's chunks are spread over as many warps as the register file allows.
 template <int BN, typename Release>
 __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t tacc, int m0, int n0, int quad, int half,
                                               uint32_t stg, int lane, float a_scale, float o_inv, Release release) {
@@ -162,22 +166,23 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t tacc
   const int rsub = lane >> 2;  // ... of rows rsub, rsub + 8, rsub + 16, rsub + 24
   const bool gate_uniform = (p.tokens % 32) == 0;  // the warp's 32 rows then belong to one sample
   constexpr int CHUNKS = BN / 32;
-  constexpr int LAST_EVEN = ((CHUNKS - 1) / 2) * 2, LAST_ODD = ((CHUNKS - 2) / 2) * 2 + 1;
-  const int c_last = half ? LAST_ODD : LAST_EVEN;
+  // this warp takes chunks half, half + EPI_SPLIT, ...; c_last = the last of them (-1: none)
+  const int c_last = half < CHUNKS ? half + ((CHUNKS - 1 - half) / EPI_SPLIT) * EPI_SPLIT : -1;
+  if (c_last < 0) {  // nothing to read: hand the accumulator stage back untouched
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) release();
+    return;
+  }
   const int row_base = m0 + quad * 32;
   const uint32_t taddr = tacc + (static_cast<uint32_t>(quad * 32) << 16);
 
-#ifndef QDIT_EPI_PIPELINE
-#define QDIT_EPI_PIPELINE 0
-#endif
-#if QDIT_EPI_PIPELINE == 0
   // plain order per chunk: global loads -> TMEM load -> transpose -> math and stores
-  int buf = 0;
 #pragma unroll 1
-  for (int c = half; c < CHUNKS; c += 2, buf ^= 1) {
+  for (int c = half; c < CHUNKS; c += EPI_SPLIT) {
     const int n = n0 + c * 32 + cg * 8;
     const bool col_ok = n < p.N;
-    const uint32_t patch = stg + static_cast<uint32_t>(buf * 4096);
+    const uint32_t patch = stg;
     ChunkInputs cur;
     prefetch_chunk(p, n, row_base, rsub, a_scale, cur);
     uint32_t v[32];
@@ -213,58 +218,6 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t tacc
       }
     }
   }
-#else
-  ChunkInputs cur, nxt;
-  uint32_t v[32];
-  prefetch_chunk(p, n0 + half * 32 + cg * 8, row_base, rsub, a_scale, cur);
-  __syncwarp();
-  tmem_ld_32x32(taddr + static_cast<uint32_t>(half * 32), v);
-  int buf = 0;
-#pragma unroll 1
-  for (int c = half; c < CHUNKS; c += 2, buf ^= 1) {
-    const int n = n0 + c * 32 + cg * 8;
-    const bool col_ok = n < p.N;
-    const uint32_t patch = stg + static_cast<uint32_t>(buf * 4096);
-    tmem_ld_wait();  // chunk c is in v
-    // ---- registers (one row per thread) -> swizzled staging patch; the patch was last read two chunks ago
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const uint32_t addr = patch + static_cast<uint32_t>(lane * 128 + ((j ^ (lane & 7)) << 4));
-      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v[4 * j]), "r"(v[4 * j + 1]),
-                   "r"(v[4 * j + 2]), "r"(v[4 * j + 3])
-                   : "memory");
-    }
-    if (c == c_last) {
-      // this warp has read all of its share of the accumulator stage: hand it back to the MMA warp
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) release();
-    } else {
-      // next chunk: global loads and the TMEM load fly while this chunk is processed
-      prefetch_chunk(p, n + 64, row_base, rsub, a_scale, nxt);
-      __syncwarp();
-      tmem_ld_32x32(taddr + static_cast<uint32_t>((c + 2) * 32), v);
-    }
-    __syncwarp();
-    // ---- transposed ownership: 8 columns of 4 rows per lane
-#pragma unroll
-    for (int sidx = 0; sidx < 4; ++sidx) {
-      const int r = sidx * 8 + rsub;
-      const int row = row_base + r;
-      uint4 lo, hi;
-      const uint32_t a_lo = patch + static_cast<uint32_t>(r * 128 + (((2 * cg) ^ (r & 7)) << 4));
-      const uint32_t a_hi = patch + static_cast<uint32_t>(r * 128 + (((2 * cg + 1) ^ (r & 7)) << 4));
-      asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(lo.x), "=r"(lo.y), "=r"(lo.z), "=r"(lo.w) : "r"(a_lo));
-      asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(hi.x), "=r"(hi.y), "=r"(hi.z), "=r"(hi.w) : "r"(a_hi));
-      if (row < p.M && col_ok) {
-        if (!gate_uniform && (p.flags & QDIT_EPI_GATE))
-          Load8<float>::load(p.gate + static_cast<int64_t>(row / p.tokens) * p.ld_gate + n, cur.cp.gt);
-        epilogue8(p, lo, hi, cur.cp, cur.res[sidx], row, n, o_inv);
-      }
-    }
-    cur = nxt;
-  }
-#endif
 }
 
 }  // namespace qgemm

@@ -1,9 +1,9 @@
 // W8A8 linear layer: persistent tcgen05 kind::i8 GEMM with TMEM int32 accumulators and a fused
 // de-quantising epilogue (bias / GELU / cache store / adaLN gate / residual / re-quantisation).
 //
-// CTA = 10 warps: warp 0 lane 0  TMA producer  (A and W tiles -> 128B-swizzled smem ring, mbarrier tx)
+// CTA = 2 + NUM_EPI_WARPS warps: warp 0 lane 0  TMA producer  (A and W tiles -> 128B-swizzled smem ring, mbarrier tx)
 //                 warp 1 lane 0  MMA issuer    (tcgen05.mma into one of two TMEM accumulator stages)
-//                 warps 2..9     epilogue      (two warps per TMEM lane quadrant, alternating 32-column chunks)
+//                 warps 2..      epilogue      (EPI_SPLIT warps per TMEM lane quadrant, taking 32-column chunks in turn)
 // The two accumulator stages let the epilogue of tile i overlap the main loop of tile i+1.
 // Tiles are 128 x BN, K is consumed in blocks of 128 bytes (4 MMAs of K = 32 each).
 //
@@ -135,8 +135,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     // -------------------------------------------------------------------- epilogue warps
     const int e = warp - 2;
     const int quad = warp & 3;   // TMEM lane quadrant this warp may access
-    const int half = e >> 2;     // this warp takes chunks half, half + 2, ...
-    const uint32_t stg = smem_u32(staging + e * (2 * 32 * 128));  // [32 rows][8 x 16 B], 16-byte index XOR (row & 7)
+    const int half = e >> 2;     // this warp takes chunks half, half + EPI_SPLIT, ...
+    const uint32_t stg = smem_u32(staging + e * (32 * 128));  // [32 rows][8 x 16 B], 16-byte index XOR (row & 7)
     const float a_scale = p.a_scale_dev ? __ldg(p.a_scale_dev) : p.a_scale;
     float o_inv = 0.0f;
     if (p.flags & QDIT_EPI_QUANT_OUT) o_inv = __fdiv_rn(1.0f, p.o_scale_dev ? __ldg(p.o_scale_dev) : p.o_scale);

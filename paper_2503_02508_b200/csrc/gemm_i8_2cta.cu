@@ -141,7 +141,7 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     const int e = warp - 2;
     const int quad = warp & 3;
     const int half = e >> 2;
-    const uint32_t stg = smem_u32(staging + e * (2 * 32 * 128));
+    const uint32_t stg = smem_u32(staging + e * (32 * 128));
     const float a_scale = p.a_scale_dev ? __ldg(p.a_scale_dev) : p.a_scale;
     float o_inv = 0.0f;
     if (p.flags & QDIT_EPI_QUANT_OUT) o_inv = __fdiv_rn(1.0f, p.o_scale_dev ? __ldg(p.o_scale_dev) : p.o_scale);
