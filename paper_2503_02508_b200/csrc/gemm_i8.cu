@@ -200,7 +200,7 @@ int pick_bn(int M, int N, int num_sms) {
     const int tiles = mt * ((N + bn - 1) / bn);
     const int waves = (tiles + num_sms - 1) / num_sms;
     const double cost = static_cast<double>(waves) * (bn + 24);
-    if (cost < best_cost * 0.97) {  // keep the wider tile unless the narrower one wins clearly
+    if (cost < best_cost * 0.85) {  // measured: the wider tile wins unless the narrower one saves a whole wave or more
       best_cost = cost;
       best = bn;
     }
