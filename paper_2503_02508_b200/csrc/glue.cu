@@ -249,75 +249,117 @@ __global__ void __launch_bounds__(256) small_linear_kernel(const float* __restri
 }
 
 // ----------------------------------------------------------------------------- final layer
-// Warp per token row: LayerNorm + modulate in registers, then the D -> OUT linear and un-patchify
-// (output vector ordered (py, px, c)) into net[b, c, gy*p+py, gx*p+px].
+// LayerNorm + modulate, then the D -> OUT linear (OUT = 32 for patch 2, 8 channels) and un-patchify (output
+// vector ordered (py, px, c)) into net[b, c, gy*p+py, gx*p+px].  Persistent CTAs keep the whole weight
+// matrix in shared memory (laid out so that a lane's 16-byte reads are conflict-free); a warp normalises
+// two token rows in registers, accumulates all OUT partial dot products per lane and finishes with a
+// transposing butterfly (31 shuffles per row) after which lane o holds output o.
+constexpr int FIN_OUT = 32;
 template <int NV>
-__global__ void __launch_bounds__(256) final_kernel(const __nv_bfloat16* __restrict__ x, int64_t M, int D, int T,
-                                                    float eps, const float* __restrict__ modf,
-                                                    const float* __restrict__ w, const float* __restrict__ bias,
-                                                    float* __restrict__ net, int grid, int patch, int OUT) {
-  const int lane = threadIdx.x & 31;
-  const int64_t row = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (row >= M) return;
+__global__ void __launch_bounds__(256, 1) final_kernel(const __nv_bfloat16* __restrict__ x, int64_t M, int D, int T,
+                                                       float eps, const float* __restrict__ modf,
+                                                       const float* __restrict__ w, const float* __restrict__ bias,
+                                                       float* __restrict__ net, int grid, int patch) {
+  extern __shared__ float4 s_w[];  // [FIN_OUT][NV][2][32] float4: (o, j, h, lane) = w[o][(lane + 32 j) * 8 + 4 h ..]
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   const int nvec = D >> 3;
-  float v[NV][8];
-  float sum = 0.0f;
-#pragma unroll
-  for (int j = 0; j < NV; ++j) {
-    const int vi = lane + 32 * j;
-    if (vi < nvec) {
-      Load8<__nv_bfloat16>::load(x + row * D + vi * 8, v[j]);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) sum += v[j][i];
-    } else {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) v[j][i] = 0.0f;
-    }
+  for (int i = threadIdx.x; i < FIN_OUT * NV * 2 * 32; i += blockDim.x) {
+    const int l = i & 31, h = (i >> 5) & 1, j = (i >> 6) % NV, o = i / (64 * NV);
+    const int vi = l + 32 * j;
+    s_w[i] = vi < nvec ? *reinterpret_cast<const float4*>(w + static_cast<int64_t>(o) * D + vi * 8 + 4 * h)
+                       : make_float4(0.f, 0.f, 0.f, 0.f);
   }
-  const float mean = warp_sum(sum) / static_cast<float>(D);
-  float ss = 0.0f;
+  __syncthreads();
+  const int side = grid * patch, co = FIN_OUT / (patch * patch);
+  for (int64_t row0 = (static_cast<int64_t>(blockIdx.x) * nwarps + warp) * 2; row0 < M;
+       row0 += static_cast<int64_t>(gridDim.x) * nwarps * 2) {
+    float y[2][NV][8];
 #pragma unroll
-  for (int j = 0; j < NV; ++j) {
-    if (lane + 32 * j < nvec) {
+    for (int r = 0; r < 2; ++r) {
+      const int64_t row = row0 + r;
+      const bool live = row < M;
+      float sum = 0.0f;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const float d = v[j][i] - mean;
-        ss += d * d;
+      for (int j = 0; j < NV; ++j) {
+        const int vi = lane + 32 * j;
+        if (live && vi < nvec) {
+          Load8<__nv_bfloat16>::load(x + row * D + vi * 8, y[r][j]);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) sum += y[r][j][i];
+        } else {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) y[r][j][i] = 0.0f;
+        }
+      }
+      const float mean = warp_sum(sum) / static_cast<float>(D);
+      float ss = 0.0f;
+#pragma unroll
+      for (int j = 0; j < NV; ++j) {
+        if (lane + 32 * j < nvec) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float d = y[r][j][i] - mean;
+            ss += d * d;
+          }
+        }
+      }
+      const float rstd = 1.0f / sqrtf(warp_sum(ss) / static_cast<float>(D) + eps);
+      const int b = live ? static_cast<int>(row / T) : 0;
+      const float* sh = modf + static_cast<int64_t>(b) * 2 * D;
+      const float* sc = sh + D;
+#pragma unroll
+      for (int j = 0; j < NV; ++j) {
+        const int vi = lane + 32 * j;
+        if (live && vi < nvec) {
+          float shv[8], scv[8];
+          Load8<float>::load(sh + vi * 8, shv);
+          Load8<float>::load(sc + vi * 8, scv);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) y[r][j][i] = (y[r][j][i] - mean) * rstd * (1.0f + scv[i]) + shv[i];
+        } else {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) y[r][j][i] = 0.0f;
+        }
       }
     }
-  }
-  const float rstd = 1.0f / sqrtf(warp_sum(ss) / static_cast<float>(D) + eps);
-  const int b = static_cast<int>(row / T), t = static_cast<int>(row % T);
-  const float* sh = modf + static_cast<int64_t>(b) * 2 * D;
-  const float* sc = sh + D;
+    float p0[FIN_OUT], p1[FIN_OUT];
 #pragma unroll
-  for (int j = 0; j < NV; ++j) {
-    const int vi = lane + 32 * j;
-    if (vi < nvec) {
-      float shv[8], scv[8];
-      Load8<float>::load(sh + vi * 8, shv);
-      Load8<float>::load(sc + vi * 8, scv);
+    for (int o = 0; o < FIN_OUT; ++o) {
+      float a0 = 0.0f, a1 = 0.0f;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) v[j][i] = (v[j][i] - mean) * rstd * (1.0f + scv[i]) + shv[i];
+      for (int j = 0; j < NV; ++j) {
+        const float4 wl = s_w[((o * NV + j) * 2 + 0) * 32 + lane], wh = s_w[((o * NV + j) * 2 + 1) * 32 + lane];
+        a0 = fmaf(wl.x, y[0][j][0], a0); a0 = fmaf(wl.y, y[0][j][1], a0); a0 = fmaf(wl.z, y[0][j][2], a0); a0 = fmaf(wl.w, y[0][j][3], a0);
+        a0 = fmaf(wh.x, y[0][j][4], a0); a0 = fmaf(wh.y, y[0][j][5], a0); a0 = fmaf(wh.z, y[0][j][6], a0); a0 = fmaf(wh.w, y[0][j][7], a0);
+        a1 = fmaf(wl.x, y[1][j][0], a1); a1 = fmaf(wl.y, y[1][j][1], a1); a1 = fmaf(wl.z, y[1][j][2], a1); a1 = fmaf(wl.w, y[1][j][3], a1);
+        a1 = fmaf(wh.x, y[1][j][4], a1); a1 = fmaf(wh.y, y[1][j][5], a1); a1 = fmaf(wh.z, y[1][j][6], a1); a1 = fmaf(wh.w, y[1][j][7], a1);
+      }
+      p0[o] = a0;
+      p1[o] = a1;
     }
-  }
-  const int gy = t / grid, gx = t % grid, side = grid * patch, co = OUT / (patch * patch);
-  for (int o = 0; o < OUT; ++o) {
-    float acc = 0.0f;
+    // transposing reduction: after the round with stride s, a lane with bit s set keeps the upper half
 #pragma unroll
-    for (int j = 0; j < NV; ++j) {
-      const int vi = lane + 32 * j;
-      if (vi < nvec) {
-        float wv[8];
-        Load8<float>::load(w + static_cast<int64_t>(o) * D + vi * 8, wv);
+    for (int sft = 16; sft >= 1; sft >>= 1) {
+      const bool up = (lane & sft) != 0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) acc = fmaf(wv[i], v[j][i], acc);
+      for (int i = 0; i < sft; ++i) {
+        const float send0 = up ? p0[i] : p0[i + sft], keep0 = up ? p0[i + sft] : p0[i];
+        const float send1 = up ? p1[i] : p1[i + sft], keep1 = up ? p1[i + sft] : p1[i];
+        p0[i] = keep0 + __shfl_xor_sync(0xffffffffu, send0, sft);
+        p1[i] = keep1 + __shfl_xor_sync(0xffffffffu, send1, sft);
       }
     }
-    acc = warp_sum(acc);
-    if (lane == 0) {
-      const int c = o % co, px = (o / co) % patch, py = o / (co * patch);
-      net[((static_cast<int64_t>(b) * co + c) * side + gy * patch + py) * side + gx * patch + px] = acc + bias[o];
+    const int o = lane;  // lane o now holds output o of both rows
+    const int c = o % co, px = (o / co) % patch, py = o / (co * patch);
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      const int64_t row = row0 + r;
+      if (row < M) {
+        const int b = static_cast<int>(row / T), t = static_cast<int>(row % T);
+        const int gy = t / grid, gx = t % grid;
+        net[((static_cast<int64_t>(b) * co + c) * side + gy * patch + py) * side + gx * patch + px] =
+            (r == 0 ? p0[0] : p1[0]) + bias[o];
+      }
     }
   }
 }
@@ -363,16 +405,25 @@ int32_t launch_cond1(qdit_ctx* ctx, const float* t, const float* w1, const float
 
 int32_t launch_final(qdit_ctx* ctx, const void* x, int64_t M, int D, int T, float eps, const float* modf,
                      const float* w, const float* bias, float* net, int grid, int patch, int OUT) {
-  const int warps = 8;
-  const unsigned g = static_cast<unsigned>((M + warps - 1) / warps);
+  if (OUT != FIN_OUT) return qdit_fail(ctx, QDIT_ERR_SHAPE, "final layer width %d not supported (needs patch*patch*2*channels = %d)", OUT, FIN_OUT);
   const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
   const int nv = (D / 8 + 31) / 32;
-#define QDIT_FINAL_CASE(NV) \
-  case NV: final_kernel<NV><<<g, warps * 32, 0, ctx->stream>>>(xb, M, D, T, eps, modf, w, bias, net, grid, patch, OUT); break;
+  const size_t smem = static_cast<size_t>(FIN_OUT) * nv * 2 * 32 * sizeof(float4);
+  int64_t want = (M + 15) / 16;
+  const unsigned g = static_cast<unsigned>(want < ctx->num_sms ? want : ctx->num_sms);
+#define QDIT_FINAL_CASE(NV)                                                                                             \
+  case NV: {                                                                                                            \
+    static bool attr_set[64] = {};                                                                                      \
+    if (!attr_set[ctx->device & 63]) {                                                                                  \
+      QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(final_kernel<NV>, cudaFuncAttributeMaxDynamicSharedMemorySize,          \
+                                                FIN_OUT * NV * 2 * 32 * static_cast<int>(sizeof(float4))));             \
+      attr_set[ctx->device & 63] = true;                                                                                \
+    }                                                                                                                   \
+    final_kernel<NV><<<g, 256, smem, ctx->stream>>>(xb, M, D, T, eps, modf, w, bias, net, grid, patch);                 \
+  } break;
   switch (nv) {
     QDIT_FINAL_CASE(1) QDIT_FINAL_CASE(2) QDIT_FINAL_CASE(3) QDIT_FINAL_CASE(4) QDIT_FINAL_CASE(5) QDIT_FINAL_CASE(6)
-    QDIT_FINAL_CASE(7)
-    default: final_kernel<8><<<g, warps * 32, 0, ctx->stream>>>(xb, M, D, T, eps, modf, w, bias, net, grid, patch, OUT); break;
+    default: return qdit_fail(ctx, QDIT_ERR_SHAPE, "final layer supports hidden <= 1536");
   }
 #undef QDIT_FINAL_CASE
   return qdit_after_launch(ctx, "final_kernel");

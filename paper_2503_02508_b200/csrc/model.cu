@@ -288,7 +288,7 @@ int32_t qdit_model_create(qdit_ctx* ctx, const qdit_model_desc* desc, qdit_model
     return qdit_fail(ctx, QDIT_ERR_SHAPE, "model shape fields must be positive");
   if (s.hidden % s.heads != 0 || (s.hidden / s.heads != 64 && s.hidden / s.heads != 72))
     return qdit_fail(ctx, QDIT_ERR_SHAPE, "head_dim must be 64 or 72");
-  if (s.hidden % 16 != 0 || s.mlp % 16 != 0 || s.hidden > 2048) return qdit_fail(ctx, QDIT_ERR_SHAPE, "hidden (<= 2048) and mlp must be multiples of 16");
+  if (s.hidden % 16 != 0 || s.mlp % 16 != 0 || s.hidden > 1536) return qdit_fail(ctx, QDIT_ERR_SHAPE, "hidden (<= 1536) and mlp must be multiples of 16");
   if ((s.grid * s.grid) % 64 != 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "tokens per image must be a multiple of 64");
   if (s.freq_dim % 2 != 0 || s.freq_dim % 4 != 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "freq_dim must be a multiple of 4");
   if ((s.grid * s.patch * s.grid * s.patch) % 4 != 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "latent size must be a multiple of 4");

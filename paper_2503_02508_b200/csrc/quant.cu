@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(256) weight_quant_kernel(const float* __restri
 // while every warp's row is already in flight, so the modulation parameters cost one pass over L2 per CTA
 // instead of one per row and no dependent round trip after the statistics.
 template <int NV>
-__global__ void __launch_bounds__(256) ln_modulate_kernel(const __nv_bfloat16* __restrict__ x, int64_t M, int D,
+__global__ void __launch_bounds__(256, 4) ln_modulate_kernel(const __nv_bfloat16* __restrict__ x, int64_t M, int D,
                                                           int64_t T, float eps, const float* __restrict__ shift,
                                                           const float* __restrict__ scale, int64_t ld_mod,
                                                           void* __restrict__ out, int out_dtype, QuantArgs qa) {
