@@ -1,7 +1,8 @@
 // Non-causal softmax attention in bf16 between the quantized linears.
 //
-// One CTA = 64 queries of one (sample, head); 4 warps x 16 query rows.  Q and 64-key K/V tiles are
-// staged by TMA (double-buffered, mbarrier completion) straight out of the token-major QKV matrix:
+// One CTA = 128 (or 64) queries of one (sample, head); one warp per 16 query rows.  Q and 64-key K/V tiles
+// are staged by TMA (a 4-deep ring with mbarrier completion: at 256 tokens the whole K and V of the head are
+// requested up front and the loop never synchronises) straight out of the token-major QKV matrix:
 // head_dim 64 uses 128-byte-swizzled rows, head_dim 72 keeps its natural 144-byte rows (which are
 // already bank-conflict-free for ldmatrix).  S = Q K^T and O = P V run on bf16 mma.sync with f32
 // accumulation; softmax is the online (running max / running sum) form in f32, exponentials in base 2.
@@ -13,9 +14,8 @@ namespace {
 
 using namespace qd;
 
-constexpr int BQ = 64;   // queries per CTA
-constexpr int BKV = 64;  // keys per staged tile
-constexpr int ATT_THREADS = 128;
+constexpr int BKV = 64;     // keys per staged tile
+constexpr int KV_STAGES = 4;  // ring depth
 
 struct AttnParams {
   int T, H, dh;
@@ -57,7 +57,7 @@ struct ACfg {
   static constexpr int KSTEPS = (DH + 15) / 16;      // k16 steps of Q K^T; the last one is half for DH = 72
   static constexpr bool HALF_TAIL = (DH % 16) == 8;
   static constexpr int NT_O = DH / 8;                // 8-wide column tiles of O
-  static constexpr int SMEM_BYTES = 5 * TILE_BYTES + 64 + 1024;
+  static constexpr int smem_bytes(int qw) { return (qw / 4 + 2 * KV_STAGES) * TILE_BYTES + 128 + 1024; }
 };
 
 template <int DH>
@@ -67,19 +67,20 @@ __device__ __forceinline__ uint32_t tile_addr(uint32_t base, int row, int col_el
   return base + static_cast<uint32_t>(row) * ACfg<DH>::ROW_BYTES + c;
 }
 
-template <int DH>
-__global__ void __launch_bounds__(ATT_THREADS)
+template <int DH, int QW>  // QW query warps (4 or 8) -> 16 * QW queries per CTA
+__global__ void __launch_bounds__(QW * 32, QW == 8 ? 2 : 4)
 attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
   using C = ACfg<DH>;
+  constexpr int BQ = QW * 16, QTILES = QW / 4;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sQ = smem;
-  uint8_t* sK = smem + C::TILE_BYTES;       // two stages
-  uint8_t* sV = smem + 3 * C::TILE_BYTES;   // two stages
-  uint64_t* bar_q = reinterpret_cast<uint64_t*>(smem + 5 * C::TILE_BYTES);
-  uint64_t* bar_kv = bar_q + 1;             // two stages
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_kv + 2);
+  uint8_t* sQ = smem;                                      // QTILES tiles of 64 rows
+  uint8_t* sK = smem + QTILES * C::TILE_BYTES;             // KV_STAGES tiles
+  uint8_t* sV = sK + KV_STAGES * C::TILE_BYTES;            // KV_STAGES tiles
+  uint64_t* bar_q = reinterpret_cast<uint64_t*>(sV + KV_STAGES * C::TILE_BYTES);
+  uint64_t* bar_kv = bar_q + 1;                            // one per stage
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_kv + KV_STAGES);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q0 = blockIdx.x * BQ, h = blockIdx.y, b = blockIdx.z;
@@ -89,33 +90,35 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
   if (threadIdx.x == 0) {
     mbar_init(bar_q, 1);
-    mbar_init(&bar_kv[0], 1);
-    mbar_init(&bar_kv[1], 1);
+    for (int s = 0; s < KV_STAGES; ++s) mbar_init(&bar_kv[s], 1);
     *abort_flag = 0;
     mbar_fence_init();
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    mbar_expect_tx(bar_q, C::TILE_BYTES);
-    tma_load_2d(sQ, &tm_q, col0, row0 + q0, bar_q);
-    mbar_expect_tx(&bar_kv[0], 2 * C::TILE_BYTES);
-    tma_load_2d(sK, &tm_k, col0, row0, &bar_kv[0]);
-    tma_load_2d(sV, &tm_v, col0, row0, &bar_kv[0]);
+    mbar_expect_tx(bar_q, QTILES * C::TILE_BYTES);
+    for (int t = 0; t < QTILES; ++t) tma_load_2d(sQ + t * C::TILE_BYTES, &tm_q, col0, row0 + q0 + t * 64, bar_q);
+    for (int j = 0; j < KV_STAGES && j < n_kv; ++j) {
+      mbar_expect_tx(&bar_kv[j], 2 * C::TILE_BYTES);
+      tma_load_2d(sK + j * C::TILE_BYTES, &tm_k, col0, row0 + j * BKV, &bar_kv[j]);
+      tma_load_2d(sV + j * C::TILE_BYTES, &tm_v, col0, row0 + j * BKV, &bar_kv[j]);
+    }
   }
 
   const uint32_t aQ = smem_u32(sQ);
   uint32_t qf[C::KSTEPS][4];
   bool ok = mbar_wait(bar_q, 0, abort_flag, p.status);
   if (ok) {
-    const int r = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+    const uint32_t aQw = aQ + static_cast<uint32_t>((warp >> 2) * C::TILE_BYTES);  // 64-row tile of this warp
+    const int r = (warp & 3) * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
 #pragma unroll
     for (int ks = 0; ks < C::KSTEPS; ++ks) {
       if (C::HALF_TAIL && ks == C::KSTEPS - 1) {
-        ldsm_x2(qf[ks][0], qf[ks][1], tile_addr<DH>(aQ, r, ks * 16));
+        ldsm_x2(qf[ks][0], qf[ks][1], tile_addr<DH>(aQw, r, ks * 16));
         qf[ks][2] = 0u;
         qf[ks][3] = 0u;
       } else {
-        ldsm_x4(qf[ks], tile_addr<DH>(aQ, r, ks * 16 + (lane >> 4) * 8));
+        ldsm_x4(qf[ks], tile_addr<DH>(aQw, r, ks * 16 + (lane >> 4) * 8));
       }
     }
   }
@@ -126,15 +129,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.0f, 0.0f};
 
   for (int j = 0; j < n_kv && ok; ++j) {
-    const int st = j & 1;
-    if (threadIdx.x == 0 && j + 1 < n_kv) {
-      // stage (j+1)&1 was last read in iteration j-1; every thread has passed that iteration's barrier
-      const int ns = (j + 1) & 1;
-      mbar_expect_tx(&bar_kv[ns], 2 * C::TILE_BYTES);
-      tma_load_2d(sK + ns * C::TILE_BYTES, &tm_k, col0, row0 + (j + 1) * BKV, &bar_kv[ns]);
-      tma_load_2d(sV + ns * C::TILE_BYTES, &tm_v, col0, row0 + (j + 1) * BKV, &bar_kv[ns]);
-    }
-    if (!mbar_wait(&bar_kv[st], static_cast<uint32_t>(j >> 1) & 1u, abort_flag, p.status)) {
+    const int st = j % KV_STAGES;
+    if (!mbar_wait(&bar_kv[st], static_cast<uint32_t>(j / KV_STAGES) & 1u, abort_flag, p.status)) {
       ok = false;
       break;
     }
@@ -219,7 +215,14 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         mma_bf16(o[C::NT_O - 1], a0, a1, a2, a3, b0, b1);
       }
     }
-    __syncthreads();  // everyone is done with stage st before it is refilled
+    if (j + KV_STAGES < n_kv) {
+      __syncthreads();  // everyone is done with stage st before it is refilled
+      if (threadIdx.x == 0) {
+        mbar_expect_tx(&bar_kv[st], 2 * C::TILE_BYTES);
+        tma_load_2d(sK + st * C::TILE_BYTES, &tm_k, col0, row0 + (j + KV_STAGES) * BKV, &bar_kv[st]);
+        tma_load_2d(sV + st * C::TILE_BYTES, &tm_v, col0, row0 + (j + KV_STAGES) * BKV, &bar_kv[st]);
+      }
+    }
   }
   if (!ok) return;
 
@@ -247,8 +250,11 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       if (p.out_dtype == QDIT_I8) {
         const int c0 = __float2int_rn(quantize_code(v0, q_inv, p.qa.zp, p.qa.qmin, p.qa.qmax));
         const int c1 = __float2int_rn(quantize_code(v1, q_inv, p.qa.zp, p.qa.qmin, p.qa.qmax));
-        *reinterpret_cast<uint16_t*>(static_cast<uint8_t*>(p.out) + off) =
-            static_cast<uint16_t>((c0 & 0xFF) | ((c1 & 0xFF) << 8));
+        // the 4 lanes of a quad hold 8 consecutive columns of this row: gather them into one 8-byte store
+        uint32_t w = static_cast<uint32_t>((c0 & 0xFF) | ((c1 & 0xFF) << 8));
+        w |= __shfl_down_sync(0xffffffffu, w, 1) << 16;            // lanes t = 0, 2: columns 2t .. 2t + 3
+        const uint32_t w_hi = __shfl_down_sync(0xffffffffu, w, 2);  // lane t = 0 receives lane 2's word
+        if (t == 0) *reinterpret_cast<uint2*>(static_cast<uint8_t*>(p.out) + off) = make_uint2(w, w_hi);
       } else if (p.out_dtype == QDIT_BF16) {
         *reinterpret_cast<uint32_t*>(static_cast<__nv_bfloat16*>(p.out) + off) = pack_bf16x2(v0, v1);
       } else {
@@ -258,13 +264,13 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   }
 }
 
-template <int DH>
+template <int DH, int QW>
 int32_t launch_attention(qdit_ctx* ctx, const void* q, const void* k, const void* v, int64_t ld, int B, int H, int T,
                          const AttnParams& p) {
   using C = ACfg<DH>;
   static bool attr_set[64] = {};
   if (!attr_set[ctx->device & 63]) {
-    QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(attention_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+    QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(attention_kernel<DH, QW>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::smem_bytes(QW)));
     attr_set[ctx->device & 63] = true;
   }
   const uint64_t rows = static_cast<uint64_t>(B) * T, cols = static_cast<uint64_t>(H) * DH;
@@ -272,9 +278,9 @@ int32_t launch_attention(qdit_ctx* ctx, const void* q, const void* k, const void
   QDIT_TRY(qdit_get_tmap(ctx, q, rows, cols, ld, 64, DH, C::SWZ ? 1 : 0, 2, &tq));
   QDIT_TRY(qdit_get_tmap(ctx, k, rows, cols, ld, 64, DH, C::SWZ ? 1 : 0, 2, &tk));
   QDIT_TRY(qdit_get_tmap(ctx, v, rows, cols, ld, 64, DH, C::SWZ ? 1 : 0, 2, &tv));
-  dim3 grid(T / BQ, H, B);
+  dim3 grid(T / (QW * 16), H, B);
   ProfScope prof(ctx, QDIT_PROF_ATTENTION, 4.0 * B * H * static_cast<double>(T) * T * DH);
-  attention_kernel<DH><<<grid, ATT_THREADS, C::SMEM_BYTES, ctx->stream>>>(tq, tk, tv, p);
+  attention_kernel<DH, QW><<<grid, QW * 32, C::smem_bytes(QW), ctx->stream>>>(tq, tk, tv, p);
   return qdit_after_launch(ctx, "attention_kernel");
 }
 
@@ -305,6 +311,7 @@ extern "C" int32_t qdit_attention(qdit_ctx* ctx, const void* q, const void* k, c
     QDIT_TRY(qdit_check_qparams(ctx, out_qp, out_scale_dev != nullptr));
     p.qa = make_quant_args(*out_qp, out_scale_dev);
   }
-  if (dh == 64) return launch_attention<64>(ctx, q, k, v, ld, B, H, T, p);
-  return launch_attention<72>(ctx, q, k, v, ld, B, H, T, p);
+  const bool wide = T % 128 == 0;  // 128 queries per CTA when the token count allows
+  if (dh == 64) return wide ? launch_attention<64, 8>(ctx, q, k, v, ld, B, H, T, p) : launch_attention<64, 4>(ctx, q, k, v, ld, B, H, T, p);
+  return wide ? launch_attention<72, 8>(ctx, q, k, v, ld, B, H, T, p) : launch_attention<72, 4>(ctx, q, k, v, ld, B, H, T, p);
 }

@@ -25,13 +25,9 @@ __global__ void __launch_bounds__(256) act_quant_kernel(const T* __restrict__ x,
   float a[8], b[8];
   Load8<T>::load(src, a);
   if (second) Load8<T>::load(src + 8, b);
-#pragma unroll
-  for (int i = 0; i < 8; ++i) a[i] = quantize_code(a[i], inv, qa.zp, qa.qmin, qa.qmax);
-  const uint2 lo = pack_codes8(a);
+  const uint2 lo = quantize_pack8(a, inv, qa.zp, qa.qmin, qa.qmax);
   if (second) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) b[i] = quantize_code(b[i], inv, qa.zp, qa.qmin, qa.qmax);
-    const uint2 hi = pack_codes8(b);
+    const uint2 hi = quantize_pack8(b, inv, qa.zp, qa.qmin, qa.qmax);
     if ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
       *reinterpret_cast<uint4*>(dst) = make_uint4(lo.x, lo.y, hi.x, hi.y);
     } else {
@@ -136,7 +132,7 @@ __global__ void __launch_bounds__(256) weight_quant_kernel(const float* __restri
 // while every warp's row is already in flight, so the modulation parameters cost one pass over L2 per CTA
 // instead of one per row and no dependent round trip after the statistics.
 template <int NV>
-__global__ void __launch_bounds__(256, 4) ln_modulate_kernel(const __nv_bfloat16* __restrict__ x, int64_t M, int D,
+__global__ void __launch_bounds__(256) ln_modulate_kernel(const __nv_bfloat16* __restrict__ x, int64_t M, int D,
                                                           int64_t T, float eps, const float* __restrict__ shift,
                                                           const float* __restrict__ scale, int64_t ld_mod,
                                                           void* __restrict__ out, int out_dtype, QuantArgs qa) {
@@ -210,9 +206,7 @@ __global__ void __launch_bounds__(256, 4) ln_modulate_kernel(const __nv_bfloat16
       for (int i = 0; i < 8; ++i) y[i] = (v[j][i] - mean) * rstd * (1.0f + scv[i]) + shv[i];
       const int64_t o = row * D + vi * 8;
       if (out_dtype == QDIT_I8) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) y[i] = quantize_code(y[i], inv, qa.zp, qa.qmin, qa.qmax);
-        *reinterpret_cast<uint2*>(static_cast<uint8_t*>(out) + o) = pack_codes8(y);
+        *reinterpret_cast<uint2*>(static_cast<uint8_t*>(out) + o) = quantize_pack8(y, inv, qa.zp, qa.qmin, qa.qmax);
       } else if (out_dtype == QDIT_BF16) {
         *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(out) + o) = pack_bf16x8(y);
       } else {
