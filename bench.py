@@ -105,6 +105,31 @@ def workload_inputs(name):
     return cfg, seed, steps, batch, guidance, interval, latent, labels, vc_table
 
 
+def rank_inputs(name, rank, world):
+    """Inputs of one rank: the model (seed) is the same on every rank, the batch is the rank's own
+    (rank 0 of a 1-GPU run gets exactly the workload's seeded batch)."""
+    cfg, seed, steps, batch, guidance, interval, latent, labels, vc_table = workload_inputs(name)
+    if world > 1:
+        latent = synth.normal(seed + rank, "latent", latent.shape)
+        labels = synth.uniform_int(seed + rank, "labels", labels.shape, 0, cfg.num_classes)
+    return cfg, seed, steps, batch, guidance, interval, latent, labels, vc_table
+
+
+def reduce_max_ms(ms, dist, device=None):
+    """Slowest rank's time (the job is done when the last replica is)."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def images_per_second(world, batch, n_traj, ms):
+    """Whole-job throughput: every rank finished n_traj trajectories of `batch` images in `ms`."""
+    return world * batch * n_traj / (ms * 1e-3)
+
+
 # ------------------------------------------------------------------------------------------ CPU oracle leg
 def oracle_sample_rate(name, n_images=1, n_steps=2):
     """Times the oracle on `n_images` images for the first `n_steps` sampling steps (one refresh + one reuse
@@ -192,10 +217,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     import paper_2503_02508_b200 as q
 
-    cfg, seed, steps, batch, guidance, interval, latent, labels, vc_table = workload_inputs(args.workload)
-    if world > 1:  # every rank samples its own batch (different noise, same model)
-        latent = synth.normal(seed + rank, "latent", latent.shape)
-        labels = synth.uniform_int(seed + rank, "labels", labels.shape, 0, cfg.num_classes)
+    cfg, seed, steps, batch, guidance, interval, latent, labels, vc_table = rank_inputs(args.workload, rank, world)
     stream = torch.cuda.Stream()
     ctx = q.qdit_create(local, stream.cuda_stream)
     weights = synth.model_weights(seed, cfg)
@@ -246,12 +268,7 @@ def run_ours(args):
         e1.record(stream)
         q.qdit_sync(ctx)
         barrier()
-        ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return reduce_max_ms(e0.elapsed_time(e1), dist, "cuda")
 
     n_warm = args.warmup if args.short_warmup else max(args.warmup, 3)
     for _ in range(n_warm):
@@ -263,11 +280,11 @@ def run_ours(args):
     ms = timed(trajectory_device, args.steps)
     launches = q.qdit_launch_count(ctx) - l0
     clock_info = clocks.stop()
-    value = world * batch * args.steps / (ms * 1e-3)
+    value = images_per_second(world, batch, args.steps, ms)
 
     trajectory_host()
     ms_e2e = timed(trajectory_host, args.steps)
-    e2e_value = world * batch * args.steps / (ms_e2e * 1e-3)
+    e2e_value = images_per_second(world, batch, args.steps, ms_e2e)
     final = out_h.numpy()
     if not np.isfinite(final).all():
         raise SystemExit("non-finite latent after sampling")
