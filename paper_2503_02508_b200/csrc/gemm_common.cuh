@@ -43,6 +43,20 @@ struct GemmParams {
   int num_m_tiles, num_n_tiles;
 };
 
+// Epilogue classes.  The three block-level layers get kernels whose epilogue flags are compile-time
+// constants (no flag branches, no dead registers, a smaller instruction footprint: instruction-fetch stalls
+// were a top stall reason of the all-in-one kernel); class 0 keeps the flags as run-time values.
+constexpr uint32_t EPI_FLAGS_QKV = QDIT_EPI_BIAS | QDIT_EPI_OUT_BF16;
+constexpr uint32_t EPI_FLAGS_FC1 = QDIT_EPI_BIAS | QDIT_EPI_GELU | QDIT_EPI_QUANT_OUT;
+constexpr uint32_t EPI_FLAGS_GATED = QDIT_EPI_BIAS | QDIT_EPI_GATE | QDIT_EPI_RESIDUAL | QDIT_EPI_CACHE_STORE | QDIT_EPI_OUT_BF16;
+template <int EPI>
+__device__ __forceinline__ uint32_t epi_flags(const GemmParams& p) {
+  return EPI == 1 ? EPI_FLAGS_QKV : EPI == 2 ? EPI_FLAGS_FC1 : EPI == 3 ? EPI_FLAGS_GATED : p.flags;
+}
+inline int epi_class(uint32_t flags) {
+  return flags == EPI_FLAGS_QKV ? 1 : flags == EPI_FLAGS_FC1 ? 2 : flags == EPI_FLAGS_GATED ? 3 : 0;
+}
+
 // Per-column parameters of the 8 columns a lane owns within a chunk.
 struct ColParams {
   float sc[8];  // s_a * s_w[n]
@@ -50,20 +64,24 @@ struct ColParams {
   float gt[8];
 };
 
+template <int EPI>
 __device__ __forceinline__ void load_col_params(const GemmParams& p, int n, int b, float a_scale, ColParams& cp) {
+  const uint32_t flags = epi_flags<EPI>(p);
   float t[8];
   Load8<float>::load(p.w_scale + n, t);
 #pragma unroll
   for (int i = 0; i < 8; ++i) cp.sc[i] = __fmul_rn(a_scale, t[i]);
-  if (p.flags & QDIT_EPI_BIAS) Load8<float>::load(p.bias + n, cp.bi);
-  if (p.flags & QDIT_EPI_GATE) Load8<float>::load(p.gate + static_cast<int64_t>(b) * p.ld_gate + n, cp.gt);
+  if (flags & QDIT_EPI_BIAS) Load8<float>::load(p.bias + n, cp.bi);
+  if (flags & QDIT_EPI_GATE) Load8<float>::load(p.gate + static_cast<int64_t>(b) * p.ld_gate + n, cp.gt);
 }
 
 // Epilogue for 8 consecutive columns of one row; `res` holds the residual's 8 bf16 values (if used).
+template <int EPI>
 __device__ __forceinline__ void epilogue8(const GemmParams& p, const uint4 lo, const uint4 hi, const ColParams& cp,
                                           const uint4 res, int row, int n, float o_inv) {
+  const uint32_t flags = epi_flags<EPI>(p);
   const int64_t o = static_cast<int64_t>(row) * p.ldo + n;
-  if (p.flags & QDIT_EPI_OUT_I32) {
+  if (flags & QDIT_EPI_OUT_I32) {
     int32_t* op = static_cast<int32_t*>(p.out) + o;
     *reinterpret_cast<uint4*>(op) = lo;
     *reinterpret_cast<uint4*>(op + 4) = hi;
@@ -78,7 +96,7 @@ __device__ __forceinline__ void epilogue8(const GemmParams& p, const uint4 lo, c
     acc[4] -= p.a_zp * c1.x; acc[5] -= p.a_zp * c1.y; acc[6] -= p.a_zp * c1.z; acc[7] -= p.a_zp * c1.w;
   }
   float f[8];
-  if (p.flags & QDIT_EPI_GELU) {
+  if (flags & QDIT_EPI_GELU) {
     // the GELU path keeps the conversion unit for exp and reciprocal: convert on the FMA pipe instead
 #pragma unroll
     for (int i = 0; i < 8; ++i) f[i] = int_to_float_rn(acc[i]) * cp.sc[i];
@@ -86,21 +104,21 @@ __device__ __forceinline__ void epilogue8(const GemmParams& p, const uint4 lo, c
 #pragma unroll
     for (int i = 0; i < 8; ++i) f[i] = static_cast<float>(acc[i]) * cp.sc[i];
   }
-  if (p.flags & QDIT_EPI_BIAS) {
+  if (flags & QDIT_EPI_BIAS) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) f[i] += cp.bi[i];
   }
-  if (p.flags & QDIT_EPI_GELU) {
+  if (flags & QDIT_EPI_GELU) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) f[i] = gelu_tanh_f(f[i]);
   }
-  if (p.flags & QDIT_EPI_CACHE_STORE)
+  if (flags & QDIT_EPI_CACHE_STORE)
     *reinterpret_cast<uint4*>(p.cache_out + static_cast<int64_t>(row) * p.N + n) = pack_bf16x8(f);
-  if (p.flags & QDIT_EPI_GATE) {
+  if (flags & QDIT_EPI_GATE) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) f[i] *= cp.gt[i];
   }
-  if (p.flags & QDIT_EPI_RESIDUAL) {
+  if (flags & QDIT_EPI_RESIDUAL) {
     float r[8];
     unpack_bf16x2(res.x, r[0], r[1]);
     unpack_bf16x2(res.y, r[2], r[3]);
@@ -109,7 +127,7 @@ __device__ __forceinline__ void epilogue8(const GemmParams& p, const uint4 lo, c
 #pragma unroll
     for (int i = 0; i < 8; ++i) f[i] += r[i];
   }
-  if (p.flags & QDIT_EPI_QUANT_OUT) {
+  if (flags & QDIT_EPI_QUANT_OUT) {
     // clip(rne(t) + z, qmin, qmax) == rne(clamp(t, qmin - z, qmax - z)) + z because the bounds are integers;
     // adding 1.5 * 2^23 performs the rne and leaves the integer in the low mantissa bits (magic & 0xFF == 0)
     const float lo_f = p.o_qmin - p.o_zp, hi_f = p.o_qmax - p.o_zp;
@@ -124,7 +142,7 @@ __device__ __forceinline__ void epilogue8(const GemmParams& p, const uint4 lo, c
     packed.x = __byte_perm(__byte_perm(m[0], m[1], 0x0040), __byte_perm(m[2], m[3], 0x0040), 0x5410);
     packed.y = __byte_perm(__byte_perm(m[4], m[5], 0x0040), __byte_perm(m[6], m[7], 0x0040), 0x5410);
     *reinterpret_cast<uint2*>(static_cast<uint8_t*>(p.out) + o) = packed;
-  } else if (p.flags & QDIT_EPI_OUT_BF16) {
+  } else if (flags & QDIT_EPI_OUT_BF16) {
     *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + o) = pack_bf16x8(f);
   } else {
     float* of = static_cast<float*>(p.out) + o;
@@ -140,11 +158,13 @@ struct ChunkInputs {
   uint4 res[4];
 };
 
+template <int EPI>
 __device__ __forceinline__ void prefetch_chunk(const GemmParams& p, int n, int row_base, int rsub, float a_scale,
                                                ChunkInputs& in) {
-  if (n < p.N && !(p.flags & QDIT_EPI_OUT_I32)) {
-    load_col_params(p, n, row_base / p.tokens, a_scale, in.cp);
-    if (p.flags & QDIT_EPI_RESIDUAL) {
+  const uint32_t flags = epi_flags<EPI>(p);
+  if (n < p.N && !(flags & QDIT_EPI_OUT_I32)) {
+    load_col_params<EPI>(p, n, row_base / p.tokens, a_scale, in.cp);
+    if (flags & QDIT_EPI_RESIDUAL) {
 #pragma unroll
       for (int sidx = 0; sidx < 4; ++sidx) {
         const int row = row_base + sidx * 8 + rsub;
@@ -159,11 +179,12 @@ __device__ __forceinline__ void prefetch_chunk(const GemmParams& p, int n, int r
 // stage back to the MMA issuer once this warp has read its share.  `stg` = this warp's 4 KB staging patch.
 // The epilogue is bound by the latency chain of one chunk (global loads, TMEM load, transpose, stores), so
 // the tile's chunks are spread over as many warps as the register file allows.
-template <int BN, typename Release>
+template <int BN, int EPI, typename Release>
 __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t tacc, int m0, int n0, int quad, int half,
                                               uint32_t stg, int lane, float a_scale, float o_inv, Release release) {
   const int cg = lane & 3;     // after the transpose: column group (8 columns) ...
   const int rsub = lane >> 2;  // ... of rows rsub, rsub + 8, rsub + 16, rsub + 24
+  const uint32_t flags = epi_flags<EPI>(p);
   const bool gate_uniform = (p.tokens % 32) == 0;  // the warp's 32 rows then belong to one sample
   constexpr int CHUNKS = BN / 32;
   // this warp takes chunks half, half + EPI_SPLIT, ...; c_last = the last of them (-1: none)
@@ -184,7 +205,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t tacc
     const bool col_ok = n < p.N;
     const uint32_t patch = stg;
     ChunkInputs cur;
-    prefetch_chunk(p, n, row_base, rsub, a_scale, cur);
+    prefetch_chunk<EPI>(p, n, row_base, rsub, a_scale, cur);
     uint32_t v[32];
     __syncwarp();
     tmem_ld_32x32(taddr + static_cast<uint32_t>(c * 32), v);
@@ -212,9 +233,9 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t tacc
       asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(lo.x), "=r"(lo.y), "=r"(lo.z), "=r"(lo.w) : "r"(a_lo));
       asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(hi.x), "=r"(hi.y), "=r"(hi.z), "=r"(hi.w) : "r"(a_hi));
       if (row < p.M && col_ok) {
-        if (!gate_uniform && (p.flags & QDIT_EPI_GATE))
+        if (!gate_uniform && (flags & QDIT_EPI_GATE))
           Load8<float>::load(p.gate + static_cast<int64_t>(row / p.tokens) * p.ld_gate + n, cur.cp.gt);
-        epilogue8(p, lo, hi, cur.cp, cur.res[sidx], row, n, o_inv);
+        epilogue8<EPI>(p, lo, hi, cur.cp, cur.res[sidx], row, n, o_inv);
       }
     }
   }

@@ -32,7 +32,7 @@ struct Cfg {
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + BAR_BYTES + 1024;  // + alignment slack
 };
 
-template <int BN>
+template <int BN, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                const GemmParams p, const uint32_t idesc) {
@@ -139,7 +139,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     const uint32_t stg = smem_u32(staging + e * (32 * 128));  // [32 rows][8 x 16 B], 16-byte index XOR (row & 7)
     const float a_scale = p.a_scale_dev ? __ldg(p.a_scale_dev) : p.a_scale;
     float o_inv = 0.0f;
-    if (p.flags & QDIT_EPI_QUANT_OUT) o_inv = __fdiv_rn(1.0f, p.o_scale_dev ? __ldg(p.o_scale_dev) : p.o_scale);
+    if (epi_flags<EPI>(p) & QDIT_EPI_QUANT_OUT) o_inv = __fdiv_rn(1.0f, p.o_scale_dev ? __ldg(p.o_scale_dev) : p.o_scale);
     int it = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
       const int as = it & 1;
@@ -150,7 +150,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       __syncwarp();
       tc_fence_after();
       uint64_t* release_bar = &tempty_bar[as];
-      epilogue_tile<BN>(p, tmem_base + static_cast<uint32_t>(as * BN), m0, n0, quad, half, stg, lane, a_scale, o_inv,
+      epilogue_tile<BN, EPI>(p, tmem_base + static_cast<uint32_t>(as * BN), m0, n0, quad, half, stg, lane, a_scale, o_inv,
                         [release_bar]() { mbar_arrive_relaxed(release_bar); });
     }
   }
@@ -163,12 +163,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   }
 }
 
-template <int BN>
-int32_t launch_gemm(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p, bool a_unsigned) {
+template <int BN, int EPI>
+int32_t launch_gemm_epi(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p, bool a_unsigned) {
   using C = Cfg<BN>;
   static bool attr_set[64] = {};
   if (!attr_set[ctx->device & 63]) {
-    QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(gemm_i8_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+    QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(gemm_i8_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
     attr_set[ctx->device & 63] = true;
   }
   CUtensorMap ta, tw;
@@ -180,8 +180,19 @@ int32_t launch_gemm(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p, 
   const int grid = total < ctx->num_sms ? total : ctx->num_sms;
   const uint32_t idesc = umma_idesc_i8(BM, BN, a_unsigned);
   ProfScope prof(ctx, QDIT_PROF_GEMM, 2.0 * p.M * static_cast<double>(p.N) * p.K);
-  gemm_i8_kernel<BN><<<grid, NUM_THREADS, C::SMEM_BYTES, ctx->stream>>>(ta, tw, p, idesc);
+  gemm_i8_kernel<BN, EPI><<<grid, NUM_THREADS, C::SMEM_BYTES, ctx->stream>>>(ta, tw, p, idesc);
   return qdit_after_launch(ctx, "gemm_i8_kernel");
+}
+
+template <int BN>
+int32_t launch_gemm(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p, bool a_unsigned) {
+  const int cls = getenv("QDIT_GEMM_GENERIC_EPILOGUE") ? 0 : epi_class(p.flags);  // tuning switch
+  switch (cls) {
+    case 1: return launch_gemm_epi<BN, 1>(ctx, A, W, p, a_unsigned);
+    case 2: return launch_gemm_epi<BN, 2>(ctx, A, W, p, a_unsigned);
+    case 3: return launch_gemm_epi<BN, 3>(ctx, A, W, p, a_unsigned);
+    default: return launch_gemm_epi<BN, 0>(ctx, A, W, p, a_unsigned);
+  }
 }
 
 // Tile width: prefer 192 (divides every DiT-XL/2 layer width); fall back to narrower tiles when that

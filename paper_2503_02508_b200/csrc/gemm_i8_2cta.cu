@@ -155,7 +155,7 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       __syncwarp();
       tc_fence_after();
       const uint32_t leader_tempty = mapa_shared(smem_u32(&tempty_bar[as]), 0);
-      epilogue_tile<BN>(p, tmem_base + static_cast<uint32_t>(as * BN), m0, n0, quad, half, stg, lane, a_scale, o_inv,
+      epilogue_tile<BN, 0>(p, tmem_base + static_cast<uint32_t>(as * BN), m0, n0, quad, half, stg, lane, a_scale, o_inv,
                         [leader_tempty]() { mbar_arrive_cluster_relaxed(leader_tempty); });
     }
   }
