@@ -313,7 +313,8 @@ def run_ours(args):
             rate = w / (t * 1e-3)
             breakdown[name] = {"launches": n, "ms": round(t, 3),
                                "rate": round(rate / 1e12, 2) if k < 2 else round(rate / 1e9, 1),
-                               "unit": "TOP/s" if k == 0 else "TFLOP/s" if k == 1 else "GB/s"}
+                               "unit": "TOP/s" if k == 0 else "TFLOP/s" if k == 1 else "GB/s",
+                               "avg_us": round(1e3 * t / n, 2)}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -126,25 +126,27 @@ __global__ void __launch_bounds__(256) cfg_ddim_kernel(float* __restrict__ laten
 
 // ----------------------------------------------------------------------------- patch embedding
 // x[m,:] = bf16(W_patch . patch(m) + b_patch + pos[t,:]); patch vector ordered (c, py, px).
-// CTA = 32 token rows x 512 columns; a thread keeps the weights of its two columns in registers and walks
-// the rows, so weights are read once per CTA and the bf16 stores of a warp are 128 contiguous bytes.
+// CTA = 32 token rows x 512 columns.  The weights come TRANSPOSED (wT[j][d], made once when the model is
+// built), so a thread reads the PD weights of its two columns with coalesced 8-byte loads and keeps them
+// in registers while it walks the rows; patch values are broadcast from shared memory; the bf16 stores of
+// a warp are 128 contiguous bytes.
 constexpr int EMB_ROWS = 32;
-constexpr int EMB_MAX_PD = 64;  // patch vector length limit (C * p * p)
+template <int PD>
 __global__ void __launch_bounds__(256) embed_kernel(const float* __restrict__ latent, int latent_batch,
-                                                    const float* __restrict__ w, const float* __restrict__ bias,
+                                                    const float* __restrict__ wT, const float* __restrict__ bias,
                                                     const float* __restrict__ pos, __nv_bfloat16* __restrict__ x,
                                                     int64_t M, int D, int grid, int patch, int C) {
-  __shared__ float sp[EMB_ROWS][EMB_MAX_PD];
-  const int T = grid * grid, side = grid * patch, pd = C * patch * patch;
+  __shared__ float sp[EMB_ROWS][PD];
+  const int T = grid * grid, side = grid * patch, pp = patch * patch;
   const int64_t m0 = static_cast<int64_t>(blockIdx.x) * EMB_ROWS;
-  for (int i = threadIdx.x; i < EMB_ROWS * pd; i += blockDim.x) {
-    const int r = i / pd, j = i % pd;
+  for (int i = threadIdx.x; i < EMB_ROWS * PD; i += blockDim.x) {
+    const int r = i / PD, j = i % PD;
     const int64_t m = m0 + r;
     float v = 0.0f;
     if (m < M) {
       const int b = static_cast<int>(m / T) % latent_batch, t = static_cast<int>(m % T);
       const int gy = t / grid, gx = t % grid;
-      const int c = j / (patch * patch), py = (j / patch) % patch, px = j % patch;
+      const int c = j / pp, py = (j / patch) % patch, px = j % patch;
       v = latent[((static_cast<int64_t>(b) * C + c) * side + gy * patch + py) * side + gx * patch + px];
     }
     sp[r][j] = v;
@@ -152,28 +154,23 @@ __global__ void __launch_bounds__(256) embed_kernel(const float* __restrict__ la
   __syncthreads();
   const int d = (blockIdx.y * blockDim.x + threadIdx.x) * 2;
   if (d >= D) return;
-  float w0[EMB_MAX_PD], w1[EMB_MAX_PD];
+  float2 w[PD];
 #pragma unroll
-  for (int j = 0; j < EMB_MAX_PD; ++j) {
-    if (j < pd) {
-      w0[j] = w[static_cast<int64_t>(d) * pd + j];
-      w1[j] = w[static_cast<int64_t>(d + 1) * pd + j];
-    }
-  }
-  const float b0 = bias[d], b1 = bias[d + 1];
-  for (int r = 0; r < EMB_ROWS; ++r) {
-    const int64_t m = m0 + r;
-    if (m >= M) break;
-    float a0 = 0.0f, a1 = 0.0f;
+  for (int j = 0; j < PD; ++j) w[j] = *reinterpret_cast<const float2*>(wT + static_cast<int64_t>(j) * D + d);
+  const float2 bv = *reinterpret_cast<const float2*>(bias + d);
+  int t = static_cast<int>(m0 % T);
+  const int rows = M - m0 < EMB_ROWS ? static_cast<int>(M - m0) : EMB_ROWS;
+  for (int r = 0; r < rows; ++r) {
+    float a0 = bv.x, a1 = bv.y;
 #pragma unroll
-    for (int j = 0; j < EMB_MAX_PD; ++j) {
-      if (j < pd) {
-        a0 = fmaf(w0[j], sp[r][j], a0);
-        a1 = fmaf(w1[j], sp[r][j], a1);
-      }
+    for (int j = 0; j < PD; ++j) {
+      const float pv = sp[r][j];
+      a0 = fmaf(w[j].x, pv, a0);
+      a1 = fmaf(w[j].y, pv, a1);
     }
-    const float2 pv = *reinterpret_cast<const float2*>(pos + static_cast<int64_t>(m % T) * D + d);
-    *reinterpret_cast<uint32_t*>(x + m * D + d) = pack_bf16x2(a0 + b0 + pv.x, a1 + b1 + pv.y);
+    const float2 ps = *reinterpret_cast<const float2*>(pos + static_cast<int64_t>(t) * D + d);
+    *reinterpret_cast<uint32_t*>(x + (m0 + r) * D + d) = pack_bf16x2(a0 + ps.x, a1 + ps.y);
+    if (++t == T) t = 0;
   }
 }
 
@@ -190,59 +187,59 @@ __global__ void timestep_features_kernel(const float* __restrict__ t, float* __r
 }
 
 // out[b,n] = W[n,:] . f(in[b,:]) + bias[n] (+ table[y[b],n]), optionally passed through SiLU, and optionally
-// SiLU(out) as a second output.  The inputs of up to `bc` samples sit in shared memory; a warp owns one
-// output feature, keeps its weight row in registers and walks the samples.
+// SiLU(out) as a second output.  A warp owns one output feature for SL_BG consecutive samples: its weight
+// row sits in registers, the samples' inputs stream through L1/L2 with independent 16-byte loads.
 constexpr int SL_MAXV = 16;  // float4 per lane: K <= 2048
+constexpr int SL_BG = 4;     // samples per warp
 __global__ void __launch_bounds__(256) small_linear_kernel(const float* __restrict__ in, const float* __restrict__ w,
                                                            const float* __restrict__ bias,
                                                            const float* __restrict__ table, const int32_t* __restrict__ y,
                                                            float* __restrict__ out, float* __restrict__ out_silu, int B,
-                                                           int N, int K, int bc, int silu_input, int silu_output) {
-  extern __shared__ float s_in[];  // [bc][K]
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n = blockIdx.x * (blockDim.x >> 5) + warp;
+                                                           int N, int K, int silu_input, int silu_output) {
+  const int lane = threadIdx.x & 31;
+  const int gw = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int groups = (B + SL_BG - 1) / SL_BG;
+  if (gw >= N * groups) return;
+  const int n = gw / groups, b0 = (gw % groups) * SL_BG;
   float4 wv[SL_MAXV];
-  if (n < N) {
+#pragma unroll
+  for (int j = 0; j < SL_MAXV; ++j) {
+    const int k = lane * 4 + 128 * j;
+    wv[j] = k < K ? *reinterpret_cast<const float4*>(w + static_cast<int64_t>(n) * K + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  float acc[SL_BG];
+#pragma unroll
+  for (int g = 0; g < SL_BG; ++g) {
+    acc[g] = 0.0f;
+    const int b = b0 + g < B ? b0 + g : B - 1;  // clamp: the duplicate is not written
 #pragma unroll
     for (int j = 0; j < SL_MAXV; ++j) {
       const int k = lane * 4 + 128 * j;
-      wv[j] = k < K ? *reinterpret_cast<const float4*>(w + static_cast<int64_t>(n) * K + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+      if (k < K) {
+        float4 xv = *reinterpret_cast<const float4*>(in + static_cast<int64_t>(b) * K + k);
+        if (silu_input) {
+          xv.x = silu_f(xv.x); xv.y = silu_f(xv.y); xv.z = silu_f(xv.z); xv.w = silu_f(xv.w);
+        }
+        acc[g] = fmaf(wv[j].x, xv.x, acc[g]);
+        acc[g] = fmaf(wv[j].y, xv.y, acc[g]);
+        acc[g] = fmaf(wv[j].z, xv.z, acc[g]);
+        acc[g] = fmaf(wv[j].w, xv.w, acc[g]);
+      }
     }
   }
-  for (int b0 = 0; b0 < B; b0 += bc) {
-    const int nb = B - b0 < bc ? B - b0 : bc;
-    __syncthreads();
-    for (int i = threadIdx.x * 4; i < nb * K; i += blockDim.x * 4) {
-      float4 v = *reinterpret_cast<const float4*>(in + static_cast<int64_t>(b0) * K + i);
-      if (silu_input) {
-        v.x = silu_f(v.x); v.y = silu_f(v.y); v.z = silu_f(v.z); v.w = silu_f(v.w);
-      }
-      *reinterpret_cast<float4*>(s_in + i) = v;
-    }
-    __syncthreads();
-    if (n < N) {
-      for (int b = 0; b < nb; ++b) {
-        float acc = 0.0f;
 #pragma unroll
-        for (int j = 0; j < SL_MAXV; ++j) {
-          const int k = lane * 4 + 128 * j;
-          if (k < K) {
-            const float4 xv = *reinterpret_cast<const float4*>(s_in + b * K + k);
-            acc = fmaf(wv[j].x, xv.x, acc);
-            acc = fmaf(wv[j].y, xv.y, acc);
-            acc = fmaf(wv[j].z, xv.z, acc);
-            acc = fmaf(wv[j].w, xv.w, acc);
-          }
-        }
-        acc = warp_sum(acc);
-        if (lane == 0) {
-          const int64_t o = static_cast<int64_t>(b0 + b) * N + n;
-          float v = acc + bias[n];
-          if (table) v += table[static_cast<int64_t>(y[b0 + b]) * N + n];
-          if (silu_output) v = silu_f(v);
-          out[o] = v;
-          if (out_silu) out_silu[o] = silu_f(v);
-        }
+  for (int g = 0; g < SL_BG; ++g) acc[g] = warp_sum(acc[g]);
+  if (lane == 0) {
+#pragma unroll
+    for (int g = 0; g < SL_BG; ++g) {
+      const int b = b0 + g;
+      if (b < B) {
+        const int64_t o = static_cast<int64_t>(b) * N + n;
+        float v = acc[g] + bias[n];
+        if (table) v += table[static_cast<int64_t>(y[b]) * N + n];
+        if (silu_output) v = silu_f(v);
+        out[o] = v;
+        if (out_silu) out_silu[o] = silu_f(v);
       }
     }
   }
@@ -367,12 +364,18 @@ __global__ void __launch_bounds__(256, 1) final_kernel(const __nv_bfloat16* __re
 }  // namespace
 
 // ================================================================================ launchers
-int32_t launch_embed(qdit_ctx* ctx, const float* latent, int latent_batch, const float* w, const float* bias,
+int32_t launch_embed(qdit_ctx* ctx, const float* latent, int latent_batch, const float* wT, const float* bias,
                      const float* pos, void* x, int64_t M, int D, int grid, int patch, int C) {
-  if (C * patch * patch > EMB_MAX_PD) return qdit_fail(ctx, QDIT_ERR_SHAPE, "patch vector longer than %d", EMB_MAX_PD);
+  const int pd = C * patch * patch;
   dim3 g(static_cast<unsigned>((M + EMB_ROWS - 1) / EMB_ROWS), static_cast<unsigned>((D / 2 + 255) / 256));
-  embed_kernel<<<g, 256, 0, ctx->stream>>>(latent, latent_batch, w, bias, pos, static_cast<__nv_bfloat16*>(x), M, D, grid,
-                                           patch, C);
+  __nv_bfloat16* xb = static_cast<__nv_bfloat16*>(x);
+  ProfScope prof(ctx, QDIT_PROF_OTHER, static_cast<double>(M) * D * 2.0);
+  switch (pd) {
+    case 16: embed_kernel<16><<<g, 256, 0, ctx->stream>>>(latent, latent_batch, wT, bias, pos, xb, M, D, grid, patch, C); break;
+    case 4: embed_kernel<4><<<g, 256, 0, ctx->stream>>>(latent, latent_batch, wT, bias, pos, xb, M, D, grid, patch, C); break;
+    case 64: embed_kernel<64><<<g, 256, 0, ctx->stream>>>(latent, latent_batch, wT, bias, pos, xb, M, D, grid, patch, C); break;
+    default: return qdit_fail(ctx, QDIT_ERR_SHAPE, "patch vector length %d not supported (4, 16 or 64)", pd);
+  }
   return qdit_after_launch(ctx, "embed_kernel");
 }
 
@@ -380,18 +383,10 @@ int32_t launch_small_linear(qdit_ctx* ctx, const float* in, const float* w, cons
                             const int32_t* y, float* out, float* out_silu, int B, int N, int K, int silu_input,
                             int silu_output) {
   if (K % 4 != 0 || K > 128 * SL_MAXV) return qdit_fail(ctx, QDIT_ERR_SHAPE, "small linear needs K %% 4 == 0 and K <= %d", 128 * SL_MAXV);
-  const int smem_budget = 160 * 1024;
-  int bc = smem_budget / (K * static_cast<int>(sizeof(float)));
-  if (bc > B) bc = B;
-  if (bc < 1) bc = 1;
-  const size_t smem = static_cast<size_t>(bc) * K * sizeof(float);
-  static bool attr_set[64] = {};
-  if (!attr_set[ctx->device & 63]) {
-    QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(small_linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_budget));
-    attr_set[ctx->device & 63] = true;
-  }
-  small_linear_kernel<<<static_cast<unsigned>((N + 7) / 8), 256, smem, ctx->stream>>>(in, w, bias, table, y, out, out_silu, B, N,
-                                                                                    K, bc, silu_input, silu_output);
+  const int64_t warps = static_cast<int64_t>(N) * ((B + SL_BG - 1) / SL_BG);
+  ProfScope prof(ctx, QDIT_PROF_OTHER, static_cast<double>(N) * K * 4.0);
+  small_linear_kernel<<<static_cast<unsigned>((warps + 7) / 8), 256, 0, ctx->stream>>>(in, w, bias, table, y, out, out_silu, B, N,
+                                                                                     K, silu_input, silu_output);
   return qdit_after_launch(ctx, "small_linear_kernel");
 }
 
@@ -421,6 +416,7 @@ int32_t launch_final(qdit_ctx* ctx, const void* x, int64_t M, int D, int T, floa
     }                                                                                                                   \
     final_kernel<NV><<<g, 256, smem, ctx->stream>>>(xb, M, D, T, eps, modf, w, bias, net, grid, patch);                 \
   } break;
+  ProfScope prof(ctx, QDIT_PROF_OTHER, static_cast<double>(M) * D * 2.0);
   switch (nv) {
     QDIT_FINAL_CASE(1) QDIT_FINAL_CASE(2) QDIT_FINAL_CASE(3) QDIT_FINAL_CASE(4) QDIT_FINAL_CASE(5) QDIT_FINAL_CASE(6)
     default: return qdit_fail(ctx, QDIT_ERR_SHAPE, "final layer supports hidden <= 1536");

@@ -6,8 +6,8 @@ struct DdimCoef {
   float sqrt_ab_t, sqrt_1mab_t, sqrt_ab_prev, sqrt_1mab_prev;
 };
 
-// x[m,:] = bf16(W_patch . patch(m) + b + pos); sample b reads latent[b % latent_batch].
-int32_t launch_embed(qdit_ctx* ctx, const float* latent, int latent_batch, const float* w, const float* bias,
+// x[m,:] = bf16(W_patch . patch(m) + b + pos); sample b reads latent[b % latent_batch]; wT = W_patch transposed [pd][D].
+int32_t launch_embed(qdit_ctx* ctx, const float* latent, int latent_batch, const float* wT, const float* bias,
                      const float* pos, void* x, int64_t M, int D, int grid, int patch, int C);
 // h[b,:] = SiLU(W1 . sinusoid(t_b) + b1); feat is scratch [B, F]
 int32_t launch_cond1(qdit_ctx* ctx, const float* t, const float* w1, const float* b1, float* feat, float* h, int B, int D,

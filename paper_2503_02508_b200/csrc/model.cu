@@ -108,7 +108,15 @@ int32_t build_model(qdit_ctx* ctx, const qdit_model_desc* desc, qdit_model* m) {
   const qdit_model_shape& s = desc->shape;
   const int64_t D = s.hidden, F = s.mlp, T = static_cast<int64_t>(s.grid) * s.grid;
   const int pd = s.channels * s.patch * s.patch, od = 2 * s.channels * s.patch * s.patch;
-  QDIT_TRY(upload(ctx, m->mem, desc->w_patch, D * pd, &m->w_patch));
+  {
+    // the embedding kernel reads the patch weights transposed: [pd][D]
+    if (!desc->w_patch) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "a weight pointer in the model description is NULL");
+    std::vector<float> wt(static_cast<size_t>(D) * pd);
+    for (int64_t d = 0; d < D; ++d)
+      for (int j = 0; j < pd; ++j) wt[static_cast<size_t>(j) * D + d] = desc->w_patch[d * pd + j];
+    QDIT_TRY(upload(ctx, m->mem, wt.data(), D * pd, &m->w_patch));
+    QDIT_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));  // `wt` is a host temporary
+  }
   QDIT_TRY(upload(ctx, m->mem, desc->b_patch, D, &m->b_patch));
   QDIT_TRY(upload(ctx, m->mem, desc->pos, T * D, &m->pos));
   QDIT_TRY(upload(ctx, m->mem, desc->w_t1, D * s.freq_dim, &m->w_t1));
