@@ -187,59 +187,65 @@ __global__ void timestep_features_kernel(const float* __restrict__ t, float* __r
 }
 
 // out[b,n] = W[n,:] . f(in[b,:]) + bias[n] (+ table[y[b],n]), optionally passed through SiLU, and optionally
-// SiLU(out) as a second output.  A warp owns one output feature for SL_BG consecutive samples: its weight
-// row sits in registers, the samples' inputs stream through L1/L2 with independent 16-byte loads.
+// SiLU(out) as a second output.  One CTA per 8 output features: the inputs of up to `bc` samples are copied
+// into shared memory with cp.async (all copies in flight at once: the copy is one L2 latency, not one per
+// loop trip), f is applied in place, then a warp keeps its weight row in registers and walks the samples.
 constexpr int SL_MAXV = 16;  // float4 per lane: K <= 2048
-constexpr int SL_BG = 4;     // samples per warp
 __global__ void __launch_bounds__(256) small_linear_kernel(const float* __restrict__ in, const float* __restrict__ w,
                                                            const float* __restrict__ bias,
                                                            const float* __restrict__ table, const int32_t* __restrict__ y,
                                                            float* __restrict__ out, float* __restrict__ out_silu, int B,
-                                                           int N, int K, int silu_input, int silu_output) {
-  const int lane = threadIdx.x & 31;
-  const int gw = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const int groups = (B + SL_BG - 1) / SL_BG;
-  if (gw >= N * groups) return;
-  const int n = gw / groups, b0 = (gw % groups) * SL_BG;
+                                                           int N, int K, int bc, int silu_input, int silu_output) {
+  extern __shared__ float s_in[];  // [bc][K]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n = blockIdx.x * (blockDim.x >> 5) + warp;
   float4 wv[SL_MAXV];
-#pragma unroll
-  for (int j = 0; j < SL_MAXV; ++j) {
-    const int k = lane * 4 + 128 * j;
-    wv[j] = k < K ? *reinterpret_cast<const float4*>(w + static_cast<int64_t>(n) * K + k) : make_float4(0.f, 0.f, 0.f, 0.f);
-  }
-  float acc[SL_BG];
-#pragma unroll
-  for (int g = 0; g < SL_BG; ++g) {
-    acc[g] = 0.0f;
-    const int b = b0 + g < B ? b0 + g : B - 1;  // clamp: the duplicate is not written
+  if (n < N) {
 #pragma unroll
     for (int j = 0; j < SL_MAXV; ++j) {
       const int k = lane * 4 + 128 * j;
-      if (k < K) {
-        float4 xv = *reinterpret_cast<const float4*>(in + static_cast<int64_t>(b) * K + k);
-        if (silu_input) {
-          xv.x = silu_f(xv.x); xv.y = silu_f(xv.y); xv.z = silu_f(xv.z); xv.w = silu_f(xv.w);
-        }
-        acc[g] = fmaf(wv[j].x, xv.x, acc[g]);
-        acc[g] = fmaf(wv[j].y, xv.y, acc[g]);
-        acc[g] = fmaf(wv[j].z, xv.z, acc[g]);
-        acc[g] = fmaf(wv[j].w, xv.w, acc[g]);
-      }
+      wv[j] = k < K ? *reinterpret_cast<const float4*>(w + static_cast<int64_t>(n) * K + k) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
   }
+  const uint32_t s_base = smem_u32(s_in);
+  for (int b0 = 0; b0 < B; b0 += bc) {
+    const int nb = B - b0 < bc ? B - b0 : bc;
+    __syncthreads();  // the previous group has been consumed
+    for (int i = threadIdx.x * 4; i < nb * K; i += blockDim.x * 4)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s_base + i * 4), "l"(in + static_cast<int64_t>(b0) * K + i) : "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (silu_input) {  // own elements only: no barrier needed before
+      for (int i = threadIdx.x * 4; i < nb * K; i += blockDim.x * 4) {
+        float4 v = *reinterpret_cast<float4*>(s_in + i);
+        v.x = silu_f(v.x); v.y = silu_f(v.y); v.z = silu_f(v.z); v.w = silu_f(v.w);
+        *reinterpret_cast<float4*>(s_in + i) = v;
+      }
+    }
+    __syncthreads();
+    if (n < N) {
+      for (int b = 0; b < nb; ++b) {
+        float acc = 0.0f;
 #pragma unroll
-  for (int g = 0; g < SL_BG; ++g) acc[g] = warp_sum(acc[g]);
-  if (lane == 0) {
-#pragma unroll
-    for (int g = 0; g < SL_BG; ++g) {
-      const int b = b0 + g;
-      if (b < B) {
-        const int64_t o = static_cast<int64_t>(b) * N + n;
-        float v = acc[g] + bias[n];
-        if (table) v += table[static_cast<int64_t>(y[b]) * N + n];
-        if (silu_output) v = silu_f(v);
-        out[o] = v;
-        if (out_silu) out_silu[o] = silu_f(v);
+        for (int j = 0; j < SL_MAXV; ++j) {
+          const int k = lane * 4 + 128 * j;
+          if (k < K) {
+            const float4 xv = *reinterpret_cast<const float4*>(s_in + b * K + k);
+            acc = fmaf(wv[j].x, xv.x, acc);
+            acc = fmaf(wv[j].y, xv.y, acc);
+            acc = fmaf(wv[j].z, xv.z, acc);
+            acc = fmaf(wv[j].w, xv.w, acc);
+          }
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) {
+          const int64_t o = static_cast<int64_t>(b0 + b) * N + n;
+          float v = acc + bias[n];
+          if (table) v += table[static_cast<int64_t>(y[b0 + b]) * N + n];
+          if (silu_output) v = silu_f(v);
+          out[o] = v;
+          if (out_silu) out_silu[o] = silu_f(v);
+        }
       }
     }
   }
@@ -383,10 +389,20 @@ int32_t launch_small_linear(qdit_ctx* ctx, const float* in, const float* w, cons
                             const int32_t* y, float* out, float* out_silu, int B, int N, int K, int silu_input,
                             int silu_output) {
   if (K % 4 != 0 || K > 128 * SL_MAXV) return qdit_fail(ctx, QDIT_ERR_SHAPE, "small linear needs K %% 4 == 0 and K <= %d", 128 * SL_MAXV);
-  const int64_t warps = static_cast<int64_t>(N) * ((B + SL_BG - 1) / SL_BG);
+  if (!aligned16(in) || !aligned16(w)) return qdit_fail(ctx, QDIT_ERR_ALIGN, "small linear operands must be 16-byte aligned");
+  const int smem_budget = 160 * 1024;
+  int bc = smem_budget / (K * static_cast<int>(sizeof(float)));
+  if (bc > B) bc = B;
+  if (bc < 1) bc = 1;
+  const size_t smem = static_cast<size_t>(bc) * K * sizeof(float);
+  static bool attr_set[64] = {};
+  if (!attr_set[ctx->device & 63]) {
+    QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(small_linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_budget));
+    attr_set[ctx->device & 63] = true;
+  }
   ProfScope prof(ctx, QDIT_PROF_OTHER, static_cast<double>(N) * K * 4.0);
-  small_linear_kernel<<<static_cast<unsigned>((warps + 7) / 8), 256, 0, ctx->stream>>>(in, w, bias, table, y, out, out_silu, B, N,
-                                                                                     K, silu_input, silu_output);
+  small_linear_kernel<<<static_cast<unsigned>((N + 7) / 8), 256, smem, ctx->stream>>>(in, w, bias, table, y, out, out_silu, B, N,
+                                                                                    K, bc, silu_input, silu_output);
   return qdit_after_launch(ctx, "small_linear_kernel");
 }
 
