@@ -126,105 +126,123 @@ __global__ void __launch_bounds__(256) weight_quant_kernel(const float* __restri
 }
 
 // ----------------------------------------------------------------------------- LayerNorm + modulate (+ quantize)
-// One warp per row, 8 rows per CTA; the row lives in registers (NV vectors of 8 per lane), statistics are
-// two-pass in f32.  The CTA first copies shift and scale of its first row's sample into shared memory
-// (all its rows share them when T is a multiple of 8; a row of another sample falls back to global reads),
-// while every warp's row is already in flight, so the modulation parameters cost one pass over L2 per CTA
-// instead of one per row and no dependent round trip after the statistics.
+// A CTA owns a contiguous range of rows; its 8 warps take the rows in turn, one warp per row, the row in
+// registers (NV vectors of 8 per lane), statistics two-pass in f32.  While a warp works on one row the next
+// row's loads are already in flight.  Shift and scale of the (at most two) samples the range touches are
+// copied to shared memory once per CTA; a row of any other sample falls back to global reads.
+template <int NV>
+__device__ __forceinline__ void ln_load_row(const __nv_bfloat16* __restrict__ xr, int nvec, int lane, uint4 (&raw)[NV]) {
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    const int vi = lane + 32 * j;
+    if (vi < nvec) raw[j] = *reinterpret_cast<const uint4*>(xr + vi * 8);
+  }
+}
+
 template <int NV>
 __global__ void __launch_bounds__(256) ln_modulate_kernel(const __nv_bfloat16* __restrict__ x, int64_t M, int D,
                                                           int64_t T, float eps, const float* __restrict__ shift,
                                                           const float* __restrict__ scale, int64_t ld_mod,
-                                                          void* __restrict__ out, int out_dtype, QuantArgs qa) {
-  extern __shared__ float s_mod[];  // [2][D]: shift, scale of sample b0
-  const int lane = threadIdx.x & 31;
-  const int64_t row0 = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5);
-  const int64_t row = row0 + (threadIdx.x >> 5);
-  const bool active = row < M;
+                                                          void* __restrict__ out, int out_dtype, QuantArgs qa,
+                                                          int rows_per_cta) {
+  extern __shared__ float s_mod[];  // [2 samples][2][D]: shift, scale
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  const int64_t row_begin = static_cast<int64_t>(blockIdx.x) * rows_per_cta;
+  const int64_t row_end = row_begin + rows_per_cta < M ? row_begin + rows_per_cta : M;
+  if (row_begin >= M) return;
   const int nvec = D >> 3;
-  float v[NV][8];
-  if (active) {
-    const __nv_bfloat16* xr = x + row * D;
-#pragma unroll
-    for (int j = 0; j < NV; ++j) {
-      const int vi = lane + 32 * j;
-      if (vi < nvec) Load8<__nv_bfloat16>::load(xr + vi * 8, v[j]);
-    }
-  }
-  const int64_t b0 = row0 / T;
-  {
-    const float4* gs = reinterpret_cast<const float4*>(shift + b0 * ld_mod);
-    const float4* gc = reinterpret_cast<const float4*>(scale + b0 * ld_mod);
-    float4* ss = reinterpret_cast<float4*>(s_mod);
-    float4* sc4 = reinterpret_cast<float4*>(s_mod + D);
+  int64_t row = row_begin + warp;
+  uint4 raw[NV], raw_next[NV];
+  if (row < row_end) ln_load_row<NV>(x + row * D, nvec, lane, raw);
+  const int64_t b0 = row_begin / T;
+  for (int s = 0; s < 2; ++s) {
+    if ((b0 + s) * T >= row_end && s > 0) break;
+    const float4* gs = reinterpret_cast<const float4*>(shift + (b0 + s) * ld_mod);
+    const float4* gc = reinterpret_cast<const float4*>(scale + (b0 + s) * ld_mod);
+    float4* ss = reinterpret_cast<float4*>(s_mod + s * 2 * D);
+    float4* sc4 = reinterpret_cast<float4*>(s_mod + s * 2 * D + D);
     for (int i = threadIdx.x; i < D / 4; i += blockDim.x) {
       ss[i] = gs[i];
       sc4[i] = gc[i];
     }
   }
   __syncthreads();
-  if (!active) return;
-  float sum = 0.0f;
-#pragma unroll
-  for (int j = 0; j < NV; ++j) {
-    if (lane + 32 * j < nvec) {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) sum += v[j][i];
-    }
-  }
-  const float mean = warp_sum(sum) / static_cast<float>(D);
-  float ssq = 0.0f;
-#pragma unroll
-  for (int j = 0; j < NV; ++j) {
-    if (lane + 32 * j < nvec) {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const float d = v[j][i] - mean;
-        ssq += d * d;
-      }
-    }
-  }
-  const float var = warp_sum(ssq) / static_cast<float>(D);
-  const float rstd = 1.0f / sqrtf(var + eps);
-  const int64_t b = row / T;
-  const bool staged = b == b0;
-  const float* sh = staged ? s_mod : shift + b * ld_mod;
-  const float* sc = staged ? s_mod + D : scale + b * ld_mod;
   float inv = 0.0f;
   if (out_dtype == QDIT_I8) {
     const float s = qa.scale_dev ? __ldg(qa.scale_dev) : qa.scale;
     inv = __fdiv_rn(1.0f, s);
   }
+  for (; row < row_end; row += nwarps) {
+    const int64_t next = row + nwarps;
+    if (next < row_end) ln_load_row<NV>(x + next * D, nvec, lane, raw_next);
+    float v[NV][8];
+    float sum = 0.0f;
 #pragma unroll
-  for (int j = 0; j < NV; ++j) {
-    const int vi = lane + 32 * j;
-    if (vi < nvec) {
-      float shv[8], scv[8], y[8];
-      Load8<float>::load(sh + vi * 8, shv);
-      Load8<float>::load(sc + vi * 8, scv);
+    for (int j = 0; j < NV; ++j) {
+      if (lane + 32 * j < nvec) {
+        unpack_bf16x2(raw[j].x, v[j][0], v[j][1]);
+        unpack_bf16x2(raw[j].y, v[j][2], v[j][3]);
+        unpack_bf16x2(raw[j].z, v[j][4], v[j][5]);
+        unpack_bf16x2(raw[j].w, v[j][6], v[j][7]);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) y[i] = (v[j][i] - mean) * rstd * (1.0f + scv[i]) + shv[i];
-      const int64_t o = row * D + vi * 8;
-      if (out_dtype == QDIT_I8) {
-        *reinterpret_cast<uint2*>(static_cast<uint8_t*>(out) + o) = quantize_pack8(y, inv, qa.zp, qa.qmin, qa.qmax);
-      } else if (out_dtype == QDIT_BF16) {
-        *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(out) + o) = pack_bf16x8(y);
-      } else {
-        float* of = static_cast<float*>(out) + o;
-        *reinterpret_cast<float4*>(of) = make_float4(y[0], y[1], y[2], y[3]);
-        *reinterpret_cast<float4*>(of + 4) = make_float4(y[4], y[5], y[6], y[7]);
+        for (int i = 0; i < 8; ++i) sum += v[j][i];
       }
     }
+    const float mean = warp_sum(sum) / static_cast<float>(D);
+    float ssq = 0.0f;
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+      if (lane + 32 * j < nvec) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float d = v[j][i] - mean;
+          ssq += d * d;
+        }
+      }
+    }
+    const float var = warp_sum(ssq) / static_cast<float>(D);
+    const float rstd = 1.0f / sqrtf(var + eps);
+    const int64_t b = row / T;
+    const bool staged = b - b0 < 2;
+    const float* sh = staged ? s_mod + (b - b0) * 2 * D : shift + b * ld_mod;
+    const float* sc = staged ? s_mod + (b - b0) * 2 * D + D : scale + b * ld_mod;
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+      const int vi = lane + 32 * j;
+      if (vi < nvec) {
+        float shv[8], scv[8], y[8];
+        Load8<float>::load(sh + vi * 8, shv);
+        Load8<float>::load(sc + vi * 8, scv);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) y[i] = (v[j][i] - mean) * rstd * (1.0f + scv[i]) + shv[i];
+        const int64_t o = row * D + vi * 8;
+        if (out_dtype == QDIT_I8) {
+          *reinterpret_cast<uint2*>(static_cast<uint8_t*>(out) + o) = quantize_pack8(y, inv, qa.zp, qa.qmin, qa.qmax);
+        } else if (out_dtype == QDIT_BF16) {
+          *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(out) + o) = pack_bf16x8(y);
+        } else {
+          float* of = static_cast<float*>(out) + o;
+          *reinterpret_cast<float4*>(of) = make_float4(y[0], y[1], y[2], y[3]);
+          *reinterpret_cast<float4*>(of + 4) = make_float4(y[4], y[5], y[6], y[7]);
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < NV; ++j) raw[j] = raw_next[j];
   }
 }
 
 template <int NV>
 void launch_ln(qdit_ctx* ctx, const void* x, int64_t M, int D, int64_t T, float eps, const float* shift,
                const float* scale, int64_t ld_mod, void* out, int out_dtype, QuantArgs qa) {
-  const int warps = 8;
-  const unsigned grid = static_cast<unsigned>((M + warps - 1) / warps);
-  ln_modulate_kernel<NV><<<grid, warps * 32, 2 * D * sizeof(float), ctx->stream>>>(
-      static_cast<const __nv_bfloat16*>(x), M, D, T, eps, shift, scale, ld_mod, out, out_dtype, qa);
+  // two CTAs per SM, contiguous row ranges (at least one row per warp, at most what keeps a range within two samples)
+  int64_t ctas = 2 * static_cast<int64_t>(ctx->num_sms);
+  int64_t rows = (M + ctas - 1) / ctas;
+  if (rows < 8) rows = 8;
+  if (rows > T) rows = T;
+  const unsigned grid = static_cast<unsigned>((M + rows - 1) / rows);
+  ln_modulate_kernel<NV><<<grid, 256, 4 * D * sizeof(float), ctx->stream>>>(
+      static_cast<const __nv_bfloat16*>(x), M, D, T, eps, shift, scale, ld_mod, out, out_dtype, qa, static_cast<int>(rows));
 }
 
 }  // namespace
