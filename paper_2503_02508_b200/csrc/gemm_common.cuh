@@ -223,19 +223,22 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t tacc
                    : "memory");
     }
     __syncwarp();
+    uint4 lo[4], hi[4];  // all eight shared-memory reads are issued before the first is consumed
 #pragma unroll
     for (int sidx = 0; sidx < 4; ++sidx) {
       const int r = sidx * 8 + rsub;
-      const int row = row_base + r;
-      uint4 lo, hi;
       const uint32_t a_lo = patch + static_cast<uint32_t>(r * 128 + (((2 * cg) ^ (r & 7)) << 4));
       const uint32_t a_hi = patch + static_cast<uint32_t>(r * 128 + (((2 * cg + 1) ^ (r & 7)) << 4));
-      asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(lo.x), "=r"(lo.y), "=r"(lo.z), "=r"(lo.w) : "r"(a_lo));
-      asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(hi.x), "=r"(hi.y), "=r"(hi.z), "=r"(hi.w) : "r"(a_hi));
+      asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(lo[sidx].x), "=r"(lo[sidx].y), "=r"(lo[sidx].z), "=r"(lo[sidx].w) : "r"(a_lo));
+      asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(hi[sidx].x), "=r"(hi[sidx].y), "=r"(hi[sidx].z), "=r"(hi[sidx].w) : "r"(a_hi));
+    }
+#pragma unroll
+    for (int sidx = 0; sidx < 4; ++sidx) {
+      const int row = row_base + sidx * 8 + rsub;
       if (row < p.M && col_ok) {
         if (!gate_uniform && (flags & QDIT_EPI_GATE))
           Load8<float>::load(p.gate + static_cast<int64_t>(row / p.tokens) * p.ld_gate + n, cur.cp.gt);
-        epilogue8<EPI>(p, lo, hi, cur.cp, cur.res[sidx], row, n, o_inv);
+        epilogue8<EPI>(p, lo[sidx], hi[sidx], cur.cp, cur.res[sidx], row, n, o_inv);
       }
     }
   }
