@@ -301,6 +301,9 @@ extern "C" int32_t qdit_w8a8_linear(qdit_ctx* ctx, const void* A, const void* W,
     const int bn = atoi(env);
     if (bn == 128 || bn == 192 || bn == 256) return qdit_launch_gemm_pair(ctx, A, W, p, a_unsigned, bn);
   }
+  // Wide outputs on many rows: the CTA-pair kernel (256 x 256 tiles; each CTA stages only half of the weight
+  // tile) measured 4-10 % faster on the QKV and fc1 shapes; narrow outputs (N = hidden) stay on 128 x 192.
+  if (!getenv("QDIT_GEMM_BN") && p.M >= 1024 && p.N >= 2304) return qdit_launch_gemm_pair(ctx, A, W, p, a_unsigned, 256);
   switch (pick_bn(p.M, p.N, ctx->num_sms)) {
     case 64: return launch_gemm<64>(ctx, A, W, p, a_unsigned);
     case 128: return launch_gemm<128>(ctx, A, W, p, a_unsigned);

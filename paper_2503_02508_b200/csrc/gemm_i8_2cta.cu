@@ -33,7 +33,7 @@ struct PairCfg {
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + BAR_BYTES + 1024;
 };
 
-template <int BN>
+template <int BN, int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                     const GemmParams p, const uint32_t idesc) {
@@ -144,7 +144,7 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     const uint32_t stg = smem_u32(staging + e * (32 * 128));
     const float a_scale = p.a_scale_dev ? __ldg(p.a_scale_dev) : p.a_scale;
     float o_inv = 0.0f;
-    if (p.flags & QDIT_EPI_QUANT_OUT) o_inv = __fdiv_rn(1.0f, p.o_scale_dev ? __ldg(p.o_scale_dev) : p.o_scale);
+    if (epi_flags<EPI>(p) & QDIT_EPI_QUANT_OUT) o_inv = __fdiv_rn(1.0f, p.o_scale_dev ? __ldg(p.o_scale_dev) : p.o_scale);
     int it = 0;
     for (int tile = pair_id; tile < total_tiles; tile += num_pairs, ++it) {
       const int as = it & 1;
@@ -155,7 +155,7 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       __syncwarp();
       tc_fence_after();
       const uint32_t leader_tempty = mapa_shared(smem_u32(&tempty_bar[as]), 0);
-      epilogue_tile<BN, 0>(p, tmem_base + static_cast<uint32_t>(as * BN), m0, n0, quad, half, stg, lane, a_scale, o_inv,
+      epilogue_tile<BN, EPI>(p, tmem_base + static_cast<uint32_t>(as * BN), m0, n0, quad, half, stg, lane, a_scale, o_inv,
                         [leader_tempty]() { mbar_arrive_cluster_relaxed(leader_tempty); });
     }
   }
@@ -169,12 +169,12 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   }
 }
 
-template <int BN>
-int32_t launch_pair(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p, bool a_unsigned) {
+template <int BN, int EPI>
+int32_t launch_pair_epi(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p, bool a_unsigned) {
   using C = PairCfg<BN>;
   static bool attr_set[64] = {};
   if (!attr_set[ctx->device & 63]) {
-    QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(gemm_i8_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+    QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(gemm_i8_pair_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
     attr_set[ctx->device & 63] = true;
   }
   CUtensorMap ta, tw;
@@ -187,8 +187,18 @@ int32_t launch_pair(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p, 
   const int pairs = total < max_pairs ? total : max_pairs;
   const uint32_t idesc = umma_idesc_i8(2 * BM, BN, a_unsigned);
   ProfScope prof(ctx, QDIT_PROF_GEMM, 2.0 * p.M * static_cast<double>(p.N) * p.K);
-  gemm_i8_pair_kernel<BN><<<2 * pairs, NUM_THREADS, C::SMEM_BYTES, ctx->stream>>>(ta, tw, p, idesc);
+  gemm_i8_pair_kernel<BN, EPI><<<2 * pairs, NUM_THREADS, C::SMEM_BYTES, ctx->stream>>>(ta, tw, p, idesc);
   return qdit_after_launch(ctx, "gemm_i8_pair_kernel");
+}
+
+template <int BN>
+int32_t launch_pair(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p, bool a_unsigned) {
+  switch (getenv("QDIT_GEMM_GENERIC_EPILOGUE") ? 0 : epi_class(p.flags)) {
+    case 1: return launch_pair_epi<BN, 1>(ctx, A, W, p, a_unsigned);
+    case 2: return launch_pair_epi<BN, 2>(ctx, A, W, p, a_unsigned);
+    case 3: return launch_pair_epi<BN, 3>(ctx, A, W, p, a_unsigned);
+    default: return launch_pair_epi<BN, 0>(ctx, A, W, p, a_unsigned);
+  }
 }
 
 }  // namespace
