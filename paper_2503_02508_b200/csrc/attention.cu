@@ -7,6 +7,8 @@
 // already bank-conflict-free for ldmatrix).  S = Q K^T and O = P V run on bf16 mma.sync with f32
 // accumulation; softmax is the online (running max / running sum) form in f32, exponentials in base 2.
 // The output can be written as f32, bf16, or directly as the projection's 8-bit activation codes.
+#include <cstdlib>
+
 #include "common.cuh"
 #include "internal.h"
 
@@ -286,6 +288,9 @@ int32_t launch_attention(qdit_ctx* ctx, const void* q, const void* k, const void
 
 }  // namespace
 
+int32_t qdit_launch_attention_tc(qdit_ctx* ctx, const void* q, const void* k, const void* v, int64_t ld, int B, int H,
+                                 int T, int dh, float softmax_scale, void* out, int out_dtype, QuantArgs qa);
+
 extern "C" int32_t qdit_attention(qdit_ctx* ctx, const void* q, const void* k, const void* v, int64_t ld, int B, int H,
                                   int T, int dh, float softmax_scale, void* out, int out_dtype,
                                   const qdit_qparams* out_qp, const float* out_scale_dev) {
@@ -311,6 +316,9 @@ extern "C" int32_t qdit_attention(qdit_ctx* ctx, const void* q, const void* k, c
     QDIT_TRY(qdit_check_qparams(ctx, out_qp, out_scale_dev != nullptr));
     p.qa = make_quant_args(*out_qp, out_scale_dev);
   }
+  // token counts that fill 128-query tiles run on the tcgen05 kernel; the mma.sync kernel covers the rest
+  if (T % 128 == 0 && !getenv("QDIT_ATTN_LEGACY"))
+    return qdit_launch_attention_tc(ctx, q, k, v, ld, B, H, T, dh, softmax_scale, out, out_dtype, p.qa);
   const bool wide = T % 128 == 0;  // 128 queries per CTA when the token count allows
   if (dh == 64) return wide ? launch_attention<64, 8>(ctx, q, k, v, ld, B, H, T, p) : launch_attention<64, 4>(ctx, q, k, v, ld, B, H, T, p);
   return wide ? launch_attention<72, 8>(ctx, q, k, v, ld, B, H, T, p) : launch_attention<72, 4>(ctx, q, k, v, ld, B, H, T, p);

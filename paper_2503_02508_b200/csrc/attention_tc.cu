@@ -1,0 +1,317 @@
+// Non-causal softmax attention on the 5th-generation tensor cores (tcgen05 kind::f16, bf16 operands).
+//
+// One CTA = 128 queries of one (sample, head).  Keys are consumed in blocks of 128:
+//   S = Q K^T     tcgen05.mma, A = Q and B = K tiles (K-major, TMA-staged), accumulator in tensor memory
+//   softmax       one thread per query row: tcgen05.ld S, running max / sum in f32 (no shuffles needed),
+//                 P = exp2(..) written as bf16 into a 128B-swizzled shared-memory tile
+//   O_blk = P V   tcgen05.mma, A = P (K-major), B = V tile used MN-major (its head-dim index is contiguous),
+//                 accumulator re-uses the S columns; the row thread folds it into its f32 registers
+// Head dim 72 does not fill a 128-byte swizzle row: every operand is staged as a 64-column tile (128B
+// swizzle) plus a 16-column tail tile (32B swizzle, columns 64..79).  The tail's columns 72..79 belong to the
+// next head; they are zeroed in the Q tail, so they add nothing to S, and in V they only produce output
+// columns 72..79, which are dropped.
+// Warps 0-3: softmax rows; warp 4 lane 0: TMA producer; warp 5 lane 0: MMA issuer (warp 5 owns the TMEM
+// allocation).  Two CTAs fit per SM (92 KB shared memory, 128 TMEM columns each) and overlap each other's phases.
+#include "common.cuh"
+#include "internal.h"
+
+namespace {
+
+using namespace qd;
+
+constexpr int TQ = 128;   // queries per CTA
+constexpr int TK = 128;   // keys per block
+constexpr int TC_THREADS = 192;
+
+struct AttnTcParams {
+  int T, H;
+  float scale_log2;  // softmax_scale * log2(e)
+  void* out;
+  int out_dtype;
+  QuantArgs qa;
+  int* status;
+};
+
+template <int DH>
+struct TCfg {
+  static constexpr bool TAIL = DH > 64;                 // 64 < DH <= 80: a 16-column tail tile
+  static constexpr int MAIN_BYTES = 128 * 128;          // 128 rows x 64 bf16
+  static constexpr int TAIL_BYTES = TAIL ? 128 * 32 : 0;
+  static constexpr int OP_BYTES = MAIN_BYTES + TAIL_BYTES;
+  static constexpr int P_BYTES = 2 * MAIN_BYTES;        // 128 rows x 128 keys bf16 = two 64-key tiles
+  static constexpr int SMEM_BYTES = 3 * OP_BYTES + P_BYTES + 256 + 1024;
+  static constexpr int O_COLS = TAIL ? 80 : 64;
+};
+
+template <int DH>
+__global__ void __launch_bounds__(TC_THREADS, 2)
+attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_qt,
+                    const __grid_constant__ CUtensorMap tm_kt, const __grid_constant__ CUtensorMap tm_vt,
+                    const AttnTcParams p) {
+  using C = TCfg<DH>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sQ = smem;
+  uint8_t* sK = sQ + C::MAIN_BYTES;
+  uint8_t* sV = sK + C::MAIN_BYTES;
+  uint8_t* sP = sV + C::MAIN_BYTES;             // two 64-key tiles
+  uint8_t* sQt = sP + C::P_BYTES;               // tails (256-byte aligned: 32B-swizzle atoms)
+  uint8_t* sKt = sQt + C::TAIL_BYTES;
+  uint8_t* sVt = sKt + C::TAIL_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sVt + C::TAIL_BYTES);
+  uint64_t* bar_q = bars + 0;      // Q tiles landed (tx)
+  uint64_t* bar_qz = bars + 1;     // Q tail padding zeroed (128 arrivals)
+  uint64_t* bar_kfull = bars + 2;  // K block landed (tx)
+  uint64_t* bar_vfull = bars + 3;  // V block landed (tx)
+  uint64_t* bar_kfree = bars + 4;  // S MMAs done reading K (commit)
+  uint64_t* bar_vfree = bars + 5;  // PV MMAs done reading V and P (commit)
+  uint64_t* bar_s = bars + 6;      // S complete (commit)
+  uint64_t* bar_p = bars + 7;      // P written (128 arrivals)
+  uint64_t* bar_o = bars + 8;      // O_blk complete (commit)
+  uint64_t* bar_sfree = bars + 9;  // O_blk read: the accumulator columns may be overwritten (128 arrivals)
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 10);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int q0 = blockIdx.x * TQ, h = blockIdx.y, b = blockIdx.z;
+  const int row0 = b * p.T, col0 = h * DH;
+  const int n_blk = p.T / TK;
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar_q, 1);
+    mbar_init(bar_qz, 128);
+    mbar_init(bar_kfull, 1);
+    mbar_init(bar_vfull, 1);
+    mbar_init(bar_kfree, 1);
+    mbar_init(bar_vfree, 1);
+    mbar_init(bar_s, 1);
+    mbar_init(bar_p, 128);
+    mbar_init(bar_o, 1);
+    mbar_init(bar_sfree, 128);
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  if (warp == 5) {
+    tmem_alloc(tmem_holder, 128);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_holder;
+
+  if (warp == 4) {
+    if (lane == 0) {
+      // ---------------------------------------------------------------- TMA producer
+      mbar_expect_tx(bar_q, C::OP_BYTES);
+      tma_load_2d(sQ, &tm_q, col0, row0 + q0, bar_q);
+      if (C::TAIL) tma_load_2d(sQt, &tm_qt, col0 + 64, row0 + q0, bar_q);
+      for (int j = 0; j < n_blk; ++j) {
+        if (j > 0 && !mbar_wait(bar_kfree, (j - 1) & 1, abort_flag, p.status)) break;
+        mbar_expect_tx(bar_kfull, C::OP_BYTES);
+        tma_load_2d(sK, &tm_k, col0, row0 + j * TK, bar_kfull);
+        if (C::TAIL) tma_load_2d(sKt, &tm_kt, col0 + 64, row0 + j * TK, bar_kfull);
+        if (j > 0 && !mbar_wait(bar_vfree, (j - 1) & 1, abort_flag, p.status)) break;
+        mbar_expect_tx(bar_vfull, C::OP_BYTES);
+        tma_load_2d(sV, &tm_v, col0, row0 + j * TK, bar_vfull);
+        if (C::TAIL) tma_load_2d(sVt, &tm_vt, col0 + 64, row0 + j * TK, bar_vfull);
+      }
+    }
+  } else if (warp == 5) {
+    if (lane == 0) {
+      // ---------------------------------------------------------------- MMA issuer
+      const uint32_t id_s = umma_idesc_bf16(128, TK, false);
+      const uint32_t id_o = umma_idesc_bf16(128, 64, true);
+      const uint32_t id_ot = umma_idesc_bf16(128, 16, true);
+      bool ok = mbar_wait(bar_qz, 0, abort_flag, p.status);
+      for (int j = 0; j < n_blk && ok; ++j) {
+        const uint32_t ph = j & 1;
+        if (!mbar_wait(bar_kfull, ph, abort_flag, p.status)) break;
+        if (j > 0 && !mbar_wait(bar_sfree, (j - 1) & 1, abort_flag, p.status)) break;
+        tc_fence_after();
+        // S = Q K^T: 4 k-steps of 16 out of the 64-column tiles, one out of the tails
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          umma_bf16(tmem, umma_desc(smem_u32(sQ) + k * 32, 1024, 2), umma_desc(smem_u32(sK) + k * 32, 1024, 2), id_s, k ? 1u : 0u);
+        if (C::TAIL) umma_bf16(tmem, umma_desc(smem_u32(sQt), 256, 6), umma_desc(smem_u32(sKt), 256, 6), id_s, 1u);
+        umma_commit(bar_s);
+        umma_commit(bar_kfree);
+        if (!mbar_wait(bar_p, ph, abort_flag, p.status)) break;
+        if (!mbar_wait(bar_vfull, ph, abort_flag, p.status)) break;
+        tc_fence_after();
+        // O_blk = P V: 8 k-steps of 16 keys; V's 8-key groups are 1024 (main) / 256 (tail) bytes apart
+#pragma unroll
+        for (int k = 0; k < TK / 16; ++k) {
+          const uint64_t a = umma_desc(smem_u32(sP) + (k >> 2) * C::MAIN_BYTES + (k & 3) * 32, 1024, 2);
+          umma_bf16(tmem, a, umma_desc(smem_u32(sV) + k * 2048, 1024, 2), id_o, k ? 1u : 0u);
+          if (C::TAIL) umma_bf16(tmem + 64, a, umma_desc(smem_u32(sVt) + k * 512, 256, 6), id_ot, k ? 1u : 0u);
+        }
+        umma_commit(bar_o);
+        umma_commit(bar_vfree);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax rows (thread = query row)
+    const int r = warp * 32 + lane;
+    const uint32_t trow = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+    bool ok = mbar_wait(bar_q, 0, abort_flag, p.status);
+    if (ok) {
+      if (C::TAIL) {  // zero columns 72..79 of this row of the Q tail (second 16-byte slot, 32B swizzle)
+        const uint32_t addr = smem_u32(sQt) + static_cast<uint32_t>(r * 32) + ((1u ^ ((static_cast<uint32_t>(r) >> 2) & 1u)) << 4);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
+        fence_async_smem();
+      }
+      mbar_arrive(bar_qz);
+    }
+    float o[C::O_COLS];
+#pragma unroll
+    for (int i = 0; i < C::O_COLS; ++i) o[i] = 0.0f;
+    float m_run = -INFINITY, l_run = 0.0f;
+    for (int j = 0; j < n_blk && ok; ++j) {
+      const uint32_t ph = j & 1;
+      if (!mbar_wait(bar_s, ph, abort_flag, p.status)) { ok = false; break; }
+      __syncwarp();
+      tc_fence_after();
+      // pass 1: row maximum of this block
+      float mx = -INFINITY;
+#pragma unroll 1
+      for (int c = 0; c < TK / 32; ++c) {
+        uint32_t v[32];
+        tmem_ld_32x32(trow + c * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
+      }
+      const float m_new = fmaxf(m_run, mx * p.scale_log2);
+      const float alpha = ex2_approx(m_run - m_new);
+      m_run = m_new;
+      // pass 2: P = exp2(s * scale - m), row sum, bf16 into the swizzled tiles
+      float rs = 0.0f;
+#pragma unroll 1
+      for (int c = 0; c < TK / 32; ++c) {
+        uint32_t v[32];
+        tmem_ld_32x32(trow + c * 32, v);
+        tmem_ld_wait();
+        float pv[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          pv[i] = ex2_approx(fmaf(__uint_as_float(v[i]), p.scale_log2, -m_new));
+          rs += pv[i];
+        }
+        const uint32_t tile = smem_u32(sP) + static_cast<uint32_t>((c >> 1) * C::MAIN_BYTES + r * 128);
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {  // 8 keys = one 16-byte slot; slot index within the 64-key tile
+          const uint32_t slot = static_cast<uint32_t>((c & 1) * 4 + g);
+          const uint32_t addr = tile + ((slot ^ (static_cast<uint32_t>(r) & 7u)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pack_bf16x2(pv[8 * g], pv[8 * g + 1])),
+                       "r"(pack_bf16x2(pv[8 * g + 2], pv[8 * g + 3])), "r"(pack_bf16x2(pv[8 * g + 4], pv[8 * g + 5])),
+                       "r"(pack_bf16x2(pv[8 * g + 6], pv[8 * g + 7]))
+                       : "memory");
+        }
+      }
+      l_run = l_run * alpha + rs;
+      fence_async_smem();   // P is read by the tensor core through the async proxy
+      tc_fence_before();    // and the S columns are about to be overwritten by O_blk
+      mbar_arrive(bar_p);
+      // fold O_blk into the running output
+      if (!mbar_wait(bar_o, ph, abort_flag, p.status)) { ok = false; break; }
+      __syncwarp();
+      tc_fence_after();
+      {
+        uint32_t v[32];
+        tmem_ld_32x32(trow, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[i] = fmaf(o[i], alpha, __uint_as_float(v[i]));
+        tmem_ld_32x32(trow + 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[32 + i] = fmaf(o[32 + i], alpha, __uint_as_float(v[i]));
+        if (C::TAIL) {
+          uint32_t w[16];
+          tmem_ld_32x16(trow + 64, w);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) o[64 + i] = fmaf(o[64 + i], alpha, __uint_as_float(w[i]));
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(bar_sfree);
+    }
+    if (ok) {
+      const float inv_l = 1.0f / l_run;
+      const int64_t row = static_cast<int64_t>(row0) + q0 + r;
+      const int64_t base = row * (static_cast<int64_t>(p.H) * DH) + col0;
+      float q_inv = 0.0f;
+      if (p.out_dtype == QDIT_I8) q_inv = __fdiv_rn(1.0f, p.qa.scale_dev ? __ldg(p.qa.scale_dev) : p.qa.scale);
+#pragma unroll
+      for (int g = 0; g < DH / 8; ++g) {
+        float y[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) y[i] = o[8 * g + i] * inv_l;
+        if (p.out_dtype == QDIT_I8) {
+          *reinterpret_cast<uint2*>(static_cast<uint8_t*>(p.out) + base + 8 * g) = quantize_pack8(y, q_inv, p.qa.zp, p.qa.qmin, p.qa.qmax);
+        } else if (p.out_dtype == QDIT_BF16) {
+          *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + base + 8 * g) = pack_bf16x8(y);
+        } else {
+          float* of = static_cast<float*>(p.out) + base + 8 * g;
+          *reinterpret_cast<float4*>(of) = make_float4(y[0], y[1], y[2], y[3]);
+          *reinterpret_cast<float4*>(of + 4) = make_float4(y[4], y[5], y[6], y[7]);
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 128);
+  }
+}
+
+template <int DH>
+int32_t launch_tc(qdit_ctx* ctx, const void* q, const void* k, const void* v, int64_t ld, int B, int H, int T,
+                  const AttnTcParams& p) {
+  using C = TCfg<DH>;
+  static bool attr_set[64] = {};
+  if (!attr_set[ctx->device & 63]) {
+    QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(attention_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+    attr_set[ctx->device & 63] = true;
+  }
+  const uint64_t rows = static_cast<uint64_t>(B) * T, cols = static_cast<uint64_t>(H) * DH;
+  CUtensorMap tq, tk, tv, tqt, tkt, tvt;
+  QDIT_TRY(qdit_get_tmap(ctx, q, rows, cols, ld, 128, 64, 1, 2, &tq));
+  QDIT_TRY(qdit_get_tmap(ctx, k, rows, cols, ld, 128, 64, 1, 2, &tk));
+  QDIT_TRY(qdit_get_tmap(ctx, v, rows, cols, ld, 128, 64, 1, 2, &tv));
+  tqt = tq;
+  tkt = tk;
+  tvt = tv;
+  if (C::TAIL) {
+    QDIT_TRY(qdit_get_tmap(ctx, q, rows, cols, ld, 128, 16, 3, 2, &tqt));
+    QDIT_TRY(qdit_get_tmap(ctx, k, rows, cols, ld, 128, 16, 3, 2, &tkt));
+    QDIT_TRY(qdit_get_tmap(ctx, v, rows, cols, ld, 128, 16, 3, 2, &tvt));
+  }
+  dim3 grid(T / TQ, H, B);
+  ProfScope prof(ctx, QDIT_PROF_ATTENTION, 4.0 * B * H * static_cast<double>(T) * T * DH);
+  attention_tc_kernel<DH><<<grid, TC_THREADS, C::SMEM_BYTES, ctx->stream>>>(tq, tk, tv, tqt, tkt, tvt, p);
+  return qdit_after_launch(ctx, "attention_tc_kernel");
+}
+
+}  // namespace
+
+// Tensor-core attention for T % 128 == 0 and head dim 64 or 72 (arguments already validated by qdit_attention).
+int32_t qdit_launch_attention_tc(qdit_ctx* ctx, const void* q, const void* k, const void* v, int64_t ld, int B, int H,
+                                 int T, int dh, float softmax_scale, void* out, int out_dtype, QuantArgs qa) {
+  AttnTcParams p{};
+  p.T = T;
+  p.H = H;
+  p.scale_log2 = softmax_scale * 1.4426950408889634f;
+  p.out = out;
+  p.out_dtype = out_dtype;
+  p.qa = qa;
+  p.status = ctx->d_status;
+  if (dh == 64) return launch_tc<64>(ctx, q, k, v, ld, B, H, T, p);
+  return launch_tc<72>(ctx, q, k, v, ld, B, H, T, p);
+}

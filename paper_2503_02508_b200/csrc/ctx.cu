@@ -208,7 +208,7 @@ int32_t qdit_get_tmap(qdit_ctx* ctx, const void* ptr, uint64_t rows, uint64_t co
                                         : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
   CUtensorMap tm;
   CUresult r = encode(&tm, dt, 2, const_cast<void*>(ptr), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                      swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                      swizzle == 1 ? CU_TENSOR_MAP_SWIZZLE_128B : swizzle == 2 ? CU_TENSOR_MAP_SWIZZLE_64B : swizzle == 3 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE,
                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return qdit_fail(ctx, QDIT_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", static_cast<int>(r));
   if (ctx->tmaps.size() > 4096) ctx->tmaps.clear();

@@ -75,7 +75,8 @@ int32_t qdit_after_launch(qdit_ctx* ctx, const char* what);
   } while (0)
 
 // 2-D tensor map over a row-major matrix [rows, cols] of `esize`-byte elements with row pitch `ld`
-// elements; box = box_rows x box_cols elements; swizzle: 0 none, 1 = 128-byte.  Cached per context.
+// elements; box = box_rows x box_cols elements; swizzle: 0 none, 1 = 128-byte, 2 = 64-byte, 3 = 32-byte.
+// Cached per context.
 int32_t qdit_get_tmap(qdit_ctx* ctx, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows,
                       uint32_t box_cols, uint32_t swizzle, uint32_t esize, CUtensorMap* out);
 
