@@ -10,8 +10,9 @@
 // swizzle) plus a 16-column tail tile (32B swizzle, columns 64..79).  The tail's columns 72..79 belong to the
 // next head; they are zeroed in the Q tail, so they add nothing to S, and in V they only produce output
 // columns 72..79, which are dropped.
-// Warps 0-3: softmax rows; warp 4 lane 0: TMA producer; warp 5 lane 0: MMA issuer (warp 5 owns the TMEM
-// allocation).  Two CTAs fit per SM (92 KB shared memory, 128 TMEM columns each) and overlap each other's phases.
+// Warps 0-7: softmax (two threads per query row: both find the row maximum over the whole block, then each
+// exponentiates, stores and accumulates its half of the columns); warp 8 lane 0: TMA producer; warp 9 lane 0:
+// MMA issuer (warp 9 owns the TMEM allocation).  Two CTAs fit per SM (92 KB shared memory, 128 TMEM columns each) and overlap each other's phases.
 #include "common.cuh"
 #include "internal.h"
 
@@ -21,7 +22,8 @@ using namespace qd;
 
 constexpr int TQ = 128;   // queries per CTA
 constexpr int TK = 128;   // keys per block
-constexpr int TC_THREADS = 192;
+constexpr int SM_WARPS = 8;                    // softmax warps: two threads share a query row
+constexpr int TC_THREADS = (SM_WARPS + 2) * 32;
 
 struct AttnTcParams {
   int T, H;
@@ -39,8 +41,9 @@ struct TCfg {
   static constexpr int TAIL_BYTES = TAIL ? 128 * 32 : 0;
   static constexpr int OP_BYTES = MAIN_BYTES + TAIL_BYTES;
   static constexpr int P_BYTES = 2 * MAIN_BYTES;        // 128 rows x 128 keys bf16 = two 64-key tiles
-  static constexpr int SMEM_BYTES = 3 * OP_BYTES + P_BYTES + 256 + 1024;
+  static constexpr int SMEM_BYTES = 3 * OP_BYTES + P_BYTES + 2048 + 1024;
   static constexpr int O_COLS = TAIL ? 80 : 64;
+  static constexpr int O_HALF = O_COLS / 2;             // accumulator columns per thread of a row pair (40 or 32)
 };
 
 template <int DH>
@@ -70,8 +73,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   uint64_t* bar_p = bars + 7;      // P written (128 arrivals)
   uint64_t* bar_o = bars + 8;      // O_blk complete (commit)
   uint64_t* bar_sfree = bars + 9;  // O_blk read: the accumulator columns may be overwritten (128 arrivals)
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 10);
+  uint64_t* bar_l = bars + 10;     // row sums exchanged (256 arrivals)
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 11);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  float* s_l = reinterpret_cast<float*>(tmem_holder + 4);  // [2][128] partial row sums
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q0 = blockIdx.x * TQ, h = blockIdx.y, b = blockIdx.z;
@@ -80,19 +85,20 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
   if (threadIdx.x == 0) {
     mbar_init(bar_q, 1);
-    mbar_init(bar_qz, 128);
+    mbar_init(bar_qz, SM_WARPS * 32);
     mbar_init(bar_kfull, 1);
     mbar_init(bar_vfull, 1);
     mbar_init(bar_kfree, 1);
     mbar_init(bar_vfree, 1);
     mbar_init(bar_s, 1);
-    mbar_init(bar_p, 128);
+    mbar_init(bar_p, SM_WARPS * 32);
     mbar_init(bar_o, 1);
-    mbar_init(bar_sfree, 128);
+    mbar_init(bar_sfree, SM_WARPS * 32);
+    mbar_init(bar_l, SM_WARPS * 32);
     *abort_flag = 0;
     mbar_fence_init();
   }
-  if (warp == 5) {
+  if (warp == SM_WARPS + 1) {
     tmem_alloc(tmem_holder, 128);
     tmem_relinquish();
   }
@@ -101,7 +107,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   tc_fence_after();
   const uint32_t tmem = *tmem_holder;
 
-  if (warp == 4) {
+  if (warp == SM_WARPS) {
     if (lane == 0) {
       // ---------------------------------------------------------------- TMA producer
       mbar_expect_tx(bar_q, C::OP_BYTES);
@@ -118,7 +124,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (C::TAIL) tma_load_2d(sVt, &tm_vt, col0 + 64, row0 + j * TK, bar_vfull);
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == SM_WARPS + 1) {
     if (lane == 0) {
       // ---------------------------------------------------------------- MMA issuer
       const uint32_t id_s = umma_idesc_bf16(128, TK, false);
@@ -152,61 +158,63 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       }
     }
   } else {
-    // ------------------------------------------------------------------ softmax rows (thread = query row)
-    const int r = warp * 32 + lane;
-    const uint32_t trow = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+    // ------------------------------------------------------------------ softmax (two threads per query row)
+    const int quad = warp & 3, half = warp >> 2;
+    const int r = quad * 32 + lane;
+    const uint32_t trow = tmem + (static_cast<uint32_t>(quad * 32) << 16);
     bool ok = mbar_wait(bar_q, 0, abort_flag, p.status);
     if (ok) {
-      if (C::TAIL) {  // zero columns 72..79 of this row of the Q tail (second 16-byte slot, 32B swizzle)
+      if (C::TAIL && half == 0) {  // zero columns 72..79 of this row of the Q tail (second 16-byte slot, 32B swizzle)
         const uint32_t addr = smem_u32(sQt) + static_cast<uint32_t>(r * 32) + ((1u ^ ((static_cast<uint32_t>(r) >> 2) & 1u)) << 4);
         asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
         fence_async_smem();
       }
       mbar_arrive(bar_qz);
     }
-    float o[C::O_COLS];
+    float o[C::O_HALF];
 #pragma unroll
-    for (int i = 0; i < C::O_COLS; ++i) o[i] = 0.0f;
+    for (int i = 0; i < C::O_HALF; ++i) o[i] = 0.0f;
     float m_run = -INFINITY, l_run = 0.0f;
     for (int j = 0; j < n_blk && ok; ++j) {
       const uint32_t ph = j & 1;
       if (!mbar_wait(bar_s, ph, abort_flag, p.status)) { ok = false; break; }
       __syncwarp();
       tc_fence_after();
-      // pass 1: row maximum of this block
+      // pass 1: row maximum over the whole block (both threads of the row compute the same value)
       float mx = -INFINITY;
 #pragma unroll 1
-      for (int c = 0; c < TK / 32; ++c) {
-        uint32_t v[32];
-        tmem_ld_32x32(trow + c * 32, v);
+      for (int c = 0; c < TK / 16; ++c) {
+        uint32_t v[16];
+        tmem_ld_32x16(trow + c * 16, v);
         tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
+        for (int i = 0; i < 16; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
       }
       const float m_new = fmaxf(m_run, mx * p.scale_log2);
       const float alpha = ex2_approx(m_run - m_new);
       m_run = m_new;
-      // pass 2: P = exp2(s * scale - m), row sum, bf16 into the swizzled tiles
+      // pass 2 (this thread's 64 keys): P = exp2(s * scale - m), row sum, bf16 into the swizzled tile
       float rs = 0.0f;
+      const uint32_t tile = smem_u32(sP) + static_cast<uint32_t>(half * C::MAIN_BYTES + r * 128);
 #pragma unroll 1
-      for (int c = 0; c < TK / 32; ++c) {
-        uint32_t v[32];
-        tmem_ld_32x32(trow + c * 32, v);
+      for (int c = 0; c < 4; ++c) {  // 16 keys = two 16-byte slots
+        uint32_t v[16];
+        tmem_ld_32x16(trow + half * 64 + c * 16, v);
         tmem_ld_wait();
-        float pv[32];
+        uint32_t pk[8];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          pv[i] = ex2_approx(fmaf(__uint_as_float(v[i]), p.scale_log2, -m_new));
-          rs += pv[i];
+        for (int i = 0; i < 8; ++i) {
+          const float p0 = ex2_approx(fmaf(__uint_as_float(v[2 * i]), p.scale_log2, -m_new));
+          const float p1 = ex2_approx(fmaf(__uint_as_float(v[2 * i + 1]), p.scale_log2, -m_new));
+          rs += p0 + p1;
+          pk[i] = pack_bf16x2(p0, p1);
         }
-        const uint32_t tile = smem_u32(sP) + static_cast<uint32_t>((c >> 1) * C::MAIN_BYTES + r * 128);
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {  // 8 keys = one 16-byte slot; slot index within the 64-key tile
-          const uint32_t slot = static_cast<uint32_t>((c & 1) * 4 + g);
+        for (int g = 0; g < 2; ++g) {
+          const uint32_t slot = static_cast<uint32_t>(c * 2 + g);
           const uint32_t addr = tile + ((slot ^ (static_cast<uint32_t>(r) & 7u)) << 4);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pack_bf16x2(pv[8 * g], pv[8 * g + 1])),
-                       "r"(pack_bf16x2(pv[8 * g + 2], pv[8 * g + 3])), "r"(pack_bf16x2(pv[8 * g + 4], pv[8 * g + 5])),
-                       "r"(pack_bf16x2(pv[8 * g + 6], pv[8 * g + 7]))
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[4 * g]), "r"(pk[4 * g + 1]),
+                       "r"(pk[4 * g + 2]), "r"(pk[4 * g + 3])
                        : "memory");
         }
       }
@@ -214,50 +222,58 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       fence_async_smem();   // P is read by the tensor core through the async proxy
       tc_fence_before();    // and the S columns are about to be overwritten by O_blk
       mbar_arrive(bar_p);
-      // fold O_blk into the running output
+      // fold this thread's half of O_blk into its running output
       if (!mbar_wait(bar_o, ph, abort_flag, p.status)) { ok = false; break; }
       __syncwarp();
       tc_fence_after();
       {
-        uint32_t v[32];
-        tmem_ld_32x32(trow, v);
-        tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) o[i] = fmaf(o[i], alpha, __uint_as_float(v[i]));
-        tmem_ld_32x32(trow + 32, v);
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) o[32 + i] = fmaf(o[32 + i], alpha, __uint_as_float(v[i]));
-        if (C::TAIL) {
-          uint32_t w[16];
-          tmem_ld_32x16(trow + 64, w);
+        for (int c = 0; c < 2; ++c) {
+          uint32_t v[16];
+          tmem_ld_32x16(trow + half * C::O_HALF + c * 16, v);
           tmem_ld_wait();
 #pragma unroll
-          for (int i = 0; i < 16; ++i) o[64 + i] = fmaf(o[64 + i], alpha, __uint_as_float(w[i]));
+          for (int i = 0; i < 16; ++i) o[c * 16 + i] = fmaf(o[c * 16 + i], alpha, __uint_as_float(v[i]));
+        }
+        if (C::TAIL) {
+          uint32_t w[8];
+          tmem_ld_32x8(trow + half * C::O_HALF + 32, w);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 8; ++i) o[32 + i] = fmaf(o[32 + i], alpha, __uint_as_float(w[i]));
         }
       }
       tc_fence_before();
       mbar_arrive(bar_sfree);
     }
+    // the two threads of a row exchange their partial sums
     if (ok) {
-      const float inv_l = 1.0f / l_run;
+      s_l[half * 128 + r] = l_run;
+      mbar_arrive(bar_l);
+      ok = mbar_wait(bar_l, 0, abort_flag, p.status);
+    }
+    if (ok) {
+      const float inv_l = 1.0f / (s_l[r] + s_l[128 + r]);
       const int64_t row = static_cast<int64_t>(row0) + q0 + r;
-      const int64_t base = row * (static_cast<int64_t>(p.H) * DH) + col0;
+      const int64_t base = row * (static_cast<int64_t>(p.H) * DH) + col0 + half * C::O_HALF;
+      const int ngroups = half == 0 ? C::O_HALF / 8 : (DH - C::O_HALF) / 8;  // output columns beyond DH are padding
       float q_inv = 0.0f;
       if (p.out_dtype == QDIT_I8) q_inv = __fdiv_rn(1.0f, p.qa.scale_dev ? __ldg(p.qa.scale_dev) : p.qa.scale);
 #pragma unroll
-      for (int g = 0; g < DH / 8; ++g) {
-        float y[8];
+      for (int g = 0; g < C::O_HALF / 8; ++g) {
+        if (g < ngroups) {
+          float y[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) y[i] = o[8 * g + i] * inv_l;
-        if (p.out_dtype == QDIT_I8) {
-          *reinterpret_cast<uint2*>(static_cast<uint8_t*>(p.out) + base + 8 * g) = quantize_pack8(y, q_inv, p.qa.zp, p.qa.qmin, p.qa.qmax);
-        } else if (p.out_dtype == QDIT_BF16) {
-          *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + base + 8 * g) = pack_bf16x8(y);
-        } else {
-          float* of = static_cast<float*>(p.out) + base + 8 * g;
-          *reinterpret_cast<float4*>(of) = make_float4(y[0], y[1], y[2], y[3]);
-          *reinterpret_cast<float4*>(of + 4) = make_float4(y[4], y[5], y[6], y[7]);
+          for (int i = 0; i < 8; ++i) y[i] = o[8 * g + i] * inv_l;
+          if (p.out_dtype == QDIT_I8) {
+            *reinterpret_cast<uint2*>(static_cast<uint8_t*>(p.out) + base + 8 * g) = quantize_pack8(y, q_inv, p.qa.zp, p.qa.qmin, p.qa.qmax);
+          } else if (p.out_dtype == QDIT_BF16) {
+            *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + base + 8 * g) = pack_bf16x8(y);
+          } else {
+            float* of = static_cast<float*>(p.out) + base + 8 * g;
+            *reinterpret_cast<float4*>(of) = make_float4(y[0], y[1], y[2], y[3]);
+            *reinterpret_cast<float4*>(of + 4) = make_float4(y[4], y[5], y[6], y[7]);
+          }
         }
       }
     }
@@ -265,7 +281,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) {
+  if (warp == SM_WARPS + 1) {
     tc_fence_after();
     tmem_dealloc(tmem, 128);
   }
