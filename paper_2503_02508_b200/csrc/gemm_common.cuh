@@ -248,3 +248,6 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t tacc
 
 // CTA-pair kernel (gemm_i8_2cta.cu): tiles of 256 x bn, bn in {128, 192, 256}.
 int32_t qdit_launch_gemm_pair(qdit_ctx* ctx, const void* A, const void* W, qgemm::GemmParams& p, bool a_unsigned, int bn);
+
+// Channel-major accumulator kernel (gemm_i8_t.cu): tiles of 128 channels x bt tokens, bt in {128, 256}.
+int32_t qdit_launch_gemm_t(qdit_ctx* ctx, const void* A, const void* W, qgemm::GemmParams& p, bool a_unsigned, int bt);

@@ -296,6 +296,11 @@ extern "C" int32_t qdit_w8a8_linear(qdit_ctx* ctx, const void* A, const void* W,
       p.o_qmax = static_cast<float>(epi->out_qp.qmax);
     }
   }
+  // QDIT_GEMM_T=<bt> selects the channel-major kernel with 128 x bt tiles (experimental switch while tuning)
+  if (const char* env = getenv("QDIT_GEMM_T")) {
+    const int bt = atoi(env);
+    if (bt == 128 || bt == 256) return qdit_launch_gemm_t(ctx, A, W, p, a_unsigned, bt);
+  }
   // QDIT_GEMM_PAIR=<bn> selects the CTA-pair kernel with 256 x bn tiles (experimental switch while tuning)
   if (const char* env = getenv("QDIT_GEMM_PAIR")) {
     const int bn = atoi(env);

@@ -47,13 +47,16 @@ SHAPES = [(1, 8, 16), (128, 192, 128), (130, 200, 272), (256, 384, 1152), (517, 
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)
-@pytest.mark.parametrize("bn", ["auto", "64", "128", "192", "pair128", "pair192", "pair256"])
+@pytest.mark.parametrize("bn", ["auto", "64", "128", "192", "pair128", "pair192", "pair256", "t128", "t256"])
 def test_accumulators_bit_exact(q, ctx, M, N, K, bn):
     # "pairNNN": the CTA-pair kernel (256 x NNN tiles); plain numbers: the single-CTA kernel (128 x NNN)
     os.environ.pop("QDIT_GEMM_BN", None)
     os.environ.pop("QDIT_GEMM_PAIR", None)
+    os.environ.pop("QDIT_GEMM_T", None)
     if bn.startswith("pair"):
         os.environ["QDIT_GEMM_PAIR"] = bn[4:]
+    elif bn.startswith("t"):
+        os.environ["QDIT_GEMM_T"] = bn[1:]          # channel-major accumulator kernel, 128 x NNN tiles
     elif bn != "auto":
         os.environ["QDIT_GEMM_BN"] = bn
     try:
@@ -63,6 +66,7 @@ def test_accumulators_bit_exact(q, ctx, M, N, K, bn):
     finally:
         os.environ.pop("QDIT_GEMM_BN", None)
         os.environ.pop("QDIT_GEMM_PAIR", None)
+        os.environ.pop("QDIT_GEMM_T", None)
     np.testing.assert_array_equal(got, linear.gemm_i8(qa, qw))
 
 
@@ -127,13 +131,17 @@ def test_dequant_bias_f32(q, ctx, M, N, K, T, a_qp):
     assert max_rel_err(out.cpu().numpy(), ref) < 1e-5      # ... and what f32 arithmetic actually gives
 
 
-@pytest.fixture(params=["single", "pair192", "pair256"])
+@pytest.fixture(params=["single", "pair192", "pair256", "t128", "t256"])
 def kernel_variant(request):
     os.environ.pop("QDIT_GEMM_PAIR", None)
+    os.environ.pop("QDIT_GEMM_T", None)
     if request.param.startswith("pair"):
         os.environ["QDIT_GEMM_PAIR"] = request.param[4:]
+    elif request.param.startswith("t"):
+        os.environ["QDIT_GEMM_T"] = request.param[1:]
     yield request.param
     os.environ.pop("QDIT_GEMM_PAIR", None)
+    os.environ.pop("QDIT_GEMM_T", None)
 
 
 def test_gate_residual_cache_epilogue(q, ctx, kernel_variant):
@@ -158,6 +166,23 @@ def test_gate_residual_cache_epilogue(q, ctx, kernel_variant):
     assert (got_c != dit.round_bf16(f)).mean() < 1e-3
     assert (got_x != dit.round_bf16(want_x)).mean() < 1e-3
     assert max_rel_err(got_x, want_x) < 2.0 ** -8
+
+
+def test_bias_bf16_epilogue(q, ctx, kernel_variant):
+    # the QKV layer's epilogue, on ragged sizes (M, N not multiples of the tiles)
+    M, N, K, T = 300, 1096, 384, 100
+    a_qp = QParams(0.045, 0, -127, 127)
+    L = _layer(45, M, N, K, T, a_qp)
+    A, W = dev_i8(L["qa"]), dev_i8(L["qw"])
+    ws, bi = dev(L["s_w"]), dev(L["bias"])
+    out = torch.full((M, N), 7.0, dtype=torch.bfloat16, device="cuda")
+    q.qdit_w8a8_linear(ctx, A, W, M, N, K, q.qparams(a_qp.scale), None, q.QDIT_EPI_BIAS | q.QDIT_EPI_OUT_BF16,
+                       q.epilogue(w_scale=ws, bias=bi), out, N)
+    q.qdit_sync(ctx)
+    f = linear.w8a8_linear(L["qa"], a_qp, L["qw"], L["s_w"], L["cs"], L["bias"])
+    got = bf16_to_f64(out)
+    assert (got != dit.round_bf16(f)).mean() < 1e-3
+    assert np.abs(got - f).max() <= 2.0 ** -8 * np.abs(f).max()
 
 
 def test_gelu_requant_epilogue(q, ctx, kernel_variant):
