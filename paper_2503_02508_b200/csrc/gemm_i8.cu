@@ -306,9 +306,14 @@ extern "C" int32_t qdit_w8a8_linear(qdit_ctx* ctx, const void* A, const void* W,
     const int bn = atoi(env);
     if (bn == 128 || bn == 192 || bn == 256) return qdit_launch_gemm_pair(ctx, A, W, p, a_unsigned, bn);
   }
-  // Wide outputs on many rows: the CTA-pair kernel (256 x 256 tiles; each CTA stages only half of the weight
-  // tile) measured 4-10 % faster on the QKV and fc1 shapes; narrow outputs (N = hidden) stay on 128 x 192.
-  if (!getenv("QDIT_GEMM_BN") && p.M >= 1024 && p.N >= 2304) return qdit_launch_gemm_pair(ctx, A, W, p, a_unsigned, 256);
+  // Kernel choice (measured at M = 8192 on the DiT-XL/2 layers, see profiles/):
+  //  - layers whose epilogue neither reads a residual nor writes the cache (QKV: bias -> bf16; fc1: bias + GELU ->
+  //    8-bit) run channel-major with 128 x 256 tiles (1.96 / 1.45 POP/s vs 1.84 / 1.38 token-major; the CTA-pair
+  //    kernel is within 3 % of it);
+  //  - gated layers (proj, fc2) stay token-major on 128 x 192 tiles: their epilogue moves three tensors and the
+  //    shuffle transposes of the channel-major form cost more than the shared-memory transpose.
+  if (!getenv("QDIT_GEMM_BN") && p.M >= 1024 && p.N >= 2304 && (epi_class(p.flags) == 1 || epi_class(p.flags) == 2))
+    return qdit_launch_gemm_t(ctx, A, W, p, a_unsigned, 256);
   switch (pick_bn(p.M, p.N, ctx->num_sms)) {
     case 64: return launch_gemm<64>(ctx, A, W, p, a_unsigned);
     case 128: return launch_gemm<128>(ctx, A, W, p, a_unsigned);

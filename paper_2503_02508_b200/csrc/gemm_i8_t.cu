@@ -183,6 +183,61 @@ __device__ __forceinline__ void epilogue_chunk_t_packed(const GemmParams& p, con
   }
 }
 
+// Gated epilogue (bias, cache store, x gate, + residual -> bf16) in the same style: the branch value and its
+// gated copy are computed channel-major with scalar parameters; the bf16 cache copy travels through two word
+// transposes, the gated f32 value through four, and the residual is then added token-major, where a lane loads
+// and stores 8 consecutive channels of a token (16 bytes).  Needs the chunk inside one sample (tokens % 32 == 0).
+__device__ __forceinline__ void epilogue_chunk_t_gated(const GemmParams& p, const uint32_t (&v)[32], int n, int lane,
+                                                       int m_base, float sc, float bias, int zcs) {
+  const int i8 = lane & 7;
+  const int n8 = n - i8;
+  const bool n8_ok = n8 < p.N;
+  float f[32];
+#pragma unroll
+  for (int j = 0; j < 32; ++j) f[j] = static_cast<float>(static_cast<int>(v[j]) - zcs) * sc + bias;
+  // cache copy (pre-gate), bf16
+#pragma unroll
+  for (int s2 = 0; s2 < 4; s2 += 2) {
+    uint32_t w[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) w[t] = pack_bf16x2(f[8 * s2 + t], f[8 * (s2 + 1) + t]);
+    transpose8(w, lane);
+    if (n8_ok) {
+      const int64_t m_lo = m_base + 8 * s2 + i8, m_hi = m_lo + 8;
+      if (m_lo < p.M)
+        *reinterpret_cast<uint4*>(p.cache_out + m_lo * p.N + n8) =
+            make_uint4(__byte_perm(w[0], w[1], 0x5410), __byte_perm(w[2], w[3], 0x5410), __byte_perm(w[4], w[5], 0x5410),
+                       __byte_perm(w[6], w[7], 0x5410));
+      if (m_hi < p.M)
+        *reinterpret_cast<uint4*>(p.cache_out + m_hi * p.N + n8) =
+            make_uint4(__byte_perm(w[0], w[1], 0x7632), __byte_perm(w[2], w[3], 0x7632), __byte_perm(w[4], w[5], 0x7632),
+                       __byte_perm(w[6], w[7], 0x7632));
+    }
+  }
+  const float gate = n < p.N ? p.gate[static_cast<int64_t>(m_base / p.tokens) * p.ld_gate + n] : 0.0f;
+#pragma unroll
+  for (int s4 = 0; s4 < 4; ++s4) {
+    const int64_t m = m_base + 8 * s4 + i8;
+    const bool live = n8_ok && m < p.M;
+    uint4 rv = make_uint4(0u, 0u, 0u, 0u);
+    if (live) rv = *reinterpret_cast<const uint4*>(p.residual + m * p.ldo + n8);  // in flight during the shuffles
+    uint32_t w[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) w[t] = __float_as_uint(f[8 * s4 + t] * gate);
+    transpose8(w, lane);  // w[c] = gated value of channel n8 + c, token m
+    if (live) {
+      float r[8];
+      unpack_bf16x2(rv.x, r[0], r[1]);
+      unpack_bf16x2(rv.y, r[2], r[3]);
+      unpack_bf16x2(rv.z, r[4], r[5]);
+      unpack_bf16x2(rv.w, r[6], r[7]);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) r[c] += __uint_as_float(w[c]);
+      *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + m * p.ldo + n8) = pack_bf16x8(r);
+    }
+  }
+}
+
 template <int BT, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
@@ -330,6 +385,7 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
         const int m_base = t0 + c * 32;
         if (m_base < p.M) {
           if (EPI == 1 || EPI == 2) epilogue_chunk_t_packed<EPI>(p, v, n, lane, m_base, sc, bias, zcs, o_inv);
+          else if (EPI == 3 && (p.tokens % 32) == 0) epilogue_chunk_t_gated(p, v, n, lane, m_base, sc, bias, zcs);
           else if (n_ok) epilogue_chunk_t<EPI>(p, v, n, m_base, sc, bias, zcs, o_inv);
         }
       }
