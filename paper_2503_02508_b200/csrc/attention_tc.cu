@@ -106,6 +106,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_holder;
+  // shared and tensor memory only so far; Q, K and V come from the previous kernel of the stream
+  grid_dependency_wait();
+  grid_dependency_release();
 
   if (warp == SM_WARPS) {
     if (lane == 0) {
@@ -311,7 +314,7 @@ int32_t launch_tc(qdit_ctx* ctx, const void* q, const void* k, const void* v, in
   }
   dim3 grid(T / TQ, H, B);
   ProfScope prof(ctx, QDIT_PROF_ATTENTION, 4.0 * B * H * static_cast<double>(T) * T * DH);
-  attention_tc_kernel<DH><<<grid, TC_THREADS, C::SMEM_BYTES, ctx->stream>>>(tq, tk, tv, tqt, tkt, tvt, p);
+  QDIT_CUDA_CHECK(ctx, qdit_launch_overlapped(ctx, attention_tc_kernel<DH>, grid, dim3(TC_THREADS), C::SMEM_BYTES, tq, tk, tv, tqt, tkt, tvt, p));
   return qdit_after_launch(ctx, "attention_tc_kernel");
 }
 

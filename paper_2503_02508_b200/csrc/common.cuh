@@ -32,6 +32,14 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 __device__ __forceinline__ void mbar_arrive_relaxed(uint64_t* bar) {
   asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// Programmatic dependent launch.  A kernel launched with the programmatic-stream-serialization attribute may
+// begin (CTA scheduling, barrier set-up, tensor-memory allocation, descriptor prefetch) while the kernel
+// before it in the stream is still running.  grid_dependency_wait() returns once that kernel has completed
+// and its writes are visible; nothing before it may touch global memory that another kernel writes or reads.
+// grid_dependency_release() lets the NEXT kernel of the stream start its own preamble.  Both are no-ops for
+// a kernel launched without the attribute.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(

@@ -1,6 +1,7 @@
 // Context, status reporting and tensor-map creation.
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <new>
 
 #include "internal.h"
@@ -115,6 +116,7 @@ int32_t qdit_create(qdit_ctx** out, int device, void* cuda_stream) {
   ctx->device = device;
   ctx->stream = static_cast<cudaStream_t>(cuda_stream);
   ctx->num_sms = prop.multiProcessorCount;
+  if (const char* env = getenv("QDIT_PDL")) ctx->overlap_launches = atoi(env) != 0;
   if (cudaMalloc(&ctx->d_status, sizeof(int)) != cudaSuccess ||
       cudaMemset(ctx->d_status, 0, sizeof(int)) != cudaSuccess ||
       cudaMallocHost(&ctx->h_status, sizeof(int)) != cudaSuccess) {

@@ -73,6 +73,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
+  // everything above touched only this CTA's shared and tensor memory; from here on the kernel reads what
+  // the previous kernel of the stream wrote
+  grid_dependency_wait();
+  grid_dependency_release();
 
   const int num_kb = (p.K + BK - 1) / BK;
   const int total_tiles = p.num_m_tiles * p.num_n_tiles;
@@ -180,7 +184,7 @@ int32_t launch_gemm_epi(qdit_ctx* ctx, const void* A, const void* W, GemmParams&
   const int grid = total < ctx->num_sms ? total : ctx->num_sms;
   const uint32_t idesc = umma_idesc_i8(BM, BN, a_unsigned);
   ProfScope prof(ctx, QDIT_PROF_GEMM, 2.0 * p.M * static_cast<double>(p.N) * p.K);
-  gemm_i8_kernel<BN, EPI><<<grid, NUM_THREADS, C::SMEM_BYTES, ctx->stream>>>(ta, tw, p, idesc);
+  QDIT_CUDA_CHECK(ctx, qdit_launch_overlapped(ctx, gemm_i8_kernel<BN, EPI>, dim3(grid), dim3(NUM_THREADS), C::SMEM_BYTES, ta, tw, p, idesc));
   return qdit_after_launch(ctx, "gemm_i8_kernel");
 }
 

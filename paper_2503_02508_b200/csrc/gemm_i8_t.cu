@@ -278,6 +278,9 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
+  // the preamble above used only this CTA's shared and tensor memory; global memory is read from here on
+  grid_dependency_wait();
+  grid_dependency_release();
 
   const int num_kb = (p.K + BK - 1) / BK;
   // tiles: channel block fastest, so CTAs running together share the activation tile
@@ -419,7 +422,7 @@ int32_t launch_t_epi(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p,
   const uint32_t idesc = (2u << 4) | (1u << 7) | ((a_unsigned ? 0u : 1u) << 10) | ((static_cast<uint32_t>(BT) >> 3) << 17) |
                          ((static_cast<uint32_t>(BC) >> 4) << 24);
   ProfScope prof(ctx, QDIT_PROF_GEMM, 2.0 * p.M * static_cast<double>(p.N) * p.K);
-  gemm_i8_t_kernel<BT, EPI><<<grid, NUM_THREADS, C::SMEM_BYTES, ctx->stream>>>(tw, tx, p, idesc);
+  QDIT_CUDA_CHECK(ctx, qdit_launch_overlapped(ctx, gemm_i8_t_kernel<BT, EPI>, dim3(grid), dim3(NUM_THREADS), C::SMEM_BYTES, tw, tx, p, idesc));
   return qdit_after_launch(ctx, "gemm_i8_t_kernel");
 }
 

@@ -39,6 +39,7 @@ struct qdit_ctx {
   int* h_status = nullptr;  // pinned host mirror
   int num_sms = 0;
   int64_t launches = 0;
+  bool overlap_launches = true;  // programmatic dependent launch for the kernels that support it (QDIT_PDL=0 turns it off)
   std::string last_error;
   void* encode_fn = nullptr;  // cuTensorMapEncodeTiled
   std::unordered_map<TmapKey, CUtensorMap, TmapKeyHash> tmaps;
@@ -57,6 +58,25 @@ struct ProfScope {
   ProfScope(qdit_ctx* c, int kind, double work);
   ~ProfScope();
 };
+
+// Launches `kernel` on the context's stream.  With ctx->overlap_launches the launch carries the
+// programmatic-stream-serialization attribute: the kernel may start its preamble before the previous kernel
+// of the stream has finished, and MUST call grid_dependency_wait() before its first global-memory access.
+template <typename... KArgs, typename... Args>
+cudaError_t qdit_launch_overlapped(qdit_ctx* ctx, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                   Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = ctx->stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = ctx->overlap_launches ? 1 : 0;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 // Records a formatted message on the context and returns `code`.
 int32_t qdit_fail(qdit_ctx* ctx, int32_t code, const char* fmt, ...);

@@ -150,6 +150,8 @@ __global__ void __launch_bounds__(256) ln_modulate_kernel(const __nv_bfloat16* _
   const int64_t row_begin = static_cast<int64_t>(blockIdx.x) * rows_per_cta;
   const int64_t row_end = row_begin + rows_per_cta < M ? row_begin + rows_per_cta : M;
   if (row_begin >= M) return;
+  grid_dependency_wait();  // x and the modulation come from earlier kernels of the stream
+  grid_dependency_release();
   const int nvec = D >> 3;
   int64_t row = row_begin + warp;
   uint4 raw[NV], raw_next[NV];
@@ -241,8 +243,9 @@ void launch_ln(qdit_ctx* ctx, const void* x, int64_t M, int D, int64_t T, float 
   if (rows < 8) rows = 8;
   if (rows > T) rows = T;
   const unsigned grid = static_cast<unsigned>((M + rows - 1) / rows);
-  ln_modulate_kernel<NV><<<grid, 256, 4 * D * sizeof(float), ctx->stream>>>(
-      static_cast<const __nv_bfloat16*>(x), M, D, T, eps, shift, scale, ld_mod, out, out_dtype, qa, static_cast<int>(rows));
+  qdit_launch_overlapped(ctx, ln_modulate_kernel<NV>, dim3(grid), dim3(256), 4 * D * sizeof(float),
+                         static_cast<const __nv_bfloat16*>(x), M, D, T, eps, shift, scale, ld_mod, out, out_dtype, qa,
+                         static_cast<int>(rows));
 }
 
 }  // namespace
