@@ -186,7 +186,7 @@ __global__ void timestep_features_kernel(const float* __restrict__ t, float* __r
   feat[i] = static_cast<float>(j < half ? cos(arg) : sin(arg));
 }
 
-// out[b,n] = W[n,:] . f(in[b,:]) + bias[n] (+ table[y[b],n]), optionally passed through SiLU, and optionally
+// out[b,n] = W[n,:] . f(in[b,:]) + bias[n] (+ table[y[b % y_period],n]), optionally passed through SiLU, and optionally
 // SiLU(out) as a second output.  One CTA per 8 output features: the inputs of up to `bc` samples are copied
 // into shared memory with cp.async (all copies in flight at once: the copy is one L2 latency, not one per
 // loop trip), f is applied in place, then a warp keeps its weight row in registers and walks the samples.
@@ -195,7 +195,8 @@ __global__ void __launch_bounds__(256) small_linear_kernel(const float* __restri
                                                            const float* __restrict__ bias,
                                                            const float* __restrict__ table, const int32_t* __restrict__ y,
                                                            float* __restrict__ out, float* __restrict__ out_silu, int B,
-                                                           int N, int K, int bc, int silu_input, int silu_output) {
+                                                           int N, int K, int bc, int silu_input, int silu_output,
+                                                           int y_period) {
   extern __shared__ float s_in[];  // [bc][K]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n = blockIdx.x * (blockDim.x >> 5) + warp;
@@ -241,13 +242,103 @@ __global__ void __launch_bounds__(256) small_linear_kernel(const float* __restri
         if (lane == 0) {
           const int64_t o = static_cast<int64_t>(b0 + b) * N + n;
           float v = acc + bias[n];
-          if (table) v += table[static_cast<int64_t>(y[b0 + b]) * N + n];
+          if (table) v += table[static_cast<int64_t>(y[(b0 + b) % y_period]) * N + n];
           if (silu_output) v = silu_f(v);
           out[o] = v;
           if (out_silu) out_silu[o] = silu_f(v);
         }
       }
     }
+  }
+}
+
+// The same linear for many rows (the conditioning of a whole trajectory): a register-tiled f32 GEMM,
+// out[r, n] = g(sum_k f(in[r, k]) W[n, k] + bias[n] (+ table[y[r % y_period], n])).  Tiles of 128 rows x 64 features
+// x 16 k; each thread owns 8 x 4 outputs and sums over k in ascending order, so an output's value does not
+// depend on how many rows the call has or where the row sits.
+constexpr int BL_BM = 128, BL_BN = 64, BL_BK = 16;
+__global__ void __launch_bounds__(256) batched_linear_kernel(const float* __restrict__ in, const float* __restrict__ w,
+                                                             const float* __restrict__ bias, const float* __restrict__ table,
+                                                             const int32_t* __restrict__ y, float* __restrict__ out,
+                                                             float* __restrict__ out_silu, int R, int N, int K, int silu_input,
+                                                             int silu_output, int y_period) {
+  __shared__ __align__(16) float sA[2][BL_BK][BL_BM + 4];
+  __shared__ __align__(16) float sW[2][BL_BK][BL_BN + 4];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int r0 = blockIdx.y * BL_BM, n0 = blockIdx.x * BL_BN;
+  const int lr = tid >> 2, lk = (tid & 3) * 4;  // loader coordinates: row (or feature) within the tile, k offset
+  float4 ra[2], rw;
+  auto load = [&](int k0) {
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int r = r0 + lr + 64 * j;
+      ra[j] = r < R ? *reinterpret_cast<const float4*>(in + static_cast<int64_t>(r) * K + k0 + lk) : make_float4(0.f, 0.f, 0.f, 0.f);
+      if (silu_input) { ra[j].x = silu_f(ra[j].x); ra[j].y = silu_f(ra[j].y); ra[j].z = silu_f(ra[j].z); ra[j].w = silu_f(ra[j].w); }
+    }
+    const int n = n0 + lr;
+    rw = n < N ? *reinterpret_cast<const float4*>(w + static_cast<int64_t>(n) * K + k0 + lk) : make_float4(0.f, 0.f, 0.f, 0.f);
+  };
+  auto stash = [&](int buf) {
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      sA[buf][lk + 0][lr + 64 * j] = ra[j].x;
+      sA[buf][lk + 1][lr + 64 * j] = ra[j].y;
+      sA[buf][lk + 2][lr + 64 * j] = ra[j].z;
+      sA[buf][lk + 3][lr + 64 * j] = ra[j].w;
+    }
+    sW[buf][lk + 0][lr] = rw.x;
+    sW[buf][lk + 1][lr] = rw.y;
+    sW[buf][lk + 2][lr] = rw.z;
+    sW[buf][lk + 3][lr] = rw.w;
+  };
+  float acc[8][4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
+  load(0);
+  stash(0);
+  __syncthreads();
+  const int nk = K / BL_BK;
+  for (int kb = 0; kb < nk; ++kb) {
+    const int buf = kb & 1;
+    if (kb + 1 < nk) load((kb + 1) * BL_BK);
+#pragma unroll
+    for (int k = 0; k < BL_BK; ++k) {
+      const float4 a0 = *reinterpret_cast<const float4*>(&sA[buf][k][ty * 8]);
+      const float4 a1 = *reinterpret_cast<const float4*>(&sA[buf][k][ty * 8 + 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&sW[buf][k][tx * 4]);
+      const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+      const float bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+    if (kb + 1 < nk) {
+      stash(buf ^ 1);  // the other buffer was last read before the previous barrier
+      __syncthreads();
+    }
+  }
+  const int n = n0 + tx * 4;
+  if (n >= N) return;
+  const float4 bz = *reinterpret_cast<const float4*>(bias + n);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = r0 + ty * 8 + i;
+    if (r >= R) break;
+    float v[4] = {acc[i][0] + bz.x, acc[i][1] + bz.y, acc[i][2] + bz.z, acc[i][3] + bz.w};
+    if (table) {
+      const float4 tv = *reinterpret_cast<const float4*>(table + static_cast<int64_t>(y[r % y_period]) * N + n);
+      v[0] += tv.x; v[1] += tv.y; v[2] += tv.z; v[3] += tv.w;
+    }
+    if (silu_output) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) v[j] = silu_f(v[j]);
+    }
+    const int64_t o = static_cast<int64_t>(r) * N + n;
+    *reinterpret_cast<float4*>(out + o) = make_float4(v[0], v[1], v[2], v[3]);
+    if (out_silu) *reinterpret_cast<float4*>(out_silu + o) = make_float4(silu_f(v[0]), silu_f(v[1]), silu_f(v[2]), silu_f(v[3]));
   }
 }
 
@@ -387,7 +478,7 @@ int32_t launch_embed(qdit_ctx* ctx, const float* latent, int latent_batch, const
 
 int32_t launch_small_linear(qdit_ctx* ctx, const float* in, const float* w, const float* bias, const float* table,
                             const int32_t* y, float* out, float* out_silu, int B, int N, int K, int silu_input,
-                            int silu_output) {
+                            int silu_output, int y_period) {
   if (K % 4 != 0 || K > 128 * SL_MAXV) return qdit_fail(ctx, QDIT_ERR_SHAPE, "small linear needs K %% 4 == 0 and K <= %d", 128 * SL_MAXV);
   if (!aligned16(in) || !aligned16(w)) return qdit_fail(ctx, QDIT_ERR_ALIGN, "small linear operands must be 16-byte aligned");
   const int smem_budget = 160 * 1024;
@@ -402,16 +493,36 @@ int32_t launch_small_linear(qdit_ctx* ctx, const float* in, const float* w, cons
   }
   ProfScope prof(ctx, QDIT_PROF_OTHER, static_cast<double>(N) * K * 4.0);
   small_linear_kernel<<<static_cast<unsigned>((N + 7) / 8), 256, smem, ctx->stream>>>(in, w, bias, table, y, out, out_silu, B, N,
-                                                                                    K, bc, silu_input, silu_output);
+                                                                                    K, bc, silu_input, silu_output,
+                                                                                    y_period > 0 ? y_period : B);
   return qdit_after_launch(ctx, "small_linear_kernel");
+}
+
+int32_t launch_batched_linear(qdit_ctx* ctx, const float* in, const float* w, const float* bias, const float* table,
+                              const int32_t* y, float* out, float* out_silu, int R, int N, int K, int silu_input,
+                              int silu_output, int y_period) {
+  if (K % BL_BK != 0 || N % 4 != 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "batched linear needs K %% 16 == 0 and N %% 4 == 0");
+  if (!aligned16(in) || !aligned16(w) || !aligned16(bias) || !aligned16(out) || (table && !aligned16(table)) ||
+      (out_silu && !aligned16(out_silu)))
+    return qdit_fail(ctx, QDIT_ERR_ALIGN, "batched linear operands must be 16-byte aligned");
+  if (R <= 0) return QDIT_OK;
+  ProfScope prof(ctx, QDIT_PROF_OTHER, static_cast<double>(N) * K * 4.0);
+  dim3 grid(static_cast<unsigned>((N + BL_BN - 1) / BL_BN), static_cast<unsigned>((R + BL_BM - 1) / BL_BM));
+  batched_linear_kernel<<<grid, 256, 0, ctx->stream>>>(in, w, bias, table, y, out, out_silu, R, N, K, silu_input, silu_output,
+                                                       y_period > 0 ? y_period : R);
+  return qdit_after_launch(ctx, "batched_linear_kernel");
+}
+
+int32_t launch_timestep_features(qdit_ctx* ctx, const float* t, float* feat, int B, int F) {
+  timestep_features_kernel<<<(B * F + 255) / 256, 256, 0, ctx->stream>>>(t, feat, B, F);
+  return qdit_after_launch(ctx, "timestep_features_kernel");
 }
 
 // h[b,:] = SiLU(W1 . sinusoid(t_b) + b1); feat: scratch [B, F]
 int32_t launch_cond1(qdit_ctx* ctx, const float* t, const float* w1, const float* b1, float* feat, float* h, int B, int D,
                      int F) {
-  timestep_features_kernel<<<(B * F + 255) / 256, 256, 0, ctx->stream>>>(t, feat, B, F);
-  QDIT_TRY(qdit_after_launch(ctx, "timestep_features_kernel"));
-  return launch_small_linear(ctx, feat, w1, b1, nullptr, nullptr, h, nullptr, B, D, F, 0, 1);
+  QDIT_TRY(launch_timestep_features(ctx, t, feat, B, F));
+  return launch_small_linear(ctx, feat, w1, b1, nullptr, nullptr, h, nullptr, B, D, F, 0, 1, 0);
 }
 
 int32_t launch_final(qdit_ctx* ctx, const void* x, int64_t M, int D, int T, float eps, const float* modf,

@@ -9,14 +9,20 @@ struct DdimCoef {
 // x[m,:] = bf16(W_patch . patch(m) + b + pos); sample b reads latent[b % latent_batch]; wT = W_patch transposed [pd][D].
 int32_t launch_embed(qdit_ctx* ctx, const float* latent, int latent_batch, const float* wT, const float* bias,
                      const float* pos, void* x, int64_t M, int D, int grid, int patch, int C);
+// feat[b, :] = (cos(t_b w_j), sin(t_b w_j)), w_j = 10000^(-j / (F/2))
+int32_t launch_timestep_features(qdit_ctx* ctx, const float* t, float* feat, int B, int F);
 // h[b,:] = SiLU(W1 . sinusoid(t_b) + b1); feat is scratch [B, F]
 int32_t launch_cond1(qdit_ctx* ctx, const float* t, const float* w1, const float* b1, float* feat, float* h, int B, int D,
                      int F);
-// out[b,n] = g(W[n,:] . f(in[b,:]) + bias[n] (+ table[y[b],n])); f = SiLU if silu_input, g = SiLU if silu_output;
-// out_silu (optional) = SiLU(out)
+// out[b,n] = g(W[n,:] . f(in[b,:]) + bias[n] (+ table[y[b % y_period],n])); f = SiLU if silu_input, g = SiLU if
+// silu_output; out_silu (optional) = SiLU(out); y_period 0 means B (one label per row)
 int32_t launch_small_linear(qdit_ctx* ctx, const float* in, const float* w, const float* bias, const float* table,
                             const int32_t* y, float* out, float* out_silu, int B, int N, int K, int silu_input,
-                            int silu_output);
+                            int silu_output, int y_period);
+// The same operation as launch_small_linear for many rows (register-tiled f32 GEMM; K % 16 == 0, N % 4 == 0).
+int32_t launch_batched_linear(qdit_ctx* ctx, const float* in, const float* w, const float* bias, const float* table,
+                              const int32_t* y, float* out, float* out_silu, int R, int N, int K, int silu_input,
+                              int silu_output, int y_period);
 // LayerNorm + modulate + linear D->OUT + un-patchify into net [B, OUT/p^2, side, side]
 int32_t launch_final(qdit_ctx* ctx, const void* x, int64_t M, int D, int T, float eps, const float* modf,
                      const float* w, const float* bias, float* net, int grid, int patch, int OUT);

@@ -1,6 +1,7 @@
 // Model (quantized weights + activation scales) and sampler (workspace, cache, trajectory state):
 // host-side orchestration of one network evaluation and of one denoising step.
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -66,6 +67,11 @@ struct qdit_sampler {
   float* dyn_absmax;             // [1 + 4*depth] this pass's ranges (calibration)
   float* dyn_scale;              // [1 + 4*depth] and the scales derived from them
   float* vc_table;               // device [S, C] or null
+  // Conditioning of the whole trajectory, evaluated at step 0: the conditioning vector, and with it every block's
+  // modulation, depends on the timestep and the label only, never on the latent.  Rows are (step, sample).
+  float *traj_c, *traj_sc, *traj_hidden, *traj_feat, *traj_mod, *traj_modf;
+  uint8_t* traj_ca;
+  bool traj_cond;                // buffers allocated (the trajectory's modulation fits the memory budget)
   qdit_cache* cache;
   std::vector<DdimCoef> ddim;
   std::vector<float> t_host;
@@ -189,8 +195,11 @@ int32_t dyn_quant(qdit_ctx* ctx, qdit_sampler* s, int slot, const float* x, int6
 
 }  // namespace
 
+// `pre_mod` / `pre_modf`: modulation [B, depth*6D] and final-layer modulation [B, 2D] evaluated beforehand for this
+// step (both or neither); without them the conditioning path runs here.
 static int32_t forward_impl(qdit_ctx* ctx, qdit_sampler* s, const float* latent, int latent_batch, const float* t,
-                            const int32_t* y, int B, float* out, uint32_t flags) {
+                            const int32_t* y, int B, float* out, uint32_t flags, const float* pre_mod = nullptr,
+                            const float* pre_modf = nullptr) {
   qdit_model* m = s->model;
   const qdit_model_shape& sh = m->s;
   const int D = sh.hidden, F = sh.mlp, T = sh.grid * sh.grid, depth = sh.depth;
@@ -204,24 +213,26 @@ static int32_t forward_impl(qdit_ctx* ctx, qdit_sampler* s, const float* latent,
   const float* scales = calib ? s->dyn_scale : m->d_scales;
 
   QDIT_TRY(launch_embed(ctx, latent, latent_batch, m->w_patch, m->b_patch, m->pos, s->x, M, D, sh.grid, sh.patch, sh.channels));
-  QDIT_TRY(launch_cond1(ctx, t, m->w_t1, m->b_t1, s->feat, s->hidden, B, D, sh.freq_dim));
-  QDIT_TRY(launch_small_linear(ctx, s->hidden, m->w_t2, m->b_t2, m->y_table, y, s->c, s->sc, B, D, D, 0, 0));
-  // modulation of every block in one stacked GEMM (the conditioning does not depend on the tokens)
-  if (calib) {
-    QDIT_TRY(dyn_quant(ctx, s, 0, s->sc, B, D, s->ca));
-  } else {
-    QDIT_TRY(qdit_quantize_act_dev(ctx, s->sc, B, D, sym_qp(), scales + 0, s->ca));
-  }
-  {
+  const float* mod_all = pre_mod;
+  if (!pre_mod) {
+    QDIT_TRY(launch_cond1(ctx, t, m->w_t1, m->b_t1, s->feat, s->hidden, B, D, sh.freq_dim));
+    QDIT_TRY(launch_small_linear(ctx, s->hidden, m->w_t2, m->b_t2, m->y_table, y, s->c, s->sc, B, D, D, 0, 0, 0));
+    // modulation of every block in one stacked GEMM (the conditioning does not depend on the tokens)
+    if (calib) {
+      QDIT_TRY(dyn_quant(ctx, s, 0, s->sc, B, D, s->ca));
+    } else {
+      QDIT_TRY(qdit_quantize_act_dev(ctx, s->sc, B, D, sym_qp(), scales + 0, s->ca));
+    }
     qdit_epilogue epi{};
     QDIT_TRY(run_linear(ctx, s->ca, m->ada_all, B, scales + 0, QDIT_EPI_OUT_F32, epi, s->mod));
+    mod_all = s->mod;
   }
 
   if (reuse) {
-    QDIT_TRY(qdit_cache_reuse_all(ctx, s->cache, s->mod, ld_mod, T, s->x));
+    QDIT_TRY(qdit_cache_reuse_all(ctx, s->cache, mod_all, ld_mod, T, s->x));
   } else {
     for (int i = 0; i < depth; ++i) {
-      const float* mod = s->mod + static_cast<int64_t>(i) * 6 * D;
+      const float* mod = mod_all + static_cast<int64_t>(i) * 6 * D;
       const float* sc_qkv = scales + 1 + 4 * i;
       const float* sc_proj = sc_qkv + 1;
       const float* sc_fc1 = sc_qkv + 2;
@@ -278,10 +289,27 @@ static int32_t forward_impl(qdit_ctx* ctx, qdit_sampler* s, const float* latent,
     }
   }
   // final layer (f32): modulation from SiLU(c), LayerNorm, linear, un-patchify
-  QDIT_TRY(launch_small_linear(ctx, s->c, m->w_ada_f, m->b_ada_f, nullptr, nullptr, s->modf, nullptr, B, 2 * D, D, 1, 0));
-  QDIT_TRY(launch_final(ctx, s->x, M, D, T, 1e-6f, s->modf, m->w_out, m->b_out, out, sh.grid, sh.patch,
+  if (!pre_modf) QDIT_TRY(launch_small_linear(ctx, s->c, m->w_ada_f, m->b_ada_f, nullptr, nullptr, s->modf, nullptr, B, 2 * D, D, 1, 0, 0));
+  QDIT_TRY(launch_final(ctx, s->x, M, D, T, 1e-6f, pre_modf ? pre_modf : s->modf, m->w_out, m->b_out, out, sh.grid, sh.patch,
                         2 * sh.channels * sh.patch * sh.patch));
   return QDIT_OK;
+}
+
+// Conditioning and modulation of every step of the trajectory in one batch of S * Beff rows (step-major).
+static int32_t trajectory_conditioning(qdit_ctx* ctx, qdit_sampler* s) {
+  qdit_model* m = s->model;
+  const qdit_model_shape& sh = m->s;
+  const int D = sh.hidden, rows = s->d.num_steps * s->Beff;
+  if (!m->scales_set) return qdit_fail(ctx, QDIT_ERR_STATE, "activation scales are not set (set them or calibrate)");
+  QDIT_TRY(launch_timestep_features(ctx, s->t_all, s->traj_feat, rows, sh.freq_dim));
+  QDIT_TRY(launch_batched_linear(ctx, s->traj_feat, m->w_t1, m->b_t1, nullptr, nullptr, s->traj_hidden, nullptr, rows, D,
+                                 sh.freq_dim, 0, 1, 0));
+  QDIT_TRY(launch_batched_linear(ctx, s->traj_hidden, m->w_t2, m->b_t2, m->y_table, s->y, s->traj_c, s->traj_sc, rows, D, D, 0, 0,
+                                 s->Beff));
+  QDIT_TRY(qdit_quantize_act_dev(ctx, s->traj_sc, rows, D, sym_qp(), m->d_scales + 0, s->traj_ca));
+  qdit_epilogue epi{};
+  QDIT_TRY(run_linear(ctx, s->traj_ca, m->ada_all, rows, m->d_scales + 0, QDIT_EPI_OUT_F32, epi, s->traj_mod));
+  return launch_batched_linear(ctx, s->traj_c, m->w_ada_f, m->b_ada_f, nullptr, nullptr, s->traj_modf, nullptr, rows, 2 * D, D, 1, 0, 0);
 }
 
 extern "C" {
@@ -430,7 +458,25 @@ int32_t qdit_sampler_create(qdit_ctx* ctx, qdit_model* m, const qdit_sampler_des
   s->tmpf = a.alloc<float>(M * F);
   s->dyn_absmax = a.alloc<float>(m->n_scales());
   s->dyn_scale = a.alloc<float>(m->n_scales());
-  bool ok = s->x && s->qkv && s->h && s->a && s->u && s->ca && s->c && s->sc && s->hidden && s->feat && s->mod && s->modf && s->net &&
+  // whole-trajectory conditioning when its modulation table fits 4 GB; otherwise it is evaluated step by step
+  bool traj_ok = true;
+  {
+    const int64_t rows = B * d->num_steps;
+    s->traj_cond = rows * sh.depth * 6 * D * static_cast<int64_t>(sizeof(float)) <= (int64_t(4) << 30) && !getenv("QDIT_STEPWISE_CONDITIONING");
+    s->traj_c = s->traj_sc = s->traj_hidden = s->traj_feat = s->traj_mod = s->traj_modf = nullptr;
+    s->traj_ca = nullptr;
+    if (s->traj_cond) {
+      s->traj_c = a.alloc<float>(rows * D);
+      s->traj_sc = a.alloc<float>(rows * D);
+      s->traj_hidden = a.alloc<float>(rows * D);
+      s->traj_feat = a.alloc<float>(rows * sh.freq_dim);
+      s->traj_mod = a.alloc<float>(rows * sh.depth * 6 * D);
+      s->traj_modf = a.alloc<float>(rows * 2 * D);
+      s->traj_ca = a.alloc<uint8_t>(rows * D);
+      if (!s->traj_c || !s->traj_sc || !s->traj_hidden || !s->traj_feat || !s->traj_mod || !s->traj_modf || !s->traj_ca) traj_ok = false;
+    }
+  }
+  bool ok = traj_ok && s->x && s->qkv && s->h && s->a && s->u && s->ca && s->c && s->sc && s->hidden && s->feat && s->mod && s->modf && s->net &&
             s->latent && s->t_all && s->y && s->labels && s->tmpf && s->dyn_absmax && s->dyn_scale;
   if (ok && d->vc_mode != QDIT_VC_NONE) {
     s->vc_table = a.alloc<float>(static_cast<int64_t>(d->num_steps) * C);
@@ -535,7 +581,15 @@ int32_t qdit_sample_step(qdit_ctx* ctx, qdit_sampler* s, int i) {
   const int HW = sh.grid * sh.patch * sh.grid * sh.patch, B = s->d.batch;
   uint32_t flags = 0;
   if (s->d.cache_interval > 1) flags = qdit_cache_should_refresh(i, s->d.cache_interval) ? QDIT_FWD_STORE_CACHE : QDIT_FWD_REUSE;
-  QDIT_TRY(forward_impl(ctx, s, s->latent, B, s->t_all + static_cast<int64_t>(i) * s->Beff, s->y, s->Beff, s->net, flags));
+  const float *pre_mod = nullptr, *pre_modf = nullptr;
+  if (s->traj_cond) {
+    if (i == 0) QDIT_TRY(trajectory_conditioning(ctx, s));
+    const int64_t row0 = static_cast<int64_t>(i) * s->Beff;
+    pre_mod = s->traj_mod + row0 * sh.depth * 6 * sh.hidden;
+    pre_modf = s->traj_modf + row0 * 2 * sh.hidden;
+  }
+  QDIT_TRY(forward_impl(ctx, s, s->latent, B, s->t_all + static_cast<int64_t>(i) * s->Beff, s->y, s->Beff, s->net, flags, pre_mod,
+                        pre_modf));
   QDIT_TRY(launch_cfg_ddim(ctx, s->latent, s->net, B, sh.channels, HW, s->d.use_cfg, s->d.guidance, s->ddim[i]));
   if (s->d.vc_mode != QDIT_VC_NONE)
     QDIT_TRY(qdit_vc_correct(ctx, s->latent, B, sh.channels, HW, i, s->d.vc_mode, s->vc_table, s->d.vc_eps));

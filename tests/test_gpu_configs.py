@@ -151,10 +151,11 @@ def test_ddim50_guided_cached_sampler_batch16(q, ctx, xl256):
         print(f"ddim50 step {i} latent rel-L2 vs oracle: {err:.3e}")
         assert err < 2e-2, (i, err)
     assert np.isfinite(final).all()
-    # launch accounting: refresh steps run 7 kernels per block, reuse steps one kernel for all blocks
-    per_refresh = 6 + 7 * cfg.depth + 2 + 2          # network + guidance/DDIM + VC
-    per_reuse = 6 + 1 + 2 + 2
-    assert launches == 25 * per_refresh + 25 * per_reuse
+    # launch accounting: the conditioning of all steps is evaluated once (6 kernels); refresh steps run 7 kernels
+    # per block, reuse steps one kernel for all blocks
+    per_refresh = 1 + 7 * cfg.depth + 1 + 2          # embed + blocks + final layer + guidance/DDIM + VC
+    per_reuse = 1 + 1 + 1 + 2
+    assert launches == 6 + 25 * per_refresh + 25 * per_reuse
     # batch independence over the WHOLE trajectory: image 7 alone gives bit-identical latents
     _, final1, _ = _gpu_trajectory(q, ctx, xl256, latent[7:8], labels[7:8], S, interval, guidance, K, set())
     np.testing.assert_array_equal(final1, final[7:8])
@@ -182,7 +183,7 @@ def test_ddim100_512_cached_sampler_batch8(q, ctx):
             print(f"ddim100_512 step {i} latent rel-L2 vs oracle: {err:.3e}")
             assert err < 2e-2, (i, err)
         assert np.isfinite(final).all()
-        assert launches == 34 * (6 + 7 * cfg.depth + 2 + 2) + 66 * (6 + 1 + 2 + 2)
+        assert launches == 6 + 34 * (1 + 7 * cfg.depth + 1 + 2) + 66 * (1 + 1 + 1 + 2)
         _, final1, _ = _gpu_trajectory(q, ctx, rig, latent[2:3], labels[2:3], S, interval, None, K, set())
         np.testing.assert_array_equal(final1, final[2:3])
     finally:
