@@ -353,19 +353,26 @@ __device__ __forceinline__ uint2 pack_codes8_i(const int (&c)[8]) {
 // clip(rne(t) + z, qmin, qmax) == rne(clamp(t, qmin - z, qmax - z)) + z because the bounds are integers, and
 // adding 1.5 * 2^23 to a float of magnitude < 2^22 rounds it to the nearest integer (ties to even) and
 // leaves that integer in the low mantissa bits.  Same codes as quantize_code for every input (NaN -> qmin).
-__device__ __forceinline__ uint2 quantize_pack8(const float (&x)[8], float inv_scale, float zp, float qmin, float qmax) {
+// quantize_pack8_scaled takes t = x / s already formed.
+__device__ __forceinline__ uint2 quantize_pack8_scaled(const float (&t)[8], float zp, float qmin, float qmax) {
   const float lo_f = qmin - zp, hi_f = qmax - zp;
   const int z = static_cast<int>(zp);
   uint32_t m[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    const float t = fminf(fmaxf(__fmul_rn(x[i], inv_scale), lo_f), hi_f);
-    m[i] = static_cast<uint32_t>(__float_as_int(__fadd_rn(t, 12582912.0f)) + z);
+    const float c = fminf(fmaxf(t[i], lo_f), hi_f);
+    m[i] = static_cast<uint32_t>(__float_as_int(__fadd_rn(c, 12582912.0f)) + z);
   }
   uint2 r;
   r.x = __byte_perm(__byte_perm(m[0], m[1], 0x0040), __byte_perm(m[2], m[3], 0x0040), 0x5410);
   r.y = __byte_perm(__byte_perm(m[4], m[5], 0x0040), __byte_perm(m[6], m[7], 0x0040), 0x5410);
   return r;
+}
+__device__ __forceinline__ uint2 quantize_pack8(const float (&x)[8], float inv_scale, float zp, float qmin, float qmax) {
+  float t[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) t[i] = __fmul_rn(x[i], inv_scale);
+  return quantize_pack8_scaled(t, zp, qmin, qmax);
 }
 __device__ __forceinline__ uint4 pack_bf16x8(const float (&y)[8]) {
   return make_uint4(pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]), pack_bf16x2(y[4], y[5]), pack_bf16x2(y[6], y[7]));

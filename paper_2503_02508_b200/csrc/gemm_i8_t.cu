@@ -11,9 +11,9 @@
 // tile be 256 wide (one MMA of N = 256) and makes every DiT-XL/2 layer width (multiples of 128 channels)
 // tile without remainder.
 //
-// CTA = 2 + NUM_EPI_WARPS warps, roles and barriers as in gemm_i8.cu: warp 0 lane 0 TMA producer (weight
+// CTA = 2 + T_EPI_WARPS warps, roles and barriers as in gemm_i8.cu: warp 0 lane 0 TMA producer (weight
 // tile 128 x 128 B as operand A, activation tile BT x 128 B as operand B, both K-major, 128B swizzle), warp 1
-// lane 0 MMA issuer (two TMEM accumulator stages of BT columns), epilogue warps: EPI_SPLIT per lane quadrant,
+// lane 0 MMA issuer (two TMEM accumulator stages of BT columns), epilogue warps: T_EPI_SPLIT per lane quadrant,
 // taking 32-token chunks in turn.
 #include "gemm_common.cuh"
 
@@ -22,6 +22,14 @@ namespace {
 using namespace qgemm;
 
 constexpr int BC = 128;  // channels per tile = TMEM lanes
+// This kernel has no per-warp staging buffer, so its epilogue can be wider than the token-major kernel's:
+// 16 warps = 4 per lane quadrant, which also divides the 8 (or 4) token chunks of a tile evenly.
+#ifndef QDIT_T_EPI_WARPS
+#define QDIT_T_EPI_WARPS 12
+#endif
+constexpr int T_EPI_WARPS = QDIT_T_EPI_WARPS;
+constexpr int T_EPI_SPLIT = T_EPI_WARPS / 4;
+constexpr int T_NUM_THREADS = 64 + T_EPI_WARPS * 32;
 
 template <int BT>
 struct TCfg {
@@ -239,7 +247,7 @@ __device__ __forceinline__ void epilogue_chunk_t_gated(const GemmParams& p, cons
 }
 
 template <int BT, int EPI>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(T_NUM_THREADS, 1)
 gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                  const GemmParams p, const uint32_t idesc) {
   using C = TCfg<BT>;
@@ -265,7 +273,7 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&tfull_bar[s], 1);
-      mbar_init(&tempty_bar[s], NUM_EPI_WARPS);
+      mbar_init(&tempty_bar[s], T_EPI_WARPS);
     }
     *abort_flag = 0;
     mbar_fence_init();
@@ -342,13 +350,13 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     // -------------------------------------------------------------------- epilogue warps
     const int e = warp - 2;
     const int quad = warp & 3;   // TMEM lane quadrant = 32 channels
-    const int part = e >> 2;     // this warp takes token chunks part, part + EPI_SPLIT, ...
+    const int part = e >> 2;     // this warp takes token chunks part, part + T_EPI_SPLIT, ...
     const uint32_t flags = epi_flags<EPI>(p);
     const float a_scale = p.a_scale_dev ? __ldg(p.a_scale_dev) : p.a_scale;
     float o_inv = 0.0f;
     if (flags & QDIT_EPI_QUANT_OUT) o_inv = __fdiv_rn(1.0f, p.o_scale_dev ? __ldg(p.o_scale_dev) : p.o_scale);
     constexpr int CHUNKS = BT / 32;
-    const int c_last = part < CHUNKS ? part + ((CHUNKS - 1 - part) / EPI_SPLIT) * EPI_SPLIT : -1;
+    const int c_last = part < CHUNKS ? part + ((CHUNKS - 1 - part) / T_EPI_SPLIT) * T_EPI_SPLIT : -1;
     int it = 0;
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
       const int as = it & 1;
@@ -375,7 +383,7 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
         continue;
       }
 #pragma unroll 1
-      for (int c = part; c < CHUNKS; c += EPI_SPLIT) {
+      for (int c = part; c < CHUNKS; c += T_EPI_SPLIT) {
         uint32_t v[32];
         __syncwarp();
         tmem_ld_32x32(taddr + static_cast<uint32_t>(c * 32), v);
@@ -422,7 +430,7 @@ int32_t launch_t_epi(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p,
   const uint32_t idesc = (2u << 4) | (1u << 7) | ((a_unsigned ? 0u : 1u) << 10) | ((static_cast<uint32_t>(BT) >> 3) << 17) |
                          ((static_cast<uint32_t>(BC) >> 4) << 24);
   ProfScope prof(ctx, QDIT_PROF_GEMM, 2.0 * p.M * static_cast<double>(p.N) * p.K);
-  QDIT_CUDA_CHECK(ctx, qdit_launch_overlapped(ctx, gemm_i8_t_kernel<BT, EPI>, dim3(grid), dim3(NUM_THREADS), C::SMEM_BYTES, tw, tx, p, idesc));
+  QDIT_CUDA_CHECK(ctx, qdit_launch_overlapped(ctx, gemm_i8_t_kernel<BT, EPI>, dim3(grid), dim3(T_NUM_THREADS), C::SMEM_BYTES, tw, tx, p, idesc));
   return qdit_after_launch(ctx, "gemm_i8_t_kernel");
 }
 

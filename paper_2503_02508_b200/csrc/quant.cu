@@ -128,8 +128,12 @@ __global__ void __launch_bounds__(256) weight_quant_kernel(const float* __restri
 // ----------------------------------------------------------------------------- LayerNorm + modulate (+ quantize)
 // A CTA owns a contiguous range of rows; its 8 warps take the rows in turn, one warp per row, the row in
 // registers (NV vectors of 8 per lane), statistics two-pass in f32.  While a warp works on one row the next
-// row's loads are already in flight.  Shift and scale of the (at most two) samples the range touches are
-// copied to shared memory once per CTA; a row of any other sample falls back to global reads.
+// row's loads are already in flight.  The kernel is bound by instruction issue, so everything that does not
+// depend on the row is done once per CTA: for the (at most two) samples its range touches, the per-column
+// factors  mul = (1 + scale) / s_out  and  add = shift / s_out  (s_out = 1 unless the output is quantized) are
+// staged in shared memory, laid out so that a lane's 16-byte reads are conflict-free.  Per element that leaves
+// y / s_out = (x - mean) * (rstd * mul) + add: one multiply and one fused multiply-add.  A row of a third
+// sample (only when a sample has fewer rows than a CTA's minimum range) computes its factors from global memory.
 template <int NV>
 __device__ __forceinline__ void ln_load_row(const __nv_bfloat16* __restrict__ xr, int nvec, int lane, uint4 (&raw)[NV]) {
 #pragma unroll
@@ -140,43 +144,46 @@ __device__ __forceinline__ void ln_load_row(const __nv_bfloat16* __restrict__ xr
 }
 
 template <int NV>
-__global__ void __launch_bounds__(256) ln_modulate_kernel(const __nv_bfloat16* __restrict__ x, int64_t M, int D,
-                                                          int64_t T, float eps, const float* __restrict__ shift,
+__global__ void __launch_bounds__(256) ln_modulate_kernel(const __nv_bfloat16* __restrict__ x, int M, int D, int T,
+                                                          float eps, const float* __restrict__ shift,
                                                           const float* __restrict__ scale, int64_t ld_mod,
                                                           void* __restrict__ out, int out_dtype, QuantArgs qa,
                                                           int rows_per_cta) {
-  extern __shared__ float s_mod[];  // [2 samples][2][D]: shift, scale
+  extern __shared__ float4 s_par[];  // [2 samples][mul, add][NV][2 halves][32 lanes]
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-  const int64_t row_begin = static_cast<int64_t>(blockIdx.x) * rows_per_cta;
-  const int64_t row_end = row_begin + rows_per_cta < M ? row_begin + rows_per_cta : M;
+  const int row_begin = blockIdx.x * rows_per_cta;
+  const int row_end = row_begin + rows_per_cta < M ? row_begin + rows_per_cta : M;
   if (row_begin >= M) return;
   grid_dependency_wait();  // x and the modulation come from earlier kernels of the stream
   grid_dependency_release();
   const int nvec = D >> 3;
-  int64_t row = row_begin + warp;
+  int row = row_begin + warp;
   uint4 raw[NV], raw_next[NV];
-  if (row < row_end) ln_load_row<NV>(x + row * D, nvec, lane, raw);
-  const int64_t b0 = row_begin / T;
+  if (row < row_end) ln_load_row<NV>(x + static_cast<int64_t>(row) * D, nvec, lane, raw);
+  float inv = 1.0f;
+  if (out_dtype == QDIT_I8) inv = __fdiv_rn(1.0f, qa.scale_dev ? __ldg(qa.scale_dev) : qa.scale);
+  const int b0 = row_begin / T;
   for (int s = 0; s < 2; ++s) {
-    if ((b0 + s) * T >= row_end && s > 0) break;
-    const float4* gs = reinterpret_cast<const float4*>(shift + (b0 + s) * ld_mod);
-    const float4* gc = reinterpret_cast<const float4*>(scale + (b0 + s) * ld_mod);
-    float4* ss = reinterpret_cast<float4*>(s_mod + s * 2 * D);
-    float4* sc4 = reinterpret_cast<float4*>(s_mod + s * 2 * D + D);
-    for (int i = threadIdx.x; i < D / 4; i += blockDim.x) {
-      ss[i] = gs[i];
-      sc4[i] = gc[i];
+    if (static_cast<int64_t>(b0 + s) * T >= row_end) break;
+    const float* gs = shift + (b0 + s) * ld_mod;
+    const float* gc = scale + (b0 + s) * ld_mod;
+    for (int i = threadIdx.x; i < NV * 64; i += blockDim.x) {
+      const int l = i & 31, h = (i >> 5) & 1, j = i >> 6;
+      const int vi = l + 32 * j;
+      if (vi < nvec) {
+        const float4 c4 = *reinterpret_cast<const float4*>(gc + vi * 8 + 4 * h);
+        const float4 h4 = *reinterpret_cast<const float4*>(gs + vi * 8 + 4 * h);
+        s_par[(s * 2 + 0) * NV * 64 + i] = make_float4((1.0f + c4.x) * inv, (1.0f + c4.y) * inv, (1.0f + c4.z) * inv, (1.0f + c4.w) * inv);
+        s_par[(s * 2 + 1) * NV * 64 + i] = make_float4(h4.x * inv, h4.y * inv, h4.z * inv, h4.w * inv);
+      }
     }
   }
   __syncthreads();
-  float inv = 0.0f;
-  if (out_dtype == QDIT_I8) {
-    const float s = qa.scale_dev ? __ldg(qa.scale_dev) : qa.scale;
-    inv = __fdiv_rn(1.0f, s);
-  }
+  const float inv_d = 1.0f / static_cast<float>(D);
+  const int64_t second = static_cast<int64_t>(b0 + 1) * T;  // first row of the second staged sample
   for (; row < row_end; row += nwarps) {
-    const int64_t next = row + nwarps;
-    if (next < row_end) ln_load_row<NV>(x + next * D, nvec, lane, raw_next);
+    const int next = row + nwarps;
+    if (next < row_end) ln_load_row<NV>(x + static_cast<int64_t>(next) * D, nvec, lane, raw_next);
     float v[NV][8];
     float sum = 0.0f;
 #pragma unroll
@@ -190,36 +197,46 @@ __global__ void __launch_bounds__(256) ln_modulate_kernel(const __nv_bfloat16* _
         for (int i = 0; i < 8; ++i) sum += v[j][i];
       }
     }
-    const float mean = warp_sum(sum) / static_cast<float>(D);
+    const float mean = warp_sum(sum) * inv_d;
     float ssq = 0.0f;
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
       if (lane + 32 * j < nvec) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          const float d = v[j][i] - mean;
-          ssq += d * d;
+          v[j][i] -= mean;
+          ssq = fmaf(v[j][i], v[j][i], ssq);
         }
       }
     }
-    const float var = warp_sum(ssq) / static_cast<float>(D);
-    const float rstd = 1.0f / sqrtf(var + eps);
-    const int64_t b = row / T;
-    const bool staged = b - b0 < 2;
-    const float* sh = staged ? s_mod + (b - b0) * 2 * D : shift + b * ld_mod;
-    const float* sc = staged ? s_mod + (b - b0) * 2 * D + D : scale + b * ld_mod;
+    const float rstd = rsqrtf(warp_sum(ssq) * inv_d + eps);
+    const int sidx = row < second ? 0 : (row - second < T ? 1 : 2);
+    const float4* pm = s_par + (sidx * 2 + 0) * NV * 64 + lane;
+    const float4* pa = s_par + (sidx * 2 + 1) * NV * 64 + lane;
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
       const int vi = lane + 32 * j;
       if (vi < nvec) {
-        float shv[8], scv[8], y[8];
-        Load8<float>::load(sh + vi * 8, shv);
-        Load8<float>::load(sc + vi * 8, scv);
+        float mul[8], add[8], y[8];
+        if (sidx < 2) {
+          const float4 m0 = pm[j * 64], m1 = pm[j * 64 + 32], a0 = pa[j * 64], a1 = pa[j * 64 + 32];
+          mul[0] = m0.x; mul[1] = m0.y; mul[2] = m0.z; mul[3] = m0.w; mul[4] = m1.x; mul[5] = m1.y; mul[6] = m1.z; mul[7] = m1.w;
+          add[0] = a0.x; add[1] = a0.y; add[2] = a0.z; add[3] = a0.w; add[4] = a1.x; add[5] = a1.y; add[6] = a1.z; add[7] = a1.w;
+        } else {
+          const int b = row / T;
+          Load8<float>::load(scale + b * ld_mod + vi * 8, mul);
+          Load8<float>::load(shift + b * ld_mod + vi * 8, add);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) y[i] = (v[j][i] - mean) * rstd * (1.0f + scv[i]) + shv[i];
-        const int64_t o = row * D + vi * 8;
+          for (int i = 0; i < 8; ++i) {
+            mul[i] = (1.0f + mul[i]) * inv;
+            add[i] *= inv;
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) y[i] = fmaf(v[j][i], rstd * mul[i], add[i]);
+        const int64_t o = static_cast<int64_t>(row) * D + vi * 8;
         if (out_dtype == QDIT_I8) {
-          *reinterpret_cast<uint2*>(static_cast<uint8_t*>(out) + o) = quantize_pack8(y, inv, qa.zp, qa.qmin, qa.qmax);
+          *reinterpret_cast<uint2*>(static_cast<uint8_t*>(out) + o) = quantize_pack8_scaled(y, qa.zp, qa.qmin, qa.qmax);
         } else if (out_dtype == QDIT_BF16) {
           *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(out) + o) = pack_bf16x8(y);
         } else {
@@ -243,9 +260,9 @@ void launch_ln(qdit_ctx* ctx, const void* x, int64_t M, int D, int64_t T, float 
   if (rows < 8) rows = 8;
   if (rows > T) rows = T;
   const unsigned grid = static_cast<unsigned>((M + rows - 1) / rows);
-  qdit_launch_overlapped(ctx, ln_modulate_kernel<NV>, dim3(grid), dim3(256), 4 * D * sizeof(float),
-                         static_cast<const __nv_bfloat16*>(x), M, D, T, eps, shift, scale, ld_mod, out, out_dtype, qa,
-                         static_cast<int>(rows));
+  qdit_launch_overlapped(ctx, ln_modulate_kernel<NV>, dim3(grid), dim3(256), static_cast<size_t>(NV) * 4096,
+                         static_cast<const __nv_bfloat16*>(x), static_cast<int>(M), D, static_cast<int>(T), eps, shift, scale,
+                         ld_mod, out, out_dtype, qa, static_cast<int>(rows));
 }
 
 }  // namespace
@@ -335,6 +352,7 @@ int32_t qdit_adaln_modulate(qdit_ctx* ctx, const void* x, int64_t M, int64_t D, 
                             const qdit_qparams* out_qp, const float* out_scale_dev) {
   if (!ctx) return QDIT_ERR_INVALID_ARG;
   if (M < 0 || D <= 0 || T <= 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "bad sizes");
+  if (M > (int64_t(1) << 30) || T > (int64_t(1) << 30)) return qdit_fail(ctx, QDIT_ERR_SHAPE, "M and T must be at most 2^30");
   if (M == 0) return QDIT_OK;
   if (!x || !shift || !scale || !out) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "NULL argument");
   if (D % 8 != 0 || D > 2048) return qdit_fail(ctx, QDIT_ERR_SHAPE, "D must be a multiple of 8 and <= 2048");
