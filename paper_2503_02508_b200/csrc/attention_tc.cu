@@ -10,9 +10,14 @@
 // swizzle) plus a 16-column tail tile (32B swizzle, columns 64..79).  The tail's columns 72..79 belong to the
 // next head; they are zeroed in the Q tail, so they add nothing to S, and in V they only produce output
 // columns 72..79, which are dropped.
-// Warps 0-7: softmax (two threads per query row: both find the row maximum over the whole block, then each
-// exponentiates, stores and accumulates its half of the columns); warp 8 lane 0: TMA producer; warp 9 lane 0:
-// MMA issuer (warp 9 owns the TMEM allocation).  Two CTAs fit per SM (92 KB shared memory, 128 TMEM columns each) and overlap each other's phases.
+// Warps 0-7: softmax, two threads per query row: each reads its 64 columns of S, the two exchange their maxima
+// through shared memory, then each exponentiates, stores and accumulates its half.  Warp 8 lane 0: TMA producer;
+// warp 9 lane 0: MMA issuer (warp 9 owns the TMEM allocation).
+// S is double-buffered in tensor memory (2 x 128 columns): S of the next key block is issued as soon as its K
+// tile has landed, so it is computed while the softmax of the current block runs; O_blk of block j re-uses the
+// columns of S_j, is folded into the registers during the next block (after that block's row maximum is known),
+// and only then is the buffer handed back for S of block j + 2.
+// Two CTAs fit per SM (97 KB shared memory, 256 TMEM columns each) and overlap each other's phases.
 #include "common.cuh"
 #include "internal.h"
 
@@ -41,7 +46,7 @@ struct TCfg {
   static constexpr int TAIL_BYTES = TAIL ? 128 * 32 : 0;
   static constexpr int OP_BYTES = MAIN_BYTES + TAIL_BYTES;
   static constexpr int P_BYTES = 2 * MAIN_BYTES;        // 128 rows x 128 keys bf16 = two 64-key tiles
-  static constexpr int SMEM_BYTES = 3 * OP_BYTES + P_BYTES + 2048 + 1024;
+  static constexpr int SMEM_BYTES = 3 * OP_BYTES + P_BYTES + 4096 + 1024;
   static constexpr int O_COLS = TAIL ? 80 : 64;
   static constexpr int O_HALF = O_COLS / 2;             // accumulator columns per thread of a row pair (40 or 32)
 };
@@ -64,19 +69,21 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   uint8_t* sVt = sKt + C::TAIL_BYTES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(sVt + C::TAIL_BYTES);
   uint64_t* bar_q = bars + 0;      // Q tiles landed (tx)
-  uint64_t* bar_qz = bars + 1;     // Q tail padding zeroed (128 arrivals)
+  uint64_t* bar_qz = bars + 1;     // Q tail padding zeroed (256 arrivals)
   uint64_t* bar_kfull = bars + 2;  // K block landed (tx)
   uint64_t* bar_vfull = bars + 3;  // V block landed (tx)
   uint64_t* bar_kfree = bars + 4;  // S MMAs done reading K (commit)
   uint64_t* bar_vfree = bars + 5;  // PV MMAs done reading V and P (commit)
-  uint64_t* bar_s = bars + 6;      // S complete (commit)
-  uint64_t* bar_p = bars + 7;      // P written (128 arrivals)
-  uint64_t* bar_o = bars + 8;      // O_blk complete (commit)
-  uint64_t* bar_sfree = bars + 9;  // O_blk read: the accumulator columns may be overwritten (128 arrivals)
-  uint64_t* bar_l = bars + 10;     // row sums exchanged (256 arrivals)
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 11);
+  uint64_t* bar_s = bars + 6;      // [2] S complete in buffer 0 / 1 (commit)
+  uint64_t* bar_p = bars + 8;      // P written (256 arrivals)
+  uint64_t* bar_o = bars + 9;      // O_blk complete (commit)
+  uint64_t* bar_sfree = bars + 10; // O_blk folded: its buffer may take the S of two blocks later (256 arrivals)
+  uint64_t* bar_l = bars + 11;     // row sums exchanged (256 arrivals)
+  uint64_t* bar_mx = bars + 12;    // [4] row maxima exchanged between the two warps of a lane quadrant (64 arrivals)
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 16);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
   float* s_l = reinterpret_cast<float*>(tmem_holder + 4);  // [2][128] partial row sums
+  float* s_m = s_l + 256;                                  // [2 (block parity)][2][128] partial row maxima
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q0 = blockIdx.x * TQ, h = blockIdx.y, b = blockIdx.z;
@@ -90,16 +97,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     mbar_init(bar_vfull, 1);
     mbar_init(bar_kfree, 1);
     mbar_init(bar_vfree, 1);
-    mbar_init(bar_s, 1);
+    mbar_init(&bar_s[0], 1);
+    mbar_init(&bar_s[1], 1);
     mbar_init(bar_p, SM_WARPS * 32);
     mbar_init(bar_o, 1);
     mbar_init(bar_sfree, SM_WARPS * 32);
     mbar_init(bar_l, SM_WARPS * 32);
+    for (int i = 0; i < 4; ++i) mbar_init(&bar_mx[i], 64);
     *abort_flag = 0;
     mbar_fence_init();
   }
   if (warp == SM_WARPS + 1) {
-    tmem_alloc(tmem_holder, 128);
+    tmem_alloc(tmem_holder, 256);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -133,28 +142,40 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       const uint32_t id_s = umma_idesc_bf16(128, TK, false);
       const uint32_t id_o = umma_idesc_bf16(128, 64, true);
       const uint32_t id_ot = umma_idesc_bf16(128, 16, true);
-      bool ok = mbar_wait(bar_qz, 0, abort_flag, p.status);
-      for (int j = 0; j < n_blk && ok; ++j) {
-        const uint32_t ph = j & 1;
-        if (!mbar_wait(bar_kfull, ph, abort_flag, p.status)) break;
-        if (j > 0 && !mbar_wait(bar_sfree, (j - 1) & 1, abort_flag, p.status)) break;
-        tc_fence_after();
-        // S = Q K^T: 4 k-steps of 16 out of the 64-column tiles, one out of the tails
+      // S_j = Q K_j^T into buffer j & 1: 4 k-steps of 16 out of the 64-column tiles, one out of the tails
+      auto issue_s = [&](int j) {
+        const uint32_t d = tmem + static_cast<uint32_t>((j & 1) * 128);
 #pragma unroll
         for (int k = 0; k < 4; ++k)
-          umma_bf16(tmem, umma_desc(smem_u32(sQ) + k * 32, 1024, 2), umma_desc(smem_u32(sK) + k * 32, 1024, 2), id_s, k ? 1u : 0u);
-        if (C::TAIL) umma_bf16(tmem, umma_desc(smem_u32(sQt), 256, 6), umma_desc(smem_u32(sKt), 256, 6), id_s, 1u);
-        umma_commit(bar_s);
+          umma_bf16(d, umma_desc(smem_u32(sQ) + k * 32, 1024, 2), umma_desc(smem_u32(sK) + k * 32, 1024, 2), id_s, k ? 1u : 0u);
+        if (C::TAIL) umma_bf16(d, umma_desc(smem_u32(sQt), 256, 6), umma_desc(smem_u32(sKt), 256, 6), id_s, 1u);
+        umma_commit(&bar_s[j & 1]);
         umma_commit(bar_kfree);
+      };
+      bool ok = mbar_wait(bar_qz, 0, abort_flag, p.status) && mbar_wait(bar_kfull, 0, abort_flag, p.status);
+      if (ok) {
+        tc_fence_after();
+        issue_s(0);
+      }
+      for (int j = 0; j < n_blk && ok; ++j) {
+        const uint32_t ph = j & 1;
+        if (j + 1 < n_blk) {
+          // the next block's S goes into the other buffer, which held O_blk of block j - 1
+          if (!mbar_wait(bar_kfull, (j + 1) & 1, abort_flag, p.status)) break;
+          if (j >= 1 && !mbar_wait(bar_sfree, (j - 1) & 1, abort_flag, p.status)) break;
+          tc_fence_after();
+          issue_s(j + 1);
+        }
         if (!mbar_wait(bar_p, ph, abort_flag, p.status)) break;
         if (!mbar_wait(bar_vfull, ph, abort_flag, p.status)) break;
         tc_fence_after();
-        // O_blk = P V: 8 k-steps of 16 keys; V's 8-key groups are 1024 (main) / 256 (tail) bytes apart
+        // O_blk = P V over the columns of S_j: 8 k-steps of 16 keys; V's 8-key groups are 1024 (main) / 256 (tail) bytes apart
+        const uint32_t d = tmem + static_cast<uint32_t>((j & 1) * 128);
 #pragma unroll
         for (int k = 0; k < TK / 16; ++k) {
           const uint64_t a = umma_desc(smem_u32(sP) + (k >> 2) * C::MAIN_BYTES + (k & 3) * 32, 1024, 2);
-          umma_bf16(tmem, a, umma_desc(smem_u32(sV) + k * 2048, 1024, 2), id_o, k ? 1u : 0u);
-          if (C::TAIL) umma_bf16(tmem + 64, a, umma_desc(smem_u32(sVt) + k * 512, 256, 6), id_ot, k ? 1u : 0u);
+          umma_bf16(d, a, umma_desc(smem_u32(sV) + k * 2048, 1024, 2), id_o, k ? 1u : 0u);
+          if (C::TAIL) umma_bf16(d + 64, a, umma_desc(smem_u32(sVt) + k * 512, 256, 6), id_ot, k ? 1u : 0u);
         }
         umma_commit(bar_o);
         umma_commit(bar_vfree);
@@ -177,44 +198,75 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     float o[C::O_HALF];
 #pragma unroll
     for (int i = 0; i < C::O_HALF; ++i) o[i] = 0.0f;
-    float m_run = -INFINITY, l_run = 0.0f;
-    for (int j = 0; j < n_blk && ok; ++j) {
-      const uint32_t ph = j & 1;
-      if (!mbar_wait(bar_s, ph, abort_flag, p.status)) { ok = false; break; }
-      __syncwarp();
-      tc_fence_after();
-      // pass 1: row maximum over the whole block (both threads of the row compute the same value)
-      float mx = -INFINITY;
-#pragma unroll 1
-      for (int c = 0; c < TK / 16; ++c) {
-        uint32_t v[16];
-        tmem_ld_32x16(trow + c * 16, v);
+    // o = o * alpha + O_blk for this thread's half of the output columns (O_blk sits in buffer `buf`)
+    auto fold = [&](int buf, float alpha) {
+      const uint32_t src = trow + static_cast<uint32_t>(buf * 128 + half * C::O_HALF);
+      uint32_t v[32];
+      tmem_ld_32x32(src, v);
+      tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 32; ++i) o[i] = fmaf(o[i], alpha, __uint_as_float(v[i]));
+      if (C::TAIL) {
+        uint32_t w[8];
+        tmem_ld_32x8(src + 32, w);
         tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 16; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
+        for (int i = 0; i < 8; ++i) o[32 + i] = fmaf(o[32 + i], alpha, __uint_as_float(w[i]));
       }
+    };
+    float m_run = -INFINITY, l_run = 0.0f, alpha_prev = 0.0f;
+    ok = ok && mbar_wait(&bar_s[0], 0, abort_flag, p.status);
+    for (int j = 0; j < n_blk && ok; ++j) {
+      const uint32_t sbuf = trow + static_cast<uint32_t>((j & 1) * 128 + half * 64);
+      __syncwarp();
+      tc_fence_after();
+      // pass 1: maximum over this thread's 64 keys, then over the row with the other thread's value
+      float mx = -INFINITY;
+#pragma unroll 1
+      for (int c = 0; c < 2; ++c) {
+        uint32_t v[32];
+        tmem_ld_32x32(sbuf + c * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
+      }
+      s_m[((j & 1) * 2 + half) * 128 + r] = mx;
+      mbar_arrive(&bar_mx[quad]);
+      if (!mbar_wait(&bar_mx[quad], j & 1, abort_flag, p.status)) { ok = false; break; }
+      mx = fmaxf(mx, s_m[((j & 1) * 2 + (half ^ 1)) * 128 + r]);
       const float m_new = fmaxf(m_run, mx * p.scale_log2);
       const float alpha = ex2_approx(m_run - m_new);
       m_run = m_new;
+      if (j > 0) {
+        // O_blk of the previous block: fold it, then its buffer is free for S of block j + 1; its completion
+        // also means that the tensor core has finished reading P, which pass 2 is about to overwrite
+        if (!mbar_wait(bar_o, (j - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+        __syncwarp();
+        tc_fence_after();
+        fold((j - 1) & 1, alpha_prev);
+        tc_fence_before();
+        mbar_arrive(bar_sfree);
+      }
+      alpha_prev = alpha;
       // pass 2 (this thread's 64 keys): P = exp2(s * scale - m), row sum, bf16 into the swizzled tile
       float rs = 0.0f;
       const uint32_t tile = smem_u32(sP) + static_cast<uint32_t>(half * C::MAIN_BYTES + r * 128);
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {  // 16 keys = two 16-byte slots
-        uint32_t v[16];
-        tmem_ld_32x16(trow + half * 64 + c * 16, v);
+      for (int c = 0; c < 2; ++c) {  // 32 keys = four 16-byte slots
+        uint32_t v[32];
+        tmem_ld_32x32(sbuf + c * 32, v);
         tmem_ld_wait();
-        uint32_t pk[8];
+        uint32_t pk[16];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < 16; ++i) {
           const float p0 = ex2_approx(fmaf(__uint_as_float(v[2 * i]), p.scale_log2, -m_new));
           const float p1 = ex2_approx(fmaf(__uint_as_float(v[2 * i + 1]), p.scale_log2, -m_new));
           rs += p0 + p1;
           pk[i] = pack_bf16x2(p0, p1);
         }
 #pragma unroll
-        for (int g = 0; g < 2; ++g) {
-          const uint32_t slot = static_cast<uint32_t>(c * 2 + g);
+        for (int g = 0; g < 4; ++g) {
+          const uint32_t slot = static_cast<uint32_t>(c * 4 + g);
           const uint32_t addr = tile + ((slot ^ (static_cast<uint32_t>(r) & 7u)) << 4);
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[4 * g]), "r"(pk[4 * g + 1]),
                        "r"(pk[4 * g + 2]), "r"(pk[4 * g + 3])
@@ -225,29 +277,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       fence_async_smem();   // P is read by the tensor core through the async proxy
       tc_fence_before();    // and the S columns are about to be overwritten by O_blk
       mbar_arrive(bar_p);
-      // fold this thread's half of O_blk into its running output
-      if (!mbar_wait(bar_o, ph, abort_flag, p.status)) { ok = false; break; }
+      if (j + 1 < n_blk && !mbar_wait(&bar_s[(j + 1) & 1], ((j + 1) >> 1) & 1, abort_flag, p.status)) { ok = false; break; }
+    }
+    if (ok && mbar_wait(bar_o, (n_blk - 1) & 1, abort_flag, p.status)) {
       __syncwarp();
       tc_fence_after();
-      {
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t v[16];
-          tmem_ld_32x16(trow + half * C::O_HALF + c * 16, v);
-          tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 16; ++i) o[c * 16 + i] = fmaf(o[c * 16 + i], alpha, __uint_as_float(v[i]));
-        }
-        if (C::TAIL) {
-          uint32_t w[8];
-          tmem_ld_32x8(trow + half * C::O_HALF + 32, w);
-          tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 8; ++i) o[32 + i] = fmaf(o[32 + i], alpha, __uint_as_float(w[i]));
-        }
-      }
-      tc_fence_before();
-      mbar_arrive(bar_sfree);
+      fold((n_blk - 1) & 1, alpha_prev);
+    } else {
+      ok = false;
     }
     // the two threads of a row exchange their partial sums
     if (ok) {
@@ -286,7 +323,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   __syncthreads();
   if (warp == SM_WARPS + 1) {
     tc_fence_after();
-    tmem_dealloc(tmem, 128);
+    tmem_dealloc(tmem, 256);
   }
 }
 
