@@ -268,14 +268,6 @@ __device__ __forceinline__ int quantize_code_i(float x, float inv_scale, int zp,
   const int r = __float_as_int(__fadd_rn(t, 12582912.0f)) - 0x4B400000;
   return min(max(r + zp, qmin), qmax);
 }
-// Exact int32 -> float32 conversion (round to nearest even, as cvt.rn.f32.s32) on the FMA pipe:
-// split into a multiple of 4096 and a 12-bit remainder, both exactly representable, and join with one fma.
-__device__ __forceinline__ float int_to_float_rn(int v) {
-  const int hi = v >> 12, lo = v & 0xFFF;
-  const float fhi = __int_as_float(0x4B400000 + hi) - 12582912.0f;
-  const float flo = __int_as_float(0x4B400000 + lo) - 12582912.0f;
-  return fmaf(fhi, 4096.0f, flo);
-}
 __device__ __forceinline__ float gelu_tanh_f(float x) {
   // 0.5 x (1 + tanh(u)) = x / (1 + exp(-2u)),  u = sqrt(2/pi) (x + 0.044715 x^3)
   //                     = x / (1 + 2^(x (a + b x^2))),  a = -2 sqrt(2/pi) log2(e),  b = 0.044715 a

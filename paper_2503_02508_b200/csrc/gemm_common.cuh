@@ -96,14 +96,8 @@ __device__ __forceinline__ void epilogue8(const GemmParams& p, const uint4 lo, c
     acc[4] -= p.a_zp * c1.x; acc[5] -= p.a_zp * c1.y; acc[6] -= p.a_zp * c1.z; acc[7] -= p.a_zp * c1.w;
   }
   float f[8];
-  if (flags & QDIT_EPI_GELU) {
-    // the GELU path keeps the conversion unit for exp and reciprocal: convert on the FMA pipe instead
 #pragma unroll
-    for (int i = 0; i < 8; ++i) f[i] = int_to_float_rn(acc[i]) * cp.sc[i];
-  } else {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) f[i] = static_cast<float>(acc[i]) * cp.sc[i];
-  }
+  for (int i = 0; i < 8; ++i) f[i] = static_cast<float>(acc[i]) * cp.sc[i];
   if (flags & QDIT_EPI_BIAS) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) f[i] += cp.bi[i];

@@ -17,6 +17,10 @@
 // taking 32-token chunks in turn.
 #include "gemm_common.cuh"
 
+#ifndef QDIT_FC1_BYTE_STORES
+#define QDIT_FC1_BYTE_STORES 0
+#endif
+
 namespace {
 
 using namespace qgemm;
@@ -72,7 +76,7 @@ __device__ __forceinline__ void epilogue_chunk_t(const GemmParams& p, const uint
     for (int i = 0; i < 8; ++i) {
       const int j = j0 + i;
       const int acc = static_cast<int>(v[j]) - zcs;
-      float f = ((flags & QDIT_EPI_GELU) ? int_to_float_rn(acc) : static_cast<float>(acc)) * sc;
+      float f = static_cast<float>(acc) * sc;
       if (flags & QDIT_EPI_BIAS) f += bias;
       if (flags & QDIT_EPI_GELU) f = gelu_tanh_f(f);
       if (j < m_end) {
@@ -129,11 +133,18 @@ __device__ __forceinline__ void epilogue_chunk_t_packed(const GemmParams& p, con
   const uint32_t flags = epi_flags<EPI>(p);
   const int i8 = lane & 7;
   const int n8 = n - i8;  // first channel of this lane group
+  // The epilogue of the GELU layer is bound by instruction issue, so work that a symmetric quantizer does not
+  // need (zero-point terms) is skipped through branches that are uniform over the whole grid.
   float f[32];
+  if (p.a_zp == 0) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) f[j] = static_cast<float>(static_cast<int>(v[j])) * sc;
+  } else {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) f[j] = static_cast<float>(static_cast<int>(v[j]) - zcs) * sc;
+  }
 #pragma unroll
   for (int j = 0; j < 32; ++j) {
-    const int acc = static_cast<int>(v[j]) - zcs;
-    f[j] = ((flags & QDIT_EPI_GELU) ? int_to_float_rn(acc) : static_cast<float>(acc)) * sc;
     if (flags & QDIT_EPI_BIAS) f[j] += bias;
     if (flags & QDIT_EPI_GELU) f[j] = gelu_tanh_f(f[j]);
   }
@@ -141,6 +152,17 @@ __device__ __forceinline__ void epilogue_chunk_t_packed(const GemmParams& p, con
     // one byte per token: word t = codes of tokens t, 8 + t, 16 + t, 24 + t
     const float lo_f = p.o_qmin - p.o_zp, hi_f = p.o_qmax - p.o_zp;
     const int zp = static_cast<int>(p.o_zp);
+#if QDIT_FC1_BYTE_STORES
+    if (n < p.N) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const float q = fminf(fmaxf(__fmul_rn(f[j], o_inv), lo_f), hi_f);
+        const int code = __float_as_int(__fadd_rn(q, 12582912.0f)) + zp;
+        if (m_base + j < p.M) static_cast<uint8_t*>(p.out)[static_cast<int64_t>(m_base + j) * p.ldo + n] = static_cast<uint8_t>(code);
+      }
+    }
+    return;
+#endif
     uint32_t w[8];
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
@@ -148,9 +170,10 @@ __device__ __forceinline__ void epilogue_chunk_t_packed(const GemmParams& p, con
 #pragma unroll
       for (int s4 = 0; s4 < 4; ++s4) {
         const float q = fminf(fmaxf(__fmul_rn(f[8 * s4 + t], o_inv), lo_f), hi_f);
-        m4[s4] = static_cast<uint32_t>(__float_as_int(__fadd_rn(q, 12582912.0f)) + zp);
+        m4[s4] = static_cast<uint32_t>(__float_as_int(__fadd_rn(q, 12582912.0f)));
       }
       w[t] = __byte_perm(__byte_perm(m4[0], m4[1], 0x0040), __byte_perm(m4[2], m4[3], 0x0040), 0x5410);
+      if (zp != 0) w[t] = __vadd4(w[t], static_cast<uint32_t>(zp & 0xFF) * 0x01010101u);  // code + z stays inside a byte
     }
     transpose8(w, lane);  // w[c] = codes of channel n8 + c for tokens i8, 8 + i8, 16 + i8, 24 + i8
     if (n8 < p.N) {
