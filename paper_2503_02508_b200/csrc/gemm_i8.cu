@@ -312,12 +312,17 @@ extern "C" int32_t qdit_w8a8_linear(qdit_ctx* ctx, const void* A, const void* W,
   }
   // Kernel choice (measured at M = 8192 on the DiT-XL/2 layers, see profiles/):
   //  - layers whose epilogue neither reads a residual nor writes the cache (QKV: bias -> bf16; fc1: bias + GELU ->
-  //    8-bit) run channel-major with 128 x 256 tiles (1.96 / 1.45 POP/s vs 1.84 / 1.38 token-major; the CTA-pair
-  //    kernel is within 3 % of it);
-  //  - gated layers (proj, fc2) stay token-major on 128 x 192 tiles: their epilogue moves three tensors and the
-  //    shuffle transposes of the channel-major form cost more than the shared-memory transpose.
-  if (!getenv("QDIT_GEMM_BN") && p.M >= 1024 && p.N >= 2304 && (epi_class(p.flags) == 1 || epi_class(p.flags) == 2))
-    return qdit_launch_gemm_t(ctx, A, W, p, a_unsigned, 256);
+  //    8-bit) run channel-major with 128 x 256 tiles (2.19 / 1.94 POP/s vs 1.84 / 1.38 token-major);
+  //  - the gated layer with the long reduction (fc2, K = 4608) is bound by its main loop, where the 128 x 256 tile
+  //    moves less shared-memory traffic per MAC and fills the SMs in 2 waves instead of 2.6: channel-major too
+  //    (2.21 vs 2.02 POP/s);
+  //  - the gated layer with the short reduction (proj, K = 1152) is bound by its epilogue, which is cheaper
+  //    token-major (transpose through shared memory instead of shuffles): 128 x 192 tiles (1.10 vs 0.88 POP/s).
+  if (!getenv("QDIT_GEMM_BN") && p.M >= 1024) {
+    const int cls = epi_class(p.flags);
+    if ((cls == 1 || cls == 2) && p.N >= 2304) return qdit_launch_gemm_t(ctx, A, W, p, a_unsigned, 256);
+    if (cls == 3 && p.K >= 2304 && p.N >= 1024 && p.tokens % 32 == 0) return qdit_launch_gemm_t(ctx, A, W, p, a_unsigned, 256);
+  }
   switch (pick_bn(p.M, p.N, ctx->num_sms)) {
     case 64: return launch_gemm<64>(ctx, A, W, p, a_unsigned);
     case 128: return launch_gemm<128>(ctx, A, W, p, a_unsigned);

@@ -218,8 +218,11 @@ __device__ __forceinline__ void epilogue_chunk_t_packed(const GemmParams& p, con
 // gated copy are computed channel-major with scalar parameters; the bf16 cache copy travels through two word
 // transposes, the gated f32 value through four, and the residual is then added token-major, where a lane loads
 // and stores 8 consecutive channels of a token (16 bytes).  Needs the chunk inside one sample (tokens % 32 == 0).
+// The residual words `rv` (token 8 s + i8, channels n8..n8+7) and the gate were fetched by the caller one chunk
+// ahead, so that their latency is not part of the chunk's dependency chain.
 __device__ __forceinline__ void epilogue_chunk_t_gated(const GemmParams& p, const uint32_t (&v)[32], int n, int lane,
-                                                       int m_base, float sc, float bias, int zcs) {
+                                                       int m_base, float sc, float bias, int zcs, const uint4 (&rv)[4],
+                                                       float gate) {
   const int i8 = lane & 7;
   const int n8 = n - i8;
   const bool n8_ok = n8 < p.N;
@@ -245,23 +248,20 @@ __device__ __forceinline__ void epilogue_chunk_t_gated(const GemmParams& p, cons
                        __byte_perm(w[6], w[7], 0x7632));
     }
   }
-  const float gate = n < p.N ? p.gate[static_cast<int64_t>(m_base / p.tokens) * p.ld_gate + n] : 0.0f;
 #pragma unroll
   for (int s4 = 0; s4 < 4; ++s4) {
     const int64_t m = m_base + 8 * s4 + i8;
     const bool live = n8_ok && m < p.M;
-    uint4 rv = make_uint4(0u, 0u, 0u, 0u);
-    if (live) rv = *reinterpret_cast<const uint4*>(p.residual + m * p.ldo + n8);  // in flight during the shuffles
     uint32_t w[8];
 #pragma unroll
     for (int t = 0; t < 8; ++t) w[t] = __float_as_uint(f[8 * s4 + t] * gate);
     transpose8(w, lane);  // w[c] = gated value of channel n8 + c, token m
     if (live) {
       float r[8];
-      unpack_bf16x2(rv.x, r[0], r[1]);
-      unpack_bf16x2(rv.y, r[2], r[3]);
-      unpack_bf16x2(rv.z, r[4], r[5]);
-      unpack_bf16x2(rv.w, r[6], r[7]);
+      unpack_bf16x2(rv[s4].x, r[0], r[1]);
+      unpack_bf16x2(rv[s4].y, r[2], r[3]);
+      unpack_bf16x2(rv[s4].z, r[4], r[5]);
+      unpack_bf16x2(rv[s4].w, r[6], r[7]);
 #pragma unroll
       for (int c = 0; c < 8; ++c) r[c] += __uint_as_float(w[c]);
       *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + m * p.ldo + n8) = pack_bf16x8(r);
@@ -395,6 +395,20 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
         if (flags & QDIT_EPI_BIAS) bias = p.bias[n];
         if (p.a_zp != 0) zcs = p.a_zp * p.w_colsum[n];
       }
+      // gated layers: residual and gate of a chunk are fetched one chunk ahead (the first before the accumulator is waited for)
+      const bool gated_fast = EPI == 3 && (p.tokens % 32) == 0;
+      uint4 rv_next[4] = {};
+      float gate_next = 0.0f;
+      auto prefetch_gated = [&](int c) {
+        const int mb = t0 + c * 32, i8 = lane & 7, n8 = n - i8;
+#pragma unroll
+        for (int s4 = 0; s4 < 4; ++s4) {
+          const int64_t m = mb + 8 * s4 + i8;
+          rv_next[s4] = (n8 < p.N && m < p.M) ? *reinterpret_cast<const uint4*>(p.residual + m * p.ldo + n8) : make_uint4(0u, 0u, 0u, 0u);
+        }
+        gate_next = (n_ok && mb < p.M) ? p.gate[static_cast<int64_t>(mb / p.tokens) * p.ld_gate + n] : 0.0f;
+      };
+      if (gated_fast && c_last >= 0) prefetch_gated(part);
       if (!mbar_wait(&tfull_bar[as], aphase, abort_flag, p.status)) break;
       __syncwarp();
       tc_fence_after();
@@ -408,6 +422,11 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
 #pragma unroll 1
       for (int c = part; c < CHUNKS; c += T_EPI_SPLIT) {
         uint32_t v[32];
+        uint4 rv[4];
+        float gate = gate_next;
+#pragma unroll
+        for (int s4 = 0; s4 < 4; ++s4) rv[s4] = rv_next[s4];
+        if (gated_fast && c + T_EPI_SPLIT < CHUNKS) prefetch_gated(c + T_EPI_SPLIT);
         __syncwarp();
         tmem_ld_32x32(taddr + static_cast<uint32_t>(c * 32), v);
         tmem_ld_wait();
@@ -419,7 +438,7 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
         const int m_base = t0 + c * 32;
         if (m_base < p.M) {
           if (EPI == 1 || EPI == 2) epilogue_chunk_t_packed<EPI>(p, v, n, lane, m_base, sc, bias, zcs, o_inv);
-          else if (EPI == 3 && (p.tokens % 32) == 0) epilogue_chunk_t_gated(p, v, n, lane, m_base, sc, bias, zcs);
+          else if (gated_fast) epilogue_chunk_t_gated(p, v, n, lane, m_base, sc, bias, zcs, rv, gate);
           else if (n_ok) epilogue_chunk_t<EPI>(p, v, n, m_base, sc, bias, zcs, o_inv);
         }
       }
