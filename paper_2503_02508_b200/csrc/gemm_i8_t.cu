@@ -11,9 +11,9 @@
 // tile be 256 wide (one MMA of N = 256) and makes every DiT-XL/2 layer width (multiples of 128 channels)
 // tile without remainder.
 //
-// CTA = 2 + T_EPI_WARPS warps, roles and barriers as in gemm_i8.cu: warp 0 lane 0 TMA producer (weight
+// CTA = 2 + 12 (or more, see TWarps) warps, roles and barriers as in gemm_i8.cu: warp 0 lane 0 TMA producer (weight
 // tile 128 x 128 B as operand A, activation tile BT x 128 B as operand B, both K-major, 128B swizzle), warp 1
-// lane 0 MMA issuer (two TMEM accumulator stages of BT columns), epilogue warps: T_EPI_SPLIT per lane quadrant,
+// lane 0 MMA issuer (two TMEM accumulator stages of BT columns), epilogue warps: 3 (or more) per lane quadrant,
 // taking 32-token chunks in turn.
 #include "gemm_common.cuh"
 
@@ -26,14 +26,18 @@ namespace {
 using namespace qgemm;
 
 constexpr int BC = 128;  // channels per tile = TMEM lanes
-// This kernel has no per-warp staging buffer, so its epilogue can be wider than the token-major kernel's:
-// 16 warps = 4 per lane quadrant, which also divides the 8 (or 4) token chunks of a tile evenly.
-#ifndef QDIT_T_EPI_WARPS
-#define QDIT_T_EPI_WARPS 12
+// This kernel has no per-warp staging buffer, so its epilogue could be wider than the token-major kernel's;
+// measured, 16 warps (4 per lane quadrant) are slower than 12 for every epilogue class, so 12 it is.
+#ifndef QDIT_T_GATED_WARPS
+#define QDIT_T_GATED_WARPS 12
 #endif
-constexpr int T_EPI_WARPS = QDIT_T_EPI_WARPS;
-constexpr int T_EPI_SPLIT = T_EPI_WARPS / 4;
-constexpr int T_NUM_THREADS = 64 + T_EPI_WARPS * 32;
+// Epilogue warps per epilogue class (a multiple of 4: each TMEM lane quadrant is read by warps with warp % 4 = quadrant).
+template <int EPI>
+struct TWarps {
+  static constexpr int EPI_WARPS = EPI == 3 ? QDIT_T_GATED_WARPS : 12;
+  static constexpr int SPLIT = EPI_WARPS / 4;
+  static constexpr int THREADS = 64 + EPI_WARPS * 32;
+};
 
 template <int BT>
 struct TCfg {
@@ -270,7 +274,7 @@ __device__ __forceinline__ void epilogue_chunk_t_gated(const GemmParams& p, cons
 }
 
 template <int BT, int EPI>
-__global__ void __launch_bounds__(T_NUM_THREADS, 1)
+__global__ void __launch_bounds__(TWarps<EPI>::THREADS, 1)
 gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                  const GemmParams p, const uint32_t idesc) {
   using C = TCfg<BT>;
@@ -296,7 +300,7 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&tfull_bar[s], 1);
-      mbar_init(&tempty_bar[s], T_EPI_WARPS);
+      mbar_init(&tempty_bar[s], TWarps<EPI>::EPI_WARPS);
     }
     *abort_flag = 0;
     mbar_fence_init();
@@ -373,6 +377,7 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     // -------------------------------------------------------------------- epilogue warps
     const int e = warp - 2;
     const int quad = warp & 3;   // TMEM lane quadrant = 32 channels
+    constexpr int T_EPI_SPLIT = TWarps<EPI>::SPLIT;
     const int part = e >> 2;     // this warp takes token chunks part, part + T_EPI_SPLIT, ...
     const uint32_t flags = epi_flags<EPI>(p);
     const float a_scale = p.a_scale_dev ? __ldg(p.a_scale_dev) : p.a_scale;
@@ -472,7 +477,7 @@ int32_t launch_t_epi(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p,
   const uint32_t idesc = (2u << 4) | (1u << 7) | ((a_unsigned ? 0u : 1u) << 10) | ((static_cast<uint32_t>(BT) >> 3) << 17) |
                          ((static_cast<uint32_t>(BC) >> 4) << 24);
   ProfScope prof(ctx, QDIT_PROF_GEMM, 2.0 * p.M * static_cast<double>(p.N) * p.K);
-  QDIT_CUDA_CHECK(ctx, qdit_launch_overlapped(ctx, gemm_i8_t_kernel<BT, EPI>, dim3(grid), dim3(T_NUM_THREADS), C::SMEM_BYTES, tw, tx, p, idesc));
+  QDIT_CUDA_CHECK(ctx, qdit_launch_overlapped(ctx, gemm_i8_t_kernel<BT, EPI>, dim3(grid), dim3(TWarps<EPI>::THREADS), C::SMEM_BYTES, tw, tx, p, idesc));
   return qdit_after_launch(ctx, "gemm_i8_t_kernel");
 }
 
