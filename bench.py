@@ -36,6 +36,12 @@ WORKLOADS = {
 }
 
 
+# DRAM bytes (read + written) per GEMM launch, from the ncu capture summarised in
+# profiles/gemm_i8_layers_m8192_sections.txt: QKV 18.9 MB, proj 29.9 MB, fc1 15.3 MB, fc2 65.7 MB per launch at
+# M = 8192 (the shapes of the 50-step workload); each layer is 700 of the trajectory's 2801 GEMM launches.
+NCU_GEMM_DRAM_BYTES_PER_LAUNCH = 700 * (18.9e6 + 29.9e6 + 15.3e6 + 65.7e6) / 2801
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -298,8 +304,10 @@ def run_ours(args):
     g_n, g_ms, g_ops = prof[q.QDIT_PROF_GEMM]
     int8_peak = 2.0 * peaks["bf16_sustained"]          # dense int8 : bf16 nominal ratio 4.5 : 2.25
     achieved = g_ops / (g_ms * 1e-3) / 1e12 if g_ms > 0 else 0.0
-    roofline = {"bound": "tensor", "kernel": "gemm_i8_kernel", "achieved": achieved, "peak": int8_peak, "unit": "TOP/s",
-                "frac": achieved / int8_peak, "traffic": None,
+    roofline = {"bound": "tensor", "kernel": "int8 GEMMs (gemm_i8_t_kernel, gemm_i8_kernel)", "achieved": achieved,
+                "peak": int8_peak, "unit": "TOP/s", "frac": achieved / int8_peak,
+                "traffic": NCU_GEMM_DRAM_BYTES_PER_LAUNCH if args.workload == "ddim50" else None,
+                "traffic_note": "launch-weighted mean of the four block-level layers at M = 8192 (ncu, L2-warm sweep)",
                 "peak_source": f"2 x {peaks['source']} sustained bf16 ({peaks['bf16_sustained']} TFLOP/s)",
                 "launches": g_n, "avg_launch_ms": g_ms / max(g_n, 1), "share_of_profiled_time": None}
     tot_ms = sum(v[1] for v in prof.values())

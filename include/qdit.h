@@ -221,6 +221,17 @@ int32_t qdit_cache_reuse_all(qdit_ctx* ctx, qdit_cache* cache, const float* mod_
 enum { QDIT_VC_NONE = 0, QDIT_VC_K_TABLE = 1, QDIT_VC_VAR_RATIO = 2 };
 int32_t qdit_vc_correct(qdit_ctx* ctx, float* latent, int B, int C, int HW, int step_index, int mode,
                         const float* table, float eps);
+/* Fitting the factor of one step (same section, the closed form below "variance compensation ... using the
+ * rQNSR-MSE metric"): from N calibration samples x^ (accelerated trajectory) and targets x' (reference
+ * trajectory), both device f32 [N, C, HW], with mu = spatial mean of x^ per (sample, channel), a = x^ - mu,
+ * b = x' - mu, w = 1 / (x'^2 + eps), sums over the samples and positions of channel c:
+ *   QDIT_VC_FIT_DERIVED : K[c] = (sum a b + sum a b w) / (sum a^2 + sum a^2 w)   (d/dK of rQNSR^2 + MSE = 0)
+ *   QDIT_VC_FIT_PRINTED : the numerator's second term as the paper prints it, sum a / x'.
+ * workspace: caller-owned device scratch of 4 * N * C doubles (overwritten); K: device f32 [C] (one row of the
+ * K table).  Sums are taken in f64 and combined in a fixed order: the result is reproducible. */
+enum { QDIT_VC_FIT_DERIVED = 0, QDIT_VC_FIT_PRINTED = 1 };
+int32_t qdit_vc_fit(qdit_ctx* ctx, const float* x_hat, const float* x_target, int N, int C, int HW, float eps, int form,
+                    double* workspace, float* K);
 
 /* ------------------------------------------------------------------------------------------------
  * Whole model and sampler.  The DiT architecture (adaLN-Zero blocks, patch 2, learned-sigma output)

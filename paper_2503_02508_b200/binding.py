@@ -23,6 +23,7 @@ QDIT_EPI_BIAS, QDIT_EPI_GELU, QDIT_EPI_GATE, QDIT_EPI_RESIDUAL = 1, 2, 4, 8
 QDIT_EPI_CACHE_STORE, QDIT_EPI_QUANT_OUT, QDIT_EPI_OUT_BF16, QDIT_EPI_OUT_F32, QDIT_EPI_OUT_I32 = 16, 32, 64, 128, 256
 QDIT_BRANCH_ATTN, QDIT_BRANCH_MLP = 0, 1
 QDIT_VC_NONE, QDIT_VC_K_TABLE, QDIT_VC_VAR_RATIO = 0, 1, 2
+QDIT_VC_FIT_DERIVED, QDIT_VC_FIT_PRINTED = 0, 1
 QDIT_FWD_STORE_CACHE, QDIT_FWD_REUSE, QDIT_FWD_CALIBRATE = 1, 2, 4
 
 _vp, _i32, _i64, _u32, _f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_float
@@ -87,6 +88,7 @@ _SIGNATURES = {
     "qdit_cache_reuse": (_i32, [_vp, _vp, _int, _int, _vp, _i64, _i64, _vp]),
     "qdit_cache_reuse_all": (_i32, [_vp, _vp, _vp, _i64, _i64, _vp]),
     "qdit_vc_correct": (_i32, [_vp, _vp, _int, _int, _int, _int, _int, _vp, _f32]),
+    "qdit_vc_fit": (_i32, [_vp, _vp, _vp, _int, _int, _int, _f32, _int, _vp, _vp]),
     "qdit_model_create": (_i32, [_vp, C.POINTER(qdit_model_desc), C.POINTER(_vp)]),
     "qdit_model_destroy": (_i32, [_vp]),
     "qdit_model_set_act_scales": (_i32, [_vp, _vp, _vp, _vp]),
@@ -254,6 +256,10 @@ def qdit_cache_reuse_all(ctx, cache, mod_all, ld_mod, T, x):
 
 def qdit_vc_correct(ctx, latent, B, Cc, HW, step_index, mode, table, eps):
     return check(ctx, lib.qdit_vc_correct(ctx, ptr(latent), B, Cc, HW, step_index, mode, ptr(table), eps))
+
+
+def qdit_vc_fit(ctx, x_hat, x_target, N, Cc, HW, eps, form, workspace, K):
+    return check(ctx, lib.qdit_vc_fit(ctx, ptr(x_hat), ptr(x_target), N, Cc, HW, eps, form, ptr(workspace), ptr(K)))
 
 
 def qdit_model_create(ctx, cfg, weights):

@@ -105,6 +105,70 @@ __global__ void __launch_bounds__(256) vc_kernel(float* __restrict__ latent, int
   }
 }
 
+// ----------------------------------------------------------------------------- variance compensation: fitting K
+// Closed-form factor of one step from calibration samples x^ (quantized + cached trajectory) and targets x'
+// (reference trajectory): with mu = spatial mean of x^ per (sample, channel), a = x^ - mu, b = x' - mu and
+// w = 1 / (x'^2 + eps), minimising rQNSR^2 + MSE over K gives
+//   K[c] = (sum a b + sum a b w) / (sum a^2 + sum a^2 w)        (sums over samples and positions of channel c);
+// the form as printed in the paper has sum a / x' in place of sum a b w.
+// Pass 1: one CTA per (sample, channel) writes its four partial sums (f64: w reaches 1/eps where x' passes
+// through zero).  Pass 2: one thread per channel adds the samples' partials in order and divides, so the result
+// does not depend on scheduling.
+__device__ __forceinline__ double block_sum_f64(double v, double* sm) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) sm[threadIdx.x >> 5] = v;
+  __syncthreads();
+  double t = 0.0;
+  for (int i = 0; i < (blockDim.x >> 5); ++i) t += sm[i];
+  return t;
+}
+
+__global__ void __launch_bounds__(256) vc_fit_partial_kernel(const float* __restrict__ x_hat, const float* __restrict__ x_tgt,
+                                                             int HW, double eps, int printed_form,
+                                                             double* __restrict__ partial) {
+  __shared__ double sm[8];
+  const float* xh = x_hat + static_cast<int64_t>(blockIdx.x) * HW;
+  const float* xt = x_tgt + static_cast<int64_t>(blockIdx.x) * HW;
+  double s = 0.0;
+  for (int i = threadIdx.x; i < HW; i += blockDim.x) s += static_cast<double>(xh[i]);
+  const double mu = block_sum_f64(s, sm) / static_cast<double>(HW);
+  double ab = 0.0, aa = 0.0, abw = 0.0, aaw = 0.0;
+  for (int i = threadIdx.x; i < HW; i += blockDim.x) {
+    const double t = static_cast<double>(xt[i]);
+    const double a = static_cast<double>(xh[i]) - mu, b = t - mu;
+    const double w = 1.0 / (t * t + eps);
+    ab += a * b;
+    aa += a * a;
+    abw += printed_form ? a / t : a * b * w;
+    aaw += a * a * w;
+  }
+  ab = block_sum_f64(ab, sm);
+  aa = block_sum_f64(aa, sm);
+  abw = block_sum_f64(abw, sm);
+  aaw = block_sum_f64(aaw, sm);
+  if (threadIdx.x == 0) {
+    double* o = partial + static_cast<int64_t>(blockIdx.x) * 4;
+    o[0] = ab;
+    o[1] = aa;
+    o[2] = abw;
+    o[3] = aaw;
+  }
+}
+
+__global__ void vc_fit_finish_kernel(const double* __restrict__ partial, int N, int C, float* __restrict__ K) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= C) return;
+  double num = 0.0, den = 0.0;
+  for (int n = 0; n < N; ++n) {
+    const double* o = partial + (static_cast<int64_t>(n) * C + c) * 4;
+    num += o[0] + o[2];
+    den += o[1] + o[3];
+  }
+  K[c] = static_cast<float>(num / den);
+}
+
 // ----------------------------------------------------------------------------- guidance + DDIM update
 // net: [Beff, 2C, HW]; eps = first C channels; with guidance, sample b's unconditional twin is b + B.
 __global__ void __launch_bounds__(256) cfg_ddim_kernel(float* __restrict__ latent, const float* __restrict__ net, int B,
@@ -667,6 +731,21 @@ int32_t qdit_vc_correct(qdit_ctx* ctx, float* latent, int B, int C, int HW, int 
   vc_kernel<<<static_cast<unsigned>(B) * C, 256, 0, ctx->stream>>>(latent, C, HW, mode,
                                                                   table + static_cast<int64_t>(step_index) * C, eps);
   return qdit_after_launch(ctx, "vc_kernel");
+}
+
+int32_t qdit_vc_fit(qdit_ctx* ctx, const float* x_hat, const float* x_target, int N, int C, int HW, float eps, int form,
+                    double* workspace, float* K) {
+  if (!ctx) return QDIT_ERR_INVALID_ARG;
+  if (N <= 0 || C <= 0 || HW <= 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "N, C and HW must be positive");
+  if (form != QDIT_VC_FIT_DERIVED && form != QDIT_VC_FIT_PRINTED) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "unknown fit form %d", form);
+  if (!x_hat || !x_target || !workspace || !K) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "NULL argument");
+  if (reinterpret_cast<uintptr_t>(workspace) & 7u) return qdit_fail(ctx, QDIT_ERR_ALIGN, "workspace must be 8-byte aligned");
+  if (static_cast<int64_t>(N) * C > 0x7fffffff) return qdit_fail(ctx, QDIT_ERR_SHAPE, "N * C too large");
+  vc_fit_partial_kernel<<<static_cast<unsigned>(N) * C, 256, 0, ctx->stream>>>(x_hat, x_target, HW, static_cast<double>(eps),
+                                                                              form == QDIT_VC_FIT_PRINTED ? 1 : 0, workspace);
+  QDIT_TRY(qdit_after_launch(ctx, "vc_fit_partial_kernel"));
+  vc_fit_finish_kernel<<<(C + 63) / 64, 64, 0, ctx->stream>>>(workspace, N, C, K);
+  return qdit_after_launch(ctx, "vc_fit_finish_kernel");
 }
 
 }  // extern "C"

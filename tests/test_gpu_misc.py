@@ -79,6 +79,58 @@ def test_cache_store_reuse_and_state(q, ctx):
         q.qdit_cache_destroy(cache)
 
 
+@pytest.mark.parametrize("N,C,HW", [(4, 4, 1024), (2, 4, 4096), (1, 3, 64), (5, 2, 100)])
+def test_vc_fit_matches_the_closed_form(q, ctx, N, C, HW):
+    """K of one step fitted on the device against oracle.vc.fit (both forms), incl. targets that pass through zero."""
+    side = int(np.sqrt(HW))
+    xt = synth.normal(63, f"fit_t{HW}", (N, C, HW)) * np.array([0.5, 1.0, 2.0, 3.0][:C], dtype=np.float32).reshape(1, C, 1)
+    r = np.array([1.1, 0.9, 1.3, 0.8][:C], dtype=np.float32).reshape(1, C, 1)
+    xh = (xt.mean(axis=2, keepdims=True) + r * (xt - xt.mean(axis=2, keepdims=True)) +
+          0.05 * synth.normal(63, f"fit_n{HW}", (N, C, HW))).astype(np.float32)
+    ws = torch.empty(4 * N * C, dtype=torch.float64, device="cuda")
+    for form, name in ((q.QDIT_VC_FIT_DERIVED, "derived"), (q.QDIT_VC_FIT_PRINTED, "printed")):
+        kd = torch.empty(C, dtype=torch.float32, device="cuda")
+        q.qdit_vc_fit(ctx, dev(xh), dev(xt), N, C, HW, 1e-6, form, ws, kd)
+        q.qdit_sync(ctx)
+        want = vc.fit(xh.reshape(N, C, side, side), xt.reshape(N, C, side, side), eps=1e-6, form=name)
+        # f64 sums on both sides; what is left is the summation order and the final rounding of K to f32
+        np.testing.assert_allclose(kd.cpu().numpy(), want, rtol=2e-6)
+    # a trajectory that already matches its target needs no compensation
+    kd = torch.empty(C, dtype=torch.float32, device="cuda")
+    q.qdit_vc_fit(ctx, dev(xt), dev(xt), N, C, HW, 1e-6, q.QDIT_VC_FIT_DERIVED, ws, kd)
+    q.qdit_sync(ctx)
+    np.testing.assert_allclose(kd.cpu().numpy(), np.ones(C), rtol=1e-6)
+    # the fitted K minimises the objective sum (K a - b)^2 (1 + w) per channel: lower than K = 1 and than K +- 1 %
+    kd = torch.empty(C, dtype=torch.float32, device="cuda")
+    q.qdit_vc_fit(ctx, dev(xh), dev(xt), N, C, HW, 1e-6, q.QDIT_VC_FIT_DERIVED, ws, kd)
+    q.qdit_sync(ctx)
+    kf = kd.cpu().numpy().astype(np.float64).reshape(1, C, 1)
+    x64, t64 = xh.astype(np.float64), xt.astype(np.float64)
+    a = x64 - x64.mean(axis=2, keepdims=True)
+    b = t64 - x64.mean(axis=2, keepdims=True)
+    w1 = 1.0 + 1.0 / (t64 ** 2 + 1e-6)
+
+    def objective(k):
+        return (np.square(k * a - b) * w1).sum(axis=(0, 2))
+
+    j = objective(kf)
+    assert (j <= objective(np.ones_like(kf))).all()
+    assert (j <= objective(kf * 1.01)).all() and (j <= objective(kf * 0.99)).all()
+
+
+def test_vc_fit_rejects_bad_arguments(q, ctx):
+    import ctypes as C
+    x = torch.zeros(4 * 64, dtype=torch.float32, device="cuda")
+    ws = torch.zeros(16, dtype=torch.float64, device="cuda")
+    k = torch.zeros(4, dtype=torch.float32, device="cuda")
+    L = q.lib
+    assert L.qdit_vc_fit(ctx, x.data_ptr(), x.data_ptr(), 0, 4, 64, 1e-6, 0, ws.data_ptr(), k.data_ptr()) == q.QDIT_ERR_SHAPE
+    assert L.qdit_vc_fit(ctx, x.data_ptr(), x.data_ptr(), 1, 4, 64, 1e-6, 7, ws.data_ptr(), k.data_ptr()) == q.QDIT_ERR_INVALID_ARG
+    assert L.qdit_vc_fit(ctx, x.data_ptr(), None, 1, 4, 64, 1e-6, 0, ws.data_ptr(), k.data_ptr()) == q.QDIT_ERR_INVALID_ARG
+    assert L.qdit_vc_fit(ctx, x.data_ptr(), x.data_ptr(), 1, 4, 64, 1e-6, 0, None, k.data_ptr()) == q.QDIT_ERR_INVALID_ARG
+    q.qdit_sync(ctx)
+
+
 @pytest.mark.parametrize("B,C,HW", [(3, 4, 1024), (2, 4, 4096), (1, 3, 64)])
 def test_vc_correct(q, ctx, B, C, HW):
     S = 5
