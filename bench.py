@@ -29,6 +29,7 @@ sys.path.insert(0, ROOT)
 import synth  # noqa: E402
 
 METRIC = "DiT-XL/2 W8A8+cache images/s (256^2, 50 steps)"
+METRICS = {"ddim50": METRIC, "ddim100_512": "DiT-XL/2 W8A8+cache images/s (512^2, 100 steps)"}
 WORKLOADS = {
     # name: (config, seed key, steps, batch, guidance, interval)
     "ddim50": (synth.DIT_XL2, "ddim50_xl2", 50, 16, 1.5, 2),
@@ -197,7 +198,7 @@ def run_reference(args):
     value = float(np.mean(vals))
     cfg, seed, steps, batch, guidance, interval, *_ = workload_inputs(args.workload)
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": "images/s", "n_gpus": args.gpus,
+        "impl": "reference", "metric": METRICS.get(args.workload, METRIC), "value": value, "unit": "images/s", "n_gpus": args.gpus,
         "steps": len(vals), "warmup": 0, "ms_per_step": 1e3 * (time.perf_counter() - t_all) / len(vals),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
         "config": {"workload": args.workload, "model": "DiT-XL/2", "batch": batch, "sampling_steps": steps,
@@ -227,7 +228,7 @@ def run_ours(args):
     stream = torch.cuda.Stream()
     ctx = q.qdit_create(local, stream.cuda_stream)
     weights = synth.model_weights(seed, cfg)
-    model = q.qdit_model_create(ctx, cfg, weights)
+    model = q.qdit_model_create(ctx, cfg, weights, args.weight_bits)
     del weights
     sampler = q.qdit_sampler_create(ctx, model, batch=batch, num_steps=steps, cache_interval=interval,
                                     use_cfg=guidance is not None, guidance=guidance or 1.0,
@@ -331,12 +332,12 @@ def run_ours(args):
 
     if rank == 0:
         line = {
-            "metric": METRIC, "value": value, "unit": "images/s", "n_gpus": world, "steps": args.steps,
+            "metric": METRICS.get(args.workload, METRIC).replace("W8A8", f"W{args.weight_bits}A8"), "value": value, "unit": "images/s", "n_gpus": world, "steps": args.steps,
             "warmup": n_warm, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int8", "data": "synthetic",
             "config": {"workload": args.workload, "model": "DiT-XL/2", "batch_per_gpu": batch, "network_batch": beff,
                        "sampling_steps": steps, "cache_interval": interval, "guidance": guidance,
-                       "vc": "k_table every step", "residual_stream": "bf16",
+                       "vc": "k_table every step", "residual_stream": "bf16", "weight_bits": args.weight_bits,
                        "l2": "per-step working set (0.45 GB weights + 1.06 GB cache) exceeds L2; no flush needed",
                        "roofline_pass": "one extra trajectory with per-launch CUDA events, outside the timed region"},
             "clocks": clock_info,
@@ -438,6 +439,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="ddim50", choices=sorted(WORKLOADS) + ["gemm_sweep"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--weight-bits", type=int, default=8, help="code width of the quantized weights (4 = the paper's W4A8 setting)")
     ap.add_argument("--m", type=lambda v: [int(x) for x in v.split(",")], default=[256, 1024, 4096, 8192, 16384, 65536],
                     help="row counts of the GEMM sweep")
     ap.add_argument("--short-warmup", action="store_true",

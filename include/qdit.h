@@ -158,9 +158,14 @@ int32_t qdit_w8a8_linear(qdit_ctx* ctx, const void* A, const void* W, int64_t M,
 
 /* Channel-wise symmetric weight quantizer (the weight side of Eq. 1): for each output row n of
  * w[N,K] (f32, device), s[n] = max_k|w| / 127 (1 if the row is zero), q = clip(round(w * (1/s)),-127,127),
- * colsum[n] = sum_k q[n,k].  q: [N,K] bytes, w_scale: [N] f32, w_colsum: [N] int32.  K % 4 == 0. */
+ * colsum[n] = sum_k q[n,k].  q: [N,K] bytes, w_scale: [N] f32, w_colsum: [N] int32.  K % 4 == 0.
+ * qdit_quantize_weight_bits is the same with b-bit codes (2 <= bits <= 8): top = 2^(bits-1) - 1 replaces 127.
+ * With bits = 4 this is the weight side of the paper's W4A8 setting (Table 2); the codes are still stored one
+ * per byte, so every kernel that takes 8-bit weights takes them unchanged. */
 int32_t qdit_quantize_weight(qdit_ctx* ctx, const float* w, int64_t N, int64_t K, void* q, float* w_scale,
                              int32_t* w_colsum);
+int32_t qdit_quantize_weight_bits(qdit_ctx* ctx, const float* w, int64_t N, int64_t K, int bits, void* q,
+                                  float* w_scale, int32_t* w_colsum);
 
 /* ------------------------------------------------------------------------------------------------
  * Self-attention between the quantized linears (kept in bf16, not quantized):
@@ -239,6 +244,7 @@ int32_t qdit_vc_fit(qdit_ctx* ctx, const float* x_hat, const float* x_target, in
  * modulation linear, QKV, projection, fc1 and fc2; embedders and the final layer stay in f32. */
 typedef struct {
   int32_t hidden, heads, mlp, depth, grid, patch, channels, num_classes, freq_dim;
+  int32_t weight_bits; /* code width of the quantized linears' weights: 0 or 8 = W8A8, 4 = W4A8 (Table 2) */
 } qdit_model_shape;
 
 typedef struct { /* HOST f32 arrays, each linear [out_features, in_features] row-major */

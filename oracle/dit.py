@@ -106,8 +106,8 @@ class QLinear:
     w: np.ndarray        # original float32 weights (un-quantized mode only)
 
 
-def make_qlinear(w, b) -> QLinear:
-    q, s, cs = quantize_weight_per_channel(w)
+def make_qlinear(w, b, bits: int = 8) -> QLinear:
+    q, s, cs = quantize_weight_per_channel(w, bits)
     return QLinear(q.astype(np.int8), s, cs, np.asarray(b, dtype=F32), np.asarray(w, dtype=F32))
 
 
@@ -120,8 +120,8 @@ class QBlock:
     fc2: QLinear
 
 
-def make_qblock(bw: dict) -> QBlock:
-    return QBlock(*(make_qlinear(bw["w_" + n], bw["b_" + n]) for n in LINEARS))
+def make_qblock(bw: dict, bits: int = 8) -> QBlock:
+    return QBlock(*(make_qlinear(bw["w_" + n], bw["b_" + n], bits) for n in LINEARS))
 
 
 @dataclass
@@ -241,9 +241,10 @@ class QModel:
     w: dict                # float parameters of the un-quantized layers
 
 
-def make_qmodel(cfg, weights: dict) -> QModel:
+def make_qmodel(cfg, weights: dict, weight_bits: int = 8) -> QModel:
+    """weight_bits = 4 gives the W4A8 setting of Table 2 (4-bit channel-wise weights, 8-bit activations)."""
     fl = {k: np.asarray(v, dtype=np.float64) for k, v in weights.items() if k != "blocks"}
-    return QModel(cfg, [make_qblock(bw) for bw in weights["blocks"]], fl)
+    return QModel(cfg, [make_qblock(bw, weight_bits) for bw in weights["blocks"]], fl)
 
 
 def timestep_features(t, dim: int):

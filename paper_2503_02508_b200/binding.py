@@ -42,7 +42,7 @@ class qdit_epilogue(C.Structure):
 
 class qdit_model_shape(C.Structure):
     _fields_ = [(n, _i32) for n in ("hidden", "heads", "mlp", "depth", "grid", "patch", "channels", "num_classes",
-                                    "freq_dim")]
+                                    "freq_dim", "weight_bits")]
 
 
 class qdit_block_weights(C.Structure):
@@ -75,6 +75,7 @@ _SIGNATURES = {
     "qdit_w8a8_linear": (_i32, [_vp, _vp, _vp, _i64, _i64, _i64, qdit_qparams, _vp, _u32, C.POINTER(qdit_epilogue),
                                 _vp, _i64]),
     "qdit_quantize_weight": (_i32, [_vp, _vp, _i64, _i64, _vp, _vp, _vp]),
+    "qdit_quantize_weight_bits": (_i32, [_vp, _vp, _i64, _i64, _int, _vp, _vp, _vp]),
     "qdit_attention": (_i32, [_vp, _vp, _vp, _vp, _i64, _int, _int, _int, _int, _f32, _vp, _int,
                               C.POINTER(qdit_qparams), _vp]),
     "qdit_adaln_modulate": (_i32, [_vp, _vp, _i64, _i64, _i64, _f32, _vp, _vp, _i64, _vp, _int,
@@ -208,6 +209,10 @@ def qdit_quantize_weight(ctx, w, N, K, q, w_scale, w_colsum):
     return check(ctx, lib.qdit_quantize_weight(ctx, ptr(w), N, K, ptr(q), ptr(w_scale), ptr(w_colsum)))
 
 
+def qdit_quantize_weight_bits(ctx, w, N, K, bits, q, w_scale, w_colsum):
+    return check(ctx, lib.qdit_quantize_weight_bits(ctx, ptr(w), N, K, bits, ptr(q), ptr(w_scale), ptr(w_colsum)))
+
+
 def qdit_attention(ctx, q, k, v, ld, B, H, T, dh, softmax_scale, out, out_dtype, out_qp=None, out_scale_dev=None):
     return check(ctx, lib.qdit_attention(ctx, ptr(q), ptr(k), ptr(v), ld, B, H, T, dh, softmax_scale, ptr(out),
                                          out_dtype, C.byref(out_qp) if out_qp is not None else None,
@@ -262,9 +267,10 @@ def qdit_vc_fit(ctx, x_hat, x_target, N, Cc, HW, eps, form, workspace, K):
     return check(ctx, lib.qdit_vc_fit(ctx, ptr(x_hat), ptr(x_target), N, Cc, HW, eps, form, ptr(workspace), ptr(K)))
 
 
-def qdit_model_create(ctx, cfg, weights):
+def qdit_model_create(ctx, cfg, weights, weight_bits=8):
     """cfg: object with hidden, heads, mlp, depth, grid, patch, channels, num_classes, freq_dim;
-    weights: dict of contiguous float32 numpy arrays laid out as qdit_model_desc documents."""
+    weights: dict of contiguous float32 numpy arrays laid out as qdit_model_desc documents;
+    weight_bits: code width of the quantized linears' weights (8 = W8A8, 4 = W4A8)."""
     import numpy as np
 
     keep = []
@@ -280,7 +286,7 @@ def qdit_model_create(ctx, cfg, weights):
             setattr(blocks[i], n, hp(bw[n]))
     desc = qdit_model_desc()
     desc.shape = qdit_model_shape(cfg.hidden, cfg.heads, cfg.mlp, cfg.depth, cfg.grid, cfg.patch, cfg.channels,
-                                  cfg.num_classes, cfg.freq_dim)
+                                  cfg.num_classes, cfg.freq_dim, weight_bits)
     for n in ("w_patch", "b_patch", "pos", "w_t1", "b_t1", "w_t2", "b_t2", "y_table", "w_ada_f", "b_ada_f", "w_out",
               "b_out"):
         setattr(desc, n, hp(weights[n]))

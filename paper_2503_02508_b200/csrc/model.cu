@@ -102,10 +102,10 @@ int32_t alloc_qlinear(qdit_ctx* ctx, DeviceArena& mem, int64_t N, int64_t K, QLi
 
 // Uploads one f32 linear through the staging buffer and quantizes rows [row0, row0+N) of `l` on the device.
 int32_t quantize_into(qdit_ctx* ctx, float* staging, const float* w, const float* b, int64_t N, int64_t K,
-                      QLinearDev* l, int64_t row0) {
+                      QLinearDev* l, int64_t row0, int bits) {
   if (!w || !b) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "a block weight pointer is NULL");
   QDIT_CUDA_CHECK(ctx, cudaMemcpyAsync(staging, w, static_cast<size_t>(N) * K * sizeof(float), cudaMemcpyHostToDevice, ctx->stream));
-  QDIT_TRY(qdit_quantize_weight(ctx, staging, N, K, l->q + row0 * K, l->scale + row0, l->colsum + row0));
+  QDIT_TRY(qdit_quantize_weight_bits(ctx, staging, N, K, bits, l->q + row0 * K, l->scale + row0, l->colsum + row0));
   QDIT_CUDA_CHECK(ctx, cudaMemcpyAsync(l->bias + row0, b, static_cast<size_t>(N) * sizeof(float), cudaMemcpyHostToDevice, ctx->stream));
   return QDIT_OK;
 }
@@ -135,6 +135,7 @@ int32_t build_model(qdit_ctx* ctx, const qdit_model_desc* desc, qdit_model* m) {
   QDIT_TRY(upload(ctx, m->mem, desc->w_out, od * D, &m->w_out));
   QDIT_TRY(upload(ctx, m->mem, desc->b_out, od, &m->b_out));
 
+  const int wbits = s.weight_bits == 0 ? 8 : s.weight_bits;
   const int64_t big = 6 * D > F ? 6 * D : F;
   float* staging = nullptr;
   if (cudaMalloc(&staging, static_cast<size_t>(big) * (D > F ? D : F) * sizeof(float)) != cudaSuccess) {
@@ -152,11 +153,11 @@ int32_t build_model(qdit_ctx* ctx, const qdit_model_desc* desc, qdit_model* m) {
     if ((st = alloc_qlinear(ctx, m->mem, D, D, &m->proj[i])) != QDIT_OK) break;
     if ((st = alloc_qlinear(ctx, m->mem, F, D, &m->fc1[i])) != QDIT_OK) break;
     if ((st = alloc_qlinear(ctx, m->mem, D, F, &m->fc2[i])) != QDIT_OK) break;
-    if ((st = quantize_into(ctx, staging, b.w_ada, b.b_ada, 6 * D, D, &m->ada_all, static_cast<int64_t>(i) * 6 * D)) != QDIT_OK) break;
-    if ((st = quantize_into(ctx, staging, b.w_qkv, b.b_qkv, 3 * D, D, &m->qkv[i], 0)) != QDIT_OK) break;
-    if ((st = quantize_into(ctx, staging, b.w_proj, b.b_proj, D, D, &m->proj[i], 0)) != QDIT_OK) break;
-    if ((st = quantize_into(ctx, staging, b.w_fc1, b.b_fc1, F, D, &m->fc1[i], 0)) != QDIT_OK) break;
-    if ((st = quantize_into(ctx, staging, b.w_fc2, b.b_fc2, D, F, &m->fc2[i], 0)) != QDIT_OK) break;
+    if ((st = quantize_into(ctx, staging, b.w_ada, b.b_ada, 6 * D, D, &m->ada_all, static_cast<int64_t>(i) * 6 * D, wbits)) != QDIT_OK) break;
+    if ((st = quantize_into(ctx, staging, b.w_qkv, b.b_qkv, 3 * D, D, &m->qkv[i], 0, wbits)) != QDIT_OK) break;
+    if ((st = quantize_into(ctx, staging, b.w_proj, b.b_proj, D, D, &m->proj[i], 0, wbits)) != QDIT_OK) break;
+    if ((st = quantize_into(ctx, staging, b.w_fc1, b.b_fc1, F, D, &m->fc1[i], 0, wbits)) != QDIT_OK) break;
+    if ((st = quantize_into(ctx, staging, b.w_fc2, b.b_fc2, D, F, &m->fc2[i], 0, wbits)) != QDIT_OK) break;
   }
   if (st == QDIT_OK) {
     m->d_scales = m->mem.alloc<float>(m->n_scales());
@@ -322,6 +323,8 @@ int32_t qdit_model_create(qdit_ctx* ctx, const qdit_model_desc* desc, qdit_model
   if (s.hidden <= 0 || s.heads <= 0 || s.mlp <= 0 || s.depth <= 0 || s.grid <= 0 || s.patch <= 0 || s.channels <= 0 ||
       s.num_classes <= 0 || s.freq_dim <= 0)
     return qdit_fail(ctx, QDIT_ERR_SHAPE, "model shape fields must be positive");
+  if (s.weight_bits != 0 && (s.weight_bits < 2 || s.weight_bits > 8))
+    return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "weight_bits = %d outside 2..8 (0 = 8)", s.weight_bits);
   if (s.hidden % s.heads != 0 || (s.hidden / s.heads != 64 && s.hidden / s.heads != 72))
     return qdit_fail(ctx, QDIT_ERR_SHAPE, "head_dim must be 64 or 72");
   if (s.hidden % 16 != 0 || s.mlp % 16 != 0 || s.hidden > 1536) return qdit_fail(ctx, QDIT_ERR_SHAPE, "hidden (<= 1536) and mlp must be multiples of 16");

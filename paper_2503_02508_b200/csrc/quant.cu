@@ -84,7 +84,7 @@ __global__ void absmax_to_scale_kernel(const float* __restrict__ absmax, float* 
 // One CTA per output row: abs-max over K, then codes and their sum.
 __global__ void __launch_bounds__(256) weight_quant_kernel(const float* __restrict__ w, int64_t K,
                                                            int8_t* __restrict__ q, float* __restrict__ w_scale,
-                                                           int32_t* __restrict__ w_colsum) {
+                                                           int32_t* __restrict__ w_colsum, float top) {
   const int64_t n = blockIdx.x;
   const float* row = w + n * K;
   __shared__ float sm[8];
@@ -99,16 +99,16 @@ __global__ void __launch_bounds__(256) weight_quant_kernel(const float* __restri
   __syncthreads();
   m = 0.0f;
   for (int i = 0; i < (blockDim.x >> 5); ++i) m = fmaxf(m, sm[i]);
-  float s = __fdiv_rn(m, 127.0f);
+  float s = __fdiv_rn(m, top);
   if (!(s > 0.0f)) s = 1.0f;
   const float inv = __fdiv_rn(1.0f, s);
   int sum = 0;
   for (int64_t k = threadIdx.x * 4; k < K; k += blockDim.x * 4) {
     const float4 v = *reinterpret_cast<const float4*>(row + k);
-    const int c0 = __float2int_rn(quantize_code(v.x, inv, 0.0f, -127.0f, 127.0f));
-    const int c1 = __float2int_rn(quantize_code(v.y, inv, 0.0f, -127.0f, 127.0f));
-    const int c2 = __float2int_rn(quantize_code(v.z, inv, 0.0f, -127.0f, 127.0f));
-    const int c3 = __float2int_rn(quantize_code(v.w, inv, 0.0f, -127.0f, 127.0f));
+    const int c0 = __float2int_rn(quantize_code(v.x, inv, 0.0f, -top, top));
+    const int c1 = __float2int_rn(quantize_code(v.y, inv, 0.0f, -top, top));
+    const int c2 = __float2int_rn(quantize_code(v.z, inv, 0.0f, -top, top));
+    const int c3 = __float2int_rn(quantize_code(v.w, inv, 0.0f, -top, top));
     sum += c0 + c1 + c2 + c3;
     const uint32_t packed = (c0 & 0xFF) | ((c1 & 0xFF) << 8) | ((c2 & 0xFF) << 16) | (static_cast<uint32_t>(c3 & 0xFF) << 24);
     *reinterpret_cast<uint32_t*>(q + n * K + k) = packed;
@@ -335,16 +335,23 @@ int32_t qdit_quantize_act(qdit_ctx* ctx, const void* x, int x_dtype, int64_t M, 
   return qdit_after_launch(ctx, "act_quant_kernel");
 }
 
-int32_t qdit_quantize_weight(qdit_ctx* ctx, const float* w, int64_t N, int64_t K, void* q, float* w_scale,
+int32_t qdit_quantize_weight_bits(qdit_ctx* ctx, const float* w, int64_t N, int64_t K, int bits, void* q, float* w_scale,
                              int32_t* w_colsum) {
   if (!ctx) return QDIT_ERR_INVALID_ARG;
+  if (bits < 2 || bits > 8) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "bits = %d outside 2..8", bits);
   if (N < 0 || K < 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "negative size");
   if (N == 0 || K == 0) return QDIT_OK;
   if (!w || !q || !w_scale || !w_colsum) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "NULL argument");
   if (K % 4 != 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "K must be a multiple of 4");
   if (!aligned16(w) || (reinterpret_cast<uintptr_t>(q) & 3u)) return qdit_fail(ctx, QDIT_ERR_ALIGN, "w must be 16-byte, q 4-byte aligned");
-  weight_quant_kernel<<<static_cast<unsigned>(N), 256, 0, ctx->stream>>>(w, K, static_cast<int8_t*>(q), w_scale, w_colsum);
+  weight_quant_kernel<<<static_cast<unsigned>(N), 256, 0, ctx->stream>>>(w, K, static_cast<int8_t*>(q), w_scale, w_colsum,
+                                                                         static_cast<float>((1 << (bits - 1)) - 1));
   return qdit_after_launch(ctx, "weight_quant_kernel");
+}
+
+int32_t qdit_quantize_weight(qdit_ctx* ctx, const float* w, int64_t N, int64_t K, void* q, float* w_scale,
+                             int32_t* w_colsum) {
+  return qdit_quantize_weight_bits(ctx, w, N, K, 8, q, w_scale, w_colsum);
 }
 
 int32_t qdit_adaln_modulate(qdit_ctx* ctx, const void* x, int64_t M, int64_t D, int64_t T, float eps,

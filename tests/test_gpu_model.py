@@ -32,11 +32,11 @@ def ctx(q):
 class Rig:
     """GPU model + oracle model built from the same seeded float weights."""
 
-    def __init__(self, q, ctx, cfg, seed):
+    def __init__(self, q, ctx, cfg, seed, weight_bits=8):
         self.q, self.ctx, self.cfg = q, ctx, cfg
         self.w = synth.model_weights(seed, cfg)
-        self.om = dit.make_qmodel(cfg, self.w)
-        self.gm = q.qdit_model_create(ctx, cfg, self.w)
+        self.om = dit.make_qmodel(cfg, self.w, weight_bits)
+        self.gm = q.qdit_model_create(ctx, cfg, self.w, weight_bits)
         self.samplers = []
 
     def set_scales(self, scales):
@@ -184,6 +184,35 @@ def test_forward_tiny_matches_oracle(q, ctx):
         # a smaller batch through the same workspace gives the same per-sample result
         got1 = rig.forward(s, latent[1:2], t[1:2], y[1:2])
         np.testing.assert_array_equal(got1, got[1:2])
+    finally:
+        rig.close()
+
+
+def test_forward_tiny_w4a8_matches_oracle(q, ctx):
+    """4-bit channel-wise weights, 8-bit activations (the W4A8 setting of Table 2) through the same kernels."""
+    cfg = synth.DIT_TINY
+    rig = Rig(q, ctx, cfg, 74, weight_bits=4)
+    try:
+        latent, t, y = _inputs(cfg, 74, 3)
+        scales = calib.calibrate_model(rig.om, [(latent, t, y)])
+        rig.set_scales(scales)
+        s = rig.sampler(batch=3, num_steps=2)
+        got = rig.forward(s, latent, t, y)
+        ref = dit.forward(rig.om, dit.Context(quant="static", scales=scales), latent, t, y)
+        assert rel_l2(got, ref) < 5e-3, rel_l2(got, ref)
+        # the 4-bit model is a different function from the 8-bit one (the option is not silently ignored) ...
+        rig8 = Rig(q, ctx, cfg, 74)
+        try:
+            rig8.set_scales(scales)
+            got8 = rig8.forward(rig8.sampler(batch=3, num_steps=2), latent, t, y)
+        finally:
+            rig8.close()
+        d = rel_l2(got, got8)
+        assert 1e-3 < d < 0.5, d
+        # ... whose weight codes stay inside the 4-bit range
+        lin = q.qdit_model_linear(rig.gm, 0, LINEAR_IDS["fc1"])
+        codes = host_codes(view(lin["w_q"], (lin["N"], lin["K"]), "|i1"))
+        assert codes.min() >= -7 and codes.max() <= 7 and np.abs(codes).max() == 7
     finally:
         rig.close()
 

@@ -114,6 +114,30 @@ def test_quantize_weight_bit_exact(q, ctx, N, K):
     np.testing.assert_array_equal(co.cpu().numpy().astype(np.int64), wc)
 
 
+@pytest.mark.parametrize("bits", [4, 6, 2])
+def test_quantize_weight_bits_bit_exact(q, ctx, bits):
+    """b-bit channel-wise weights (bits = 4: the W4A8 setting of Table 2): codes, scales and code sums."""
+    N, K = 384, 1536
+    W = synth.normal(8, f"w{bits}b", (N, K), 0.02)
+    W[5] = 0
+    qo = torch.empty((N, K), dtype=torch.int8, device="cuda")
+    so = torch.empty(N, dtype=torch.float32, device="cuda")
+    co = torch.empty(N, dtype=torch.int32, device="cuda")
+    q.qdit_quantize_weight_bits(ctx, dev(W), N, K, bits, qo, so, co)
+    q.qdit_sync(ctx)
+    wq, ws, wc = quant.quantize_weight_per_channel(W, bits)
+    top = (1 << (bits - 1)) - 1
+    got = qo.cpu().numpy().astype(np.int32)
+    np.testing.assert_array_equal(got, wq)
+    np.testing.assert_array_equal(so.cpu().numpy(), ws)
+    np.testing.assert_array_equal(co.cpu().numpy().astype(np.int64), wc)
+    assert got.min() == -top and got.max() == top
+    import ctypes as C
+    assert q.lib.qdit_quantize_weight_bits(ctx, dev(W).data_ptr(), N, K, 9, qo.data_ptr(), so.data_ptr(), co.data_ptr()) == q.QDIT_ERR_INVALID_ARG
+    assert q.lib.qdit_quantize_weight_bits(ctx, dev(W).data_ptr(), N, K, 1, qo.data_ptr(), so.data_ptr(), co.data_ptr()) == q.QDIT_ERR_INVALID_ARG
+    q.qdit_sync(ctx)
+
+
 @pytest.mark.parametrize("B,T,D", [(2, 256, 384), (3, 64, 1152), (2, 8, 144), (1, 5, 2048), (5, 7, 8)])
 def test_adaln_modulate_float_outputs(q, ctx, B, T, D):
     M = B * T

@@ -105,6 +105,29 @@ def test_degenerate_range_takes_unit_scale():
     assert quant.qparams_minmax(np.full(5, 2.0, dtype=np.float32)).scale == 1.0
 
 
+@pytest.mark.parametrize("bits", [4, 6, 2])
+def test_weight_per_channel_low_bit(bits):
+    """b-bit weights (bits = 4: the W4A8 setting of Table 2): the grid has 2^bits - 1 levels around zero."""
+    rng = np.random.default_rng(5)
+    W = (rng.standard_normal((7, 64)) * 0.02).astype(np.float32)
+    top = (1 << (bits - 1)) - 1
+    q, s, cs = quant.quantize_weight_per_channel(W, bits)
+    assert q.min() == -top or q.max() == top
+    assert np.abs(q).max() == top and set(np.unique(q)) <= set(range(-top, top + 1))
+    for n in range(7):
+        assert s[n] == np.float32(np.abs(W[n]).max()) / np.float32(top)
+        assert np.abs(W[n] - s[n] * q[n]).max() <= s[n] / 2 * (1 + 1e-5)      # inside the range: half a step
+        assert cs[n] == int(q[n].sum())
+    # a value already on the grid is reproduced exactly; brute force against the definition of Eq. 1
+    Wg = (np.arange(-top, top + 1, dtype=np.float32) * np.float32(0.25)).reshape(1, -1)
+    qg, sg, _ = quant.quantize_weight_per_channel(Wg, bits)
+    np.testing.assert_array_equal(qg[0], np.arange(-top, top + 1))
+    for n in range(2):
+        for k in range(64):
+            want = int(np.clip(np.rint(np.float32(W[n, k]) * (np.float32(1.0) / s[n])), -top, top))
+            assert q[n, k] == want
+
+
 def test_weight_per_channel():
     rng = np.random.default_rng(3)
     W = (rng.standard_normal((9, 40)) * 0.02).astype(np.float32)
