@@ -308,6 +308,14 @@ float* qdit_sampler_latent(qdit_sampler* s);
  * embed -> modulation for all blocks -> blocks computed (i mod N == 0, cache refreshed) or served
  * from the cache -> final layer -> guidance -> DDIM update -> VC. */
 int32_t qdit_sample_step(qdit_ctx* ctx, qdit_sampler* s, int step_index);
+/* Per-block, per-branch cache schedule in place of the global rule (the layer-wise schedules of the cache
+ * methods the paper compares with and builds on, Related Work "Cache"): schedule is a HOST byte array
+ * [num_steps][blocks][2] (attention branch, MLP branch), non-zero = serve that branch's cached output under the
+ * current step's gate, zero = evaluate the branch and refresh its cache entry.  A step whose entries are all
+ * non-zero is the fused skipped step, all zero the refresh step; a mixed step walks the blocks in order.
+ * The array is copied; NULL returns to the global rule.  Reusing an entry that was never stored makes the step
+ * fail with QDIT_ERR_STATE. */
+int32_t qdit_sampler_set_schedule(qdit_ctx* ctx, qdit_sampler* s, const uint8_t* schedule);
 /* Whole trajectory from HOST buffers: copies latent_host/labels_host in, runs steps 0..S-1, copies the
  * final latent to out_host, and synchronises. */
 int32_t qdit_sample(qdit_ctx* ctx, qdit_sampler* s, const float* latent_host, const int32_t* labels_host,

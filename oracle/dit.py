@@ -201,20 +201,29 @@ def gated_residual(ctx: Context, x, gate, branch, tokens: int):
     return store(x + np.asarray(gate, dtype=np.float64)[b] * branch, ctx.storage.resid)
 
 
-def block_forward(ctx: Context, blk: QBlock, x, c, tokens: int, heads: int, index: int = 0, cache=None):
+def block_forward(ctx: Context, blk: QBlock, x, c, tokens: int, heads: int, index: int = 0, cache=None,
+                  reuse_attn: bool = False, reuse_mlp: bool = False):
     """One DiT block.  If `cache` is a dict, the pre-gate branch outputs are written
-    to cache[(index, "attn")] and cache[(index, "mlp")] in the cache storage format."""
+    to cache[(index, "attn")] and cache[(index, "mlp")] in the cache storage format.
+    reuse_attn / reuse_mlp (per-block, per-branch cache schedules): the branch is not evaluated; its cached
+    output enters the residual under the current step's gate, and the cache entry is left as it is."""
     sh_a, sc_a, g_a, sh_m, sc_m, g_m = modulation(ctx, blk, c, index)
-    A = attn_branch(ctx, blk, x, sh_a, sc_a, tokens, heads, index)
-    ctx.emit(f"blk{index}.attn_branch", A)
-    if cache is not None:
-        cache[(index, "attn")] = store(A, ctx.storage.cache)
+    if reuse_attn:
+        A = cache[(index, "attn")]
+    else:
+        A = attn_branch(ctx, blk, x, sh_a, sc_a, tokens, heads, index)
+        ctx.emit(f"blk{index}.attn_branch", A)
+        if cache is not None:
+            cache[(index, "attn")] = store(A, ctx.storage.cache)
     x = gated_residual(ctx, x, g_a, A, tokens)
     ctx.emit(f"blk{index}.x_mid", x)
-    Mo = mlp_branch(ctx, blk, x, sh_m, sc_m, tokens, index)
-    ctx.emit(f"blk{index}.mlp_branch", Mo)
-    if cache is not None:
-        cache[(index, "mlp")] = store(Mo, ctx.storage.cache)
+    if reuse_mlp:
+        Mo = cache[(index, "mlp")]
+    else:
+        Mo = mlp_branch(ctx, blk, x, sh_m, sc_m, tokens, index)
+        ctx.emit(f"blk{index}.mlp_branch", Mo)
+        if cache is not None:
+            cache[(index, "mlp")] = store(Mo, ctx.storage.cache)
     x = gated_residual(ctx, x, g_m, Mo, tokens)
     ctx.emit(f"blk{index}.x_out", x)
     return x
@@ -295,12 +304,20 @@ def final_layer(model: QModel, x, c, B: int):
     return unpatchify(model.cfg, h @ w["w_out"].T + w["b_out"], B)
 
 
-def forward(model: QModel, ctx: Context, latent, t, y, cache=None, reuse: bool = False):
+def forward(model: QModel, ctx: Context, latent, t, y, cache=None, reuse: bool = False, mask=None):
     """One network evaluation -> [B, 2C, Hl, Wl] (noise prediction in the first C channels).
 
     reuse=False: every block is computed (and written to `cache` if given).
     reuse=True : every block is skipped and served from `cache`.
+    mask       : optional [blocks, 2] booleans (attention branch, MLP branch), True = serve that branch from the
+                 cache.  All True is the fully skipped step above, all False the refresh step; a mixed mask walks
+                 the blocks in order, each reused branch entering the residual like a computed one.
     """
+    if mask is not None:
+        mask = np.asarray(mask, dtype=bool).reshape(len(model.blocks), 2)
+        reuse = bool(mask.all())
+        if reuse or not mask.any():
+            mask = None
     cfg = model.cfg
     B = latent.shape[0]
     x = embed(model, ctx, latent)
@@ -311,6 +328,7 @@ def forward(model: QModel, ctx: Context, latent, t, y, cache=None, reuse: bool =
         x = blocks_reuse(ctx, model.blocks, x, c, cfg.tokens, cache)
     else:
         for i, blk in enumerate(model.blocks):
-            x = block_forward(ctx, blk, x, c, cfg.tokens, cfg.heads, i, cache)
+            ra, rm = (bool(mask[i, 0]), bool(mask[i, 1])) if mask is not None else (False, False)
+            x = block_forward(ctx, blk, x, c, cfg.tokens, cfg.heads, i, cache, ra, rm)
     ctx.emit("x_final", x)
     return final_layer(model, x, c, B)

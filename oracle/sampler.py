@@ -72,6 +72,8 @@ class SamplerConfig:
     vc_mode: str = "k_table"               # or "var_ratio" (table = target variances)
     vc_eps: float = 1e-6
     use_cache: bool = True                 # False: plain un-cached loop (every step computes, nothing stored)
+    schedule: Optional[np.ndarray] = None  # [S, blocks, 2] booleans: per step, block and branch, True = reuse the
+                                           # cached output (replaces the global rule "i mod N == 0 refreshes")
 
 
 def sample(model: dit.QModel, ctx: dit.Context, scfg: SamplerConfig, latent, labels, on_step=None):
@@ -90,7 +92,11 @@ def sample(model: dit.QModel, ctx: dit.Context, scfg: SamplerConfig, latent, lab
         else:
             xin, tin, yin = x, t, labels
         reuse = scfg.use_cache and not should_refresh(i, scfg.cache_interval)
-        out = dit.forward(model, ctx, xin, tin, yin, cache=cache, reuse=reuse)
+        mask = None
+        if scfg.use_cache and scfg.schedule is not None:
+            mask = np.asarray(scfg.schedule, dtype=bool)[i]
+            reuse = bool(mask.all())
+        out = dit.forward(model, ctx, xin, tin, yin, cache=cache, reuse=reuse, mask=mask)
         eps = out[:, :C]
         if scfg.guidance is not None:
             eps = cfg_combine(eps, scfg.guidance)

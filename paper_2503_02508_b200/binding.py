@@ -100,6 +100,7 @@ _SIGNATURES = {
     "qdit_sampler_destroy": (_i32, [_vp]),
     "qdit_sampler_reset": (_i32, [_vp, _vp, _vp, _vp]),
     "qdit_sampler_latent": (_vp, [_vp]),
+    "qdit_sampler_set_schedule": (_i32, [_vp, _vp, _vp]),
     "qdit_sample_step": (_i32, [_vp, _vp, _int]),
     "qdit_sample": (_i32, [_vp, _vp, _vp, _vp, _vp]),
     "qdit_forward": (_i32, [_vp, _vp, _vp, _vp, _vp, _int, _vp, _u32]),
@@ -347,6 +348,15 @@ def qdit_sampler_reset(ctx, s, latent, labels):
 
 def qdit_sampler_latent(s):
     return lib.qdit_sampler_latent(s)
+
+
+def qdit_sampler_set_schedule(ctx, s, schedule):
+    """schedule: array-like [num_steps, blocks, 2] of reuse flags, or None for the global rule."""
+    import numpy as np
+    if schedule is None:
+        return check(ctx, lib.qdit_sampler_set_schedule(ctx, s, None))
+    a = np.ascontiguousarray(np.asarray(schedule) != 0, dtype=np.uint8)
+    return check(ctx, lib.qdit_sampler_set_schedule(ctx, s, a.ctypes.data))
 
 
 def qdit_sample_step(ctx, s, step_index):

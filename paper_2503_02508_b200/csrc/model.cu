@@ -75,6 +75,7 @@ struct qdit_sampler {
   qdit_cache* cache;
   std::vector<DdimCoef> ddim;
   std::vector<float> t_host;
+  std::vector<uint8_t> schedule;  // [S][depth][2] per-branch reuse flags; empty = global rule
   int next_step;
 };
 
@@ -198,9 +199,11 @@ int32_t dyn_quant(qdit_ctx* ctx, qdit_sampler* s, int slot, const float* x, int6
 
 // `pre_mod` / `pre_modf`: modulation [B, depth*6D] and final-layer modulation [B, 2D] evaluated beforehand for this
 // step (both or neither); without them the conditioning path runs here.
+// `mask`: [depth][2] per-branch reuse flags of a mixed step (needs STORE_CACHE; a flagged branch is not evaluated,
+// its cached output enters the residual under this step's gate).
 static int32_t forward_impl(qdit_ctx* ctx, qdit_sampler* s, const float* latent, int latent_batch, const float* t,
                             const int32_t* y, int B, float* out, uint32_t flags, const float* pre_mod = nullptr,
-                            const float* pre_modf = nullptr) {
+                            const float* pre_modf = nullptr, const uint8_t* mask = nullptr) {
   qdit_model* m = s->model;
   const qdit_model_shape& sh = m->s;
   const int D = sh.hidden, F = sh.mlp, T = sh.grid * sh.grid, depth = sh.depth;
@@ -247,24 +250,32 @@ static int32_t forward_impl(qdit_ctx* ctx, qdit_sampler* s, const float* latent,
       uint32_t gflags = QDIT_EPI_GATE | QDIT_EPI_RESIDUAL | QDIT_EPI_OUT_BF16 | (store ? QDIT_EPI_CACHE_STORE : 0u);
       if (!calib) {
         // ---- attention branch, fused quantizers
-        QDIT_TRY(qdit_adaln_modulate(ctx, s->x, M, D, T, 1e-6f, mod, mod + D, ld_mod, s->h, QDIT_I8, &qp, sc_qkv));
-        qdit_epilogue e0{};
-        QDIT_TRY(run_linear(ctx, s->h, m->qkv[i], M, sc_qkv, QDIT_EPI_OUT_BF16, e0, s->qkv));
-        const __nv_bfloat16* qkv = static_cast<const __nv_bfloat16*>(s->qkv);
-        QDIT_TRY(qdit_attention(ctx, qkv, qkv + D, qkv + 2 * D, 3 * D, B, sh.heads, T, D / sh.heads, att_scale, s->a,
-                                QDIT_I8, &qp, sc_proj));
-        gated.gate = mod + 2 * D;
-        gated.cache_out = store ? qdit_cache_slot(s->cache, i, QDIT_BRANCH_ATTN, 1) : nullptr;
-        QDIT_TRY(run_linear(ctx, s->a, m->proj[i], M, sc_proj, gflags, gated, s->x));
+        if (mask && mask[2 * i]) {
+          QDIT_TRY(qdit_cache_reuse(ctx, s->cache, i, QDIT_BRANCH_ATTN, mod + 2 * D, ld_mod, T, s->x));
+        } else {
+          QDIT_TRY(qdit_adaln_modulate(ctx, s->x, M, D, T, 1e-6f, mod, mod + D, ld_mod, s->h, QDIT_I8, &qp, sc_qkv));
+          qdit_epilogue e0{};
+          QDIT_TRY(run_linear(ctx, s->h, m->qkv[i], M, sc_qkv, QDIT_EPI_OUT_BF16, e0, s->qkv));
+          const __nv_bfloat16* qkv = static_cast<const __nv_bfloat16*>(s->qkv);
+          QDIT_TRY(qdit_attention(ctx, qkv, qkv + D, qkv + 2 * D, 3 * D, B, sh.heads, T, D / sh.heads, att_scale, s->a,
+                                  QDIT_I8, &qp, sc_proj));
+          gated.gate = mod + 2 * D;
+          gated.cache_out = store ? qdit_cache_slot(s->cache, i, QDIT_BRANCH_ATTN, 1) : nullptr;
+          QDIT_TRY(run_linear(ctx, s->a, m->proj[i], M, sc_proj, gflags, gated, s->x));
+        }
         // ---- MLP branch
-        QDIT_TRY(qdit_adaln_modulate(ctx, s->x, M, D, T, 1e-6f, mod + 3 * D, mod + 4 * D, ld_mod, s->h, QDIT_I8, &qp, sc_fc1));
-        qdit_epilogue e1{};
-        e1.out_qp = qp;
-        e1.out_scale_dev = sc_fc2;
-        QDIT_TRY(run_linear(ctx, s->h, m->fc1[i], M, sc_fc1, QDIT_EPI_GELU | QDIT_EPI_QUANT_OUT, e1, s->u));
-        gated.gate = mod + 5 * D;
-        gated.cache_out = store ? qdit_cache_slot(s->cache, i, QDIT_BRANCH_MLP, 1) : nullptr;
-        QDIT_TRY(run_linear(ctx, s->u, m->fc2[i], M, sc_fc2, gflags, gated, s->x));
+        if (mask && mask[2 * i + 1]) {
+          QDIT_TRY(qdit_cache_reuse(ctx, s->cache, i, QDIT_BRANCH_MLP, mod + 5 * D, ld_mod, T, s->x));
+        } else {
+          QDIT_TRY(qdit_adaln_modulate(ctx, s->x, M, D, T, 1e-6f, mod + 3 * D, mod + 4 * D, ld_mod, s->h, QDIT_I8, &qp, sc_fc1));
+          qdit_epilogue e1{};
+          e1.out_qp = qp;
+          e1.out_scale_dev = sc_fc2;
+          QDIT_TRY(run_linear(ctx, s->h, m->fc1[i], M, sc_fc1, QDIT_EPI_GELU | QDIT_EPI_QUANT_OUT, e1, s->u));
+          gated.gate = mod + 5 * D;
+          gated.cache_out = store ? qdit_cache_slot(s->cache, i, QDIT_BRANCH_MLP, 1) : nullptr;
+          QDIT_TRY(run_linear(ctx, s->u, m->fc2[i], M, sc_fc2, gflags, gated, s->x));
+        }
       } else {
         // ---- calibration: every quantizer input is materialised in f32, its range reduced, then quantized
         QDIT_TRY(qdit_adaln_modulate(ctx, s->x, M, D, T, 1e-6f, mod, mod + D, ld_mod, s->tmpf, QDIT_F32, nullptr, nullptr));
@@ -576,6 +587,17 @@ int32_t qdit_sampler_reset(qdit_ctx* ctx, qdit_sampler* s, const float* latent, 
   return QDIT_OK;
 }
 
+int32_t qdit_sampler_set_schedule(qdit_ctx* ctx, qdit_sampler* s, const uint8_t* schedule) {
+  if (!ctx || !s) return QDIT_ERR_INVALID_ARG;
+  if (!schedule) {
+    s->schedule.clear();
+    return QDIT_OK;
+  }
+  const size_t n = static_cast<size_t>(s->d.num_steps) * s->model->s.depth * 2;
+  s->schedule.assign(schedule, schedule + n);
+  return QDIT_OK;
+}
+
 int32_t qdit_sample_step(qdit_ctx* ctx, qdit_sampler* s, int i) {
   if (!ctx || !s) return QDIT_ERR_INVALID_ARG;
   if (s->next_step < 0) return qdit_fail(ctx, QDIT_ERR_STATE, "qdit_sampler_reset has not been called");
@@ -584,6 +606,19 @@ int32_t qdit_sample_step(qdit_ctx* ctx, qdit_sampler* s, int i) {
   const int HW = sh.grid * sh.patch * sh.grid * sh.patch, B = s->d.batch;
   uint32_t flags = 0;
   if (s->d.cache_interval > 1) flags = qdit_cache_should_refresh(i, s->d.cache_interval) ? QDIT_FWD_STORE_CACHE : QDIT_FWD_REUSE;
+  const uint8_t* mask = nullptr;
+  if (!s->schedule.empty()) {
+    // per-branch schedule: all flags set = the fused skipped step, none = the refresh step, else a mixed step
+    const uint8_t* row = s->schedule.data() + static_cast<size_t>(i) * sh.depth * 2;
+    int set = 0;
+    for (int j = 0; j < 2 * sh.depth; ++j) set += row[j] != 0;
+    if (set == 2 * sh.depth) {
+      flags = QDIT_FWD_REUSE;
+    } else {
+      flags = QDIT_FWD_STORE_CACHE;
+      if (set > 0) mask = row;
+    }
+  }
   const float *pre_mod = nullptr, *pre_modf = nullptr;
   if (s->traj_cond) {
     if (i == 0) QDIT_TRY(trajectory_conditioning(ctx, s));
@@ -592,7 +627,7 @@ int32_t qdit_sample_step(qdit_ctx* ctx, qdit_sampler* s, int i) {
     pre_modf = s->traj_modf + row0 * 2 * sh.hidden;
   }
   QDIT_TRY(forward_impl(ctx, s, s->latent, B, s->t_all + static_cast<int64_t>(i) * s->Beff, s->y, s->Beff, s->net, flags, pre_mod,
-                        pre_modf));
+                        pre_modf, mask));
   QDIT_TRY(launch_cfg_ddim(ctx, s->latent, s->net, B, sh.channels, HW, s->d.use_cfg, s->d.guidance, s->ddim[i]));
   if (s->d.vc_mode != QDIT_VC_NONE)
     QDIT_TRY(qdit_vc_correct(ctx, s->latent, B, sh.channels, HW, i, s->d.vc_mode, s->vc_table, s->d.vc_eps));

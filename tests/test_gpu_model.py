@@ -297,6 +297,64 @@ def test_sampler_tiny_matches_oracle(q, ctx, interval, guidance, use_vc):
         rig.close()
 
 
+def test_sampler_per_branch_schedule_matches_oracle(q, ctx):
+    """Per-block, per-branch reuse schedule ([steps, blocks, 2]) against the oracle, and its two reductions."""
+    cfg = synth.DIT_TINY
+    S, B = 8, 2
+    rig, latent, t, y, scales = _forward_case(q, ctx, cfg, 78, B)
+    try:
+        sched = synth.uniform_int(78, "schedule", (S, cfg.depth, 2), 0, 2).astype(bool)
+        sched[0] = False            # the first step fills the cache
+        sched[3] = True             # one fully skipped step
+        sched[5] = False            # one full refresh
+        assert sched[1].any() and not sched[1].all()
+        K = (1.0 + 0.03 * synth.normal(78, "K", (S, cfg.channels))).astype(np.float32)
+
+        def run(schedule, interval=1):
+            sm = rig.sampler(batch=B, num_steps=S, cache_interval=interval, use_cfg=True, guidance=1.5,
+                             vc_mode=q.QDIT_VC_K_TABLE, vc_table=K)
+            q.qdit_sampler_set_schedule(ctx, sm, schedule)
+            out = np.empty_like(latent, dtype=np.float32)
+            l0 = q.qdit_launch_count(ctx)
+            q.qdit_sample(ctx, sm, np.ascontiguousarray(latent, dtype=np.float32), np.ascontiguousarray(y, dtype=np.int32), out)
+            return out.astype(np.float64), q.qdit_launch_count(ctx) - l0
+
+        got, launches = run(sched)
+        ref = sampler.sample(rig.om, dit.Context(quant="static", scales=scales),
+                             sampler.SamplerConfig(S, guidance=1.5, vc_table=K, schedule=sched), latent, y)
+        assert rel_l2(got, ref) < 5e-3, rel_l2(got, ref)
+        # launch accounting: 6 for the trajectory's conditioning; per step embed + final + DDIM + VC; a fully skipped
+        # step one kernel; otherwise 4 kernels per computed attention branch, 3 per computed MLP branch, 1 per reused
+        want = 6
+        for i in range(S):
+            want += 4
+            if sched[i].all():
+                want += 1
+            else:
+                want += int((~sched[i, :, 0]).sum()) * 4 + int((~sched[i, :, 1]).sum()) * 3 + int(sched[i].sum())
+        assert launches == want
+        # the global rule written as a schedule gives the same bits as the built-in rule
+        glob = np.zeros((S, cfg.depth, 2), dtype=bool)
+        glob[1::2] = True
+        a, _ = run(glob)
+        b, _ = run(None, interval=2)
+        np.testing.assert_array_equal(a, b)
+        # NULL schedule returns to the global rule; an all-compute schedule equals interval 1
+        c, _ = run(np.zeros((S, cfg.depth, 2), dtype=bool), interval=2)
+        d, _ = run(None, interval=1)
+        np.testing.assert_array_equal(c, d)
+        # reusing an entry that was never stored is refused
+        bad = np.zeros((S, cfg.depth, 2), dtype=bool)
+        bad[0, 1, 0] = True
+        sm = rig.sampler(batch=B, num_steps=S)
+        q.qdit_sampler_set_schedule(ctx, sm, bad)
+        q.qdit_sampler_reset(ctx, sm, dev(latent), dev(y.astype(np.int32)))
+        assert q.lib.qdit_sample_step(ctx, sm, 0) == q.QDIT_ERR_STATE
+        q.qdit_sync(ctx)
+    finally:
+        rig.close()
+
+
 def test_sampler_step_by_step_and_cache_effect(q, ctx):
     cfg = synth.DIT_TINY
     S, B = 6, 2

@@ -118,6 +118,48 @@ def test_reuse_step_closed_form_and_state_error(tiny):
 
 
 # ----------------------------------------------------------------------------- VC
+def test_per_branch_schedule_reduces_to_the_global_rule_and_to_its_closed_form(tiny):
+    """A [steps, blocks, 2] reuse schedule: the global rule written as a schedule gives the same trajectory bit for
+    bit; an all-compute schedule equals the un-cached loop; a mixed step obeys its block-by-block definition."""
+    cfg, model, latent, labels, scales = tiny
+    ctx = dit.Context(quant="static", scales=scales)
+    S, N = 6, 2
+    glob = np.zeros((S, cfg.depth, 2), dtype=bool)
+    for i in range(S):
+        glob[i] = not sampler.should_refresh(i, N)
+    a = sampler.sample(model, ctx, sampler.SamplerConfig(S, cache_interval=N, guidance=1.5), latent, labels)
+    b = sampler.sample(model, ctx, sampler.SamplerConfig(S, cache_interval=1, guidance=1.5, schedule=glob), latent, labels)
+    np.testing.assert_array_equal(a, b)
+    none = np.zeros((S, cfg.depth, 2), dtype=bool)
+    c = sampler.sample(model, ctx, sampler.SamplerConfig(S, guidance=1.5, schedule=none), latent, labels)
+    d = sampler.sample(model, ctx, sampler.SamplerConfig(S, use_cache=False, guidance=1.5), latent, labels)
+    np.testing.assert_array_equal(c, d)
+    # mixed mask in exact storage: reusing only block 1's attention branch replaces exactly that branch output
+    ex = dit.Context(quant="static", scales=scales, storage=dit.Storage.exact())
+    t0, t1 = np.full(2, 900.0), np.full(2, 800.0)
+    cache = {}
+    dit.forward(model, ex, latent, t0, labels, cache=cache)
+    kept = cache[(1, "attn")].copy()
+    mask = np.zeros((cfg.depth, 2), dtype=bool)
+    mask[1, 0] = True
+    taps = {}
+    ex2 = dit.Context(quant="static", scales=scales, storage=dit.Storage.exact(),
+                      tap=lambda n, v: taps.__setitem__(n, np.array(v)))
+    lat1 = latent * 0.9 + 0.05
+    dit.forward(model, ex2, lat1, t1, labels, cache=cache, mask=mask)
+    np.testing.assert_array_equal(cache[(1, "attn")], kept)                       # a reused entry is not rewritten
+    assert "blk1.attn_branch" not in taps and "blk0.attn_branch" in taps and "blk1.mlp_branch" in taps
+    rows = np.arange(2 * cfg.tokens) // cfg.tokens
+    D = cfg.hidden
+    want_mid = taps["blk0.x_out"] + taps["blk1.mod"][rows, 2 * D:3 * D] * kept    # x + gate_msa(current step) * cached A
+    np.testing.assert_allclose(taps["blk1.x_mid"], want_mid, rtol=1e-13, atol=1e-13)
+    # the other entries were refreshed with this step's values
+    np.testing.assert_array_equal(cache[(1, "mlp")], taps["blk1.mlp_branch"])
+    # a branch that was never stored cannot be reused
+    with pytest.raises(KeyError):
+        dit.forward(model, ex, latent, t1, labels, cache={}, mask=mask)
+
+
 def test_vc_apply_identities():
     rng = np.random.default_rng(3)
     x = rng.standard_normal((3, 4, 8, 8)) * np.array([0.5, 1, 2, 3]).reshape(1, 4, 1, 1) + 0.7
