@@ -51,6 +51,12 @@ int32_t qdit_create(qdit_ctx** out, int device, void* cuda_stream);
 int32_t qdit_destroy(qdit_ctx* ctx);
 /* Waits for the stream; returns QDIT_ERR_TIMEOUT / QDIT_ERR_CUDA if work since the last sync failed. */
 int32_t qdit_sync(qdit_ctx* ctx);
+/* Self-test of the device-side time-out path (the paper has no counterpart): launches one small kernel in which
+ * a bounded wait of `polls` polls (1..2^20) on a barrier that nobody signals runs out, and a second waiting
+ * thread leaves through the CTA's abort flag, exactly as the roles of the pipelined kernels do.  The kernel ends
+ * normally; the next qdit_sync returns QDIT_ERR_TIMEOUT once and the context stays usable.
+ * observed_dev: device int[2], set to {1, 1} when both threads left their wait the intended way. */
+int32_t qdit_selftest_wait_timeout(qdit_ctx* ctx, uint32_t polls, int* observed_dev);
 const char* qdit_status_string(int32_t status);
 const char* qdit_last_error(const qdit_ctx* ctx);
 /* Number of kernels this context has launched since creation (for launch accounting). */

@@ -88,6 +88,7 @@ _SIGNATURES = {
     "qdit_cache_slot": (_vp, [_vp, _int, _int, _int]),
     "qdit_cache_reuse": (_i32, [_vp, _vp, _int, _int, _vp, _i64, _i64, _vp]),
     "qdit_cache_reuse_all": (_i32, [_vp, _vp, _vp, _i64, _i64, _vp]),
+    "qdit_selftest_wait_timeout": (_i32, [_vp, C.c_uint32, _vp]),
     "qdit_vc_correct": (_i32, [_vp, _vp, _int, _int, _int, _int, _int, _vp, _f32]),
     "qdit_vc_fit": (_i32, [_vp, _vp, _vp, _int, _int, _int, _f32, _int, _vp, _vp]),
     "qdit_model_create": (_i32, [_vp, C.POINTER(qdit_model_desc), C.POINTER(_vp)]),
@@ -258,6 +259,10 @@ def qdit_cache_reuse(ctx, cache, block, branch, gate, ld_gate, T, x):
 
 def qdit_cache_reuse_all(ctx, cache, mod_all, ld_mod, T, x):
     return check(ctx, lib.qdit_cache_reuse_all(ctx, cache, ptr(mod_all), ld_mod, T, ptr(x)))
+
+
+def qdit_selftest_wait_timeout(ctx, polls, observed):
+    return check(ctx, lib.qdit_selftest_wait_timeout(ctx, polls, ptr(observed)))
 
 
 def qdit_vc_correct(ctx, latent, B, Cc, HW, step_index, mode, table, eps):

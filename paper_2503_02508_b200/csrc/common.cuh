@@ -56,14 +56,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // (shared) and the device status word (global) and returns false; it also returns false as soon as
 // another thread of the CTA has raised the abort flag, so every role drains to the common exit.
 constexpr uint32_t kSpinLimit = 1u << 24;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+__device__ __forceinline__ bool mbar_wait_limited(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                                  uint32_t limit) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 63u) == 63u && *abort_flag) return false;
   }
   *abort_flag = 1;
   atomicExch(status, 1);
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  return mbar_wait_limited(bar, parity, abort_flag, status, kSpinLimit);
 }
 
 // ----------------------------------------------------------------------------- TMA (no multicast anywhere)

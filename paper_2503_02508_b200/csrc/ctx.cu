@@ -4,6 +4,7 @@
 #include <cstdlib>
 #include <new>
 
+#include "common.cuh"
 #include "internal.h"
 
 int32_t qdit_fail(qdit_ctx* ctx, int32_t code, const char* fmt, ...) {
@@ -62,7 +63,39 @@ ProfScope::~ProfScope() {
   if (on) cudaEventRecord(stop, ctx->stream);
 }
 
+// Self-test of the bounded wait that every pipelined kernel uses: warp 1 waits (with a small poll limit) on a
+// barrier that nobody arrives at, so the wait runs out, raises the CTA's abort flag and the device status word;
+// warp 0 waits on a second such barrier with the full limit and leaves as soon as it sees the abort flag.  The
+// kernel then exits normally: the context stays usable and the next qdit_sync reports the time-out.
+__global__ void wait_timeout_selftest_kernel(uint32_t polls, int* status, int* observed) {
+  __shared__ uint64_t bars[2];
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    qd::mbar_init(&bars[0], 1);
+    qd::mbar_init(&bars[1], 1);
+    abort_flag = 0;
+    qd::mbar_fence_init();
+  }
+  __syncthreads();
+  volatile int* af = &abort_flag;
+  if (threadIdx.x == 32) {
+    const bool ok = qd::mbar_wait_limited(&bars[0], 0, af, status, polls);
+    observed[0] = ok ? 0 : 1;  // 1: the limited wait ran out
+  } else if (threadIdx.x == 0) {
+    const bool ok = qd::mbar_wait(&bars[1], 0, af, status);
+    observed[1] = ok ? 0 : 1;  // 1: left through the abort flag
+  }
+}
+
 extern "C" {
+
+int32_t qdit_selftest_wait_timeout(qdit_ctx* ctx, uint32_t polls, int* observed_dev) {
+  if (!ctx) return QDIT_ERR_INVALID_ARG;
+  if (!observed_dev) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "observed_dev is NULL");
+  if (polls == 0 || polls > (1u << 20)) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "polls must be in 1..2^20");
+  wait_timeout_selftest_kernel<<<1, 64, 0, ctx->stream>>>(polls, ctx->d_status, observed_dev);
+  return qdit_after_launch(ctx, "wait_timeout_selftest_kernel");
+}
 
 int32_t qdit_profile_enable(qdit_ctx* ctx, int enable) {
   if (!ctx) return QDIT_ERR_INVALID_ARG;

@@ -95,22 +95,24 @@ __device__ __forceinline__ void epilogue8(const GemmParams& p, const uint4 lo, c
     acc[0] -= p.a_zp * c0.x; acc[1] -= p.a_zp * c0.y; acc[2] -= p.a_zp * c0.z; acc[3] -= p.a_zp * c0.w;
     acc[4] -= p.a_zp * c1.x; acc[5] -= p.a_zp * c1.y; acc[6] -= p.a_zp * c1.z; acc[7] -= p.a_zp * c1.w;
   }
+  // de-quantisation: one fused multiply-add acc * (s_a s_w) + bias in every kernel and epilogue class (explicit,
+  // so that the result does not depend on what the compiler contracts)
   float f[8];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) f[i] = static_cast<float>(acc[i]) * cp.sc[i];
-  if (flags & QDIT_EPI_BIAS) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) f[i] += cp.bi[i];
-  }
+  for (int i = 0; i < 8; ++i)
+    f[i] = (flags & QDIT_EPI_BIAS) ? __fmaf_rn(static_cast<float>(acc[i]), cp.sc[i], cp.bi[i])
+                                   : __fmul_rn(static_cast<float>(acc[i]), cp.sc[i]);
   if (flags & QDIT_EPI_GELU) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) f[i] = gelu_tanh_f(f[i]);
   }
   if (flags & QDIT_EPI_CACHE_STORE)
     *reinterpret_cast<uint4*>(p.cache_out + static_cast<int64_t>(row) * p.N + n) = pack_bf16x8(f);
+  // gate and residual: one rounded multiply and one rounded add, never a fused multiply-add, so that the
+  // token-major and the channel-major kernels (which add the residual after a transpose) give the same bits
   if (flags & QDIT_EPI_GATE) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) f[i] *= cp.gt[i];
+    for (int i = 0; i < 8; ++i) f[i] = __fmul_rn(f[i], cp.gt[i]);
   }
   if (flags & QDIT_EPI_RESIDUAL) {
     float r[8];
@@ -119,7 +121,7 @@ __device__ __forceinline__ void epilogue8(const GemmParams& p, const uint4 lo, c
     unpack_bf16x2(res.z, r[4], r[5]);
     unpack_bf16x2(res.w, r[6], r[7]);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) f[i] += r[i];
+    for (int i = 0; i < 8; ++i) f[i] = __fadd_rn(f[i], r[i]);
   }
   if (flags & QDIT_EPI_QUANT_OUT) {
     // clip(rne(t) + z, qmin, qmax) == rne(clamp(t, qmin - z, qmax - z)) + z because the bounds are integers;

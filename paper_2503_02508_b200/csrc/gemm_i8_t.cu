@@ -17,9 +17,6 @@
 // taking 32-token chunks in turn.
 #include "gemm_common.cuh"
 
-#ifndef QDIT_FC1_BYTE_STORES
-#define QDIT_FC1_BYTE_STORES 0
-#endif
 
 namespace {
 
@@ -80,17 +77,16 @@ __device__ __forceinline__ void epilogue_chunk_t(const GemmParams& p, const uint
     for (int i = 0; i < 8; ++i) {
       const int j = j0 + i;
       const int acc = static_cast<int>(v[j]) - zcs;
-      float f = static_cast<float>(acc) * sc;
-      if (flags & QDIT_EPI_BIAS) f += bias;
+      float f = (flags & QDIT_EPI_BIAS) ? __fmaf_rn(static_cast<float>(acc), sc, bias) : __fmul_rn(static_cast<float>(acc), sc);
       if (flags & QDIT_EPI_GELU) f = gelu_tanh_f(f);
       if (j < m_end) {
         const int64_t m = m_base + j;
         if (flags & QDIT_EPI_CACHE_STORE) p.cache_out[m * p.N + n] = __float2bfloat16_rn(f);
         if (flags & QDIT_EPI_GATE) {
           if (!gate_uniform) gate = p.gate[(m / p.tokens) * p.ld_gate + n];
-          f *= gate;
+          f = __fmul_rn(f, gate);
         }
-        if (flags & QDIT_EPI_RESIDUAL) f += res[i];
+        if (flags & QDIT_EPI_RESIDUAL) f = __fadd_rn(f, res[i]);
         const int64_t o = m * p.ldo + n;
         if (flags & QDIT_EPI_QUANT_OUT) {
           // clip(rne(t) + z, qmin, qmax) == rne(clamp(t, qmin - z, qmax - z)) + z; adding 1.5 * 2^23 rounds to
@@ -142,31 +138,20 @@ __device__ __forceinline__ void epilogue_chunk_t_packed(const GemmParams& p, con
   float f[32];
   if (p.a_zp == 0) {
 #pragma unroll
-    for (int j = 0; j < 32; ++j) f[j] = static_cast<float>(static_cast<int>(v[j])) * sc;
+    for (int j = 0; j < 32; ++j) f[j] = static_cast<float>(static_cast<int>(v[j]));
   } else {
 #pragma unroll
-    for (int j = 0; j < 32; ++j) f[j] = static_cast<float>(static_cast<int>(v[j]) - zcs) * sc;
+    for (int j = 0; j < 32; ++j) f[j] = static_cast<float>(static_cast<int>(v[j]) - zcs);
   }
 #pragma unroll
   for (int j = 0; j < 32; ++j) {
-    if (flags & QDIT_EPI_BIAS) f[j] += bias;
+    f[j] = (flags & QDIT_EPI_BIAS) ? __fmaf_rn(f[j], sc, bias) : __fmul_rn(f[j], sc);
     if (flags & QDIT_EPI_GELU) f[j] = gelu_tanh_f(f[j]);
   }
   if (flags & QDIT_EPI_QUANT_OUT) {
     // one byte per token: word t = codes of tokens t, 8 + t, 16 + t, 24 + t
     const float lo_f = p.o_qmin - p.o_zp, hi_f = p.o_qmax - p.o_zp;
     const int zp = static_cast<int>(p.o_zp);
-#if QDIT_FC1_BYTE_STORES
-    if (n < p.N) {
-#pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const float q = fminf(fmaxf(__fmul_rn(f[j], o_inv), lo_f), hi_f);
-        const int code = __float_as_int(__fadd_rn(q, 12582912.0f)) + zp;
-        if (m_base + j < p.M) static_cast<uint8_t*>(p.out)[static_cast<int64_t>(m_base + j) * p.ldo + n] = static_cast<uint8_t>(code);
-      }
-    }
-    return;
-#endif
     uint32_t w[8];
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
@@ -232,7 +217,7 @@ __device__ __forceinline__ void epilogue_chunk_t_gated(const GemmParams& p, cons
   const bool n8_ok = n8 < p.N;
   float f[32];
 #pragma unroll
-  for (int j = 0; j < 32; ++j) f[j] = static_cast<float>(static_cast<int>(v[j]) - zcs) * sc + bias;
+  for (int j = 0; j < 32; ++j) f[j] = __fmaf_rn(static_cast<float>(static_cast<int>(v[j]) - zcs), sc, bias);
   // cache copy (pre-gate), bf16
 #pragma unroll
   for (int s2 = 0; s2 < 4; s2 += 2) {
@@ -258,7 +243,7 @@ __device__ __forceinline__ void epilogue_chunk_t_gated(const GemmParams& p, cons
     const bool live = n8_ok && m < p.M;
     uint32_t w[8];
 #pragma unroll
-    for (int t = 0; t < 8; ++t) w[t] = __float_as_uint(f[8 * s4 + t] * gate);
+    for (int t = 0; t < 8; ++t) w[t] = __float_as_uint(__fmul_rn(f[8 * s4 + t], gate));
     transpose8(w, lane);  // w[c] = gated value of channel n8 + c, token m
     if (live) {
       float r[8];
@@ -267,7 +252,7 @@ __device__ __forceinline__ void epilogue_chunk_t_gated(const GemmParams& p, cons
       unpack_bf16x2(rv[s4].z, r[4], r[5]);
       unpack_bf16x2(rv[s4].w, r[6], r[7]);
 #pragma unroll
-      for (int c = 0; c < 8; ++c) r[c] += __uint_as_float(w[c]);
+      for (int c = 0; c < 8; ++c) r[c] = __fadd_rn(__uint_as_float(w[c]), r[c]);
       *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + m * p.ldo + n8) = pack_bf16x8(r);
     }
   }

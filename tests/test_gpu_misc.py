@@ -118,6 +118,28 @@ def test_vc_fit_matches_the_closed_form(q, ctx, N, C, HW):
     assert (j <= objective(kf * 1.01)).all() and (j <= objective(kf * 0.99)).all()
 
 
+def test_bounded_wait_times_out_and_context_stays_usable(q, ctx):
+    """The time-out path of the pipelined kernels, exercised without hanging anything: a wait with a small poll
+    limit on a barrier that nobody signals runs out, a second waiter leaves through the abort flag, the kernel
+    ends normally, qdit_sync reports the time-out once, and the context keeps working."""
+    q.qdit_sync(ctx)
+    obs = torch.zeros(2, dtype=torch.int32, device="cuda")
+    q.qdit_selftest_wait_timeout(ctx, 4096, obs)
+    assert q.lib.qdit_sync(ctx) == q.QDIT_ERR_TIMEOUT
+    assert b"wait" in q.lib.qdit_last_error(ctx)
+    assert obs.cpu().tolist() == [1, 1]
+    assert q.lib.qdit_sync(ctx) == q.QDIT_OK
+    x = synth.normal(64, "after_timeout", (64, 128))
+    out = torch.empty((64, 128), dtype=torch.uint8, device="cuda")
+    q.qdit_quantize_act(ctx, dev(x), q.QDIT_F32, 64, 128, 128, q.QDIT_QUANT_STATIC, q.qparams(0.02), None, out, 128)
+    q.qdit_sync(ctx)
+    want = np.clip(np.rint(x * (np.float32(1.0) / np.float32(0.02))), -127, 127).astype(np.int32)
+    got = out.cpu().numpy().view(np.int8).astype(np.int32)
+    np.testing.assert_array_equal(got, want)
+    assert q.lib.qdit_selftest_wait_timeout(ctx, 0, obs.data_ptr()) == q.QDIT_ERR_INVALID_ARG
+    assert q.lib.qdit_selftest_wait_timeout(ctx, 1 << 21, obs.data_ptr()) == q.QDIT_ERR_INVALID_ARG
+
+
 def test_vc_fit_rejects_bad_arguments(q, ctx):
     import ctypes as C
     x = torch.zeros(4 * 64, dtype=torch.float32, device="cuda")
