@@ -1,4 +1,6 @@
-// Non-causal softmax attention in bf16 between the quantized linears.
+// Non-causal softmax attention in bf16 between the quantized linears: the entry point qdit_attention and the
+// mma.sync kernel that serves token counts that are not a multiple of 128 (the tcgen05 kernel in attention_tc.cu
+// takes all others, among them both image sizes of the paper's experiments).
 //
 // One CTA = 128 (or 64) queries of one (sample, head); one warp per 16 query rows.  Q and 64-key K/V tiles
 // are staged by TMA (a 4-deep ring with mbarrier completion: at 256 tokens the whole K and V of the head are

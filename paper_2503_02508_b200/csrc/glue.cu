@@ -1,5 +1,6 @@
-// Small HBM-/latency-bound kernels around the blocks: block-output cache, variance compensation,
-// guidance + DDIM update, patch embedding, conditioning MLP, final layer.
+// Small HBM-/latency-bound kernels around the blocks: block-output cache, variance compensation (correction and
+// the closed-form fit of its factors), guidance + DDIM update, patch embedding, conditioning MLP (per call and
+// batched over a whole trajectory), final layer.
 #include <cmath>
 #include <new>
 
