@@ -29,18 +29,22 @@ sys.path.insert(0, ROOT)
 import synth  # noqa: E402
 
 METRIC = "DiT-XL/2 W8A8+cache images/s (256^2, 50 steps)"
-METRICS = {"ddim50": METRIC, "ddim100_512": "DiT-XL/2 W8A8+cache images/s (512^2, 100 steps)"}
+METRICS = {"ddim50": METRIC, "ddim100_512": "DiT-XL/2 W8A8+cache images/s (512^2, 100 steps)",
+           "ddpm250": "DiT-XL/2 W8A8+cache images/s (256^2, 250 DDPM steps)"}
 WORKLOADS = {
     # name: (config, seed key, steps, batch, guidance, interval)
     "ddim50": (synth.DIT_XL2, "ddim50_xl2", 50, 16, 1.5, 2),
     "ddim100_512": (synth.DIT_XL2_512, "ddim100_xl2_512", 100, 8, None, 3),
+    # the stochastic 250-step sampler of the paper's baseline row (noise supplied as an input), W8A8 + cache
+    "ddpm250": (synth.DIT_XL2, "ddim50_xl2", 250, 16, 1.5, 2),
 }
+STOCHASTIC = {"ddpm250"}
 
 
 # DRAM bytes (read + written) per GEMM launch, from the ncu capture summarised in
-# profiles/gemm_i8_layers_m8192_sections.txt: QKV 18.9 MB, proj 29.9 MB, fc1 15.3 MB, fc2 65.7 MB per launch at
+# profiles/gemm_i8_layers_m8192_sections.txt: QKV 17.2 MB, proj 30.0 MB, fc1 15.5 MB, fc2 65.4 MB per launch at
 # M = 8192 (the shapes of the 50-step workload); each layer is 700 of the trajectory's 2801 GEMM launches.
-NCU_GEMM_DRAM_BYTES_PER_LAUNCH = 700 * (18.9e6 + 29.9e6 + 15.3e6 + 65.7e6) / 2801
+NCU_GEMM_DRAM_BYTES_PER_LAUNCH = 700 * (17.2e6 + 30.0e6 + 15.5e6 + 65.4e6) / 2801
 
 
 def measured_peaks():
@@ -146,11 +150,13 @@ def oracle_sample_rate(name, n_images=1, n_steps=2):
     weights = synth.model_weights(seed, cfg)
     model = dit.make_qmodel(cfg, weights)
     lat, lab = latent[:n_images], labels[:n_images]
-    t0 = np.full(n_images, 980.0 if steps == 50 else 990.0)
+    t0 = np.full(n_images, float((steps - 1) * (1000 // steps)))
     scales = calib.calibrate_model(model, [(lat, t0, lab)])
     ctx = dit.Context(quant="static", scales=scales)
     stamps = []
-    full = osampler.SamplerConfig(steps, cache_interval=interval, guidance=guidance, vc_table=vc_table)
+    kind = "ddpm" if name in STOCHASTIC else "ddim"
+    noise = synth.normal(seed, "noise", (n_steps, n_images) + latent.shape[1:]) if kind == "ddpm" else None
+    full = osampler.SamplerConfig(steps, cache_interval=interval, guidance=guidance, vc_table=vc_table, kind=kind, noise=noise)
 
     class Stop(Exception):
         pass
@@ -249,6 +255,13 @@ def run_ours(args):
     q.qdit_model_finish_calibration(ctx, model)
     q.qdit_sync(ctx)
 
+    if args.workload in STOCHASTIC:
+        gen = torch.Generator(device="cuda")
+        gen.manual_seed(seed + rank)
+        noise_d = torch.randn((steps, batch, cfg.channels, cfg.latent_side, cfg.latent_side), generator=gen,
+                              dtype=torch.float32, device="cuda")
+        q.qdit_sampler_set_ddpm(ctx, sampler, noise_d)
+
     def trajectory_device():
         q.qdit_sampler_reset(ctx, sampler, lat_d, lab_d)
         for i in range(steps):
@@ -338,6 +351,7 @@ def run_ours(args):
             "config": {"workload": args.workload, "model": "DiT-XL/2", "batch_per_gpu": batch, "network_batch": beff,
                        "sampling_steps": steps, "cache_interval": interval, "guidance": guidance,
                        "vc": "k_table every step", "residual_stream": "bf16", "weight_bits": args.weight_bits,
+                       "sampler": "ddpm (noise supplied)" if args.workload in STOCHASTIC else "ddim",
                        "l2": "per-step working set (0.45 GB weights + 1.06 GB cache) exceeds L2; no flush needed",
                        "roofline_pass": "one extra trajectory with per-launch CUDA events, outside the timed region"},
             "clocks": clock_info,

@@ -322,6 +322,16 @@ int32_t qdit_sample_step(qdit_ctx* ctx, qdit_sampler* s, int step_index);
  * The array is copied; NULL returns to the global rule.  Reusing an entry that was never stored makes the step
  * fail with QDIT_ERR_STATE. */
 int32_t qdit_sampler_set_schedule(qdit_ctx* ctx, qdit_sampler* s, const uint8_t* schedule);
+/* The stochastic sampler of the Experimental Settings ("DDPM") in place of the deterministic update: the
+ * ancestral step of the cited DDPM papers on the same evenly spaced timestep subset, betas re-derived for the
+ * subset (beta'_k = 1 - ab_k / ab_{k-1}):
+ *   x0 = x / sqrt(ab_k) - sqrt(1/ab_k - 1) eps,   mean = coef_x0 x0 + coef_xt x   (posterior q(x_{k-1} | x_k, x0)),
+ *   log var = f log beta'_k + (1 - f) log beta~_k,  f = (v + 1)/2,  v = the network's second output group
+ *   (learned variance; of the conditional half under guidance),   x <- mean + [k > 0] exp(log var / 2) * noise.
+ * noise: DEVICE f32 [num_steps, batch, C, Hl*Wl] standard-normal numbers supplied by the caller (borrowed: must
+ * stay valid while the sampler steps; the last step's slice is not read); NULL returns to DDIM.  Needs
+ * num_steps >= 2.  Guidance, cache schedule and VC apply as with DDIM. */
+int32_t qdit_sampler_set_ddpm(qdit_ctx* ctx, qdit_sampler* s, const float* noise);
 /* Whole trajectory from HOST buffers: copies latent_host/labels_host in, runs steps 0..S-1, copies the
  * final latent to out_host, and synchronises. */
 int32_t qdit_sample(qdit_ctx* ctx, qdit_sampler* s, const float* latent_host, const int32_t* labels_host,

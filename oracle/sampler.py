@@ -15,6 +15,14 @@ the last step alpha_bar_prev = 1.  Classifier-free guidance evaluates the
 network on [conditional; unconditional (label = num_classes)] and combines
 eps = eps_u + g * (eps_c - eps_u) on the C noise channels.  VC (module vc) is
 applied to the latent after every update.
+
+The stochastic sampler of the Experimental Settings ("DDPM") is available as kind="ddpm": the ancestral step of
+the cited DDPM / improved-DDPM papers on the same timestep subset, with the betas re-derived for the subset
+(beta'_k = 1 - ab_k / ab_{k-1}), the mean from the predicted noise and the variance interpolated in the log
+domain between beta'_k and the posterior variance by the network's second output group (the "learned sigma"
+channels), v in [-1, 1].  The Gaussian noise of every step is an INPUT ([S, B, C, H, W]), so that both
+implementations see the same numbers.  Readings: under guidance v is taken from the conditional half; no
+clipping of the predicted x0.
 """
 from __future__ import annotations
 
@@ -49,6 +57,41 @@ def ddim_table(num_steps: int):
     return rows
 
 
+def ddpm_table(num_steps: int):
+    """Per sampling step i (t descending): (t_i, 1/sqrt(ab), sqrt(1/ab - 1), coef_x0, coef_xt, log beta',
+    log posterior variance (clipped at the last step), noise factor 0/1), float64, betas re-derived for the subset."""
+    if num_steps < 2:
+        raise ValueError("the stochastic sampler needs at least two steps")
+    betas = np.linspace(1e-4, 2e-2, TRAIN_STEPS, dtype=np.float64)
+    ab_full = np.cumprod(1.0 - betas)
+    stride = TRAIN_STEPS // num_steps
+    ts = np.array([k * stride for k in range(num_steps)])          # ascending
+    ab = ab_full[ts]
+    ab_prev = np.concatenate([[1.0], ab[:-1]])
+    beta = 1.0 - ab / ab_prev
+    post_var = beta * (1.0 - ab_prev) / (1.0 - ab)
+    log_post = np.log(np.concatenate([post_var[1:2], post_var[1:]]))
+    coef_x0 = beta * np.sqrt(ab_prev) / (1.0 - ab)
+    coef_xt = (1.0 - ab_prev) * np.sqrt(1.0 - beta) / (1.0 - ab)
+    rows = []
+    for i in range(num_steps):
+        k = num_steps - 1 - i
+        rows.append((int(ts[k]), 1.0 / np.sqrt(ab[k]), np.sqrt(1.0 / ab[k] - 1.0), coef_x0[k], coef_xt[k],
+                     np.log(beta[k]), log_post[k], 1.0 if k > 0 else 0.0))
+    return rows
+
+
+def ddpm_update(x, eps, v, row, noise):
+    """x_prev = mean + [k > 0] exp(0.5 logvar) noise;  x0 = x/sqrt(ab) - sqrt(1/ab - 1) eps,
+    mean = coef_x0 x0 + coef_xt x,  logvar = f log beta' + (1 - f) log beta~,  f = (v + 1)/2."""
+    _, sr, srm1, c0, ct, lb, lp, nz = row
+    x0 = sr * x - srm1 * eps
+    mean = c0 * x0 + ct * x
+    f = (np.asarray(v, dtype=np.float64) + 1.0) / 2.0
+    logvar = f * lb + (1.0 - f) * lp
+    return mean + nz * np.exp(0.5 * logvar) * np.asarray(noise, dtype=np.float64)
+
+
 def cfg_combine(eps_both, guidance: float):
     """eps_both [2B,C,...] = [cond; uncond] -> eps_u + g*(eps_c - eps_u)  [B,C,...]."""
     B = eps_both.shape[0] // 2
@@ -72,6 +115,8 @@ class SamplerConfig:
     vc_mode: str = "k_table"               # or "var_ratio" (table = target variances)
     vc_eps: float = 1e-6
     use_cache: bool = True                 # False: plain un-cached loop (every step computes, nothing stored)
+    kind: str = "ddim"                     # or "ddpm": stochastic ancestral step with learned variance
+    noise: Optional[np.ndarray] = None     # ddpm: standard-normal noise [S, B, C, Hl, Wl]
     schedule: Optional[np.ndarray] = None  # [S, blocks, 2] booleans: per step, block and branch, True = reuse the
                                            # cached output (replaces the global rule "i mod N == 0 refreshes")
 
@@ -81,7 +126,9 @@ def sample(model: dit.QModel, ctx: dit.Context, scfg: SamplerConfig, latent, lab
     x = np.asarray(latent, dtype=np.float64)
     B, C = x.shape[0], model.cfg.channels
     labels = np.asarray(labels, dtype=np.int64)
-    table = ddim_table(scfg.num_steps)
+    if scfg.kind not in ("ddim", "ddpm"):
+        raise ValueError(scfg.kind)
+    table = ddim_table(scfg.num_steps) if scfg.kind == "ddim" else ddpm_table(scfg.num_steps)
     cache = {} if scfg.use_cache else None
     for i, row in enumerate(table):
         t = np.full(B, row[0], dtype=np.float64)
@@ -98,9 +145,13 @@ def sample(model: dit.QModel, ctx: dit.Context, scfg: SamplerConfig, latent, lab
             reuse = bool(mask.all())
         out = dit.forward(model, ctx, xin, tin, yin, cache=cache, reuse=reuse, mask=mask)
         eps = out[:, :C]
+        v = out[:B, C:2 * C]                # learned-variance channels (of the conditional half under guidance)
         if scfg.guidance is not None:
             eps = cfg_combine(eps, scfg.guidance)
-        x = ddim_update(x, eps, row)
+        if scfg.kind == "ddim":
+            x = ddim_update(x, eps, row)
+        else:
+            x = ddpm_update(x, eps, v, row, scfg.noise[i])
         if scfg.vc_table is not None:
             x = vc.apply(x, scfg.vc_table[i], mode=scfg.vc_mode, eps=scfg.vc_eps)
         x = dit.store(x, "f32")            # the latent lives in float32 between steps

@@ -102,6 +102,7 @@ _SIGNATURES = {
     "qdit_sampler_reset": (_i32, [_vp, _vp, _vp, _vp]),
     "qdit_sampler_latent": (_vp, [_vp]),
     "qdit_sampler_set_schedule": (_i32, [_vp, _vp, _vp]),
+    "qdit_sampler_set_ddpm": (_i32, [_vp, _vp, _vp]),
     "qdit_sample_step": (_i32, [_vp, _vp, _int]),
     "qdit_sample": (_i32, [_vp, _vp, _vp, _vp, _vp]),
     "qdit_forward": (_i32, [_vp, _vp, _vp, _vp, _vp, _int, _vp, _u32]),
@@ -353,6 +354,11 @@ def qdit_sampler_reset(ctx, s, latent, labels):
 
 def qdit_sampler_latent(s):
     return lib.qdit_sampler_latent(s)
+
+
+def qdit_sampler_set_ddpm(ctx, s, noise):
+    """noise: device tensor [num_steps, batch, C, Hl, Wl] f32 (kept alive by the caller), or None for DDIM."""
+    return check(ctx, lib.qdit_sampler_set_ddpm(ctx, s, ptr(noise)))
 
 
 def qdit_sampler_set_schedule(ctx, s, schedule):

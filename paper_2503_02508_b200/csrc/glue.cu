@@ -189,6 +189,30 @@ __global__ void __launch_bounds__(256) cfg_ddim_kernel(float* __restrict__ laten
   latent[idx] = k.sqrt_ab_prev * x0 + k.sqrt_1mab_prev * eps;
 }
 
+// Stochastic (ancestral) step with learned variance: the network's second output group v in [-1, 1] interpolates
+// the log variance between beta' and the posterior variance; v comes from the conditional half under guidance.
+__global__ void __launch_bounds__(256) cfg_ddpm_kernel(float* __restrict__ latent, const float* __restrict__ net,
+                                                       const float* __restrict__ noise, int B, int C, int HW, int use_cfg,
+                                                       float guidance, DdpmCoef k) {
+  const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int64_t per_sample = static_cast<int64_t>(C) * HW;
+  if (idx >= B * per_sample) return;
+  const int64_t b = idx / per_sample;
+  const int64_t r = idx - b * per_sample;  // c*HW + i
+  float eps = net[b * 2 * per_sample + r];
+  const float v = net[b * 2 * per_sample + per_sample + r];
+  if (use_cfg) {
+    const float eu = net[(b + B) * 2 * per_sample + r];
+    eps = eu + guidance * (eps - eu);
+  }
+  const float x = latent[idx];
+  const float x0 = k.rs * x - k.rsm1 * eps;
+  const float mean = k.c_x0 * x0 + k.c_xt * x;
+  const float f = (v + 1.0f) * 0.5f;
+  const float logvar = f * k.log_beta + (1.0f - f) * k.log_post;
+  latent[idx] = k.nz != 0.0f ? mean + expf(0.5f * logvar) * noise[idx] : mean;  // the last step draws no noise
+}
+
 // ----------------------------------------------------------------------------- patch embedding
 // x[m,:] = bf16(W_patch . patch(m) + b_patch + pos[t,:]); patch vector ordered (c, py, px).
 // CTA = 32 token rows x 512 columns.  The weights come TRANSPOSED (wT[j][d], made once when the model is
@@ -623,6 +647,14 @@ int32_t launch_cfg_ddim(qdit_ctx* ctx, float* latent, const float* net, int B, i
   cfg_ddim_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, ctx->stream>>>(latent, net, B, C, HW, use_cfg,
                                                                                   guidance, k);
   return qdit_after_launch(ctx, "cfg_ddim_kernel");
+}
+
+int32_t launch_cfg_ddpm(qdit_ctx* ctx, float* latent, const float* net, const float* noise, int B, int C, int HW,
+                        int use_cfg, float guidance, const DdpmCoef& k) {
+  const int64_t n = static_cast<int64_t>(B) * C * HW;
+  cfg_ddpm_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, ctx->stream>>>(latent, net, noise, B, C, HW, use_cfg,
+                                                                                  guidance, k);
+  return qdit_after_launch(ctx, "cfg_ddpm_kernel");
 }
 
 // ================================================================================ cache object

@@ -6,6 +6,12 @@ struct DdimCoef {
   float sqrt_ab_t, sqrt_1mab_t, sqrt_ab_prev, sqrt_1mab_prev;
 };
 
+// Coefficients of one stochastic (DDPM) step: x0 = rs * x - rsm1 * eps, mean = c_x0 * x0 + c_xt * x,
+// log variance = f * log_beta + (1 - f) * log_post with f = (v + 1) / 2, noise factor nz (0 at the last step).
+struct DdpmCoef {
+  float rs, rsm1, c_x0, c_xt, log_beta, log_post, nz;
+};
+
 // x[m,:] = bf16(W_patch . patch(m) + b + pos); sample b reads latent[b % latent_batch]; wT = W_patch transposed [pd][D].
 int32_t launch_embed(qdit_ctx* ctx, const float* latent, int latent_batch, const float* wT, const float* bias,
                      const float* pos, void* x, int64_t M, int D, int grid, int patch, int C);
@@ -29,3 +35,6 @@ int32_t launch_final(qdit_ctx* ctx, const void* x, int64_t M, int D, int T, floa
 // guidance combine + DDIM (eta = 0) update of latent [B,C,HW] from net [Beff,2C,HW]
 int32_t launch_cfg_ddim(qdit_ctx* ctx, float* latent, const float* net, int B, int C, int HW, int use_cfg,
                         float guidance, const DdimCoef& k);
+// guidance combine + stochastic step with learned variance; noise: f32 [B,C,HW] standard normal for this step
+int32_t launch_cfg_ddpm(qdit_ctx* ctx, float* latent, const float* net, const float* noise, int B, int C, int HW,
+                        int use_cfg, float guidance, const DdpmCoef& k);

@@ -74,6 +74,8 @@ struct qdit_sampler {
   bool traj_cond;                // buffers allocated (the trajectory's modulation fits the memory budget)
   qdit_cache* cache;
   std::vector<DdimCoef> ddim;
+  std::vector<DdpmCoef> ddpm;    // filled when the stochastic sampler is selected
+  const float* noise;            // device [S, batch, C, HW] standard-normal noise of the stochastic sampler, or null
   std::vector<float> t_host;
   std::vector<uint8_t> schedule;  // [S][depth][2] per-branch reuse flags; empty = global rule
   int next_step;
@@ -445,6 +447,7 @@ int32_t qdit_sampler_create(qdit_ctx* ctx, qdit_model* m, const qdit_sampler_des
   s->cache = nullptr;
   s->vc_table = nullptr;
   s->next_step = -1;
+  s->noise = nullptr;
   const qdit_model_shape& sh = m->s;
   const int D = sh.hidden, F = sh.mlp, T = sh.grid * sh.grid, C = sh.channels;
   const int HW = sh.grid * sh.patch * sh.grid * sh.patch;
@@ -587,6 +590,47 @@ int32_t qdit_sampler_reset(qdit_ctx* ctx, qdit_sampler* s, const float* latent, 
   return QDIT_OK;
 }
 
+int32_t qdit_sampler_set_ddpm(qdit_ctx* ctx, qdit_sampler* s, const float* noise) {
+  if (!ctx || !s) return QDIT_ERR_INVALID_ARG;
+  s->noise = noise;
+  if (!noise) return QDIT_OK;
+  const int S = s->d.num_steps;
+  if (S < 2) {
+    s->noise = nullptr;
+    return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "the stochastic sampler needs at least two steps");
+  }
+  // alpha_bar of the kept timesteps (ascending), betas re-derived for the subset, posterior q(x_{k-1} | x_k, x0)
+  std::vector<double> ab_full(1000);
+  double prod = 1.0;
+  for (int j = 0; j < 1000; ++j) {
+    prod *= 1.0 - (1e-4 + (2e-2 - 1e-4) * static_cast<double>(j) / 999.0);
+    ab_full[j] = prod;
+  }
+  const int stride = 1000 / S;
+  std::vector<double> ab(S), beta(S), post(S);
+  for (int k = 0; k < S; ++k) {
+    ab[k] = ab_full[k * stride];
+    const double abp = k > 0 ? ab[k - 1] : 1.0;
+    beta[k] = 1.0 - ab[k] / abp;
+    post[k] = beta[k] * (1.0 - abp) / (1.0 - ab[k]);
+  }
+  s->ddpm.resize(S);
+  for (int i = 0; i < S; ++i) {
+    const int k = S - 1 - i;
+    const double abp = k > 0 ? ab[k - 1] : 1.0;
+    DdpmCoef c;
+    c.rs = static_cast<float>(1.0 / std::sqrt(ab[k]));
+    c.rsm1 = static_cast<float>(std::sqrt(1.0 / ab[k] - 1.0));
+    c.c_x0 = static_cast<float>(beta[k] * std::sqrt(abp) / (1.0 - ab[k]));
+    c.c_xt = static_cast<float>((1.0 - abp) * std::sqrt(1.0 - beta[k]) / (1.0 - ab[k]));
+    c.log_beta = static_cast<float>(std::log(beta[k]));
+    c.log_post = static_cast<float>(std::log(post[k > 0 ? k : 1]));
+    c.nz = k > 0 ? 1.0f : 0.0f;
+    s->ddpm[i] = c;
+  }
+  return QDIT_OK;
+}
+
 int32_t qdit_sampler_set_schedule(qdit_ctx* ctx, qdit_sampler* s, const uint8_t* schedule) {
   if (!ctx || !s) return QDIT_ERR_INVALID_ARG;
   if (!schedule) {
@@ -628,7 +672,12 @@ int32_t qdit_sample_step(qdit_ctx* ctx, qdit_sampler* s, int i) {
   }
   QDIT_TRY(forward_impl(ctx, s, s->latent, B, s->t_all + static_cast<int64_t>(i) * s->Beff, s->y, s->Beff, s->net, flags, pre_mod,
                         pre_modf, mask));
-  QDIT_TRY(launch_cfg_ddim(ctx, s->latent, s->net, B, sh.channels, HW, s->d.use_cfg, s->d.guidance, s->ddim[i]));
+  if (s->noise) {
+    QDIT_TRY(launch_cfg_ddpm(ctx, s->latent, s->net, s->noise + static_cast<int64_t>(i) * B * sh.channels * HW, B, sh.channels,
+                             HW, s->d.use_cfg, s->d.guidance, s->ddpm[i]));
+  } else {
+    QDIT_TRY(launch_cfg_ddim(ctx, s->latent, s->net, B, sh.channels, HW, s->d.use_cfg, s->d.guidance, s->ddim[i]));
+  }
   if (s->d.vc_mode != QDIT_VC_NONE)
     QDIT_TRY(qdit_vc_correct(ctx, s->latent, B, sh.channels, HW, i, s->d.vc_mode, s->vc_table, s->d.vc_eps));
   s->next_step = i + 1;

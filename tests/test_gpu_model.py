@@ -355,6 +355,46 @@ def test_sampler_per_branch_schedule_matches_oracle(q, ctx):
         rig.close()
 
 
+@pytest.mark.parametrize("guidance", [None, 1.5])
+def test_ddpm_sampler_tiny_matches_oracle(q, ctx, guidance):
+    """Stochastic sampler with learned variance; the noise of every step is an input shared with the oracle."""
+    cfg = synth.DIT_TINY
+    S, B = 8, 3
+    rig, latent, t, y, scales = _forward_case(q, ctx, cfg, 79, B)
+    try:
+        noise = synth.normal(79, "ddpm_noise", (S,) + latent.shape)
+        K = (1.0 + 0.03 * synth.normal(79, "K", (S, cfg.channels))).astype(np.float32)
+        nd = dev(noise)
+
+        def run(noise_dev):
+            sm = rig.sampler(batch=B, num_steps=S, cache_interval=2, use_cfg=guidance is not None, guidance=guidance or 1.0,
+                             vc_mode=q.QDIT_VC_K_TABLE, vc_table=K)
+            q.qdit_sampler_set_ddpm(ctx, sm, noise_dev)
+            out = np.empty_like(latent, dtype=np.float32)
+            q.qdit_sample(ctx, sm, np.ascontiguousarray(latent, dtype=np.float32), np.ascontiguousarray(y, dtype=np.int32), out)
+            return out.astype(np.float64)
+
+        got = run(nd)
+        ref = sampler.sample(rig.om, dit.Context(quant="static", scales=scales),
+                             sampler.SamplerConfig(S, cache_interval=2, guidance=guidance, vc_table=K, kind="ddpm", noise=noise),
+                             latent, y)
+        assert rel_l2(got, ref) < 5e-3, rel_l2(got, ref)
+        # NULL noise returns to the deterministic sampler
+        ddim = run(None)
+        ref_ddim = sampler.sample(rig.om, dit.Context(quant="static", scales=scales),
+                                  sampler.SamplerConfig(S, cache_interval=2, guidance=guidance, vc_table=K), latent, y)
+        assert rel_l2(ddim, ref_ddim) < 5e-3 and rel_l2(got, ddim) > 1e-2
+        # the last step draws no noise
+        n2 = noise.copy()
+        n2[-1] = 1e6
+        np.testing.assert_array_equal(run(dev(n2)), got)
+        # a one-step trajectory has no stochastic form
+        s1 = rig.sampler(batch=B, num_steps=1)
+        assert q.lib.qdit_sampler_set_ddpm(ctx, s1, nd.data_ptr()) == q.QDIT_ERR_INVALID_ARG
+    finally:
+        rig.close()
+
+
 def test_sampler_step_by_step_and_cache_effect(q, ctx):
     cfg = synth.DIT_TINY
     S, B = 6, 2

@@ -45,6 +45,76 @@ def test_ddim_table_and_identities():
     np.testing.assert_allclose(sampler.ddim_update(xt, eps, row), alt, atol=1e-12)
 
 
+def test_ddpm_table_and_posterior_identities():
+    """The stochastic step against the Gaussian algebra it comes from (cited DDPM papers): re-derived betas,
+    posterior mean and variance of q(x_{k-1} | x_k, x0), the log-domain variance interpolation, the last step."""
+    # all 1000 steps kept: the re-derived betas are the original linear schedule
+    full = sampler.ddpm_table(1000)
+    betas = np.linspace(1e-4, 2e-2, 1000)
+    np.testing.assert_allclose([np.exp(r[5]) for r in full], betas[::-1], rtol=1e-12)
+    tab = sampler.ddpm_table(50)
+    assert [r[0] for r in tab[:3]] == [980, 960, 940] and tab[-1][0] == 0       # same timestep subset as DDIM
+    ddim = sampler.ddim_table(50)
+    ab = np.array([r[1] ** 2 for r in ddim])            # alpha_bar of the kept steps, descending t
+    ab_prev = np.array([r[3] ** 2 for r in ddim])
+    for i, r in enumerate(tab):
+        _, sr, srm1, c0, ct, lb, lp, nz = r
+        a, ap = ab[i], ab_prev[i]
+        beta = 1 - a / ap
+        assert abs(sr - 1 / np.sqrt(a)) < 1e-12 and abs(srm1 - np.sqrt(1 / a - 1)) < 1e-9
+        assert abs(np.exp(lb) - beta) < 1e-14
+        # q(x_{k-1} | x_k, x0) from the joint Gaussian: x_{k-1} = sqrt(ap) x0 + sqrt(1-ap) e1,  x_k = sqrt(1-beta) x_{k-1} + sqrt(beta) e2
+        #   precision = (1-beta)/beta + 1/(1-ap);  mean = var * (sqrt(1-beta)/beta x_k + sqrt(ap)/(1-ap) x0)
+        if i < len(tab) - 1:
+            var = 1.0 / ((1 - beta) / beta + 1.0 / (1 - ap))
+            assert abs(np.exp(lp) - var) < 1e-12 * var + 1e-18
+            assert abs(ct - var * np.sqrt(1 - beta) / beta) < 1e-10 and abs(c0 - var * np.sqrt(ap) / (1 - ap)) < 1e-10
+            assert nz == 1.0
+        else:
+            assert nz == 0.0 and abs(c0 - 1.0) < 1e-12 and abs(ct) < 1e-12      # alpha_bar_prev = 1: the mean is x0
+            assert lp == tab[-2][6]                                              # clipped log variance
+        # a noise-free x0 maps to the mean of q(x_{k-1} | x0): coef_x0 + coef_xt sqrt(ab) = sqrt(ab_prev)
+        assert abs(c0 + ct * np.sqrt(a) - np.sqrt(ap)) < 1e-12
+    # update rule: true noise in -> exact x0 and its posterior mean; v = +1 / -1 select beta' / posterior variance
+    rng = np.random.default_rng(11)
+    x0 = rng.standard_normal((2, 4, 8, 8))
+    e = rng.standard_normal(x0.shape)
+    z = rng.standard_normal(x0.shape)
+    r = tab[7]
+    a = ab[7]
+    xk = np.sqrt(a) * x0 + np.sqrt(1 - a) * e
+    mean = r[3] * x0 + r[4] * xk
+    up = sampler.ddpm_update(xk, e, np.ones_like(x0), r, z)
+    np.testing.assert_allclose(up, mean + np.sqrt(np.exp(r[5])) * z, rtol=1e-10, atol=1e-10)
+    lo = sampler.ddpm_update(xk, e, -np.ones_like(x0), r, z)
+    np.testing.assert_allclose(lo, mean + np.sqrt(np.exp(r[6])) * z, rtol=1e-10, atol=1e-10)
+    mid = sampler.ddpm_update(xk, e, np.zeros_like(x0), r, z)
+    np.testing.assert_allclose(mid, mean + np.exp(0.25 * (r[5] + r[6])) * z, rtol=1e-10, atol=1e-10)   # geometric mean
+    last = sampler.ddpm_update(xk, e, np.zeros_like(x0), tab[-1], z)
+    x0_last = tab[-1][1] * xk - tab[-1][2] * e
+    np.testing.assert_allclose(last, x0_last, rtol=1e-12, atol=1e-12)            # no noise at the last step
+    with pytest.raises(ValueError):
+        sampler.ddpm_table(1)
+
+
+def test_ddpm_sampler_runs_and_uses_the_noise(tiny):
+    cfg, model, latent, labels, scales = tiny
+    ctx = dit.Context(quant="static", scales=scales)
+    S = 5
+    rng = np.random.default_rng(12)
+    noise = rng.standard_normal((S,) + latent.shape)
+    a = sampler.sample(model, ctx, sampler.SamplerConfig(S, cache_interval=2, guidance=1.5, kind="ddpm", noise=noise), latent, labels)
+    b = sampler.sample(model, ctx, sampler.SamplerConfig(S, cache_interval=2, guidance=1.5, kind="ddpm", noise=noise), latent, labels)
+    np.testing.assert_array_equal(a, b)                                           # deterministic given the noise
+    c = sampler.sample(model, ctx, sampler.SamplerConfig(S, cache_interval=2, guidance=1.5, kind="ddpm", noise=-noise), latent, labels)
+    assert np.isfinite(a).all() and not np.allclose(a, c)
+    # the last step's noise is never used
+    n2 = noise.copy()
+    n2[-1] = 0
+    d = sampler.sample(model, ctx, sampler.SamplerConfig(S, cache_interval=2, guidance=1.5, kind="ddpm", noise=n2), latent, labels)
+    np.testing.assert_array_equal(a, d)
+
+
 def test_cfg_combine():
     rng = np.random.default_rng(1)
     e = rng.standard_normal((6, 4, 2, 2))
