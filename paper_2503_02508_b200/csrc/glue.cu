@@ -439,7 +439,7 @@ __global__ void __launch_bounds__(256) batched_linear_kernel(const float* __rest
 // transposing butterfly (31 shuffles per row) after which lane o holds output o.
 constexpr int FIN_OUT = 32;
 template <int NV>
-__global__ void __launch_bounds__(256, 1) final_kernel(const __nv_bfloat16* __restrict__ x, int64_t M, int D, int T,
+__global__ void __launch_bounds__(512, 1) final_kernel(const __nv_bfloat16* __restrict__ x, int64_t M, int D, int T,
                                                        float eps, const float* __restrict__ modf,
                                                        const float* __restrict__ w, const float* __restrict__ bias,
                                                        float* __restrict__ net, int grid, int patch) {
@@ -620,7 +620,7 @@ int32_t launch_final(qdit_ctx* ctx, const void* x, int64_t M, int D, int T, floa
   const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
   const int nv = (D / 8 + 31) / 32;
   const size_t smem = static_cast<size_t>(FIN_OUT) * nv * 2 * 32 * sizeof(float4);
-  int64_t want = (M + 15) / 16;
+  int64_t want = (M + 31) / 32;
   const unsigned g = static_cast<unsigned>(want < ctx->num_sms ? want : ctx->num_sms);
 #define QDIT_FINAL_CASE(NV)                                                                                             \
   case NV: {                                                                                                            \
@@ -630,7 +630,7 @@ int32_t launch_final(qdit_ctx* ctx, const void* x, int64_t M, int D, int T, floa
                                                 FIN_OUT * NV * 2 * 32 * static_cast<int>(sizeof(float4))));             \
       attr_set[ctx->device & 63] = true;                                                                                \
     }                                                                                                                   \
-    final_kernel<NV><<<g, 256, smem, ctx->stream>>>(xb, M, D, T, eps, modf, w, bias, net, grid, patch);                 \
+    final_kernel<NV><<<g, 512, smem, ctx->stream>>>(xb, M, D, T, eps, modf, w, bias, net, grid, patch);                 \
   } break;
   ProfScope prof(ctx, QDIT_PROF_OTHER, static_cast<double>(M) * D * 2.0);
   switch (nv) {

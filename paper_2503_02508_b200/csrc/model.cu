@@ -71,7 +71,7 @@ struct qdit_sampler {
   // modulation, depends on the timestep and the label only, never on the latent.  Rows are (step, sample).
   float *traj_c, *traj_sc, *traj_hidden, *traj_feat, *traj_mod, *traj_modf;
   uint8_t* traj_ca;
-  bool traj_cond;                // buffers allocated (the trajectory's modulation fits the memory budget)
+  int traj_chunk;                // steps whose conditioning is evaluated together (0: per step, inside forward_impl)
   qdit_cache* cache;
   std::vector<DdimCoef> ddim;
   std::vector<DdpmCoef> ddpm;    // filled when the stochastic sampler is selected
@@ -309,13 +309,15 @@ static int32_t forward_impl(qdit_ctx* ctx, qdit_sampler* s, const float* latent,
   return QDIT_OK;
 }
 
-// Conditioning and modulation of every step of the trajectory in one batch of S * Beff rows (step-major).
-static int32_t trajectory_conditioning(qdit_ctx* ctx, qdit_sampler* s) {
+// Conditioning and modulation of `n_steps` steps of the trajectory, from step `first`, in one batch of
+// n_steps * Beff rows (step-major).
+static int32_t trajectory_conditioning(qdit_ctx* ctx, qdit_sampler* s, int first, int n_steps) {
   qdit_model* m = s->model;
   const qdit_model_shape& sh = m->s;
-  const int D = sh.hidden, rows = s->d.num_steps * s->Beff;
+  const int D = sh.hidden, rows = n_steps * s->Beff;
   if (!m->scales_set) return qdit_fail(ctx, QDIT_ERR_STATE, "activation scales are not set (set them or calibrate)");
-  QDIT_TRY(launch_timestep_features(ctx, s->t_all, s->traj_feat, rows, sh.freq_dim));
+  const float* t = s->t_all + static_cast<int64_t>(first) * s->Beff;
+  QDIT_TRY(launch_timestep_features(ctx, t, s->traj_feat, rows, sh.freq_dim));
   QDIT_TRY(launch_batched_linear(ctx, s->traj_feat, m->w_t1, m->b_t1, nullptr, nullptr, s->traj_hidden, nullptr, rows, D,
                                  sh.freq_dim, 0, 1, 0));
   QDIT_TRY(launch_batched_linear(ctx, s->traj_hidden, m->w_t2, m->b_t2, m->y_table, s->y, s->traj_c, s->traj_sc, rows, D, D, 0, 0,
@@ -475,14 +477,23 @@ int32_t qdit_sampler_create(qdit_ctx* ctx, qdit_model* m, const qdit_sampler_des
   s->tmpf = a.alloc<float>(M * F);
   s->dyn_absmax = a.alloc<float>(m->n_scales());
   s->dyn_scale = a.alloc<float>(m->n_scales());
-  // whole-trajectory conditioning when its modulation table fits 4 GB; otherwise it is evaluated step by step
+  // conditioning of as many steps at once as a 4 GB modulation table holds (all of them for the paper's 50- and
+  // 100-step settings; a 250-step trajectory at network batch 32 goes in chunks of 173 steps)
   bool traj_ok = true;
   {
-    const int64_t rows = B * d->num_steps;
-    s->traj_cond = rows * sh.depth * 6 * D * static_cast<int64_t>(sizeof(float)) <= (int64_t(4) << 30) && !getenv("QDIT_STEPWISE_CONDITIONING");
+    const int64_t per_step = B * sh.depth * 6 * D * static_cast<int64_t>(sizeof(float));
+    int64_t chunk = (int64_t(4) << 30) / per_step;
+    if (chunk > d->num_steps) chunk = d->num_steps;
+    if (getenv("QDIT_STEPWISE_CONDITIONING")) chunk = 0;
+    if (const char* env = getenv("QDIT_CONDITIONING_CHUNK")) {  // smaller chunks on request (memory, tests)
+      const int64_t v = atoll(env);
+      if (v > 0 && v < chunk) chunk = v;
+    }
+    s->traj_chunk = static_cast<int>(chunk);
     s->traj_c = s->traj_sc = s->traj_hidden = s->traj_feat = s->traj_mod = s->traj_modf = nullptr;
     s->traj_ca = nullptr;
-    if (s->traj_cond) {
+    if (s->traj_chunk > 0) {
+      const int64_t rows = B * s->traj_chunk;
       s->traj_c = a.alloc<float>(rows * D);
       s->traj_sc = a.alloc<float>(rows * D);
       s->traj_hidden = a.alloc<float>(rows * D);
@@ -664,9 +675,13 @@ int32_t qdit_sample_step(qdit_ctx* ctx, qdit_sampler* s, int i) {
     }
   }
   const float *pre_mod = nullptr, *pre_modf = nullptr;
-  if (s->traj_cond) {
-    if (i == 0) QDIT_TRY(trajectory_conditioning(ctx, s));
-    const int64_t row0 = static_cast<int64_t>(i) * s->Beff;
+  if (s->traj_chunk > 0) {
+    const int in_chunk = i % s->traj_chunk;
+    if (in_chunk == 0) {
+      const int left = s->d.num_steps - i;
+      QDIT_TRY(trajectory_conditioning(ctx, s, i, left < s->traj_chunk ? left : s->traj_chunk));
+    }
+    const int64_t row0 = static_cast<int64_t>(in_chunk) * s->Beff;
     pre_mod = s->traj_mod + row0 * sh.depth * 6 * sh.hidden;
     pre_modf = s->traj_modf + row0 * 2 * sh.hidden;
   }
