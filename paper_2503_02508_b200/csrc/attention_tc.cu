@@ -2,10 +2,10 @@
 //
 // One CTA = 128 queries of one (sample, head).  Keys are consumed in blocks of 128:
 //   S = Q K^T     tcgen05.mma, A = Q and B = K tiles (K-major, TMA-staged), accumulator in tensor memory
-//   softmax       one thread per query row: tcgen05.ld S, running max / sum in f32 (no shuffles needed),
+//   softmax       two threads per query row: tcgen05.ld S, running max / sum in f32 (no shuffles needed),
 //                 P = exp2(..) written as bf16 into a 128B-swizzled shared-memory tile
 //   O_blk = P V   tcgen05.mma, A = P (K-major), B = V tile used MN-major (its head-dim index is contiguous),
-//                 accumulator re-uses the S columns; the row thread folds it into its f32 registers
+//                 accumulator re-uses the S columns; the row's threads fold it into their f32 registers
 // Head dim 72 does not fill a 128-byte swizzle row: every operand is staged as a 64-column tile (128B
 // swizzle) plus a 16-column tail tile (32B swizzle, columns 64..79).  The tail's columns 72..79 belong to the
 // next head; they are zeroed in the Q tail, so they add nothing to S, and in V they only produce output
