@@ -33,32 +33,44 @@ __global__ void __launch_bounds__(256) cache_reuse_kernel(__nv_bfloat16* __restr
 }
 
 // Fully skipped step: x = bf16(x + sum_b gate_msa_b * A_b + gate_mlp_b * Mo_b), one pass over the cache.
-// Slot (b, branch) starts at cache + (2*b + branch) * M * D.
-__global__ void __launch_bounds__(256) cache_reuse_all_kernel(__nv_bfloat16* __restrict__ x,
-                                                              const __nv_bfloat16* __restrict__ cache,
-                                                              const float* __restrict__ mod, int64_t ld_mod, int64_t M,
-                                                              int D, int64_t T, int blocks) {
+// Slot (b, branch) starts at cache + (2*b + branch) * M * D.  A thread owns 8 columns of R consecutive rows of one
+// sample, so the two gate vectors of a block are loaded once per R rows (with R = 1 they are as many bytes from
+// L2 as the cache itself is from HBM) and 2 R independent 16-byte cache loads are in flight per block.
+template <int R>
+__global__ void __launch_bounds__(256, 2) cache_reuse_all_kernel(__nv_bfloat16* __restrict__ x,
+                                                                 const __nv_bfloat16* __restrict__ cache,
+                                                                 const float* __restrict__ mod, int64_t ld_mod, int64_t M,
+                                                                 int D, int64_t T, int blocks) {
   const int vec_per_row = D >> 3;
   const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (idx >= M * vec_per_row) return;
-  const int64_t row = idx / vec_per_row;
-  const int col = static_cast<int>(idx - row * vec_per_row) * 8;
+  const int64_t groups = M / R;  // the launcher picks R with M % R == 0 and T % R == 0
+  if (idx >= groups * vec_per_row) return;
+  const int64_t row = (idx / vec_per_row) * R;
+  const int col = static_cast<int>(idx % vec_per_row) * 8;
   const int64_t off = row * D + col;
   const int64_t slot_stride = M * D;
   const float* mrow = mod + (row / T) * ld_mod + col;
-  float acc[8];
-  Load8<__nv_bfloat16>::load(x + off, acc);
-#pragma unroll 4
+  float acc[R][8];
+#pragma unroll
+  for (int r = 0; r < R; ++r) Load8<__nv_bfloat16>::load(x + off + static_cast<int64_t>(r) * D, acc[r]);
+#pragma unroll 2
   for (int b = 0; b < blocks; ++b) {
-    float av[8], mv[8], ga[8], gm[8];
-    Load8<__nv_bfloat16>::load(cache + (2 * b) * slot_stride + off, av);
-    Load8<__nv_bfloat16>::load(cache + (2 * b + 1) * slot_stride + off, mv);
+    float ga[8], gm[8];
     Load8<float>::load(mrow + static_cast<int64_t>(b) * 6 * D + 2 * D, ga);
     Load8<float>::load(mrow + static_cast<int64_t>(b) * 6 * D + 5 * D, gm);
+    float av[R][8], mv[R][8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) acc[i] += ga[i] * av[i] + gm[i] * mv[i];
+    for (int r = 0; r < R; ++r) {
+      Load8<__nv_bfloat16>::load(cache + (2 * b) * slot_stride + off + static_cast<int64_t>(r) * D, av[r]);
+      Load8<__nv_bfloat16>::load(cache + (2 * b + 1) * slot_stride + off + static_cast<int64_t>(r) * D, mv[r]);
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[r][i] += ga[i] * av[r][i] + gm[i] * mv[r][i];
   }
-  *reinterpret_cast<uint4*>(x + off) = pack_bf16x8(acc);
+#pragma unroll
+  for (int r = 0; r < R; ++r) *reinterpret_cast<uint4*>(x + off + static_cast<int64_t>(r) * D) = pack_bf16x8(acc[r]);
 }
 
 // ----------------------------------------------------------------------------- block reductions
@@ -744,10 +756,19 @@ int32_t qdit_cache_reuse_all(qdit_ctx* ctx, qdit_cache* c, const float* mod_all,
   for (size_t i = 0; i < c->filled.size(); ++i)
     if (!c->filled[i]) return qdit_fail(ctx, QDIT_ERR_STATE, "cache slot (block %zu, branch %zu) reused before any store", i / 2, i % 2);
   if (!aligned16(mod_all) || !aligned16(x) || ld_mod % 4 != 0) return qdit_fail(ctx, QDIT_ERR_ALIGN, "mod_all and x must be 16-byte aligned, ld_mod a multiple of 4");
-  const int64_t n = c->M * (c->D / 8);
   ProfScope prof(ctx, QDIT_PROF_CACHE_REUSE, static_cast<double>(c->M) * c->D * 2.0 * (2.0 * c->blocks + 2.0));
-  cache_reuse_all_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, ctx->stream>>>(
-      static_cast<__nv_bfloat16*>(x), c->data, mod_all, ld_mod, c->M, static_cast<int>(c->D), T, c->blocks);
+  // rows per thread: 2 when samples are made of whole groups of 2 rows and there is work for every SM, else 1
+  constexpr int R = 2;
+  const bool wide = c->M % R == 0 && T % R == 0 && c->M * (c->D / 8) >= static_cast<int64_t>(R) * 256 * 4 * ctx->num_sms;
+  if (wide) {
+    const int64_t n = (c->M / R) * (c->D / 8);
+    cache_reuse_all_kernel<R><<<static_cast<unsigned>((n + 255) / 256), 256, 0, ctx->stream>>>(
+        static_cast<__nv_bfloat16*>(x), c->data, mod_all, ld_mod, c->M, static_cast<int>(c->D), T, c->blocks);
+  } else {
+    const int64_t n = c->M * (c->D / 8);
+    cache_reuse_all_kernel<1><<<static_cast<unsigned>((n + 255) / 256), 256, 0, ctx->stream>>>(
+        static_cast<__nv_bfloat16*>(x), c->data, mod_all, ld_mod, c->M, static_cast<int>(c->D), T, c->blocks);
+  }
   return qdit_after_launch(ctx, "cache_reuse_all_kernel");
 }
 
