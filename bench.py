@@ -430,10 +430,22 @@ def run_gemm_sweep(args):
             quant()
             ops = 2.0 * M * N * K
             ms_g, ms_b, ms_q = t(gemm), t(both), t(quant)
-            rows.append({"layer": name, "M": M, "K": K, "N": N, "gemm_tops": ops / ms_g / 1e9, "quant_gemm_tops": ops / ms_b / 1e9,
-                         "gemm_us": ms_g * 1e3, "act_quant_gbs": 3.0 * M * K / ms_q / 1e6,
-                         "frac_of_2x_bf16_burst": ops / ms_g / 1e9 / (2 * peaks["bf16_burst"]),
-                         "frac_of_nominal_4500": ops / ms_g / 1e9 / 4500.0})
+            row = {"layer": name, "M": M, "K": K, "N": N, "gemm_tops": ops / ms_g / 1e9, "quant_gemm_tops": ops / ms_b / 1e9,
+                   "gemm_us": ms_g * 1e3, "act_quant_gbs": 3.0 * M * K / ms_q / 1e6,
+                   "act_quant_frac_of_hbm": 3.0 * M * K / ms_q / 1e6 / peaks["hbm_gbs"],
+                   "frac_of_2x_bf16_burst": ops / ms_g / 1e9 / (2 * peaks["bf16_burst"]),
+                   "frac_of_nominal_4500": ops / ms_g / 1e9 / 4500.0}
+            if name == "qkv" and M % 256 == 0:
+                # the block's other memory-bound kernel on the same tokens: LayerNorm + adaLN modulate + quantize
+                mod = torch.from_numpy(synth.normal(seed, f"mod{M}", (M // 256, 6 * K), 0.3)).cuda()
+
+                def ln():
+                    q.qdit_adaln_modulate(ctx, x, M, K, 256, 1e-6, mod, mod[:, K:], 6 * K, a8, q.QDIT_I8, a_qp)
+
+                ms_l = t(ln)
+                row["ln_modulate_gbs"] = 3.0 * M * K / ms_l / 1e6
+                row["ln_modulate_frac_of_hbm"] = row["ln_modulate_gbs"] / peaks["hbm_gbs"]
+            rows.append(row)
     q.qdit_sync(ctx)
     q.qdit_destroy(ctx)
     best = max(r["gemm_tops"] for r in rows)
