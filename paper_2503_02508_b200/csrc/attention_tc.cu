@@ -221,14 +221,19 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       __syncwarp();
       tc_fence_after();
       // pass 1: maximum over this thread's 64 keys, then over the row with the other thread's value
-      float mx = -INFINITY;
-#pragma unroll 1
-      for (int c = 0; c < 2; ++c) {
-        uint32_t v[32];
-        tmem_ld_32x32(sbuf + c * 32, v);
+      float mx;
+      {
+        uint32_t v0[32], v1[32];  // both loads in flight, one wait
+        tmem_ld_32x32(sbuf, v0);
+        tmem_ld_32x32(sbuf + 32, v1);
         tmem_ld_wait();
+        float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
+        for (int i = 0; i < 32; ++i) {
+          m0 = fmaxf(m0, __uint_as_float(v0[i]));
+          m1 = fmaxf(m1, __uint_as_float(v1[i]));
+        }
+        mx = fmaxf(m0, m1);
       }
       s_m[((j & 1) * 2 + half) * 128 + r] = mx;
       mbar_arrive(&bar_mx[quad]);
