@@ -87,13 +87,17 @@ typedef struct {
   int32_t qmin, qmax; /* clip range; either within [-128,127] or within [0,255] */
 } qdit_qparams;
 
-enum { QDIT_QUANT_STATIC = 0, QDIT_QUANT_DYNAMIC = 1 };
+enum { QDIT_QUANT_STATIC = 0, QDIT_QUANT_DYNAMIC = 1, QDIT_QUANT_DYNAMIC_TOKEN = 2 };
 
 /* q[m,k] = Q(x[m,k]).  x: [M,K] bf16 or f32 (x_dtype), ldx elements per row; q: [M,K] bytes, ldq
  * (8-byte alignment of q and ldq suffices).
  * STATIC : *qp (host) gives s, z and the range.
  * DYNAMIC: symmetric range [-127,127]; s = max|x| / 127 is reduced on the device first (s = 1 if the
  *          tensor is all zero) and left in dyn_scale (device, 1 float, required); qp is ignored.
+ * DYNAMIC_TOKEN: the same per row (per token): s[m] = max_k|x[m,k]| / 127 left in dyn_scale (device,
+ *          M floats); the linear layer takes these scales with QDIT_EPI_ROW_SCALE.  (The paper quantizes
+ *          activations tensor-wise, Experimental Settings; the per-token form is the variant of the
+ *          quantization baselines it compares with.)
  * K must be a multiple of 8; M or K of 0 is a no-op. */
 int32_t qdit_quantize_act(qdit_ctx* ctx, const void* x, int x_dtype, int64_t M, int64_t K, int64_t ldx,
                           int mode, const qdit_qparams* qp, float* dyn_scale, void* q, int64_t ldq);
@@ -142,7 +146,8 @@ enum {
   QDIT_EPI_QUANT_OUT = 1u << 5,
   QDIT_EPI_OUT_BF16 = 1u << 6,
   QDIT_EPI_OUT_F32 = 1u << 7,
-  QDIT_EPI_OUT_I32 = 1u << 8
+  QDIT_EPI_OUT_I32 = 1u << 8,
+  QDIT_EPI_ROW_SCALE = 1u << 9 /* activation scale per row: epi->a_scale_rows[m] replaces a_qp.scale (a_qp.zero_point must be 0) */
 };
 
 typedef struct {
@@ -156,6 +161,8 @@ typedef struct {
   void* cache_out;            /* [M,N] bf16, leading dimension N */
   qdit_qparams out_qp;        /* for QDIT_EPI_QUANT_OUT */
   const float* out_scale_dev; /* optional device override of out_qp.scale */
+  const float* a_scale_rows;  /* [M] f32 device, per-token activation scales for QDIT_EPI_ROW_SCALE
+                                 (as written by qdit_quantize_act in QDIT_QUANT_DYNAMIC_TOKEN mode) */
 } qdit_epilogue;
 
 int32_t qdit_w8a8_linear(qdit_ctx* ctx, const void* A, const void* W, int64_t M, int64_t N, int64_t K,

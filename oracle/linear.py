@@ -41,6 +41,18 @@ def dequant_affine(acc: np.ndarray, a_qp: QParams, w_scale: np.ndarray, w_colsum
     return y
 
 
+def w8a8_linear_per_token(qa: np.ndarray, a_scales: np.ndarray, qw: np.ndarray, w_scale: np.ndarray,
+                          bias: np.ndarray | None) -> np.ndarray:
+    """Quantized linear whose activations carry one scale per row (symmetric, z = 0):
+    y[m,n] = (s_a[m] * s_w[n]) * acc[m,n] + bias[n], the scale product formed in float32; float64 [M,N]."""
+    acc = gemm_i8(qa, qw).astype(np.float64)
+    sprod = (np.asarray(a_scales, dtype=F32)[:, None] * np.asarray(w_scale, dtype=F32)[None, :]).astype(np.float64)
+    y = acc * sprod
+    if bias is not None:
+        y = y + np.asarray(bias, dtype=np.float64)[None, :]
+    return y
+
+
 def w8a8_linear(qa: np.ndarray, a_qp: QParams, qw: np.ndarray, w_scale: np.ndarray, w_colsum: np.ndarray,
                 bias: np.ndarray | None) -> np.ndarray:
     """Full quantized linear on already-quantized activations; float64 [M,N]."""

@@ -65,6 +65,17 @@ def quantize(X: np.ndarray, qp: QParams) -> np.ndarray:
     return np.clip(r, qp.qmin, qp.qmax).astype(np.int32)
 
 
+def quantize_per_token(X: np.ndarray):
+    """Dynamic per-token (per-row) symmetric quantizer: Eq. 1 with s[m] = max_k |X[m,k]| / 127, z = 0, range
+    [-127, 127] (s = 1 for an all-zero row).  Returns (codes int32 [M,K], scales float32 [M])."""
+    x32 = np.asarray(X).astype(F32)
+    s = (np.max(np.abs(x32), axis=1) / F32(127)).astype(F32)
+    s[~(s > 0)] = F32(1.0)
+    inv = (F32(1.0) / s).astype(F32)
+    r = np.rint(x32 * inv[:, None])
+    return np.clip(r, -127, 127).astype(np.int32), s
+
+
 def dequantize(q: np.ndarray, qp: QParams) -> np.ndarray:
     """Inverse map of Eq. 1 inside the clip range: s * (q - z), float64."""
     return np.float64(F32(qp.scale)) * (np.asarray(q, dtype=np.float64) - qp.zero_point)

@@ -18,9 +18,10 @@ QDIT_OK = 0
 QDIT_ERR_INVALID_ARG, QDIT_ERR_SHAPE, QDIT_ERR_ALIGN, QDIT_ERR_UNSUPPORTED = -1, -2, -3, -4
 QDIT_ERR_CUDA, QDIT_ERR_STATE, QDIT_ERR_TIMEOUT, QDIT_ERR_NOMEM = -5, -6, -7, -8
 QDIT_BF16, QDIT_F32, QDIT_I8, QDIT_I32 = 0, 1, 2, 3
-QDIT_QUANT_STATIC, QDIT_QUANT_DYNAMIC = 0, 1
+QDIT_QUANT_STATIC, QDIT_QUANT_DYNAMIC, QDIT_QUANT_DYNAMIC_TOKEN = 0, 1, 2
 QDIT_EPI_BIAS, QDIT_EPI_GELU, QDIT_EPI_GATE, QDIT_EPI_RESIDUAL = 1, 2, 4, 8
 QDIT_EPI_CACHE_STORE, QDIT_EPI_QUANT_OUT, QDIT_EPI_OUT_BF16, QDIT_EPI_OUT_F32, QDIT_EPI_OUT_I32 = 16, 32, 64, 128, 256
+QDIT_EPI_ROW_SCALE = 512
 QDIT_BRANCH_ATTN, QDIT_BRANCH_MLP = 0, 1
 QDIT_VC_NONE, QDIT_VC_K_TABLE, QDIT_VC_VAR_RATIO = 0, 1, 2
 QDIT_VC_FIT_DERIVED, QDIT_VC_FIT_PRINTED = 0, 1
@@ -37,7 +38,7 @@ class qdit_qparams(C.Structure):
 class qdit_epilogue(C.Structure):
     _fields_ = [("w_scale", _vp), ("w_colsum", _vp), ("bias", _vp), ("gate", _vp), ("ld_gate", _i64),
                 ("tokens_per_sample", _i64), ("residual", _vp), ("cache_out", _vp), ("out_qp", qdit_qparams),
-                ("out_scale_dev", _vp)]
+                ("out_scale_dev", _vp), ("a_scale_rows", _vp)]
 
 
 class qdit_model_shape(C.Structure):
@@ -197,10 +198,10 @@ def qdit_quantize_act_dynamic_static(ctx, x, x_dtype, M, K, ldx, dyn_scale, q, l
 
 
 def epilogue(w_scale=None, w_colsum=None, bias=None, gate=None, ld_gate=0, tokens_per_sample=0, residual=None,
-             cache_out=None, out_qp=None, out_scale_dev=None):
+             cache_out=None, out_qp=None, out_scale_dev=None, a_scale_rows=None):
     return qdit_epilogue(ptr(w_scale), ptr(w_colsum), ptr(bias), ptr(gate), ld_gate, tokens_per_sample,
                          ptr(residual), ptr(cache_out), out_qp if out_qp is not None else qparams(1.0),
-                         ptr(out_scale_dev))
+                         ptr(out_scale_dev), ptr(a_scale_rows))
 
 
 def qdit_w8a8_linear(ctx, A, W, M, N, K, a_qp, a_scale_dev, flags, epi, out, ldo):

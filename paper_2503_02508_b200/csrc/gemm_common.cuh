@@ -25,6 +25,7 @@ struct GemmParams {
   uint32_t flags;
   float a_scale;
   const float* a_scale_dev;
+  const float* a_scale_rows;  // per-row activation scales (QDIT_EPI_ROW_SCALE, generic epilogue class only)
   int a_zp;
   const float* w_scale;
   const int32_t* w_colsum;
@@ -98,10 +99,13 @@ __device__ __forceinline__ void epilogue8(const GemmParams& p, const uint4 lo, c
   // de-quantisation: one fused multiply-add acc * (s_a s_w) + bias in every kernel and epilogue class (explicit,
   // so that the result does not depend on what the compiler contracts)
   float f[8];
+  float rs = 1.0f;  // per-token activation scale (cp.sc then holds s_w alone)
+  if (flags & QDIT_EPI_ROW_SCALE) rs = p.a_scale_rows[row];
 #pragma unroll
-  for (int i = 0; i < 8; ++i)
-    f[i] = (flags & QDIT_EPI_BIAS) ? __fmaf_rn(static_cast<float>(acc[i]), cp.sc[i], cp.bi[i])
-                                   : __fmul_rn(static_cast<float>(acc[i]), cp.sc[i]);
+  for (int i = 0; i < 8; ++i) {
+    const float sc = (flags & QDIT_EPI_ROW_SCALE) ? __fmul_rn(rs, cp.sc[i]) : cp.sc[i];
+    f[i] = (flags & QDIT_EPI_BIAS) ? __fmaf_rn(static_cast<float>(acc[i]), sc, cp.bi[i]) : __fmul_rn(static_cast<float>(acc[i]), sc);
+  }
   if (flags & QDIT_EPI_GELU) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) f[i] = gelu_tanh_f(f[i]);

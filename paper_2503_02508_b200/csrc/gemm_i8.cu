@@ -291,6 +291,13 @@ extern "C" int32_t qdit_w8a8_linear(qdit_ctx* ctx, const void* A, const void* W,
       if (!aligned16(epi->cache_out)) return qdit_fail(ctx, QDIT_ERR_ALIGN, "cache_out must be 16-byte aligned");
       p.cache_out = static_cast<__nv_bfloat16*>(epi->cache_out);
     }
+    if (flags & QDIT_EPI_ROW_SCALE) {
+      if (!epi->a_scale_rows) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "ROW_SCALE set but a_scale_rows is NULL");
+      if (a_qp.zero_point != 0) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "ROW_SCALE needs a symmetric activation quantizer (zero_point 0)");
+      p.a_scale_rows = epi->a_scale_rows;
+      p.a_scale = 1.0f;
+      p.a_scale_dev = nullptr;
+    }
     if (flags & QDIT_EPI_QUANT_OUT) {
       QDIT_TRY(qdit_check_qparams(ctx, &epi->out_qp, epi->out_scale_dev != nullptr));
       p.o_scale = epi->out_qp.scale;
@@ -301,7 +308,8 @@ extern "C" int32_t qdit_w8a8_linear(qdit_ctx* ctx, const void* A, const void* W,
     }
   }
   // QDIT_GEMM_T=<bt> selects the channel-major kernel with 128 x bt tiles (experimental switch while tuning)
-  if (const char* env = getenv("QDIT_GEMM_T")) {
+  const bool row_scale = (flags & QDIT_EPI_ROW_SCALE) != 0;  // implemented by the token-major kernels' generic epilogue
+  if (const char* env = row_scale ? nullptr : getenv("QDIT_GEMM_T")) {
     const int bt = atoi(env);
     if (bt == 128 || bt == 256) return qdit_launch_gemm_t(ctx, A, W, p, a_unsigned, bt);
   }

@@ -39,6 +39,36 @@ __global__ void __launch_bounds__(256) act_quant_kernel(const T* __restrict__ x,
   }
 }
 
+// Per-token dynamic quantizer: one warp per row finds max|x| of its row, s[m] = max / 127 (1 for a zero row),
+// and writes the symmetric codes; the row is read twice (the second time from L1 / L2).
+template <typename T>
+__global__ void __launch_bounds__(256) act_quant_token_kernel(const T* __restrict__ x, int64_t M, int64_t K, int64_t ldx,
+                                                              float* __restrict__ scales, uint8_t* __restrict__ q,
+                                                              int64_t ldq) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= M) return;
+  const T* src = x + row * ldx;
+  float m = 0.0f;
+  for (int64_t k = lane * 8; k < K; k += 256) {
+    float v[8];
+    Load8<T>::load(src + k, v);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) m = fmaxf(m, fabsf(v[i]));
+  }
+  m = warp_max(m);
+  float s = __fdiv_rn(m, 127.0f);
+  if (!(s > 0.0f)) s = 1.0f;
+  const float inv = __fdiv_rn(1.0f, s);
+  if (lane == 0) scales[row] = s;
+  uint8_t* dst = q + row * ldq;
+  for (int64_t k = lane * 8; k < K; k += 256) {
+    float v[8];
+    Load8<T>::load(src + k, v);
+    *reinterpret_cast<uint2*>(dst + k) = quantize_pack8(v, inv, 0.0f, -127.0f, 127.0f);
+  }
+}
+
 // ----------------------------------------------------------------------------- abs-max reduction
 // Non-negative floats order like their bit patterns, so the global maximum is an atomicMax on uint32.
 template <typename T>
@@ -312,6 +342,16 @@ int32_t qdit_quantize_act(qdit_ctx* ctx, const void* x, int x_dtype, int64_t M, 
   if (mode == QDIT_QUANT_STATIC) {
     QDIT_TRY(qdit_check_qparams(ctx, qp, false));
     qa = make_quant_args(*qp, nullptr);
+  } else if (mode == QDIT_QUANT_DYNAMIC_TOKEN) {
+    if (!dyn_scale) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "per-token mode needs dyn_scale [M]");
+    const unsigned grid = static_cast<unsigned>((M + 7) / 8);
+    if (x_dtype == QDIT_BF16)
+      act_quant_token_kernel<__nv_bfloat16><<<grid, 256, 0, ctx->stream>>>(static_cast<const __nv_bfloat16*>(x), M, K, ldx, dyn_scale,
+                                                                        static_cast<uint8_t*>(q), ldq);
+    else
+      act_quant_token_kernel<float><<<grid, 256, 0, ctx->stream>>>(static_cast<const float*>(x), M, K, ldx, dyn_scale,
+                                                                   static_cast<uint8_t*>(q), ldq);
+    return qdit_after_launch(ctx, "act_quant_token_kernel");
   } else if (mode == QDIT_QUANT_DYNAMIC) {
     if (!dyn_scale) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "dynamic mode needs dyn_scale");
     // dyn_scale doubles as the abs-max accumulator before it is turned into the scale in place

@@ -211,6 +211,39 @@ def test_gelu_requant_epilogue(q, ctx, kernel_variant):
     np.testing.assert_array_equal(got, quant.quantize(outf.cpu().numpy(), o_qp))
 
 
+@pytest.mark.parametrize("M,N,K", [(300, 384, 1152), (1024, 2304, 256)])
+def test_per_token_scales(q, ctx, kernel_variant, M, N, K):
+    """Per-token activation scales (QDIT_EPI_ROW_SCALE): quantizer in per-token mode, then the linear layer."""
+    x = synth.outlier_activations(45, f"pt{M}", M, K) * (1.0 + (np.arange(M, dtype=np.float32)[:, None] % 5))
+    W = synth.normal(45, f"ptw{N}", (N, K), 0.02)
+    bias = synth.normal(45, f"ptb{N}", (N,), 0.02)
+    wq, ws, wc = quant.quantize_weight_per_channel(W)
+    qa, sa = quant.quantize_per_token(x)
+    ref = linear.w8a8_linear_per_token(qa, sa, wq, ws, bias)
+    a8 = torch.empty((M, K), dtype=torch.uint8, device="cuda")
+    sc = torch.empty(M, dtype=torch.float32, device="cuda")
+    q.qdit_quantize_act(ctx, dev(x), q.QDIT_F32, M, K, K, q.QDIT_QUANT_DYNAMIC_TOKEN, None, sc, a8, K)
+    out = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    ws_d, bias_d, wq_d = dev(ws), dev(bias), dev_i8(wq)     # the epilogue struct holds raw addresses: keep the tensors alive
+    epi = q.epilogue(w_scale=ws_d, bias=bias_d, a_scale_rows=sc)
+    q.qdit_w8a8_linear(ctx, a8, wq_d, M, N, K, q.qparams(1.0), None,
+                       q.QDIT_EPI_BIAS | q.QDIT_EPI_OUT_F32 | q.QDIT_EPI_ROW_SCALE, epi, out, N)
+    q.qdit_sync(ctx)
+    assert max_rel_err(out.cpu().numpy(), ref) < 1e-5
+    # closer to the un-quantized product than one tensor-wide scale is, on rows of very different magnitude
+    exact = x.astype(np.float64) @ W.astype(np.float64).T + bias
+    qp = quant.qparams_symmetric(float(np.abs(x).max()))
+    tens = linear.w8a8_linear(quant.quantize(x, qp), qp, wq, ws, wc, bias)
+    small = np.arange(M) % 5 == 0
+    assert np.abs(out.cpu().numpy()[small] - exact[small]).mean() < np.abs(tens[small] - exact[small]).mean()
+    # the flag needs its scales and a symmetric quantizer
+    L = q.lib
+    import ctypes as C
+    bad = q.epilogue(w_scale=ws_d, bias=bias_d)
+    assert L.qdit_w8a8_linear(ctx, a8.data_ptr(), wq_d.data_ptr(), M, N, K, q.qparams(1.0), None,
+                              q.QDIT_EPI_BIAS | q.QDIT_EPI_OUT_F32 | q.QDIT_EPI_ROW_SCALE, C.byref(bad), out.data_ptr(), N) == q.QDIT_ERR_INVALID_ARG
+
+
 def test_device_scale_override(q, ctx):
     M, N, K = 256, 192, 256
     a_qp = QParams(0.05, 0, -127, 127)

@@ -114,6 +114,27 @@ def test_quantize_weight_bit_exact(q, ctx, N, K):
     np.testing.assert_array_equal(co.cpu().numpy().astype(np.int64), wc)
 
 
+@pytest.mark.parametrize("M,K,dtype", [(300, 1152, "bf16"), (64, 4608, "f32"), (5, 8, "f32"), (1030, 384, "bf16")])
+def test_quantize_act_per_token_bit_exact(q, ctx, M, K, dtype):
+    """Per-token dynamic mode: one scale per row, codes and scales bit-exact against the oracle."""
+    x = synth.outlier_activations(12, f"tok{M}x{K}", M, K) * (1.0 + np.arange(M, dtype=np.float32)[:, None] % 7)
+    x[min(3, M - 1)] = 0
+    if dtype == "bf16":
+        xd = dev(x).to(torch.bfloat16)
+        xh = xd.float().cpu().numpy()
+        code = q.QDIT_BF16
+    else:
+        xd, xh, code = dev(x), x, q.QDIT_F32
+    out = torch.empty((M, K), dtype=torch.uint8, device="cuda")
+    sc = torch.empty(M, dtype=torch.float32, device="cuda")
+    q.qdit_quantize_act(ctx, xd, code, M, K, K, q.QDIT_QUANT_DYNAMIC_TOKEN, None, sc, out, K)
+    q.qdit_sync(ctx)
+    want_q, want_s = quant.quantize_per_token(xh)
+    np.testing.assert_array_equal(sc.cpu().numpy(), want_s)
+    np.testing.assert_array_equal(host_codes(out), want_q)
+    assert q.lib.qdit_quantize_act(ctx, xd.data_ptr(), code, M, K, K, q.QDIT_QUANT_DYNAMIC_TOKEN, None, None, out.data_ptr(), K) == q.QDIT_ERR_INVALID_ARG
+
+
 @pytest.mark.parametrize("bits", [4, 6, 2])
 def test_quantize_weight_bits_bit_exact(q, ctx, bits):
     """b-bit channel-wise weights (bits = 4: the W4A8 setting of Table 2): codes, scales and code sums."""

@@ -105,6 +105,41 @@ def test_degenerate_range_takes_unit_scale():
     assert quant.qparams_minmax(np.full(5, 2.0, dtype=np.float32)).scale == 1.0
 
 
+def test_per_token_quantizer_and_linear():
+    """Per-row scales: each row is the tensor-wise quantizer applied to that row alone, and the per-token linear
+    is the float product it approximates to within the quantization steps."""
+    from oracle import linear
+    rng = np.random.default_rng(21)
+    X = (rng.standard_normal((6, 48)) * np.array([0.1, 1, 10, 100, 1e-3, 0])[:, None]).astype(np.float32)
+    q, s = quant.quantize_per_token(X)
+    for m in range(6):
+        qp = quant.qparams_symmetric(float(np.abs(X[m]).max()))
+        np.testing.assert_array_equal(q[m], quant.quantize(X[m], qp))
+        assert s[m] == np.float32(qp.scale)
+        if m < 5:
+            assert np.abs(q[m]).max() == 127 and np.abs(X[m] - s[m] * q[m]).max() <= s[m] / 2 * (1 + 1e-5)
+    assert s[5] == 1.0 and not q[5].any()
+    # scaling a row by a power of two changes its scale only
+    X2 = X.copy()
+    X2[2] *= 4
+    q2, s2 = quant.quantize_per_token(X2)
+    np.testing.assert_array_equal(q2, q)
+    assert s2[2] == 4 * s[2]
+    # linear: exact on values that sit on both grids
+    W = rng.integers(-127, 128, size=(5, 48)).astype(np.int32)
+    ws = np.full(5, 0.5, dtype=np.float32)
+    Xg = (q[:5] * s[:5, None]).astype(np.float32)         # activations exactly on their grids
+    qg, sg = quant.quantize_per_token(Xg)
+    y = linear.w8a8_linear_per_token(qg, sg, W, ws, None)
+    want = (Xg.astype(np.float64)) @ (W.astype(np.float64) * 0.5).T
+    np.testing.assert_allclose(y, want, rtol=1e-6, atol=1e-9)
+    # and equals the tensor-wise linear when all rows share a scale
+    qp = quant.QParams(0.25, 0, -127, 127)
+    qa = rng.integers(-127, 128, size=(4, 48)).astype(np.int32)
+    np.testing.assert_array_equal(linear.w8a8_linear_per_token(qa, np.full(4, 0.25, dtype=np.float32), W, ws, None),
+                                  linear.w8a8_linear(qa, qp, W, ws, W.sum(axis=1), None))
+
+
 @pytest.mark.parametrize("bits", [4, 6, 2])
 def test_weight_per_channel_low_bit(bits):
     """b-bit weights (bits = 4: the W4A8 setting of Table 2): the grid has 2^bits - 1 levels around zero."""
