@@ -252,6 +252,18 @@ int32_t qdit_vc_fit(qdit_ctx* ctx, const float* x_hat, const float* x_target, in
                     double* workspace, float* K);
 
 /* ------------------------------------------------------------------------------------------------
+ * Matrix steps of Temporal-Aware Parallel Clustering for one subsample (section "Temporal-Aware Parallel
+ * Clustering for Calibration", Algorithm 1): from the n samples' features x [n,d] and timestamps t [n] (device f32)
+ *   A_spatial[k,h] = x_k.x_h / (|x_k||x_h|),  A_temporal[k,h] = exp(-|t_k - t_h|),
+ *   A = alpha A_spatial + (1 - alpha) A_temporal,   L = D^e A D^e,  D = diag(row sums of A)
+ * (A is symmetric, so the paper's row and column degree matrices coincide; the paper prints e = +1/2, the usual
+ * normalised adjacency is e = -1/2: `exponent` selects).  L: device f32 [n,n].  workspace: device f32, n*d + 2n
+ * floats, overwritten.  n % 4 == 0, d % 16 == 0.  Eigenvectors, k-means and the aggregation over subsamples are
+ * left to the host. */
+int32_t qdit_tap_laplacian(qdit_ctx* ctx, const float* x, const float* t, int n, int d, float alpha, float exponent,
+                           float* workspace, float* L);
+
+/* ------------------------------------------------------------------------------------------------
  * Whole model and sampler.  The DiT architecture (adaLN-Zero blocks, patch 2, learned-sigma output)
  * is the one the paper evaluates (Experimental Settings); quantized layers are each block's
  * modulation linear, QKV, projection, fc1 and fc2; embedders and the final layer stay in f32. */

@@ -91,6 +91,7 @@ _SIGNATURES = {
     "qdit_cache_reuse_all": (_i32, [_vp, _vp, _vp, _i64, _i64, _vp]),
     "qdit_selftest_wait_timeout": (_i32, [_vp, C.c_uint32, _vp]),
     "qdit_vc_correct": (_i32, [_vp, _vp, _int, _int, _int, _int, _int, _vp, _f32]),
+    "qdit_tap_laplacian": (_i32, [_vp, _vp, _vp, _int, _int, _f32, _f32, _vp, _vp]),
     "qdit_vc_fit": (_i32, [_vp, _vp, _vp, _int, _int, _int, _f32, _int, _vp, _vp]),
     "qdit_model_create": (_i32, [_vp, C.POINTER(qdit_model_desc), C.POINTER(_vp)]),
     "qdit_model_destroy": (_i32, [_vp]),
@@ -269,6 +270,10 @@ def qdit_selftest_wait_timeout(ctx, polls, observed):
 
 def qdit_vc_correct(ctx, latent, B, Cc, HW, step_index, mode, table, eps):
     return check(ctx, lib.qdit_vc_correct(ctx, ptr(latent), B, Cc, HW, step_index, mode, ptr(table), eps))
+
+
+def qdit_tap_laplacian(ctx, x, t, n, d, alpha, exponent, workspace, L):
+    return check(ctx, lib.qdit_tap_laplacian(ctx, ptr(x), ptr(t), n, d, alpha, exponent, ptr(workspace), ptr(L)))
 
 
 def qdit_vc_fit(ctx, x_hat, x_target, N, Cc, HW, eps, form, workspace, K):

@@ -182,6 +182,45 @@ __global__ void vc_fit_finish_kernel(const double* __restrict__ partial, int N, 
   K[c] = static_cast<float>(num / den);
 }
 
+// ----------------------------------------------------------------------------- TAP: similarity matrix and its normalisation
+// Matrix steps of Algorithm 1 for one subsample of n samples (features x [n,d], timestamps t [n]):
+//   xn = x / |x| (rows; a zero row stays zero)            tap_normalize_kernel, one CTA per row
+//   S  = xn xn^T                                            batched_linear_kernel (the register-tiled f32 GEMM)
+//   A  = alpha S + (1 - alpha) exp(-|t_k - t_h|), deg = row sums of A   tap_combine_kernel, one CTA per row
+//   L  = deg_k^e A_kh deg_h^e                               tap_scale_kernel
+// A is symmetric, so the row-sum and column-sum degrees of the paper coincide.
+__global__ void __launch_bounds__(256) tap_normalize_kernel(const float* __restrict__ x, int d, float* __restrict__ xn) {
+  __shared__ float sm[8];
+  const float* row = x + static_cast<int64_t>(blockIdx.x) * d;
+  float* out = xn + static_cast<int64_t>(blockIdx.x) * d;
+  float s = 0.0f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) s = fmaf(row[i], row[i], s);
+  const float norm = sqrtf(block_sum(s, sm));
+  const float inv = norm > 0.0f ? 1.0f / norm : 0.0f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) out[i] = row[i] * inv;
+}
+
+__global__ void __launch_bounds__(256) tap_combine_kernel(float* __restrict__ A, const float* __restrict__ t, int n, float alpha,
+                                                          float* __restrict__ deg) {
+  __shared__ float sm[8];
+  float* row = A + static_cast<int64_t>(blockIdx.x) * n;
+  const float tk = t[blockIdx.x];
+  float s = 0.0f;
+  for (int h = threadIdx.x; h < n; h += blockDim.x) {
+    const float a = alpha * row[h] + (1.0f - alpha) * expf(-fabsf(tk - t[h]));
+    row[h] = a;
+    s += a;
+  }
+  s = block_sum(s, sm);
+  if (threadIdx.x == 0) deg[blockIdx.x] = s;
+}
+
+__global__ void __launch_bounds__(256) tap_scale_kernel(float* __restrict__ A, const float* __restrict__ deg, int n, float e) {
+  float* row = A + static_cast<int64_t>(blockIdx.x) * n;
+  const float dk = powf(deg[blockIdx.x], e);
+  for (int h = threadIdx.x; h < n; h += blockDim.x) row[h] = dk * row[h] * powf(deg[h], e);
+}
+
 // ----------------------------------------------------------------------------- guidance + DDIM update
 // net: [Beff, 2C, HW]; eps = first C channels; with guidance, sample b's unconditional twin is b + B.
 __global__ void __launch_bounds__(256) cfg_ddim_kernel(float* __restrict__ latent, const float* __restrict__ net, int B,
@@ -785,6 +824,27 @@ int32_t qdit_vc_correct(qdit_ctx* ctx, float* latent, int B, int C, int HW, int 
   vc_kernel<<<static_cast<unsigned>(B) * C, 256, 0, ctx->stream>>>(latent, C, HW, mode,
                                                                   table + static_cast<int64_t>(step_index) * C, eps);
   return qdit_after_launch(ctx, "vc_kernel");
+}
+
+int32_t qdit_tap_laplacian(qdit_ctx* ctx, const float* x, const float* t, int n, int d, float alpha, float exponent,
+                           float* workspace, float* L) {
+  if (!ctx) return QDIT_ERR_INVALID_ARG;
+  if (n <= 0 || d <= 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "n and d must be positive");
+  if (n % 4 != 0 || d % 16 != 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "n must be a multiple of 4 and d a multiple of 16");
+  if (!x || !t || !workspace || !L) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "NULL argument");
+  if (!(alpha >= 0.0f && alpha <= 1.0f)) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "alpha must lie in [0, 1]");
+  if (!aligned16(x) || !aligned16(workspace) || !aligned16(L)) return qdit_fail(ctx, QDIT_ERR_ALIGN, "x, workspace and L must be 16-byte aligned");
+  float* xn = workspace;                               // [n, d]
+  float* zero = workspace + static_cast<int64_t>(n) * d;  // [n] zeros (bias of the product)
+  float* deg = zero + n;                               // [n]
+  QDIT_CUDA_CHECK(ctx, cudaMemsetAsync(zero, 0, static_cast<size_t>(n) * sizeof(float), ctx->stream));
+  tap_normalize_kernel<<<static_cast<unsigned>(n), 256, 0, ctx->stream>>>(x, d, xn);
+  QDIT_TRY(qdit_after_launch(ctx, "tap_normalize_kernel"));
+  QDIT_TRY(launch_batched_linear(ctx, xn, xn, zero, nullptr, nullptr, L, nullptr, n, n, d, 0, 0, 0));
+  tap_combine_kernel<<<static_cast<unsigned>(n), 256, 0, ctx->stream>>>(L, t, n, alpha, deg);
+  QDIT_TRY(qdit_after_launch(ctx, "tap_combine_kernel"));
+  tap_scale_kernel<<<static_cast<unsigned>(n), 256, 0, ctx->stream>>>(L, deg, n, exponent);
+  return qdit_after_launch(ctx, "tap_scale_kernel");
 }
 
 int32_t qdit_vc_fit(qdit_ctx* ctx, const float* x_hat, const float* x_target, int N, int C, int HW, float eps, int form,

@@ -118,6 +118,27 @@ def test_vc_fit_matches_the_closed_form(q, ctx, N, C, HW):
     assert (j <= objective(kf * 1.01)).all() and (j <= objective(kf * 0.99)).all()
 
 
+@pytest.mark.parametrize("n,d,alpha,e", [(64, 4096, 0.7, 0.5), (200, 1024, 0.3, -0.5), (4, 16, 1.0, 0.5)])
+def test_tap_laplacian_matches_oracle(q, ctx, n, d, alpha, e):
+    """Similarity matrix and degree normalisation of Algorithm 1 for one subsample."""
+    from oracle import tap
+    x = synth.normal(65, f"tap{n}x{d}", (n, d)) + 0.5          # a common offset: cosines well away from zero
+    if n > 8:
+        x[5] = 0                                               # a zero feature vector
+        x[7] = 3 * x[2]
+    t = synth.uniform_int(65, f"tapt{n}", (n,), 0, 20).astype(np.float32)
+    ws = torch.empty(n * d + 2 * n, dtype=torch.float32, device="cuda")
+    L = torch.empty((n, n), dtype=torch.float32, device="cuda")
+    q.qdit_tap_laplacian(ctx, dev(x), dev(t), n, d, alpha, e, ws, L)
+    q.qdit_sync(ctx)
+    want = tap.laplacian(tap.affinity(x, t, alpha), e)
+    got = L.cpu().numpy().astype(np.float64)
+    assert np.abs(got - want).max() <= 2e-5 * np.abs(want).max()
+    np.testing.assert_allclose(got, got.T, rtol=1e-5, atol=1e-6 * np.abs(want).max())
+    assert q.lib.qdit_tap_laplacian(ctx, dev(x).data_ptr(), dev(t).data_ptr(), n + 1, d, alpha, e, ws.data_ptr(), L.data_ptr()) == q.QDIT_ERR_SHAPE
+    q.qdit_sync(ctx)
+
+
 def test_bounded_wait_times_out_and_context_stays_usable(q, ctx):
     """The time-out path of the pipelined kernels, exercised without hanging anything: a wait with a small poll
     limit on a barrier that nobody signals runs out, a second waiter leaves through the abort flag, the kernel
