@@ -445,6 +445,17 @@ def run_gemm_sweep(args):
                 ms_l = t(ln)
                 row["ln_modulate_gbs"] = 3.0 * M * K / ms_l / 1e6
                 row["ln_modulate_frac_of_hbm"] = row["ln_modulate_gbs"] / peaks["hbm_gbs"]
+                # and the block's attention on the layer's output shape (16 heads of 72, 256 tokens per image)
+                qkv_t = torch.from_numpy(synth.normal(seed, f"qkv{M}", (M, N))).cuda().to(torch.bfloat16)
+
+                def attn():
+                    p0 = qkv_t.data_ptr()
+                    q.qdit_attention(ctx, p0, p0 + 2 * K, p0 + 4 * K, N, M // 256, 16, 256, K // 16, 1.0 / np.sqrt(K // 16),
+                                     a8, q.QDIT_I8, a_qp)
+
+                ms_a = t(attn)
+                row["attention_us"] = ms_a * 1e3
+                row["attention_tflops"] = 4.0 * (M // 256) * 16 * 256 * 256 * (K // 16) / ms_a / 1e9
             rows.append(row)
     q.qdit_sync(ctx)
     q.qdit_destroy(ctx)
