@@ -34,11 +34,11 @@ def ctx(q):
 
 
 class XLRig:
-    def __init__(self, q, ctx, cfg, seed):
+    def __init__(self, q, ctx, cfg, seed, weight_bits=8):
         self.q, self.ctx, self.cfg = q, ctx, cfg
         w = synth.model_weights(seed, cfg)
-        self.om = dit.make_qmodel(cfg, w)
-        self.gm = q.qdit_model_create(ctx, cfg, w)
+        self.om = dit.make_qmodel(cfg, w, weight_bits)
+        self.gm = q.qdit_model_create(ctx, cfg, w, weight_bits)
         del w
         self.samplers = []
 
@@ -163,6 +163,29 @@ def test_ddim50_guided_cached_sampler_batch16(q, ctx, xl256):
     _, nocache, _ = _gpu_trajectory(q, ctx, xl256, latent[7:8], labels[7:8], S, 1, guidance, K, set())
     d = rel_l2(final1, nocache)
     assert 0 < d < 0.5, d
+
+
+def test_forward_xl2_w4a8_matches_oracle(q, ctx):
+    """Full DiT-XL/2 forward with 4-bit channel-wise weights and 8-bit activations (the W4A8 setting of Table 2)."""
+    cfg, seed, B = synth.DIT_XL2, synth.CONFIG_SEEDS["forward_xl2"], 2
+    rig = XLRig(q, ctx, cfg, seed, weight_bits=4)
+    try:
+        latent = synth.normal(seed, "latent", (B, cfg.channels, cfg.latent_side, cfg.latent_side))
+        t = synth.uniform_int(seed, "t", (B,), 0, 1000).astype(np.float64)
+        y = synth.uniform_int(seed, "y", (B,), 0, cfg.num_classes)
+        scales = calib.calibrate_model(rig.om, [(latent, t, y)])
+        rig.set_scales(scales)
+        s = rig.sampler(batch=B, num_steps=2)
+        out = torch.empty((B, 2 * cfg.channels, cfg.latent_side, cfg.latent_side), dtype=torch.float32, device="cuda")
+        q.qdit_forward(ctx, s, dev(latent), dev(t.astype(np.float32)), dev(y.astype(np.int32)), B, out, 0)
+        q.qdit_sync(ctx)
+        got = out.cpu().numpy().astype(np.float64)
+        ref = dit.forward(rig.om, dit.Context(quant="static", scales=scales), latent, t, y)
+        err = rel_l2(got, ref)
+        print(f"forward_xl2 W4A8 rel-L2 vs oracle: {err:.3e}")
+        assert err < 2e-2, err
+    finally:
+        rig.close()
 
 
 def test_ddim100_512_cached_sampler_batch8(q, ctx):
