@@ -357,7 +357,11 @@ __device__ __forceinline__ uint2 quantize_pack8_scaled(const float (&t)[8], floa
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const float c = fminf(fmaxf(t[i], lo_f), hi_f);
-    m[i] = static_cast<uint32_t>(__float_as_int(__fadd_rn(c, 12582912.0f)) + z);
+    m[i] = static_cast<uint32_t>(__float_as_int(__fadd_rn(c, 12582912.0f)));
+  }
+  if (z != 0) {  // uniform over the grid: symmetric quantizers skip the eight adds
+#pragma unroll
+    for (int i = 0; i < 8; ++i) m[i] += static_cast<uint32_t>(z);
   }
   uint2 r;
   r.x = __byte_perm(__byte_perm(m[0], m[1], 0x0040), __byte_perm(m[2], m[3], 0x0040), 0x5410);
