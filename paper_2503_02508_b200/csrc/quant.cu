@@ -281,14 +281,124 @@ __global__ void __launch_bounds__(256) ln_modulate_kernel(const __nv_bfloat16* _
   }
 }
 
-template <int NV>
-void launch_ln(qdit_ctx* ctx, const void* x, int64_t M, int D, int64_t T, float eps, const float* shift,
-               const float* scale, int64_t ld_mod, void* out, int out_dtype, QuantArgs qa) {
-  // two CTAs per SM, contiguous row ranges (at least one row per warp, at most what keeps a range within two samples)
-  int64_t ctas = 2 * static_cast<int64_t>(ctx->num_sms);
+// The same operation for the shape the network's blocks use: 8-bit output and D = 128 * NV4.  A lane owns NV4
+// groups of 4 consecutive columns (group lane + 32 j), so all 32 lanes are busy for every group (D = 1152 has 4.5
+// groups of 8 per lane, which leaves half a warp idle for a fifth of the work), and the f32 arithmetic runs on
+// the two-wide instructions (add / mul / fma on a pair of floats: same rounding per element as the scalar forms).
+// Together that is less than half of the general kernel's instructions per row.  Values are identical to the
+// general kernel's except for the summation order of the two statistics.  A CTA's row range must lie within two
+// samples (rows_per_cta <= T).
+__device__ __forceinline__ float2 f2(float a, float b) { return make_float2(a, b); }
+
+template <int NV4>
+__global__ void __launch_bounds__(256, 2) ln_modulate_q8_kernel(const __nv_bfloat16* __restrict__ x, int M, int T, float eps,
+                                                                const float* __restrict__ shift,
+                                                                const float* __restrict__ scale, int64_t ld_mod,
+                                                                uint8_t* __restrict__ out, QuantArgs qa, int rows_per_cta) {
+  constexpr int D = NV4 * 128, D4 = D / 4;
+  extern __shared__ float4 s_par[];  // [2 samples][mul, add][D / 4]
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int row_begin = blockIdx.x * rows_per_cta;
+  const int row_end = row_begin + rows_per_cta < M ? row_begin + rows_per_cta : M;
+  if (row_begin >= M) return;
+  grid_dependency_wait();  // x and the modulation come from earlier kernels of the stream
+  grid_dependency_release();
+  int row = row_begin + warp;
+  uint2 raw[NV4], raw_next[NV4];
+  if (row < row_end) {
+    const uint2* xr = reinterpret_cast<const uint2*>(x + static_cast<int64_t>(row) * D) + lane;
+#pragma unroll
+    for (int j = 0; j < NV4; ++j) raw[j] = xr[32 * j];
+  }
+  const float inv = __fdiv_rn(1.0f, qa.scale_dev ? __ldg(qa.scale_dev) : qa.scale);
+  const int b0 = row_begin / T;
+  for (int s = 0; s < 2; ++s) {
+    if (static_cast<int64_t>(b0 + s) * T >= row_end) break;
+    const float4* gs = reinterpret_cast<const float4*>(shift + (b0 + s) * ld_mod);
+    const float4* gc = reinterpret_cast<const float4*>(scale + (b0 + s) * ld_mod);
+    for (int i = threadIdx.x; i < D4; i += 256) {
+      const float4 c4 = gc[i], h4 = gs[i];
+      s_par[(s * 2 + 0) * D4 + i] = make_float4((1.0f + c4.x) * inv, (1.0f + c4.y) * inv, (1.0f + c4.z) * inv, (1.0f + c4.w) * inv);
+      s_par[(s * 2 + 1) * D4 + i] = make_float4(h4.x * inv, h4.y * inv, h4.z * inv, h4.w * inv);
+    }
+  }
+  __syncthreads();
+  constexpr float inv_d = 1.0f / static_cast<float>(D);
+  const int second = (b0 + 1) * T;  // first row of the second staged sample
+  const float lo_f = qa.qmin - qa.zp, hi_f = qa.qmax - qa.zp;
+  const uint32_t z4 = (static_cast<uint32_t>(static_cast<int>(qa.zp)) & 0xFFu) * 0x01010101u;
+  const float2 magic = f2(12582912.0f, 12582912.0f);
+  for (; row < row_end; row += 8) {
+    const int next = row + 8;
+    if (next < row_end) {
+      const uint2* xr = reinterpret_cast<const uint2*>(x + static_cast<int64_t>(next) * D) + lane;
+#pragma unroll
+      for (int j = 0; j < NV4; ++j) raw_next[j] = xr[32 * j];
+    }
+    float2 v[NV4][2];
+    float2 s0 = f2(0.0f, 0.0f), s1 = f2(0.0f, 0.0f);
+#pragma unroll
+    for (int j = 0; j < NV4; ++j) {
+      v[j][0] = f2(__uint_as_float(raw[j].x << 16), __uint_as_float(raw[j].x & 0xFFFF0000u));
+      v[j][1] = f2(__uint_as_float(raw[j].y << 16), __uint_as_float(raw[j].y & 0xFFFF0000u));
+      s0 = __fadd2_rn(s0, v[j][0]);
+      s1 = __fadd2_rn(s1, v[j][1]);
+    }
+    const float mean = warp_sum((s0.x + s0.y) + (s1.x + s1.y)) * inv_d;
+    const float2 nmean = f2(-mean, -mean);
+    float2 q0 = f2(0.0f, 0.0f), q1 = f2(0.0f, 0.0f);
+#pragma unroll
+    for (int j = 0; j < NV4; ++j) {
+      v[j][0] = __fadd2_rn(v[j][0], nmean);
+      v[j][1] = __fadd2_rn(v[j][1], nmean);
+      q0 = __ffma2_rn(v[j][0], v[j][0], q0);
+      q1 = __ffma2_rn(v[j][1], v[j][1], q1);
+    }
+    const float rstd = rsqrtf(warp_sum((q0.x + q0.y) + (q1.x + q1.y)) * inv_d + eps);
+    const float2 r2 = f2(rstd, rstd);
+    const float4* pm = s_par + (row < second ? 0 : 2) * D4 + lane;
+    const float4* pa = pm + D4;
+    uint32_t* orow = reinterpret_cast<uint32_t*>(out + static_cast<int64_t>(row) * D) + lane;
+#pragma unroll
+    for (int j = 0; j < NV4; ++j) {
+      const float4 m4 = pm[32 * j], a4 = pa[32 * j];
+      // y / s_out = (x - mean) * (rstd * mul) + add, then Eq. 1's clip and round on the scaled value
+      float2 y0 = __ffma2_rn(v[j][0], __fmul2_rn(r2, f2(m4.x, m4.y)), f2(a4.x, a4.y));
+      float2 y1 = __ffma2_rn(v[j][1], __fmul2_rn(r2, f2(m4.z, m4.w)), f2(a4.z, a4.w));
+      y0 = __fadd2_rn(f2(fminf(fmaxf(y0.x, lo_f), hi_f), fminf(fmaxf(y0.y, lo_f), hi_f)), magic);
+      y1 = __fadd2_rn(f2(fminf(fmaxf(y1.x, lo_f), hi_f), fminf(fmaxf(y1.y, lo_f), hi_f)), magic);
+      uint32_t w = __byte_perm(__byte_perm(__float_as_uint(y0.x), __float_as_uint(y0.y), 0x0040),
+                               __byte_perm(__float_as_uint(y1.x), __float_as_uint(y1.y), 0x0040), 0x5410);
+      if (z4 != 0u) w = __vadd4(w, z4);  // code + z stays inside a byte
+      orow[32 * j] = w;
+    }
+#pragma unroll
+    for (int j = 0; j < NV4; ++j) raw[j] = raw_next[j];
+  }
+}
+
+template <int NV4>
+void launch_ln_q8(qdit_ctx* ctx, const void* x, int64_t M, const float* shift, const float* scale, int64_t ld_mod,
+                  int64_t T, float eps, void* out, QuantArgs qa, int64_t rows) {
+  const unsigned grid = static_cast<unsigned>((M + rows - 1) / rows);
+  qdit_launch_overlapped(ctx, ln_modulate_q8_kernel<NV4>, dim3(grid), dim3(256), static_cast<size_t>(NV4) * 128 * 16,
+                         static_cast<const __nv_bfloat16*>(x), static_cast<int>(M), static_cast<int>(T), eps, shift, scale,
+                         ld_mod, static_cast<uint8_t*>(out), qa, static_cast<int>(rows));
+}
+
+// Row range per CTA: two CTAs per SM, at least one row per warp, at most what keeps a range within two samples.
+int64_t ln_rows_per_cta(const qdit_ctx* ctx, int64_t M, int64_t T) {
+  const int64_t ctas = 2 * static_cast<int64_t>(ctx->num_sms);
   int64_t rows = (M + ctas - 1) / ctas;
   if (rows < 8) rows = 8;
   if (rows > T) rows = T;
+  return rows;
+}
+
+template <int NV>
+void launch_ln(qdit_ctx* ctx, const void* x, int64_t M, int D, int64_t T, float eps, const float* shift,
+               const float* scale, int64_t ld_mod, void* out, int out_dtype, QuantArgs qa) {
+  const int64_t rows = ln_rows_per_cta(ctx, M, T);
   const unsigned grid = static_cast<unsigned>((M + rows - 1) / rows);
   qdit_launch_overlapped(ctx, ln_modulate_kernel<NV>, dim3(grid), dim3(256), static_cast<size_t>(NV) * 4096,
                          static_cast<const __nv_bfloat16*>(x), static_cast<int>(M), D, static_cast<int>(T), eps, shift, scale,
@@ -416,6 +526,19 @@ int32_t qdit_adaln_modulate(qdit_ctx* ctx, const void* x, int64_t M, int64_t D, 
   const int d = static_cast<int>(D);
   const double out_bytes = out_dtype == QDIT_I8 ? 1.0 : out_dtype == QDIT_BF16 ? 2.0 : 4.0;
   ProfScope prof(ctx, QDIT_PROF_LN_MODULATE, static_cast<double>(M) * D * (2.0 + out_bytes));
+  if (out_dtype == QDIT_I8 && D % 128 == 0) {
+    // the widths of the DiT family (S 384, B 768, L 1024, XL 1152) with 8-bit output: the two-wide kernel
+    const int64_t rows = ln_rows_per_cta(ctx, M, T);
+    bool done = true;
+    switch (D / 128) {
+      case 3: launch_ln_q8<3>(ctx, x, M, shift, scale, ld_mod, T, eps, out, qa, rows); break;
+      case 6: launch_ln_q8<6>(ctx, x, M, shift, scale, ld_mod, T, eps, out, qa, rows); break;
+      case 8: launch_ln_q8<8>(ctx, x, M, shift, scale, ld_mod, T, eps, out, qa, rows); break;
+      case 9: launch_ln_q8<9>(ctx, x, M, shift, scale, ld_mod, T, eps, out, qa, rows); break;
+      default: done = false; break;
+    }
+    if (done) return qdit_after_launch(ctx, "ln_modulate_q8_kernel");
+  }
   switch (nv) {
     case 1: launch_ln<1>(ctx, x, M, d, T, eps, shift, scale, ld_mod, out, out_dtype, qa); break;
     case 2: launch_ln<2>(ctx, x, M, d, T, eps, shift, scale, ld_mod, out, out_dtype, qa); break;
