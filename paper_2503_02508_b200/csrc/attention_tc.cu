@@ -332,6 +332,285 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
   }
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// T = 256 (two key blocks): the whole score row fits the CTA's 256 tensor-memory columns, so the softmax is
+// taken in one piece instead of online.  Both K blocks and V_0 are requested at once (K_1 lands in the P tile,
+// which nobody needs before both S blocks are complete); S_0 and S_1 are issued back to back; V_1 is requested
+// into the Q tile as soon as the S products have finished reading Q.  One row maximum (one exchange between
+// the two threads of a row), no rescaling, both P.V products accumulate into the same columns (those of S_0),
+// which are read once at the end.  Same shared and tensor memory as the general kernel: two CTAs per SM.
+// Every barrier completes exactly once (phase 0).
+template <int DH>
+__global__ void __launch_bounds__(TC_THREADS, 2)
+attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                       const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_qt,
+                       const __grid_constant__ CUtensorMap tm_kt, const __grid_constant__ CUtensorMap tm_vt,
+                       const AttnTcParams p) {
+  using C = TCfg<DH>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sQ = smem;                           // Q, later V_1
+  uint8_t* sK = sQ + C::MAIN_BYTES;             // K_0
+  uint8_t* sV = sK + C::MAIN_BYTES;             // V_0
+  uint8_t* sP = sV + C::MAIN_BYTES;             // K_1 (main tile, tail tile behind it), later P (two 64-key tiles)
+  uint8_t* sQt = sP + C::P_BYTES;               // tails (256-byte aligned: 32B-swizzle atoms); Q's, later V_1's
+  uint8_t* sKt = sQt + C::TAIL_BYTES;
+  uint8_t* sVt = sKt + C::TAIL_BYTES;
+  uint8_t* sK1 = sP;
+  uint8_t* sK1t = sP + C::MAIN_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sVt + C::TAIL_BYTES);
+  uint64_t* bar_q = bars + 0;      // Q tiles landed (tx)
+  uint64_t* bar_qz = bars + 1;     // Q tail padding zeroed (256 arrivals)
+  uint64_t* bar_k = bars + 2;      // [2] K block landed (tx)
+  uint64_t* bar_v = bars + 4;      // [2] V block landed (tx)
+  uint64_t* bar_s = bars + 6;      // [2] S block complete (commit); [1] also: Q and both K blocks have been read
+  uint64_t* bar_p = bars + 8;      // [2] P block written (256 arrivals)
+  uint64_t* bar_o = bars + 10;     // [2] P.V of block 0 / of both blocks complete (commit)
+  uint64_t* bar_l = bars + 12;     // row sums exchanged (256 arrivals)
+  uint64_t* bar_mx = bars + 13;    // [4] row maxima exchanged between the two warps of a lane quadrant (64 arrivals)
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 17);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  float* s_l = reinterpret_cast<float*>(tmem_holder + 4);  // [2][128] partial row sums
+  float* s_m = s_l + 256;                                  // [2][128] partial row maxima
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int q0 = blockIdx.x * TQ, h = blockIdx.y, b = blockIdx.z;
+  const int row0 = b * p.T, col0 = h * DH;
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar_q, 1);
+    mbar_init(bar_qz, SM_WARPS * 32);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bar_k[i], 1);
+      mbar_init(&bar_v[i], 1);
+      mbar_init(&bar_s[i], 1);
+      mbar_init(&bar_p[i], SM_WARPS * 32);
+      mbar_init(&bar_o[i], 1);
+    }
+    mbar_init(bar_l, SM_WARPS * 32);
+    for (int i = 0; i < 4; ++i) mbar_init(&bar_mx[i], 64);
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  if (warp == SM_WARPS + 1) {
+    tmem_alloc(tmem_holder, 256);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_holder;
+  // shared and tensor memory only so far; Q, K and V come from the previous kernel of the stream
+  grid_dependency_wait();
+  grid_dependency_release();
+
+  if (warp == SM_WARPS) {
+    if (lane == 0) {
+      // ---------------------------------------------------------------- TMA producer
+      mbar_expect_tx(bar_q, C::OP_BYTES);
+      tma_load_2d(sQ, &tm_q, col0, row0 + q0, bar_q);
+      if (C::TAIL) tma_load_2d(sQt, &tm_qt, col0 + 64, row0 + q0, bar_q);
+      mbar_expect_tx(&bar_k[0], C::OP_BYTES);
+      tma_load_2d(sK, &tm_k, col0, row0, &bar_k[0]);
+      if (C::TAIL) tma_load_2d(sKt, &tm_kt, col0 + 64, row0, &bar_k[0]);
+      mbar_expect_tx(&bar_k[1], C::OP_BYTES);
+      tma_load_2d(sK1, &tm_k, col0, row0 + TK, &bar_k[1]);
+      if (C::TAIL) tma_load_2d(sK1t, &tm_kt, col0 + 64, row0 + TK, &bar_k[1]);
+      mbar_expect_tx(&bar_v[0], C::OP_BYTES);
+      tma_load_2d(sV, &tm_v, col0, row0, &bar_v[0]);
+      if (C::TAIL) tma_load_2d(sVt, &tm_vt, col0 + 64, row0, &bar_v[0]);
+      // V_1 takes Q's place once both S products have read Q
+      if (mbar_wait(&bar_s[1], 0, abort_flag, p.status)) {
+        mbar_expect_tx(&bar_v[1], C::OP_BYTES);
+        tma_load_2d(sQ, &tm_v, col0, row0 + TK, &bar_v[1]);
+        if (C::TAIL) tma_load_2d(sQt, &tm_vt, col0 + 64, row0 + TK, &bar_v[1]);
+      }
+    }
+  } else if (warp == SM_WARPS + 1) {
+    if (lane == 0) {
+      // ---------------------------------------------------------------- MMA issuer
+      const uint32_t id_s = umma_idesc_bf16(128, TK, false);
+      const uint32_t id_o = umma_idesc_bf16(128, 64, true);
+      const uint32_t id_ot = umma_idesc_bf16(128, 16, true);
+      // S_j = Q K_j^T into columns 128 j: 4 k-steps of 16 out of the 64-column tiles, one out of the tails
+      auto issue_s = [&](int j, const uint8_t* k_main, const uint8_t* k_tail) {
+        const uint32_t d = tmem + static_cast<uint32_t>(j * 128);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          umma_bf16(d, umma_desc(smem_u32(sQ) + k * 32, 1024, 2), umma_desc(smem_u32(k_main) + k * 32, 1024, 2), id_s, k ? 1u : 0u);
+        if (C::TAIL) umma_bf16(d, umma_desc(smem_u32(sQt), 256, 6), umma_desc(smem_u32(k_tail), 256, 6), id_s, 1u);
+        umma_commit(&bar_s[j]);
+      };
+      // O += P_j V_j over columns 0..79: 8 k-steps of 16 keys; V's 8-key groups are 1024 (main) / 256 (tail) bytes apart
+      auto issue_pv = [&](int j, const uint8_t* v_main, const uint8_t* v_tail) {
+#pragma unroll
+        for (int k = 0; k < TK / 16; ++k) {
+          const uint64_t a = umma_desc(smem_u32(sP) + (k >> 2) * C::MAIN_BYTES + (k & 3) * 32, 1024, 2);
+          const uint32_t acc = (j | k) ? 1u : 0u;
+          umma_bf16(tmem, a, umma_desc(smem_u32(v_main) + k * 2048, 1024, 2), id_o, acc);
+          if (C::TAIL) umma_bf16(tmem + 64, a, umma_desc(smem_u32(v_tail) + k * 512, 256, 6), id_ot, acc);
+        }
+        umma_commit(&bar_o[j]);
+      };
+      bool ok = mbar_wait(bar_qz, 0, abort_flag, p.status) && mbar_wait(&bar_k[0], 0, abort_flag, p.status);
+      if (ok) {
+        tc_fence_after();
+        issue_s(0, sK, sKt);
+      }
+      ok = ok && mbar_wait(&bar_k[1], 0, abort_flag, p.status);
+      if (ok) {
+        tc_fence_after();
+        issue_s(1, sK1, sK1t);
+      }
+      ok = ok && mbar_wait(&bar_p[0], 0, abort_flag, p.status) && mbar_wait(&bar_v[0], 0, abort_flag, p.status);
+      if (ok) {
+        tc_fence_after();
+        issue_pv(0, sV, sVt);
+      }
+      ok = ok && mbar_wait(&bar_p[1], 0, abort_flag, p.status) && mbar_wait(&bar_v[1], 0, abort_flag, p.status);
+      if (ok) {
+        tc_fence_after();
+        issue_pv(1, sQ, sQt);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax (two threads per query row)
+    const int quad = warp & 3, half = warp >> 2;
+    const int r = quad * 32 + lane;
+    const uint32_t trow = tmem + (static_cast<uint32_t>(quad * 32) << 16);
+    bool ok = mbar_wait(bar_q, 0, abort_flag, p.status);
+    if (ok) {
+      if (C::TAIL && half == 0) {  // zero columns 72..79 of this row of the Q tail (second 16-byte slot, 32B swizzle)
+        const uint32_t addr = smem_u32(sQt) + static_cast<uint32_t>(r * 32) + ((1u ^ ((static_cast<uint32_t>(r) >> 2) & 1u)) << 4);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
+        fence_async_smem();
+      }
+      mbar_arrive(bar_qz);
+    }
+    // row maximum over this thread's 64 keys of each block, then over the row with the other thread's value
+    float mx = -INFINITY;
+#pragma unroll 1
+    for (int j = 0; j < 2 && ok; ++j) {
+      if (!mbar_wait(&bar_s[j], 0, abort_flag, p.status)) { ok = false; break; }
+      __syncwarp();
+      tc_fence_after();
+      uint32_t v0[32], v1[32];  // both loads in flight, one wait
+      const uint32_t sbuf = trow + static_cast<uint32_t>(j * 128 + half * 64);
+      tmem_ld_32x32(sbuf, v0);
+      tmem_ld_32x32(sbuf + 32, v1);
+      tmem_ld_wait();
+      float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        m0 = fmaxf(m0, __uint_as_float(v0[i]));
+        m1 = fmaxf(m1, __uint_as_float(v1[i]));
+      }
+      mx = fmaxf(mx, fmaxf(m0, m1));
+    }
+    if (ok) {
+      s_m[half * 128 + r] = mx;
+      mbar_arrive(&bar_mx[quad]);
+      ok = mbar_wait(&bar_mx[quad], 0, abort_flag, p.status);
+    }
+    float rs = 0.0f;
+    if (ok) {
+      const float m_row = fmaxf(mx, s_m[(half ^ 1) * 128 + r]) * p.scale_log2;
+      const uint32_t tile = smem_u32(sP) + static_cast<uint32_t>(half * C::MAIN_BYTES + r * 128);
+#pragma unroll 1
+      for (int j = 0; j < 2 && ok; ++j) {
+        // P_j = exp2(s * scale - m) for this thread's 64 keys of block j: bf16, row sum in f32
+        const uint32_t sbuf = trow + static_cast<uint32_t>(j * 128 + half * 64);
+        uint32_t pk[32];
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t v[32];
+          tmem_ld_32x32(sbuf + c * 32, v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float p0 = ex2_approx(fmaf(__uint_as_float(v[2 * i]), p.scale_log2, -m_row));
+            const float p1 = ex2_approx(fmaf(__uint_as_float(v[2 * i + 1]), p.scale_log2, -m_row));
+            rs += p0 + p1;
+            pk[c * 16 + i] = pack_bf16x2(p0, p1);
+          }
+        }
+        // the P tile is free once the tensor core has read what it held: K_1 (both S complete: waited for above)
+        // for block 0, P_0 for block 1
+        if (j == 1) {
+          if (!mbar_wait(&bar_o[0], 0, abort_flag, p.status)) { ok = false; break; }
+          tc_fence_after();
+        }
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          const uint32_t addr = tile + ((static_cast<uint32_t>(g) ^ (static_cast<uint32_t>(r) & 7u)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[4 * g]), "r"(pk[4 * g + 1]),
+                       "r"(pk[4 * g + 2]), "r"(pk[4 * g + 3])
+                       : "memory");
+        }
+        fence_async_smem();   // P is read by the tensor core through the async proxy
+        tc_fence_before();    // and (block 0) the S_0 columns are about to be overwritten by O
+        mbar_arrive(&bar_p[j]);
+      }
+    }
+    // the two threads of a row exchange their partial sums
+    if (ok) {
+      s_l[half * 128 + r] = rs;
+      mbar_arrive(bar_l);
+      ok = mbar_wait(bar_l, 0, abort_flag, p.status);
+    }
+    if (ok && mbar_wait(&bar_o[1], 0, abort_flag, p.status)) {
+      __syncwarp();
+      tc_fence_after();
+      float o[C::O_HALF];
+      const uint32_t src = trow + static_cast<uint32_t>(half * C::O_HALF);
+      {
+        uint32_t v[32];
+        tmem_ld_32x32(src, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(v[i]);
+        if (C::TAIL) {
+          uint32_t w[8];
+          tmem_ld_32x8(src + 32, w);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 8; ++i) o[32 + i] = __uint_as_float(w[i]);
+        }
+      }
+      const float inv_l = 1.0f / (s_l[r] + s_l[128 + r]);
+      const int64_t row = static_cast<int64_t>(row0) + q0 + r;
+      const int64_t base = row * (static_cast<int64_t>(p.H) * DH) + col0 + half * C::O_HALF;
+      const int ngroups = half == 0 ? C::O_HALF / 8 : (DH - C::O_HALF) / 8;  // output columns beyond DH are padding
+      float q_inv = 0.0f;
+      if (p.out_dtype == QDIT_I8) q_inv = __fdiv_rn(1.0f, p.qa.scale_dev ? __ldg(p.qa.scale_dev) : p.qa.scale);
+#pragma unroll
+      for (int g = 0; g < C::O_HALF / 8; ++g) {
+        if (g < ngroups) {
+          float y[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) y[i] = o[8 * g + i] * inv_l;
+          if (p.out_dtype == QDIT_I8) {
+            *reinterpret_cast<uint2*>(static_cast<uint8_t*>(p.out) + base + 8 * g) = quantize_pack8(y, q_inv, p.qa.zp, p.qa.qmin, p.qa.qmax);
+          } else if (p.out_dtype == QDIT_BF16) {
+            *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + base + 8 * g) = pack_bf16x8(y);
+          } else {
+            float* of = static_cast<float*>(p.out) + base + 8 * g;
+            *reinterpret_cast<float4*>(of) = make_float4(y[0], y[1], y[2], y[3]);
+            *reinterpret_cast<float4*>(of + 4) = make_float4(y[4], y[5], y[6], y[7]);
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == SM_WARPS + 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 256);
+  }
+}
+
 template <int DH>
 int32_t launch_tc(qdit_ctx* ctx, const void* q, const void* k, const void* v, int64_t ld, int B, int H, int T,
                   const AttnTcParams& p) {
@@ -339,6 +618,7 @@ int32_t launch_tc(qdit_ctx* ctx, const void* q, const void* k, const void* v, in
   static bool attr_set[64] = {};
   if (!attr_set[ctx->device & 63]) {
     QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(attention_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+    QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(attention_tc256_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
     attr_set[ctx->device & 63] = true;
   }
   const uint64_t rows = static_cast<uint64_t>(B) * T, cols = static_cast<uint64_t>(H) * DH;
@@ -356,6 +636,10 @@ int32_t launch_tc(qdit_ctx* ctx, const void* q, const void* k, const void* v, in
   }
   dim3 grid(T / TQ, H, B);
   ProfScope prof(ctx, QDIT_PROF_ATTENTION, 4.0 * B * H * static_cast<double>(T) * T * DH);
+  if (T == 2 * TK && !getenv("QDIT_ATTN_ONLINE")) {  // the whole score row in tensor memory (tuning switch: the general kernel)
+    QDIT_CUDA_CHECK(ctx, qdit_launch_overlapped(ctx, attention_tc256_kernel<DH>, grid, dim3(TC_THREADS), C::SMEM_BYTES, tq, tk, tv, tqt, tkt, tvt, p));
+    return qdit_after_launch(ctx, "attention_tc256_kernel");
+  }
   QDIT_CUDA_CHECK(ctx, qdit_launch_overlapped(ctx, attention_tc_kernel<DH>, grid, dim3(TC_THREADS), C::SMEM_BYTES, tq, tk, tv, tqt, tkt, tvt, p));
   return qdit_after_launch(ctx, "attention_tc_kernel");
 }

@@ -280,14 +280,6 @@ __device__ __forceinline__ float gelu_tanh_f(float x) {
   const float e = ex2_approx(x * fmaf(x * x, b, a));
   return __fdividef(x, 1.0f + e);
 }
-// The same function for a pair: the polynomial and the 1 + e on the two-wide f32 instructions, which round each
-// element like their scalar forms, so both elements equal gelu_tanh_f of themselves bit for bit.
-__device__ __forceinline__ float2 gelu_tanh_f2(float2 x) {
-  const float2 a = make_float2(-2.3022081998f, -2.3022081998f), b = make_float2(-0.1029432396f, -0.1029432396f);
-  const float2 t = __fmul2_rn(x, __ffma2_rn(__fmul2_rn(x, x), b, a));
-  const float2 d = __fadd2_rn(make_float2(ex2_approx(t.x), ex2_approx(t.y)), make_float2(1.0f, 1.0f));
-  return make_float2(__fdividef(x.x, d.x), __fdividef(x.y, d.y));
-}
 __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + expf(-x)); }
 
 __device__ __forceinline__ float warp_sum(float v) {

@@ -135,34 +135,18 @@ __device__ __forceinline__ void epilogue_chunk_t_packed(const GemmParams& p, con
   const int n8 = n - i8;  // first channel of this lane group
   // The epilogue of the GELU layer is bound by instruction issue, so work that a symmetric quantizer does not
   // need (zero-point terms) is skipped through branches that are uniform over the whole grid.
-  // The f32 arithmetic runs on the two-wide instructions (mul / add / fma on a pair of floats, each element rounded
-  // as by the scalar instruction): tokens (2k, 2k + 1) of the chunk share an instruction.
-  float2 g[16];
+  float f[32];
   if (p.a_zp == 0) {
 #pragma unroll
-    for (int k = 0; k < 16; ++k)
-      g[k] = make_float2(static_cast<float>(static_cast<int>(v[2 * k])), static_cast<float>(static_cast<int>(v[2 * k + 1])));
+    for (int j = 0; j < 32; ++j) f[j] = static_cast<float>(static_cast<int>(v[j]));
   } else {
 #pragma unroll
-    for (int k = 0; k < 16; ++k)
-      g[k] = make_float2(static_cast<float>(static_cast<int>(v[2 * k]) - zcs), static_cast<float>(static_cast<int>(v[2 * k + 1]) - zcs));
+    for (int j = 0; j < 32; ++j) f[j] = static_cast<float>(static_cast<int>(v[j]) - zcs);
   }
-  const float2 sc2 = make_float2(sc, sc), bias2 = make_float2(bias, bias);
 #pragma unroll
-  for (int k = 0; k < 16; ++k) {
-    g[k] = (flags & QDIT_EPI_BIAS) ? __ffma2_rn(g[k], sc2, bias2) : __fmul2_rn(g[k], sc2);
-    if (flags & QDIT_EPI_GELU) g[k] = gelu_tanh_f2(g[k]);
-  }
-  if (flags & QDIT_EPI_QUANT_OUT) {
-    const float2 oi2 = make_float2(o_inv, o_inv);
-#pragma unroll
-    for (int k = 0; k < 16; ++k) g[k] = __fmul2_rn(g[k], oi2);
-  }
-  float f[32];
-#pragma unroll
-  for (int k = 0; k < 16; ++k) {
-    f[2 * k] = g[k].x;
-    f[2 * k + 1] = g[k].y;
+  for (int j = 0; j < 32; ++j) {
+    f[j] = (flags & QDIT_EPI_BIAS) ? __fmaf_rn(f[j], sc, bias) : __fmul_rn(f[j], sc);
+    if (flags & QDIT_EPI_GELU) f[j] = gelu_tanh_f(f[j]);
   }
   if (flags & QDIT_EPI_QUANT_OUT) {
     // one byte per token: word t = codes of tokens t, 8 + t, 16 + t, 24 + t
@@ -174,7 +158,7 @@ __device__ __forceinline__ void epilogue_chunk_t_packed(const GemmParams& p, con
       uint32_t m4[4];
 #pragma unroll
       for (int s4 = 0; s4 < 4; ++s4) {
-        const float q = fminf(fmaxf(f[8 * s4 + t], lo_f), hi_f);  // f is already x / s_out
+        const float q = fminf(fmaxf(__fmul_rn(f[8 * s4 + t], o_inv), lo_f), hi_f);
         m4[s4] = static_cast<uint32_t>(__float_as_int(__fadd_rn(q, 12582912.0f)));
       }
       w[t] = __byte_perm(__byte_perm(m4[0], m4[1], 0x0040), __byte_perm(m4[2], m4[3], 0x0040), 0x5410);
