@@ -291,7 +291,7 @@ __global__ void __launch_bounds__(256) ln_modulate_kernel(const __nv_bfloat16* _
 __device__ __forceinline__ float2 f2(float a, float b) { return make_float2(a, b); }
 
 template <int NV4>
-__global__ void __launch_bounds__(256, 2) ln_modulate_q8_kernel(const __nv_bfloat16* __restrict__ x, int M, int T, float eps,
+__global__ void __launch_bounds__(256, 3) ln_modulate_q8_kernel(const __nv_bfloat16* __restrict__ x, int M, int T, float eps,
                                                                 const float* __restrict__ shift,
                                                                 const float* __restrict__ scale, int64_t ld_mod,
                                                                 uint8_t* __restrict__ out, QuantArgs qa, int rows_per_cta) {
@@ -386,9 +386,9 @@ void launch_ln_q8(qdit_ctx* ctx, const void* x, int64_t M, const float* shift, c
                          ld_mod, static_cast<uint8_t*>(out), qa, static_cast<int>(rows));
 }
 
-// Row range per CTA: two CTAs per SM, at least one row per warp, at most what keeps a range within two samples.
-int64_t ln_rows_per_cta(const qdit_ctx* ctx, int64_t M, int64_t T) {
-  const int64_t ctas = 2 * static_cast<int64_t>(ctx->num_sms);
+// Row range per CTA: `per_sm` CTAs per SM, at least one row per warp, at most what keeps a range within two samples.
+int64_t ln_rows_per_cta(const qdit_ctx* ctx, int64_t M, int64_t T, int per_sm) {
+  const int64_t ctas = per_sm * static_cast<int64_t>(ctx->num_sms);
   int64_t rows = (M + ctas - 1) / ctas;
   if (rows < 8) rows = 8;
   if (rows > T) rows = T;
@@ -398,7 +398,7 @@ int64_t ln_rows_per_cta(const qdit_ctx* ctx, int64_t M, int64_t T) {
 template <int NV>
 void launch_ln(qdit_ctx* ctx, const void* x, int64_t M, int D, int64_t T, float eps, const float* shift,
                const float* scale, int64_t ld_mod, void* out, int out_dtype, QuantArgs qa) {
-  const int64_t rows = ln_rows_per_cta(ctx, M, T);
+  const int64_t rows = ln_rows_per_cta(ctx, M, T, 2);
   const unsigned grid = static_cast<unsigned>((M + rows - 1) / rows);
   qdit_launch_overlapped(ctx, ln_modulate_kernel<NV>, dim3(grid), dim3(256), static_cast<size_t>(NV) * 4096,
                          static_cast<const __nv_bfloat16*>(x), static_cast<int>(M), D, static_cast<int>(T), eps, shift, scale,
@@ -528,7 +528,7 @@ int32_t qdit_adaln_modulate(qdit_ctx* ctx, const void* x, int64_t M, int64_t D, 
   ProfScope prof(ctx, QDIT_PROF_LN_MODULATE, static_cast<double>(M) * D * (2.0 + out_bytes));
   if (out_dtype == QDIT_I8 && D % 128 == 0) {
     // the widths of the DiT family (S 384, B 768, L 1024, XL 1152) with 8-bit output: the two-wide kernel
-    const int64_t rows = ln_rows_per_cta(ctx, M, T);
+    const int64_t rows = ln_rows_per_cta(ctx, M, T, 3);  // 80 registers: three CTAs of 8 warps per SM
     bool done = true;
     switch (D / 128) {
       case 3: launch_ln_q8<3>(ctx, x, M, shift, scale, ld_mod, T, eps, out, qa, rows); break;
