@@ -61,8 +61,9 @@ def test_attention_matches_oracle(q, ctx, B, T, H, dh):
     np.testing.assert_array_equal(gb, dit.round_bf16(got))
 
 
-def test_attention_special_cases(q, ctx):
-    B, T, H, dh = 1, 128, 2, 72
+@pytest.mark.parametrize("T", [128, 256])            # one key block (online kernel) / two (whole row in tensor memory)
+def test_attention_special_cases(q, ctx, T):
+    B, H, dh = 1, 2, 72
     D = H * dh
     x = synth.normal(52, "qkv0", (B * T, 3 * D), 1.0)
     x[:, :D] = 0                                     # zero queries -> mean of V

@@ -200,3 +200,32 @@ def test_adaln_modulate_fused_quantizer(q, ctx, B, T, D):
     n_bad, ok = code_mismatch_report(got, want, pre, tol)
     assert ok and n_bad <= 1e-3 * got.size, (n_bad, got.size)
     assert np.abs(got).max() == 127 and (np.abs(want) == 127).sum() > 3
+
+
+@pytest.mark.parametrize("B,T,D,asym", [(3, 5, 384, False), (7, 33, 768, True), (2, 100, 1024, False), (5, 64, 1152, True),
+                                        (3, 64, 1152, False), (2, 8, 144, True)])
+def test_adaln_modulate_fused_quantizer_ragged_and_unsigned(q, ctx, B, T, D, asym):
+    """Row counts that leave ragged row ranges per CTA, ranges that straddle two samples, the other widths of the
+    two-wide kernel (768, 1024), a width it does not take (144), and Eq. 1's unsigned codes with a zero point."""
+    M = B * T
+    x = synth.normal(12, f"lrx{D}_{T}", (M, D), 1.3, -0.2)
+    mod = synth.normal(12, f"lrm{D}_{T}", (B, 6 * D), 0.4)
+    xd = dev(x).to(torch.bfloat16)
+    xh = bf16_to_f64(xd)
+    md = dev(mod)
+    ref = dit.layer_norm_modulate(xh, mod[:, :D], mod[:, D:2 * D], T)
+    if asym:
+        qp = quant.qparams_minmax(ref * 0.6)                              # Eq. 2-3 range, saturating at both ends
+    else:
+        qp = quant.qparams_symmetric(float(np.abs(ref).max()) * 0.6)
+    out = torch.empty((M, D), dtype=torch.uint8, device="cuda")
+    q.qdit_adaln_modulate(ctx, xd, M, D, T, 1e-6, md[:, :D], md[:, D:2 * D], 6 * D, out, q.QDIT_I8,
+                          q.qparams(qp.scale, qp.zero_point, qp.qmin, qp.qmax))
+    q.qdit_sync(ctx)
+    got = host_codes(out, signed=not asym)
+    want = quant.quantize(ref, qp)
+    pre = ref.astype(np.float32).astype(np.float64) * float(qp.inv_scale)
+    tol = 1e-4 * np.abs(pre).max() + 1e-6
+    n_bad, ok = code_mismatch_report(got, want, pre, tol)
+    assert ok and n_bad <= 2e-3 * got.size, (n_bad, got.size)
+    assert got.min() == qp.qmin and got.max() == qp.qmax
