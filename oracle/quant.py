@@ -11,8 +11,8 @@ Readings taken where the paper is silent or garbled:
     float32 once; the rounding decision is taken in float32.
   * Besides the unsigned range of Eq. 1 a symmetric signed range [-127, 127]
     with z = 0 is supported (s = max|X| / 127); weights use it per output channel
-    and activations per tensor ("channel-wise ... weights, tensor-wise ...
-    activations", Comparison on Performance).
+    and activations per tensor (granularities as stated in the section
+    "Comparison on Performance").
   * A degenerate range (u == l, or max|X| == 0) takes s = 1.
 """
 from __future__ import annotations
@@ -95,3 +95,32 @@ def quantize_weight_per_channel(W: np.ndarray, bits: int = 8):
     inv = (F32(1.0) / s).astype(F32)
     q = np.clip(np.rint(W * inv[:, None]), -top, top).astype(np.int32)
     return q, s, q.sum(axis=1, dtype=np.int64)
+
+
+def pack_int4(q: np.ndarray) -> np.ndarray:
+    """Storage form of 4-bit weight codes (the W4A8 setting of Table 2): two signed codes per byte.
+
+    q: integer codes in [-8, 7], shape [N, K] with K even.  Byte j of a row holds code 2j in its low nibble and
+    code 2j + 1 in its high nibble, each as a 4-bit two's-complement number.  Returns uint8 [N, K/2].
+    (The byte layout is this build's choice: the paper fixes the code width only.)
+    """
+    q = np.asarray(q)
+    if q.ndim != 2 or q.shape[1] % 2:
+        raise ValueError("codes must be [N, K] with K even")
+    if q.min(initial=0) < -8 or q.max(initial=0) > 7:
+        raise ValueError("codes outside the 4-bit range [-8, 7]")
+    n = (q.astype(np.int64) & 0xF).astype(np.uint8)
+    return (n[:, 0::2] | (n[:, 1::2] << 4)).astype(np.uint8)
+
+
+def unpack_int4(p: np.ndarray) -> np.ndarray:
+    """Inverse of pack_int4: uint8 [N, K/2] -> int32 codes [N, K] (nibbles sign-extended)."""
+    p = np.asarray(p, dtype=np.uint8)
+    lo = (p & 0xF).astype(np.int32)
+    hi = (p >> 4).astype(np.int32)
+    lo = np.where(lo >= 8, lo - 16, lo)
+    hi = np.where(hi >= 8, hi - 16, hi)
+    out = np.empty((p.shape[0], 2 * p.shape[1]), dtype=np.int32)
+    out[:, 0::2] = lo
+    out[:, 1::2] = hi
+    return out

@@ -185,3 +185,43 @@ def test_weight_per_channel():
     q2, s2, _ = quant.quantize_weight_per_channel(W2)
     np.testing.assert_array_equal(q2, q)
     assert s2[2] == pytest.approx(4 * s[2]) and s2[3] == s[3]
+
+
+def test_int4_pack_hand_worked_bytes_and_round_trip():
+    rows = []
+    with open(os.path.join(os.path.dirname(__file__), "golden", "int4_pack.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                a, b, h = line.split()
+                rows.append((int(a), int(b), int(h, 16)))
+    codes = np.array([[r[0], r[1]] for r in rows], dtype=np.int32)
+    np.testing.assert_array_equal(quant.pack_int4(codes)[:, 0], np.array([r[2] for r in rows], dtype=np.uint8))
+    # every byte value decodes to two codes in [-8, 7] and encodes back to itself (the map is a bijection)
+    allb = np.arange(256, dtype=np.uint8).reshape(16, 16)
+    un = quant.unpack_int4(allb)
+    assert un.shape == (16, 32) and un.min() == -8 and un.max() == 7
+    np.testing.assert_array_equal(quant.pack_int4(un), allb)
+    # definition by bit arithmetic, element by element
+    for byte in (0x00, 0x7F, 0x80, 0xE3, 0x9C):
+        lo, hi = byte & 0xF, byte >> 4
+        want = [lo - 16 if lo & 8 else lo, hi - 16 if hi & 8 else hi]
+        assert quant.unpack_int4(np.array([[byte]], dtype=np.uint8))[0].tolist() == want
+    # order inside a row: code 2j low nibble, code 2j+1 high nibble
+    q = np.array([[1, 2, 3, 4, -1, -2]], dtype=np.int32)
+    assert quant.pack_int4(q)[0].tolist() == [0x21, 0x43, 0xEF]
+    np.testing.assert_array_equal(quant.unpack_int4(quant.pack_int4(q)), q)
+    with pytest.raises(ValueError):
+        quant.pack_int4(np.array([[8, 0]]))
+    with pytest.raises(ValueError):
+        quant.pack_int4(np.array([[1, 2, 3]]))
+
+
+def test_int4_weights_survive_packing():
+    rng = np.random.default_rng(5)
+    W = (rng.standard_normal((12, 64)) * 0.02).astype(np.float32)
+    q, s, cs = quant.quantize_weight_per_channel(W, bits=4)
+    assert q.min() >= -7 and q.max() <= 7
+    back = quant.unpack_int4(quant.pack_int4(q))
+    np.testing.assert_array_equal(back, q)
+    np.testing.assert_array_equal(back.sum(axis=1), cs)
