@@ -144,6 +144,8 @@ class Context:
     scales: Optional[ActScales] = None
     storage: Storage = field(default_factory=Storage)
     tap: Optional[Callable] = None
+    reuse_walk: bool = False   # a fully skipped step walked block by block (each cached branch enters the residual
+                               # stream with its own rounding, as in a computed step) instead of accumulated once
 
     def emit(self, name, arr):
         if self.tap is not None:
@@ -324,7 +326,11 @@ def forward(model: QModel, ctx: Context, latent, t, y, cache=None, reuse: bool =
     c = conditioning(model, t, y)
     ctx.emit("c", c)
     ctx.emit("x_embed", x)
-    if reuse:
+    if reuse and ctx.reuse_walk:
+        # the cache rule taken literally, block by block: the same sum as blocks_reuse, rounded after every branch
+        for i, blk in enumerate(model.blocks):
+            x = block_forward(ctx, blk, x, c, cfg.tokens, cfg.heads, i, cache, True, True)
+    elif reuse:
         x = blocks_reuse(ctx, model.blocks, x, c, cfg.tokens, cache)
     else:
         for i, blk in enumerate(model.blocks):

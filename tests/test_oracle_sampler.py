@@ -292,3 +292,42 @@ def test_sampler_applies_vc_every_step(tiny):
     sampler.sample(model, ctx, sampler.SamplerConfig(1 * S, cache_interval=2), latent, labels,
                    on_step=lambda i, x, r: first.append(x.copy()))
     np.testing.assert_allclose(seen[0], vc.apply(first[0], K[0]), atol=1e-6)
+
+
+def test_skipped_step_walked_block_by_block_equals_the_accumulated_form(tiny):
+    """The fully skipped step has two spellings: every block adds its cached branches in turn (the cache rule
+    taken literally), or all of them are accumulated and stored once.  In exact storage they are the same sum;
+    with a bfloat16 residual stream the walked form rounds after each of the 2 * depth additions, so the two may
+    differ by a few bfloat16 steps per element (at most depth steps: 2 * depth roundings of half a step each)."""
+    cfg, model, latent, labels, scales = tiny
+    t0, t1 = np.full(2, 900.0), np.full(2, 800.0)
+    lat1 = latent * 0.9 + 0.05
+    for storage, exact in ((dit.Storage.exact(), True), (dit.Storage(), False)):
+        outs, finals = [], []
+        for walk in (False, True):
+            taps = {}
+            ctx = dit.Context(quant="static", scales=scales, storage=storage, reuse_walk=walk,
+                              tap=lambda n, a, taps=taps: taps.__setitem__(n, np.array(a)))
+            cache = {}
+            dit.forward(model, ctx, latent, t0, labels, cache=cache)
+            outs.append(dit.forward(model, ctx, lat1, t1, labels, cache=cache, reuse=True))
+            finals.append(taps["x_final"])
+        acc, walk = finals
+        if exact:
+            np.testing.assert_allclose(walk, acc, rtol=1e-13, atol=1e-13)
+            np.testing.assert_allclose(outs[1], outs[0], rtol=1e-11, atol=1e-12)
+        else:
+            # one bfloat16 step at the largest magnitude any partial sum of the element can reach
+            rows = np.arange(2 * cfg.tokens) // cfg.tokens
+            D = cfg.hidden
+            bound = np.abs(taps["x_embed"])
+            for i in range(cfg.depth):
+                mod = taps[f"blk{i}.mod"]
+                bound = bound + np.abs(mod[rows, 2 * D:3 * D] * cache[(i, "attn")]) + np.abs(mod[rows, 5 * D:6 * D] * cache[(i, "mlp")])
+            step = 2.0 ** (np.floor(np.log2(bound)) - 7)
+            steps = np.abs(walk - acc) / step
+            assert steps.max() <= cfg.depth + 1
+            assert np.mean(steps > 0) > 0.01                 # the two spellings do differ, by rounding only
+            rel = np.linalg.norm(outs[1] - outs[0]) / np.linalg.norm(outs[0])
+            print(f"walked vs accumulated skipped step, bf16 residual: max {steps.max():.1f} bf16 steps, output rel-L2 {rel:.2e}")
+            assert rel < 1e-2
