@@ -329,7 +329,7 @@ extern "C" int32_t qdit_w8a8_linear(qdit_ctx* ctx, const void* A, const void* W,
   if (!getenv("QDIT_GEMM_BN") && p.M >= 1024) {
     const int cls = epi_class(p.flags);
     if ((cls == 1 || cls == 2) && p.N >= 2304) return qdit_launch_gemm_t(ctx, A, W, p, a_unsigned, 256);
-    if (cls == 3 && p.K >= 2304 && p.N >= 1024 && p.tokens % 32 == 0) return qdit_launch_gemm_t(ctx, A, W, p, a_unsigned, 256);
+    if (cls == 3 && p.N >= 1024 && p.tokens % 32 == 0) return qdit_launch_gemm_t(ctx, A, W, p, a_unsigned, 256);
   }
   switch (pick_bn(p.M, p.N, ctx->num_sms)) {
     case 64: return launch_gemm<64>(ctx, A, W, p, a_unsigned);

@@ -11,10 +11,19 @@
 // tile be 256 wide (one MMA of N = 256) and makes every DiT-XL/2 layer width (multiples of 128 channels)
 // tile without remainder.
 //
-// CTA = 2 + 12 (or more, see TWarps) warps, roles and barriers as in gemm_i8.cu: warp 0 lane 0 TMA producer (weight
+// CTA = 2 + 8 or 12 warps (see TWarps), roles and barriers as in gemm_i8.cu: warp 0 lane 0 TMA producer (weight
 // tile 128 x 128 B as operand A, activation tile BT x 128 B as operand B, both K-major, 128B swizzle), warp 1
-// lane 0 MMA issuer (two TMEM accumulator stages of BT columns), epilogue warps: 3 (or more) per lane quadrant,
+// lane 0 MMA issuer (two TMEM accumulator stages of BT columns), epilogue warps: 2 or 3 per lane quadrant,
 // taking 32-token chunks in turn.
+//
+// Epilogues that write 16-bit outputs (bias -> bf16; the gated one: bias, cache copy, x gate, + residual -> bf16)
+// read the accumulator in the matrix-fragment layout (tcgen05.ld 16x256b: a thread holds pairs of adjacent tokens
+// of 4 channels), so that the finished bf16 pairs are exactly the operands of stmatrix.trans: four of them lay a
+// chunk of 32 tokens x 32 channels into a 2 KB shared-memory tile in token-major order (64-byte rows, 64B
+// swizzle, conflict-free), and one thread hands the tile to a TMA store.  No shuffles, no per-thread global
+// stores (warp-level stores of 64-byte row pieces reach 4.2 TB/s on this chip, TMA stores of the same tiles
+// 6.7 TB/s, and they do not hold the issuing warp), and the residual of the gated epilogue arrives the same way
+// in reverse (TMA load one chunk ahead, ldmatrix.trans).
 #include "gemm_common.cuh"
 
 
@@ -23,30 +32,33 @@ namespace {
 using namespace qgemm;
 
 constexpr int BC = 128;  // channels per tile = TMEM lanes
-// This kernel has no per-warp staging buffer, so its epilogue could be wider than the token-major kernel's;
-// measured, 16 warps (4 per lane quadrant) are slower than 12 for every epilogue class, so 12 it is.
-#ifndef QDIT_T_GATED_WARPS
-#define QDIT_T_GATED_WARPS 12
+// Epilogue warps per epilogue class (a multiple of 4: each TMEM lane quadrant is read by warps with warp % 4 =
+// quadrant).  The staged epilogues (classes 1 and 3) are light and asynchronous: 2 warps per quadrant, which split
+// the 8 chunks of a 256-token tile evenly; the others use 3 (measured: 16 warps are slower than 12 for them).
+#ifndef QDIT_T_STAGED_WARPS
+#define QDIT_T_STAGED_WARPS 8
 #endif
-// Epilogue warps per epilogue class (a multiple of 4: each TMEM lane quadrant is read by warps with warp % 4 = quadrant).
 template <int EPI>
 struct TWarps {
-  static constexpr int EPI_WARPS = EPI == 3 ? QDIT_T_GATED_WARPS : 12;
+  static constexpr bool STAGED = EPI == 1 || EPI == 3;
+  static constexpr int EPI_WARPS = STAGED ? QDIT_T_STAGED_WARPS : 12;
   static constexpr int SPLIT = EPI_WARPS / 4;
   static constexpr int THREADS = 64 + EPI_WARPS * 32;
+  static constexpr int STAGING_PER_WARP = STAGED ? 4096 : 0;  // two 2 KB tiles of 32 tokens x 32 channels bf16
+  static constexpr int STAGING_BYTES = EPI_WARPS * STAGING_PER_WARP;
 };
 
-template <int BT>
+template <int BT, int EPI>
 struct TCfg {
   static constexpr int W_BYTES = BC * BK;
   static constexpr int X_BYTES = BT * BK;
   static constexpr int STAGE_BYTES = W_BYTES + X_BYTES;
-  static constexpr int BAR_BYTES = 256;
+  static constexpr int BAR_BYTES = 512;
   static constexpr int SMEM_LIMIT = 232448;
-  static constexpr int STAGES_FIT = (SMEM_LIMIT - 1024 - BAR_BYTES) / STAGE_BYTES;
+  static constexpr int STAGES_FIT = (SMEM_LIMIT - 1024 - BAR_BYTES - TWarps<EPI>::STAGING_BYTES) / STAGE_BYTES;
   static constexpr int STAGES = STAGES_FIT > 8 ? 8 : STAGES_FIT;
   static constexpr int TMEM_COLS = 2 * BT <= 128 ? 128 : (2 * BT <= 256 ? 256 : 512);
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + TWarps<EPI>::STAGING_BYTES + BAR_BYTES + 1024;
 };
 
 // One 32-token chunk of one channel (this thread): v[j] = accumulator of token m_base + j.
@@ -122,10 +134,9 @@ __device__ __forceinline__ void transpose8(uint32_t (&x)[8], int lane) {
   }
 }
 
-// Light epilogues (bias -> bf16, bias + GELU -> 8-bit codes): the math runs channel-major with scalar
-// parameters; the finished 16-bit / 8-bit results are then transposed inside each group of 8 lanes with
-// shuffles, so that a lane stores 8 consecutive channels of a token at once (16 or 8 bytes) and a warp
-// instruction covers 8 tokens x 32 channels, without touching shared memory.
+// GELU layer (bias + GELU -> 8-bit codes): the math runs channel-major with scalar parameters; the finished codes
+// are then transposed inside each group of 8 lanes with shuffles, so that a lane stores 8 consecutive channels of a
+// token at once (8 bytes) and a warp instruction covers 8 tokens x 32 channels, without touching shared memory.
 // Lane (g, i) = (lane >> 3, lane & 7) ends up with channels 8g..8g+7 of tokens i, 8 + i, 16 + i, 24 + i.
 template <int EPI>
 __device__ __forceinline__ void epilogue_chunk_t_packed(const GemmParams& p, const uint32_t (&v)[32], int n, int lane,
@@ -148,132 +159,98 @@ __device__ __forceinline__ void epilogue_chunk_t_packed(const GemmParams& p, con
     f[j] = (flags & QDIT_EPI_BIAS) ? __fmaf_rn(f[j], sc, bias) : __fmul_rn(f[j], sc);
     if (flags & QDIT_EPI_GELU) f[j] = gelu_tanh_f(f[j]);
   }
-  if (flags & QDIT_EPI_QUANT_OUT) {
-    // one byte per token: word t = codes of tokens t, 8 + t, 16 + t, 24 + t
-    const float lo_f = p.o_qmin - p.o_zp, hi_f = p.o_qmax - p.o_zp;
-    const int zp = static_cast<int>(p.o_zp);
-    uint32_t w[8];
+  // one byte per token: word t = codes of tokens t, 8 + t, 16 + t, 24 + t
+  const float lo_f = p.o_qmin - p.o_zp, hi_f = p.o_qmax - p.o_zp;
+  const int zp = static_cast<int>(p.o_zp);
+  uint32_t w[8];
 #pragma unroll
-    for (int t = 0; t < 8; ++t) {
-      uint32_t m4[4];
+  for (int t = 0; t < 8; ++t) {
+    uint32_t m4[4];
 #pragma unroll
-      for (int s4 = 0; s4 < 4; ++s4) {
-        const float q = fminf(fmaxf(__fmul_rn(f[8 * s4 + t], o_inv), lo_f), hi_f);
-        m4[s4] = static_cast<uint32_t>(__float_as_int(__fadd_rn(q, 12582912.0f)));
-      }
-      w[t] = __byte_perm(__byte_perm(m4[0], m4[1], 0x0040), __byte_perm(m4[2], m4[3], 0x0040), 0x5410);
-      if (zp != 0) w[t] = __vadd4(w[t], static_cast<uint32_t>(zp & 0xFF) * 0x01010101u);  // code + z stays inside a byte
+    for (int s4 = 0; s4 < 4; ++s4) {
+      const float q = fminf(fmaxf(__fmul_rn(f[8 * s4 + t], o_inv), lo_f), hi_f);
+      m4[s4] = static_cast<uint32_t>(__float_as_int(__fadd_rn(q, 12582912.0f)));
     }
-    transpose8(w, lane);  // w[c] = codes of channel n8 + c for tokens i8, 8 + i8, 16 + i8, 24 + i8
-    if (n8 < p.N) {
+    w[t] = __byte_perm(__byte_perm(m4[0], m4[1], 0x0040), __byte_perm(m4[2], m4[3], 0x0040), 0x5410);
+    if (zp != 0) w[t] = __vadd4(w[t], static_cast<uint32_t>(zp & 0xFF) * 0x01010101u);  // code + z stays inside a byte
+  }
+  transpose8(w, lane);  // w[c] = codes of channel n8 + c for tokens i8, 8 + i8, 16 + i8, 24 + i8
+  if (n8 < p.N) {
 #pragma unroll
-      for (int s4 = 0; s4 < 4; ++s4) {
-        const int64_t m = m_base + 8 * s4 + i8;
-        if (m < p.M) {
-          // byte s4 of each of the 8 words
-          const uint32_t sel = 0x0000 | (s4) | ((4 + s4) << 4);  // (w_a byte s4, w_b byte s4) -> low two bytes
-          const uint32_t lo = __byte_perm(__byte_perm(w[0], w[1], sel), __byte_perm(w[2], w[3], sel), 0x5410);
-          const uint32_t hi = __byte_perm(__byte_perm(w[4], w[5], sel), __byte_perm(w[6], w[7], sel), 0x5410);
-          *reinterpret_cast<uint2*>(static_cast<uint8_t*>(p.out) + m * p.ldo + n8) = make_uint2(lo, hi);
-        }
-      }
-    }
-  } else {
-    // bf16: word t of pair (s, s + 1) = (token 8 s + t, token 8 (s + 1) + t)
-#pragma unroll
-    for (int s2 = 0; s2 < 4; s2 += 2) {
-      uint32_t w[8];
-#pragma unroll
-      for (int t = 0; t < 8; ++t) w[t] = pack_bf16x2(f[8 * s2 + t], f[8 * (s2 + 1) + t]);
-      transpose8(w, lane);  // w[c] = channel n8 + c: (token 8 s2 + i8 in the low half, token 8 (s2 + 1) + i8 in the high half)
-      if (n8 < p.N) {
-        const int64_t m_lo = m_base + 8 * s2 + i8, m_hi = m_lo + 8;
-        if (m_lo < p.M) {
-          const uint4 o = make_uint4(__byte_perm(w[0], w[1], 0x5410), __byte_perm(w[2], w[3], 0x5410),
-                                     __byte_perm(w[4], w[5], 0x5410), __byte_perm(w[6], w[7], 0x5410));
-          *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + m_lo * p.ldo + n8) = o;
-        }
-        if (m_hi < p.M) {
-          const uint4 o = make_uint4(__byte_perm(w[0], w[1], 0x7632), __byte_perm(w[2], w[3], 0x7632),
-                                     __byte_perm(w[4], w[5], 0x7632), __byte_perm(w[6], w[7], 0x7632));
-          *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + m_hi * p.ldo + n8) = o;
-        }
+    for (int s4 = 0; s4 < 4; ++s4) {
+      const int64_t m = m_base + 8 * s4 + i8;
+      if (m < p.M) {
+        // byte s4 of each of the 8 words
+        const uint32_t sel = 0x0000 | (s4) | ((4 + s4) << 4);  // (w_a byte s4, w_b byte s4) -> low two bytes
+        const uint32_t lo = __byte_perm(__byte_perm(w[0], w[1], sel), __byte_perm(w[2], w[3], sel), 0x5410);
+        const uint32_t hi = __byte_perm(__byte_perm(w[4], w[5], sel), __byte_perm(w[6], w[7], sel), 0x5410);
+        *reinterpret_cast<uint2*>(static_cast<uint8_t*>(p.out) + m * p.ldo + n8) = make_uint2(lo, hi);
       }
     }
   }
 }
 
-// Gated epilogue (bias, cache store, x gate, + residual -> bf16) in the same style: the branch value and its
-// gated copy are computed channel-major with scalar parameters; the bf16 cache copy travels through two word
-// transposes, the gated f32 value through four, and the residual is then added token-major, where a lane loads
-// and stores 8 consecutive channels of a token (16 bytes).  Needs the chunk inside one sample (tokens % 32 == 0).
-// The residual words `rv` (token 8 s + i8, channels n8..n8+7) and the gate were fetched by the caller one chunk
-// ahead, so that their latency is not part of the chunk's dependency chain.
-__device__ __forceinline__ void epilogue_chunk_t_gated(const GemmParams& p, const uint32_t (&v)[32], int n, int lane,
-                                                       int m_base, float sc, float bias, int zcs, const uint4 (&rv)[4],
-                                                       float gate) {
-  const int i8 = lane & 7;
-  const int n8 = n - i8;
-  const bool n8_ok = n8 < p.N;
-  float f[32];
+// ---------------------------------------------------------------------------------------------------------
+// Staged epilogues (classes 1 and 3).  A chunk = 32 tokens x the warp's 32 channels.  The accumulator is read as
+// two fragment loads (TMEM lanes 0..15 and 16..31 of the warp's quadrant); thread t then holds, for channel
+// k = 0..3 (channel offset t/4 + 8k) and token group i = 0..3, the token pair 8i + 2(t%4), + 1:
+//   k = 0: a[4i], a[4i+1]   k = 1: a[4i+2], a[4i+3]   k = 2: b[4i], b[4i+1]   k = 3: b[4i+2], b[4i+3]
+// stmatrix.trans of the four packed pairs of a token group writes rows 8i..8i+7 of the tile (64 bytes = 32 channels
+// per row; the 16-byte piece of channel group k sits at index k ^ ((row >> 1) & 3): the 64B swizzle of the tensor maps).
+struct FragChannels {
+  float sc[4], bias[4];
+  int zcs[4];
+};
+
+// Shared-memory offset of the row this thread addresses in stmatrix / ldmatrix for token group 0 (group i: + 512 i).
+__device__ __forceinline__ uint32_t frag_row_offset(int lane) {
+  const uint32_t row = static_cast<uint32_t>(lane & 7), piece = static_cast<uint32_t>(lane >> 3);
+  return row * 64u + ((piece ^ ((row >> 1) & 3u)) << 4);
+}
+
+// f[k][2i + e] = de-quantised value of channel k, token 8i + 2(t%4) + e:  (acc - z_a colsum) * (s_a s_w) + bias.
+__device__ __forceinline__ void frag_dequant(const uint32_t (&a)[16], const uint32_t (&b)[16], const FragChannels& fc,
+                                             float (&f)[4][8]) {
 #pragma unroll
-  for (int j = 0; j < 32; ++j) f[j] = __fmaf_rn(static_cast<float>(static_cast<int>(v[j]) - zcs), sc, bias);
-  // cache copy (pre-gate), bf16
+  for (int i = 0; i < 4; ++i) {
 #pragma unroll
-  for (int s2 = 0; s2 < 4; s2 += 2) {
-    uint32_t w[8];
-#pragma unroll
-    for (int t = 0; t < 8; ++t) w[t] = pack_bf16x2(f[8 * s2 + t], f[8 * (s2 + 1) + t]);
-    transpose8(w, lane);
-    if (n8_ok) {
-      const int64_t m_lo = m_base + 8 * s2 + i8, m_hi = m_lo + 8;
-      if (m_lo < p.M)
-        *reinterpret_cast<uint4*>(p.cache_out + m_lo * p.N + n8) =
-            make_uint4(__byte_perm(w[0], w[1], 0x5410), __byte_perm(w[2], w[3], 0x5410), __byte_perm(w[4], w[5], 0x5410),
-                       __byte_perm(w[6], w[7], 0x5410));
-      if (m_hi < p.M)
-        *reinterpret_cast<uint4*>(p.cache_out + m_hi * p.N + n8) =
-            make_uint4(__byte_perm(w[0], w[1], 0x7632), __byte_perm(w[2], w[3], 0x7632), __byte_perm(w[4], w[5], 0x7632),
-                       __byte_perm(w[6], w[7], 0x7632));
+    for (int e = 0; e < 2; ++e) {
+      f[0][2 * i + e] = __fmaf_rn(static_cast<float>(static_cast<int>(a[4 * i + e]) - fc.zcs[0]), fc.sc[0], fc.bias[0]);
+      f[1][2 * i + e] = __fmaf_rn(static_cast<float>(static_cast<int>(a[4 * i + 2 + e]) - fc.zcs[1]), fc.sc[1], fc.bias[1]);
+      f[2][2 * i + e] = __fmaf_rn(static_cast<float>(static_cast<int>(b[4 * i + e]) - fc.zcs[2]), fc.sc[2], fc.bias[2]);
+      f[3][2 * i + e] = __fmaf_rn(static_cast<float>(static_cast<int>(b[4 * i + 2 + e]) - fc.zcs[3]), fc.sc[3], fc.bias[3]);
     }
   }
+}
+
+// The chunk as bf16 into a staging tile (token-major, swizzled).
+__device__ __forceinline__ void frag_store_tile(uint32_t tile_row_addr, const float (&f)[4][8]) {
 #pragma unroll
-  for (int s4 = 0; s4 < 4; ++s4) {
-    const int64_t m = m_base + 8 * s4 + i8;
-    const bool live = n8_ok && m < p.M;
-    uint32_t w[8];
-#pragma unroll
-    for (int t = 0; t < 8; ++t) w[t] = __float_as_uint(__fmul_rn(f[8 * s4 + t], gate));
-    transpose8(w, lane);  // w[c] = gated value of channel n8 + c, token m
-    if (live) {
-      float r[8];
-      unpack_bf16x2(rv[s4].x, r[0], r[1]);
-      unpack_bf16x2(rv[s4].y, r[2], r[3]);
-      unpack_bf16x2(rv[s4].z, r[4], r[5]);
-      unpack_bf16x2(rv[s4].w, r[6], r[7]);
-#pragma unroll
-      for (int c = 0; c < 8; ++c) r[c] = __fadd_rn(__uint_as_float(w[c]), r[c]);
-      *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + m * p.ldo + n8) = pack_bf16x8(r);
-    }
-  }
+  for (int i = 0; i < 4; ++i)
+    stmatrix_x4_trans(tile_row_addr + 512u * i, pack_bf16x2(f[0][2 * i], f[0][2 * i + 1]), pack_bf16x2(f[1][2 * i], f[1][2 * i + 1]),
+                      pack_bf16x2(f[2][2 * i], f[2][2 * i + 1]), pack_bf16x2(f[3][2 * i], f[3][2 * i + 1]));
 }
 
 template <int BT, int EPI>
 __global__ void __launch_bounds__(TWarps<EPI>::THREADS, 1)
 gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
-                 const GemmParams p, const uint32_t idesc) {
-  using C = TCfg<BT>;
+                 const __grid_constant__ CUtensorMap tmap_out, const __grid_constant__ CUtensorMap tmap_cache,
+                 const __grid_constant__ CUtensorMap tmap_res, const GemmParams p, const uint32_t idesc) {
+  using C = TCfg<BT, EPI>;
+  using TW = TWarps<EPI>;
   constexpr int STAGES = C::STAGES;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sW = smem;
   uint8_t* sX = smem + STAGES * C::W_BYTES;
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + STAGES * C::STAGE_BYTES);
+  uint8_t* staging = smem + STAGES * C::STAGE_BYTES;  // [EPI_WARPS][2][2 KB] (staged epilogues only; 1024-byte aligned)
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(staging + TW::STAGING_BYTES);
   uint64_t* empty_bar = full_bar + STAGES;
   uint64_t* tfull_bar = empty_bar + STAGES;
   uint64_t* tempty_bar = tfull_bar + 2;
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tempty_bar + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  uint64_t* res_bar = full_bar + 32;  // [EPI_WARPS] residual tile of a warp landed (tx)
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -285,8 +262,9 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&tfull_bar[s], 1);
-      mbar_init(&tempty_bar[s], TWarps<EPI>::EPI_WARPS);
+      mbar_init(&tempty_bar[s], TW::EPI_WARPS);
     }
+    for (int s = 0; s < TW::EPI_WARPS; ++s) mbar_init(&res_bar[s], 1);
     *abort_flag = 0;
     mbar_fence_init();
   }
@@ -362,7 +340,7 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     // -------------------------------------------------------------------- epilogue warps
     const int e = warp - 2;
     const int quad = warp & 3;   // TMEM lane quadrant = 32 channels
-    constexpr int T_EPI_SPLIT = TWarps<EPI>::SPLIT;
+    constexpr int T_EPI_SPLIT = TW::SPLIT;
     const int part = e >> 2;     // this warp takes token chunks part, part + T_EPI_SPLIT, ...
     const uint32_t flags = epi_flags<EPI>(p);
     const float a_scale = p.a_scale_dev ? __ldg(p.a_scale_dev) : p.a_scale;
@@ -370,66 +348,201 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     if (flags & QDIT_EPI_QUANT_OUT) o_inv = __fdiv_rn(1.0f, p.o_scale_dev ? __ldg(p.o_scale_dev) : p.o_scale);
     constexpr int CHUNKS = BT / 32;
     const int c_last = part < CHUNKS ? part + ((CHUNKS - 1 - part) / T_EPI_SPLIT) * T_EPI_SPLIT : -1;
-    int it = 0;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
-      const int as = it & 1;
-      const uint32_t aphase = static_cast<uint32_t>(it >> 1) & 1u;
-      const int t0 = (tile / num_c_tiles) * BT;
-      const int n = (tile % num_c_tiles) * BC + quad * 32 + lane;
-      const bool n_ok = n < p.N;
-      // this channel's parameters: scalars, fetched before the accumulator is waited for
-      float sc = 0.0f, bias = 0.0f;
-      int zcs = 0;
-      if (n_ok && !(flags & QDIT_EPI_OUT_I32)) {
-        sc = __fmul_rn(a_scale, p.w_scale[n]);
-        if (flags & QDIT_EPI_BIAS) bias = p.bias[n];
-        if (p.a_zp != 0) zcs = p.a_zp * p.w_colsum[n];
-      }
-      // gated layers: residual and gate of a chunk are fetched one chunk ahead (the first before the accumulator is waited for)
-      const bool gated_fast = EPI == 3 && (p.tokens % 32) == 0;
-      uint4 rv_next[4] = {};
-      float gate_next = 0.0f;
-      auto prefetch_gated = [&](int c) {
-        const int mb = t0 + c * 32, i8 = lane & 7, n8 = n - i8;
-#pragma unroll
-        for (int s4 = 0; s4 < 4; ++s4) {
-          const int64_t m = mb + 8 * s4 + i8;
-          rv_next[s4] = (n8 < p.N && m < p.M) ? *reinterpret_cast<const uint4*>(p.residual + m * p.ldo + n8) : make_uint4(0u, 0u, 0u, 0u);
-        }
-        gate_next = (n_ok && mb < p.M) ? p.gate[static_cast<int64_t>(mb / p.tokens) * p.ld_gate + n] : 0.0f;
+    // the staged form of the gated epilogue needs a chunk to lie inside one sample (one gate row per chunk)
+    const bool staged = TW::STAGED && (EPI == 1 || (p.tokens % 32) == 0);
+    if (staged) {
+      // ------------------------------------------------------------ classes 1 and 3 through shared-memory tiles and TMA
+      uint8_t* stg = staging + e * TW::STAGING_PER_WARP;
+      // class 1: two output tiles used in turn; class 3: tile 0 receives the residual, tile 1 carries the cache copy and then the output
+      const uint32_t tile0 = smem_u32(stg), tile1 = tile0 + 2048u;
+      const uint32_t row_off = frag_row_offset(lane);
+      uint64_t* rbar = &res_bar[e];
+      uint32_t r_phase = 0;
+      bool r_inflight = false;
+      int out_turn = 0;
+      auto chunk_live = [&](int tile, int c) {
+        return tile < total_tiles && c < CHUNKS && (tile / num_c_tiles) * BT + 32 * c < p.M && (tile % num_c_tiles) * BC + quad * 32 < p.N;
       };
-      if (gated_fast && c_last >= 0) prefetch_gated(part);
-      if (!mbar_wait(&tfull_bar[as], aphase, abort_flag, p.status)) break;
-      __syncwarp();
-      tc_fence_after();
-      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(as * BT);
-      if (c_last < 0) {
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive_relaxed(&tempty_bar[as]);
-        continue;
+      auto issue_residual = [&](int tile, int c) {  // one lane
+        mbar_expect_tx(rbar, 2048u);
+        tma_load_2d(stg, &tmap_res, (tile % num_c_tiles) * BC + quad * 32, (tile / num_c_tiles) * BT + 32 * c, rbar);
+      };
+      if (lane == 0) {
+        tma_prefetch_desc(&tmap_out);
+        if (EPI == 3) {
+          tma_prefetch_desc(&tmap_cache);
+          tma_prefetch_desc(&tmap_res);
+        }
       }
-#pragma unroll 1
-      for (int c = part; c < CHUNKS; c += T_EPI_SPLIT) {
-        uint32_t v[32];
-        uint4 rv[4];
-        float gate = gate_next;
+      int it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+        // the residual of the tile's first chunk, unless the previous tile's last chunk has already asked for it
+        if (EPI == 3 && !r_inflight && chunk_live(tile, part)) {
+          if (lane == 0) issue_residual(tile, part);
+          r_inflight = true;
+        }
+        const int as = it & 1;
+        const uint32_t aphase = static_cast<uint32_t>(it >> 1) & 1u;
+        const int t0 = (tile / num_c_tiles) * BT;
+        const int c0q = (tile % num_c_tiles) * BC + quad * 32;   // first channel of this warp's quadrant
+        // parameters of this thread's 4 channels (channel c0q + lane / 4 + 8 k), fetched before the accumulator is waited for
+        FragChannels fc;
+        int nk[4];
 #pragma unroll
-        for (int s4 = 0; s4 < 4; ++s4) rv[s4] = rv_next[s4];
-        if (gated_fast && c + T_EPI_SPLIT < CHUNKS) prefetch_gated(c + T_EPI_SPLIT);
+        for (int k = 0; k < 4; ++k) {
+          nk[k] = c0q + (lane >> 2) + 8 * k;
+          const bool n_ok = nk[k] < p.N;
+          fc.sc[k] = n_ok ? __fmul_rn(a_scale, p.w_scale[nk[k]]) : 0.0f;
+          fc.bias[k] = n_ok ? p.bias[nk[k]] : 0.0f;
+          fc.zcs[k] = (n_ok && p.a_zp != 0) ? p.a_zp * p.w_colsum[nk[k]] : 0;
+        }
+        if (!mbar_wait(&tfull_bar[as], aphase, abort_flag, p.status)) { ok = false; break; }
         __syncwarp();
-        tmem_ld_32x32(taddr + static_cast<uint32_t>(c * 32), v);
-        tmem_ld_wait();
-        if (c == c_last) {
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(as * BT);
+        if (c_last < 0) {
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive_relaxed(&tempty_bar[as]);
+          continue;
         }
-        const int m_base = t0 + c * 32;
-        if (m_base < p.M) {
-          if (EPI == 1 || EPI == 2) epilogue_chunk_t_packed<EPI>(p, v, n, lane, m_base, sc, bias, zcs, o_inv);
-          else if (gated_fast) epilogue_chunk_t_gated(p, v, n, lane, m_base, sc, bias, zcs, rv, gate);
-          else if (n_ok) epilogue_chunk_t<EPI>(p, v, n, m_base, sc, bias, zcs, o_inv);
+#pragma unroll 1
+        for (int c = part; c < CHUNKS; c += T_EPI_SPLIT) {
+          const int m_base = t0 + c * 32;
+          const bool live = m_base < p.M && c0q < p.N;   // uniform over the warp
+          uint32_t a[16], b[16];
+          float gate[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+          if (EPI == 3 && live) {
+            const float* grow = p.gate + static_cast<int64_t>(m_base / p.tokens) * p.ld_gate;
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              if (nk[k] < p.N) gate[k] = grow[nk[k]];
+          }
+          __syncwarp();
+          if (live) {
+            tmem_ld_16x256b_x4(taddr + static_cast<uint32_t>(c * 32), a);
+            tmem_ld_16x256b_x4(taddr + (16u << 16) + static_cast<uint32_t>(c * 32), b);
+            tmem_ld_wait();
+          }
+          if (c == c_last) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_relaxed(&tempty_bar[as]);
+          }
+          if (!live) continue;
+          float f[4][8];
+          frag_dequant(a, b, fc, f);
+          if (EPI == 1) {
+            const uint32_t tile = out_turn ? tile1 : tile0;
+            if (lane == 0) tma_store_wait_read<1>();  // the store that used this tile two chunks ago has read it
+            __syncwarp();
+            frag_store_tile(tile + row_off, f);
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&tmap_out, stg + (out_turn ? 2048 : 0), c0q, m_base);
+              tma_store_commit();
+            }
+            out_turn ^= 1;
+          } else {
+            // cache copy (the branch output before the gate)
+            if (lane == 0) tma_store_wait_read<0>();  // the previous chunk's output store has read tile 1
+            __syncwarp();
+            frag_store_tile(tile1 + row_off, f);
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&tmap_cache, stg + 2048, c0q, m_base);
+              tma_store_commit();
+            }
+            // residual of this chunk (requested one chunk ahead)
+            if (!mbar_wait(rbar, r_phase, abort_flag, p.status)) { ok = false; break; }
+            r_phase ^= 1u;
+            r_inflight = false;
+            uint32_t rw[4][4];  // [token group][channel]: bf16 pair (token 8i + 2(t%4), + 1)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) ldmatrix_x4_trans(tile0 + row_off + 512u * i, rw[i][0], rw[i][1], rw[i][2], rw[i][3]);
+            // x gate, + residual: one rounded multiply and one rounded add, as in every other kernel of this layer
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                float r0, r1;
+                unpack_bf16x2(rw[i][k], r0, r1);
+                f[k][2 * i] = __fadd_rn(__fmul_rn(f[k][2 * i], gate[k]), r0);
+                f[k][2 * i + 1] = __fadd_rn(__fmul_rn(f[k][2 * i + 1], gate[k]), r1);
+              }
+            }
+            __syncwarp();  // every lane has consumed the residual tile: the next one may land
+            {
+              int nt = tile, nc = c + T_EPI_SPLIT;
+              if (!(nc < CHUNKS && t0 + 32 * nc < p.M)) {
+                nt = tile + static_cast<int>(gridDim.x);
+                nc = part;
+              }
+              if (chunk_live(nt, nc)) {
+                if (lane == 0) issue_residual(nt, nc);
+                r_inflight = true;
+              }
+            }
+            if (lane == 0) tma_store_wait_read<0>();  // the cache store has read tile 1
+            __syncwarp();
+            frag_store_tile(tile1 + row_off, f);
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&tmap_out, stg + 2048, c0q, m_base);
+              tma_store_commit();
+            }
+          }
+        }
+      }
+      // a residual tile still in flight must land before the CTA's shared memory is released
+      if (r_inflight) mbar_wait(rbar, r_phase, abort_flag, p.status);
+      if (lane == 0) tma_store_wait_all();
+    } else {
+      int it = 0;
+      for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
+        const int as = it & 1;
+        const uint32_t aphase = static_cast<uint32_t>(it >> 1) & 1u;
+        const int t0 = (tile / num_c_tiles) * BT;
+        const int n = (tile % num_c_tiles) * BC + quad * 32 + lane;
+        const bool n_ok = n < p.N;
+        // this channel's parameters: scalars, fetched before the accumulator is waited for
+        float sc = 0.0f, bias = 0.0f;
+        int zcs = 0;
+        if (n_ok && !(flags & QDIT_EPI_OUT_I32)) {
+          sc = __fmul_rn(a_scale, p.w_scale[n]);
+          if (flags & QDIT_EPI_BIAS) bias = p.bias[n];
+          if (p.a_zp != 0) zcs = p.a_zp * p.w_colsum[n];
+        }
+        if (!mbar_wait(&tfull_bar[as], aphase, abort_flag, p.status)) break;
+        __syncwarp();
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(as * BT);
+        if (c_last < 0) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_relaxed(&tempty_bar[as]);
+          continue;
+        }
+#pragma unroll 1
+        for (int c = part; c < CHUNKS; c += T_EPI_SPLIT) {
+          uint32_t v[32];
+          __syncwarp();
+          tmem_ld_32x32(taddr + static_cast<uint32_t>(c * 32), v);
+          tmem_ld_wait();
+          if (c == c_last) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_relaxed(&tempty_bar[as]);
+          }
+          const int m_base = t0 + c * 32;
+          if (m_base < p.M) {
+            if (EPI == 2) epilogue_chunk_t_packed<EPI>(p, v, n, lane, m_base, sc, bias, zcs, o_inv);
+            else if (n_ok) epilogue_chunk_t<EPI>(p, v, n, m_base, sc, bias, zcs, o_inv);
+          }
         }
       }
     }
@@ -445,7 +558,7 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
 
 template <int BT, int EPI>
 int32_t launch_t_epi(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p, bool a_unsigned) {
-  using C = TCfg<BT>;
+  using C = TCfg<BT, EPI>;
   static bool attr_set[64] = {};
   if (!attr_set[ctx->device & 63]) {
     QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(gemm_i8_t_kernel<BT, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
@@ -454,6 +567,16 @@ int32_t launch_t_epi(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p,
   CUtensorMap tw, tx;
   QDIT_TRY(qdit_get_tmap(ctx, W, p.N, p.K, p.K, BC, BK, 1, 1, &tw));
   QDIT_TRY(qdit_get_tmap(ctx, A, p.M, p.K, p.K, BT, BK, 1, 1, &tx));
+  // staged epilogues: 32 tokens x 32 channels bf16 tiles (64-byte rows, 64B swizzle) of the output, the cache slot and the residual
+  CUtensorMap to = tx, tc = tx, tr = tx;
+  if (TWarps<EPI>::STAGED) {
+    QDIT_TRY(qdit_get_tmap(ctx, p.out, p.M, p.N, p.ldo, 32, 32, 2, 2, &to));
+    tc = tr = to;
+    if (EPI == 3) {
+      QDIT_TRY(qdit_get_tmap(ctx, p.cache_out, p.M, p.N, p.N, 32, 32, 2, 2, &tc));
+      QDIT_TRY(qdit_get_tmap(ctx, p.residual, p.M, p.N, p.ldo, 32, 32, 2, 2, &tr));
+    }
+  }
   p.num_m_tiles = (p.M + BT - 1) / BT;   // token tiles
   p.num_n_tiles = (p.N + BC - 1) / BC;   // channel tiles
   const int total = p.num_m_tiles * p.num_n_tiles;
@@ -462,7 +585,7 @@ int32_t launch_t_epi(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p,
   const uint32_t idesc = (2u << 4) | (1u << 7) | ((a_unsigned ? 0u : 1u) << 10) | ((static_cast<uint32_t>(BT) >> 3) << 17) |
                          ((static_cast<uint32_t>(BC) >> 4) << 24);
   ProfScope prof(ctx, QDIT_PROF_GEMM, 2.0 * p.M * static_cast<double>(p.N) * p.K);
-  QDIT_CUDA_CHECK(ctx, qdit_launch_overlapped(ctx, gemm_i8_t_kernel<BT, EPI>, dim3(grid), dim3(TWarps<EPI>::THREADS), C::SMEM_BYTES, tw, tx, p, idesc));
+  QDIT_CUDA_CHECK(ctx, qdit_launch_overlapped(ctx, gemm_i8_t_kernel<BT, EPI>, dim3(grid), dim3(TWarps<EPI>::THREADS), C::SMEM_BYTES, tw, tx, to, tc, tr, p, idesc));
   return qdit_after_launch(ctx, "gemm_i8_t_kernel");
 }
 
