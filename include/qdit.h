@@ -62,6 +62,27 @@ const char* qdit_last_error(const qdit_ctx* ctx);
 /* Number of kernels this context has launched since creation (for launch accounting). */
 int64_t qdit_launch_count(const qdit_ctx* ctx);
 
+/* Kernel-selection options of a context (tuning and test aid; the paper has no counterpart).  Every option chooses
+ * among kernels that compute the same values.  A new context takes its initial values from the environment
+ * variables of the same names (QDIT_PDL, QDIT_GEMM_BN, QDIT_GEMM_T, QDIT_GEMM_GENERIC_EPILOGUE, QDIT_ATTN,
+ * QDIT_CONDITIONING_CHUNK), read once inside qdit_create; afterwards only qdit_set_option changes them.
+ *   QDIT_OPT_PDL                    1 (default): kernels are launched with programmatic stream serialization, so that
+ *                                   a kernel's preamble overlaps the tail of the kernel before it; 0: plain launches
+ *   QDIT_OPT_GEMM_BN                0 (default): automatic; 64 | 128 | 192: token-major GEMM kernel with 128 x BN tiles
+ *   QDIT_OPT_GEMM_T                 0 (default): automatic; 128 | 256: channel-major GEMM kernel with 128 x BT tiles
+ *   QDIT_OPT_GEMM_GENERIC_EPILOGUE  1: the GEMM kernels' run-time-flag epilogue instead of the specialised classes
+ *   QDIT_OPT_ATTN                   0 (default): automatic; 1: the mma.sync attention kernel for every token count;
+ *                                   2: the online-softmax tcgen05 kernel also at 256 tokens
+ *   QDIT_OPT_CONDITIONING_CHUNK     sampling steps whose conditioning a sampler evaluates at once: 0 (default) as many
+ *                                   as fit a 4 GB modulation table, -1 step by step, n > 0 at most n (read by
+ *                                   qdit_sampler_create) */
+enum {
+  QDIT_OPT_PDL = 0, QDIT_OPT_GEMM_BN = 1, QDIT_OPT_GEMM_T = 2, QDIT_OPT_GEMM_GENERIC_EPILOGUE = 3, QDIT_OPT_ATTN = 4,
+  QDIT_OPT_CONDITIONING_CHUNK = 5, QDIT_OPT_COUNT = 6
+};
+int32_t qdit_set_option(qdit_ctx* ctx, int option, int value);
+int32_t qdit_get_option(const qdit_ctx* ctx, int option, int* value);
+
 /* Per-kernel timing for measurement (the paper has no counterpart): while enabled, every kernel launch of
  * this context is bracketed by CUDA events on the context's stream.  qdit_profile_read synchronises the
  * stream and returns, for one kernel kind, the launches since profiling was enabled, their summed device
@@ -112,7 +133,8 @@ int32_t qdit_quantize_act(qdit_ctx* ctx, const void* x, int x_dtype, int64_t M, 
  *  - Limit: M*K <= 134,217,728 elements per call (65536 partial maxima of 2048 elements each); larger
  *    inputs are refused with QDIT_ERR_SHAPE before anything is launched.
  *  - The first call on a device looks up the array's device address (cudaGetSymbolAddress) with that
- *    device current; make that first call outside any stream capture.
+ *    device made current for the lookup (the caller's current device is put back); make that first call
+ *    outside any stream capture.  The lookup is serialised, so first calls from several threads are safe.
  *  - The array is shared by every call on the device and keeps the last call's values.  Each call
  *    overwrites all slots it later reads, so nothing needs clearing; two calls that overlap on the GPU
  *    (different streams, no ordering) race on it and must be serialised by the caller.
@@ -135,7 +157,8 @@ int32_t qdit_quantize_act_dynamic_static(qdit_ctx* ctx, const void* x, int x_dty
  * Exactly one of OUT_BF16, OUT_F32, OUT_I32, QUANT_OUT must be set.
  * A: [M,K] bytes (signed, or unsigned when a_qp.qmin >= 0 and a_qp.qmax > 127), W: [N,K] signed bytes,
  * both K-contiguous with leading dimension K.  K % 16 == 0 and N % 8 == 0 are required; M, N, K are
- * otherwise free (ragged tiles are handled).  a_scale_dev, if non-NULL, is a device float that
+ * otherwise free (ragged tiles are handled; with QDIT_EPI_GATE the gate needs one row per started sample,
+ * ceil(M / tokens_per_sample) rows, and no row beyond them is read).  a_scale_dev, if non-NULL, is a device float that
  * overrides a_qp.scale at run time (used when the scale was just reduced on the device). */
 enum {
   QDIT_EPI_BIAS = 1u << 0,
@@ -239,8 +262,8 @@ int32_t qdit_cache_reuse_all(qdit_ctx* ctx, qdit_cache* cache, const float* mod_
 enum { QDIT_VC_NONE = 0, QDIT_VC_K_TABLE = 1, QDIT_VC_VAR_RATIO = 2 };
 int32_t qdit_vc_correct(qdit_ctx* ctx, float* latent, int B, int C, int HW, int step_index, int mode,
                         const float* table, float eps);
-/* Fitting the factor of one step (same section, the closed form below "variance compensation ... using the
- * rQNSR-MSE metric"): from N calibration samples x^ (accelerated trajectory) and targets x' (reference
+/* Fitting the factor of one step (same section, the closed form for K that follows the correction formula): from
+ * N calibration samples x^ (accelerated trajectory) and targets x' (reference
  * trajectory), both device f32 [N, C, HW], with mu = spatial mean of x^ per (sample, channel), a = x^ - mu,
  * b = x' - mu, w = 1 / (x'^2 + eps), sums over the samples and positions of channel c:
  *   QDIT_VC_FIT_DERIVED : K[c] = (sum a b + sum a b w) / (sum a^2 + sum a^2 w)   (d/dK of rQNSR^2 + MSE = 0)

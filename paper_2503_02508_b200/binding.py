@@ -26,6 +26,8 @@ QDIT_BRANCH_ATTN, QDIT_BRANCH_MLP = 0, 1
 QDIT_VC_NONE, QDIT_VC_K_TABLE, QDIT_VC_VAR_RATIO = 0, 1, 2
 QDIT_VC_FIT_DERIVED, QDIT_VC_FIT_PRINTED = 0, 1
 QDIT_FWD_STORE_CACHE, QDIT_FWD_REUSE, QDIT_FWD_CALIBRATE = 1, 2, 4
+(QDIT_OPT_PDL, QDIT_OPT_GEMM_BN, QDIT_OPT_GEMM_T, QDIT_OPT_GEMM_GENERIC_EPILOGUE, QDIT_OPT_ATTN,
+ QDIT_OPT_CONDITIONING_CHUNK) = range(6)
 
 _vp, _i32, _i64, _u32, _f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_float
 _int = C.c_int
@@ -69,6 +71,8 @@ _SIGNATURES = {
     "qdit_status_string": (C.c_char_p, [_i32]),
     "qdit_last_error": (C.c_char_p, [_vp]),
     "qdit_launch_count": (_i64, [_vp]),
+    "qdit_set_option": (_i32, [_vp, _int, _int]),
+    "qdit_get_option": (_i32, [_vp, _int, _vp]),
     "qdit_profile_enable": (_i32, [_vp, _int]),
     "qdit_profile_read": (_i32, [_vp, _int, C.POINTER(_i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]),
     "qdit_quantize_act": (_i32, [_vp, _vp, _int, _i64, _i64, _i64, _int, C.POINTER(qdit_qparams), _vp, _vp, _i64]),
@@ -172,6 +176,16 @@ def qdit_sync(ctx):
 
 def qdit_launch_count(ctx):
     return lib.qdit_launch_count(ctx)
+
+
+def qdit_set_option(ctx, option, value):
+    return check(ctx, lib.qdit_set_option(ctx, option, value))
+
+
+def qdit_get_option(ctx, option):
+    v = C.c_int(0)
+    check(ctx, lib.qdit_get_option(ctx, option, C.byref(v)))
+    return v.value
 
 
 QDIT_PROF_GEMM, QDIT_PROF_ATTENTION, QDIT_PROF_LN_MODULATE, QDIT_PROF_ACT_QUANT = 0, 1, 2, 3

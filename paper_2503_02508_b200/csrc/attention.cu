@@ -272,11 +272,7 @@ template <int DH, int QW>
 int32_t launch_attention(qdit_ctx* ctx, const void* q, const void* k, const void* v, int64_t ld, int B, int H, int T,
                          const AttnParams& p) {
   using C = ACfg<DH>;
-  static bool attr_set[64] = {};
-  if (!attr_set[ctx->device & 63]) {
-    QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(attention_kernel<DH, QW>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::smem_bytes(QW)));
-    attr_set[ctx->device & 63] = true;
-  }
+  QDIT_TRY(qdit_allow_smem(ctx, attention_kernel<DH, QW>, C::smem_bytes(QW)));
   const uint64_t rows = static_cast<uint64_t>(B) * T, cols = static_cast<uint64_t>(H) * DH;
   CUtensorMap tq, tk, tv;
   QDIT_TRY(qdit_get_tmap(ctx, q, rows, cols, ld, 64, DH, C::SWZ ? 1 : 0, 2, &tq));
@@ -319,7 +315,7 @@ extern "C" int32_t qdit_attention(qdit_ctx* ctx, const void* q, const void* k, c
     p.qa = make_quant_args(*out_qp, out_scale_dev);
   }
   // token counts that fill 128-query tiles run on the tcgen05 kernel; the mma.sync kernel covers the rest
-  if (T % 128 == 0 && !getenv("QDIT_ATTN_LEGACY"))
+  if (T % 128 == 0 && ctx->opt[QDIT_OPT_ATTN] != 1)
     return qdit_launch_attention_tc(ctx, q, k, v, ld, B, H, T, dh, softmax_scale, out, out_dtype, p.qa);
   const bool wide = T % 128 == 0;  // 128 queries per CTA when the token count allows
   if (dh == 64) return wide ? launch_attention<64, 8>(ctx, q, k, v, ld, B, H, T, p) : launch_attention<64, 4>(ctx, q, k, v, ld, B, H, T, p);

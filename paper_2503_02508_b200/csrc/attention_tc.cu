@@ -615,12 +615,8 @@ template <int DH>
 int32_t launch_tc(qdit_ctx* ctx, const void* q, const void* k, const void* v, int64_t ld, int B, int H, int T,
                   const AttnTcParams& p) {
   using C = TCfg<DH>;
-  static bool attr_set[64] = {};
-  if (!attr_set[ctx->device & 63]) {
-    QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(attention_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
-    QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(attention_tc256_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
-    attr_set[ctx->device & 63] = true;
-  }
+  QDIT_TRY(qdit_allow_smem(ctx, attention_tc_kernel<DH>, C::SMEM_BYTES));
+  QDIT_TRY(qdit_allow_smem(ctx, attention_tc256_kernel<DH>, C::SMEM_BYTES));
   const uint64_t rows = static_cast<uint64_t>(B) * T, cols = static_cast<uint64_t>(H) * DH;
   CUtensorMap tq, tk, tv, tqt, tkt, tvt;
   QDIT_TRY(qdit_get_tmap(ctx, q, rows, cols, ld, 128, 64, 1, 2, &tq));
@@ -636,7 +632,7 @@ int32_t launch_tc(qdit_ctx* ctx, const void* q, const void* k, const void* v, in
   }
   dim3 grid(T / TQ, H, B);
   ProfScope prof(ctx, QDIT_PROF_ATTENTION, 4.0 * B * H * static_cast<double>(T) * T * DH);
-  if (T == 2 * TK && !getenv("QDIT_ATTN_ONLINE")) {  // the whole score row in tensor memory (tuning switch: the general kernel)
+  if (T == 2 * TK && ctx->opt[QDIT_OPT_ATTN] != 2) {  // the whole score row in tensor memory (option 2 forces the general kernel)
     QDIT_CUDA_CHECK(ctx, qdit_launch_overlapped(ctx, attention_tc256_kernel<DH>, grid, dim3(TC_THREADS), C::SMEM_BYTES, tq, tk, tv, tqt, tkt, tvt, p));
     return qdit_after_launch(ctx, "attention_tc256_kernel");
   }

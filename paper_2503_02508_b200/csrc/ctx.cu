@@ -149,7 +149,15 @@ int32_t qdit_create(qdit_ctx** out, int device, void* cuda_stream) {
   ctx->device = device;
   ctx->stream = static_cast<cudaStream_t>(cuda_stream);
   ctx->num_sms = prop.multiProcessorCount;
-  if (const char* env = getenv("QDIT_PDL")) ctx->overlap_launches = atoi(env) != 0;
+  ctx->opt[QDIT_OPT_PDL] = 1;
+  {  // initial option values from the environment, read here once and nowhere else
+    static const struct { const char* name; int opt; } kEnv[] = {
+        {"QDIT_PDL", QDIT_OPT_PDL}, {"QDIT_GEMM_BN", QDIT_OPT_GEMM_BN}, {"QDIT_GEMM_T", QDIT_OPT_GEMM_T},
+        {"QDIT_GEMM_GENERIC_EPILOGUE", QDIT_OPT_GEMM_GENERIC_EPILOGUE}, {"QDIT_ATTN", QDIT_OPT_ATTN},
+        {"QDIT_CONDITIONING_CHUNK", QDIT_OPT_CONDITIONING_CHUNK}};
+    for (const auto& e : kEnv)
+      if (const char* v = getenv(e.name)) qdit_set_option(ctx, e.opt, atoi(v));
+  }
   if (cudaMalloc(&ctx->d_status, sizeof(int)) != cudaSuccess ||
       cudaMemset(ctx->d_status, 0, sizeof(int)) != cudaSuccess ||
       cudaMallocHost(&ctx->h_status, sizeof(int)) != cudaSuccess) {
@@ -169,6 +177,30 @@ int32_t qdit_create(qdit_ctx** out, int device, void* cuda_stream) {
   }
   ctx->encode_fn = fn;
   *out = ctx;
+  return QDIT_OK;
+}
+
+int32_t qdit_set_option(qdit_ctx* ctx, int option, int value) {
+  if (!ctx) return QDIT_ERR_INVALID_ARG;
+  bool ok = false;
+  switch (option) {
+    case QDIT_OPT_PDL: ok = value == 0 || value == 1; break;
+    case QDIT_OPT_GEMM_BN: ok = value == 0 || value == 64 || value == 128 || value == 192; break;
+    case QDIT_OPT_GEMM_T: ok = value == 0 || value == 128 || value == 256; break;
+    case QDIT_OPT_GEMM_GENERIC_EPILOGUE: ok = value == 0 || value == 1; break;
+    case QDIT_OPT_ATTN: ok = value >= 0 && value <= 2; break;
+    case QDIT_OPT_CONDITIONING_CHUNK: ok = value >= -1; break;
+    default: return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "unknown option %d", option);
+  }
+  if (!ok) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "value %d not valid for option %d", value, option);
+  ctx->opt[option] = value;
+  if (option == QDIT_OPT_PDL) ctx->overlap_launches = value != 0;
+  return QDIT_OK;
+}
+
+int32_t qdit_get_option(const qdit_ctx* ctx, int option, int* value) {
+  if (!ctx || !value || option < 0 || option >= QDIT_OPT_COUNT) return QDIT_ERR_INVALID_ARG;
+  *value = ctx->opt[option];
   return QDIT_OK;
 }
 

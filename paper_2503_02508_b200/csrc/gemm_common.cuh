@@ -162,7 +162,8 @@ template <int EPI>
 __device__ __forceinline__ void prefetch_chunk(const GemmParams& p, int n, int row_base, int rsub, float a_scale,
                                                ChunkInputs& in) {
   const uint32_t flags = epi_flags<EPI>(p);
-  if (n < p.N && !(flags & QDIT_EPI_OUT_I32)) {
+  // a warp whose 32 rows lie wholly past M (ragged last tile) has no sample: it loads nothing
+  if (n < p.N && row_base < p.M && !(flags & QDIT_EPI_OUT_I32)) {
     load_col_params<EPI>(p, n, row_base / p.tokens, a_scale, in.cp);
     if (flags & QDIT_EPI_RESIDUAL) {
 #pragma unroll
@@ -245,9 +246,6 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t tacc
 }
 
 }  // namespace qgemm
-
-// CTA-pair kernel (gemm_i8_2cta.cu): tiles of 256 x bn, bn in {128, 192, 256}.
-int32_t qdit_launch_gemm_pair(qdit_ctx* ctx, const void* A, const void* W, qgemm::GemmParams& p, bool a_unsigned, int bn);
 
 // Channel-major accumulator kernel (gemm_i8_t.cu): tiles of 128 channels x bt tokens, bt in {128, 256}.
 int32_t qdit_launch_gemm_t(qdit_ctx* ctx, const void* A, const void* W, qgemm::GemmParams& p, bool a_unsigned, int bt);

@@ -170,11 +170,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 template <int BN, int EPI>
 int32_t launch_gemm_epi(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p, bool a_unsigned) {
   using C = Cfg<BN>;
-  static bool attr_set[64] = {};
-  if (!attr_set[ctx->device & 63]) {
-    QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(gemm_i8_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
-    attr_set[ctx->device & 63] = true;
-  }
+  QDIT_TRY(qdit_allow_smem(ctx, gemm_i8_kernel<BN, EPI>, C::SMEM_BYTES));
   CUtensorMap ta, tw;
   QDIT_TRY(qdit_get_tmap(ctx, A, p.M, p.K, p.K, BM, BK, 1, 1, &ta));
   QDIT_TRY(qdit_get_tmap(ctx, W, p.N, p.K, p.K, BN, BK, 1, 1, &tw));
@@ -190,7 +186,7 @@ int32_t launch_gemm_epi(qdit_ctx* ctx, const void* A, const void* W, GemmParams&
 
 template <int BN>
 int32_t launch_gemm(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p, bool a_unsigned) {
-  const int cls = getenv("QDIT_GEMM_GENERIC_EPILOGUE") ? 0 : epi_class(p.flags);  // tuning switch
+  const int cls = ctx->opt[QDIT_OPT_GEMM_GENERIC_EPILOGUE] ? 0 : epi_class(p.flags);
   switch (cls) {
     case 1: return launch_gemm_epi<BN, 1>(ctx, A, W, p, a_unsigned);
     case 2: return launch_gemm_epi<BN, 2>(ctx, A, W, p, a_unsigned);
@@ -201,12 +197,8 @@ int32_t launch_gemm(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p, 
 
 // Tile width: prefer 192 (divides every DiT-XL/2 layer width); fall back to narrower tiles when that
 // fills the SMs better.  Cost model: waves * (BN + fixed per-tile overhead).
-int pick_bn(int M, int N, int num_sms) {
-  const char* env = getenv("QDIT_GEMM_BN");
-  if (env) {
-    const int v = atoi(env);
-    if (v == 64 || v == 128 || v == 192) return v;
-  }
+int pick_bn(int M, int N, int num_sms, int forced) {
+  if (forced == 64 || forced == 128 || forced == 192) return forced;
   const int mt = (M + BM - 1) / BM;
   int best = 192;
   double best_cost = 1e30;
@@ -307,31 +299,20 @@ extern "C" int32_t qdit_w8a8_linear(qdit_ctx* ctx, const void* A, const void* W,
       p.o_qmax = static_cast<float>(epi->out_qp.qmax);
     }
   }
-  // QDIT_GEMM_T=<bt> selects the channel-major kernel with 128 x bt tiles (experimental switch while tuning)
-  const bool row_scale = (flags & QDIT_EPI_ROW_SCALE) != 0;  // implemented by the token-major kernels' generic epilogue
-  if (const char* env = row_scale ? nullptr : getenv("QDIT_GEMM_T")) {
-    const int bt = atoi(env);
-    if (bt == 128 || bt == 256) return qdit_launch_gemm_t(ctx, A, W, p, a_unsigned, bt);
-  }
-  // QDIT_GEMM_PAIR=<bn> selects the CTA-pair kernel with 256 x bn tiles (experimental switch while tuning)
-  if (const char* env = getenv("QDIT_GEMM_PAIR")) {
-    const int bn = atoi(env);
-    if (bn == 128 || bn == 192 || bn == 256) return qdit_launch_gemm_pair(ctx, A, W, p, a_unsigned, bn);
-  }
-  // Kernel choice (measured at M = 8192 on the DiT-XL/2 layers, see profiles/):
-  //  - layers whose epilogue neither reads a residual nor writes the cache (QKV: bias -> bf16; fc1: bias + GELU ->
-  //    8-bit) run channel-major with 128 x 256 tiles (2.19 / 1.94 POP/s vs 1.84 / 1.38 token-major);
-  //  - the gated layer with the long reduction (fc2, K = 4608) is bound by its main loop, where the 128 x 256 tile
-  //    moves less shared-memory traffic per MAC and fills the SMs in 2 waves instead of 2.6: channel-major too
-  //    (2.21 vs 2.02 POP/s);
-  //  - the gated layer with the short reduction (proj, K = 1152) is bound by its epilogue, which is cheaper
-  //    token-major (transpose through shared memory instead of shuffles): 128 x 192 tiles (1.10 vs 0.88 POP/s).
-  if (!getenv("QDIT_GEMM_BN") && p.M >= 1024) {
+  // QDIT_OPT_GEMM_T forces the channel-major kernel with 128 x bt tiles (per-token scales exist only in the
+  // token-major kernel's generic epilogue)
+  const bool row_scale = (flags & QDIT_EPI_ROW_SCALE) != 0;
+  if (!row_scale && ctx->opt[QDIT_OPT_GEMM_T] != 0) return qdit_launch_gemm_t(ctx, A, W, p, a_unsigned, ctx->opt[QDIT_OPT_GEMM_T]);
+  // Kernel choice (measured at M = 8192 on the DiT-XL/2 layers, see profiles/): the block's four layers run
+  // channel-major with 128 x 256 tiles (QKV: bias -> bf16 and the gated proj / fc2 through shared-memory tiles and
+  // TMA stores; fc1: bias + GELU -> 8-bit through shuffle transposes); everything else (small M, narrow N, f32 or
+  // raw outputs, per-token scales) runs token-major.
+  if (ctx->opt[QDIT_OPT_GEMM_BN] == 0 && !row_scale && p.M >= 1024) {
     const int cls = epi_class(p.flags);
     if ((cls == 1 || cls == 2) && p.N >= 2304) return qdit_launch_gemm_t(ctx, A, W, p, a_unsigned, 256);
     if (cls == 3 && p.N >= 1024 && p.tokens % 32 == 0) return qdit_launch_gemm_t(ctx, A, W, p, a_unsigned, 256);
   }
-  switch (pick_bn(p.M, p.N, ctx->num_sms)) {
+  switch (pick_bn(p.M, p.N, ctx->num_sms, ctx->opt[QDIT_OPT_GEMM_BN])) {
     case 64: return launch_gemm<64>(ctx, A, W, p, a_unsigned);
     case 128: return launch_gemm<128>(ctx, A, W, p, a_unsigned);
     default: return launch_gemm<192>(ctx, A, W, p, a_unsigned);

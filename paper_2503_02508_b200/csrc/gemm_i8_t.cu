@@ -44,7 +44,13 @@ struct TWarps {
   static constexpr int EPI_WARPS = STAGED ? QDIT_T_STAGED_WARPS : 12;
   static constexpr int SPLIT = EPI_WARPS / 4;
   static constexpr int THREADS = 64 + EPI_WARPS * 32;
-  static constexpr int STAGING_PER_WARP = STAGED ? 4096 : 0;  // two 2 KB tiles of 32 tokens x 32 channels bf16
+#ifndef QDIT_T_GATED_TILES
+#define QDIT_T_GATED_TILES 2
+#endif
+  // 2 KB tiles of 32 tokens x 32 channels bf16 per warp: class 1 two output tiles used in turn; class 3 the residual
+  // tile plus one tile shared by the cache copy and the output (2) or one tile each (3)
+  static constexpr int TILES = EPI == 3 ? QDIT_T_GATED_TILES : 2;
+  static constexpr int STAGING_PER_WARP = STAGED ? TILES * 2048 : 0;
   static constexpr int STAGING_BYTES = EPI_WARPS * STAGING_PER_WARP;
 };
 
@@ -355,6 +361,9 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
       uint8_t* stg = staging + e * TW::STAGING_PER_WARP;
       // class 1: two output tiles used in turn; class 3: tile 0 receives the residual, tile 1 carries the cache copy and then the output
       const uint32_t tile0 = smem_u32(stg), tile1 = tile0 + 2048u;
+      constexpr bool SEPARATE = TW::TILES == 3;                       // class 3: the output has a tile of its own
+      const uint32_t tile_o = SEPARATE ? tile0 + 4096u : tile1;
+      uint8_t* const stg_o = stg + (SEPARATE ? 4096 : 2048);
       const uint32_t row_off = frag_row_offset(lane);
       uint64_t* rbar = &res_bar[e];
       uint32_t r_phase = 0;
@@ -447,7 +456,11 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
             out_turn ^= 1;
           } else {
             // cache copy (the branch output before the gate)
-            if (lane == 0) tma_store_wait_read<0>();  // the previous chunk's output store has read tile 1
+            // tile 1 is free once the store that last used it has read it: the previous chunk's output store, or
+            // (separate tiles) the previous chunk's cache store, one group further back
+            if (lane == 0) {
+              if (SEPARATE) tma_store_wait_read<1>(); else tma_store_wait_read<0>();
+            }
             __syncwarp();
             frag_store_tile(tile1 + row_off, f);
             fence_async_smem();
@@ -486,13 +499,15 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                 r_inflight = true;
               }
             }
-            if (lane == 0) tma_store_wait_read<0>();  // the cache store has read tile 1
+            if (lane == 0) {  // the output tile is free: this chunk's cache store has read it, or (separate tiles) the previous chunk's output store
+              if (SEPARATE) tma_store_wait_read<1>(); else tma_store_wait_read<0>();
+            }
             __syncwarp();
-            frag_store_tile(tile1 + row_off, f);
+            frag_store_tile(tile_o + row_off, f);
             fence_async_smem();
             __syncwarp();
             if (lane == 0) {
-              tma_store_2d(&tmap_out, stg + 2048, c0q, m_base);
+              tma_store_2d(&tmap_out, stg_o, c0q, m_base);
               tma_store_commit();
             }
           }
@@ -559,11 +574,7 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
 template <int BT, int EPI>
 int32_t launch_t_epi(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p, bool a_unsigned) {
   using C = TCfg<BT, EPI>;
-  static bool attr_set[64] = {};
-  if (!attr_set[ctx->device & 63]) {
-    QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(gemm_i8_t_kernel<BT, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
-    attr_set[ctx->device & 63] = true;
-  }
+  QDIT_TRY(qdit_allow_smem(ctx, gemm_i8_t_kernel<BT, EPI>, C::SMEM_BYTES));
   CUtensorMap tw, tx;
   QDIT_TRY(qdit_get_tmap(ctx, W, p.N, p.K, p.K, BC, BK, 1, 1, &tw));
   QDIT_TRY(qdit_get_tmap(ctx, A, p.M, p.K, p.K, BT, BK, 1, 1, &tx));
@@ -591,7 +602,7 @@ int32_t launch_t_epi(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p,
 
 template <int BT>
 int32_t launch_t(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p, bool a_unsigned) {
-  switch (getenv("QDIT_GEMM_GENERIC_EPILOGUE") ? 0 : epi_class(p.flags)) {
+  switch (ctx->opt[QDIT_OPT_GEMM_GENERIC_EPILOGUE] ? 0 : epi_class(p.flags)) {
     case 1: return launch_t_epi<BT, 1>(ctx, A, W, p, a_unsigned);
     case 2: return launch_t_epi<BT, 2>(ctx, A, W, p, a_unsigned);
     case 3: return launch_t_epi<BT, 3>(ctx, A, W, p, a_unsigned);

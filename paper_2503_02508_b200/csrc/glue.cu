@@ -626,11 +626,7 @@ int32_t launch_small_linear(qdit_ctx* ctx, const float* in, const float* w, cons
   if (bc > B) bc = B;
   if (bc < 1) bc = 1;
   const size_t smem = static_cast<size_t>(bc) * K * sizeof(float);
-  static bool attr_set[64] = {};
-  if (!attr_set[ctx->device & 63]) {
-    QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(small_linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_budget));
-    attr_set[ctx->device & 63] = true;
-  }
+  QDIT_TRY(qdit_allow_smem(ctx, small_linear_kernel, smem_budget));
   ProfScope prof(ctx, QDIT_PROF_OTHER, static_cast<double>(N) * K * 4.0);
   small_linear_kernel<<<static_cast<unsigned>((N + 7) / 8), 256, smem, ctx->stream>>>(in, w, bias, table, y, out, out_silu, B, N,
                                                                                     K, bc, silu_input, silu_output,
@@ -675,12 +671,7 @@ int32_t launch_final(qdit_ctx* ctx, const void* x, int64_t M, int D, int T, floa
   const unsigned g = static_cast<unsigned>(want < ctx->num_sms ? want : ctx->num_sms);
 #define QDIT_FINAL_CASE(NV)                                                                                             \
   case NV: {                                                                                                            \
-    static bool attr_set[64] = {};                                                                                      \
-    if (!attr_set[ctx->device & 63]) {                                                                                  \
-      QDIT_CUDA_CHECK(ctx, cudaFuncSetAttribute(final_kernel<NV>, cudaFuncAttributeMaxDynamicSharedMemorySize,          \
-                                                FIN_OUT * NV * 2 * 32 * static_cast<int>(sizeof(float4))));             \
-      attr_set[ctx->device & 63] = true;                                                                                \
-    }                                                                                                                   \
+    QDIT_TRY(qdit_allow_smem(ctx, final_kernel<NV>, FIN_OUT * NV * 2 * 32 * static_cast<int>(sizeof(float4))));          \
     final_kernel<NV><<<g, 512, smem, ctx->stream>>>(xb, M, D, T, eps, modf, w, bias, net, grid, patch);                 \
   } break;
   ProfScope prof(ctx, QDIT_PROF_OTHER, static_cast<double>(M) * D * 2.0);

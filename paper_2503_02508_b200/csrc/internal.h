@@ -7,6 +7,7 @@
 
 #include <string>
 #include <unordered_map>
+#include <unordered_set>
 #include <vector>
 
 #include "qdit.h"
@@ -39,7 +40,11 @@ struct qdit_ctx {
   int* h_status = nullptr;  // pinned host mirror
   int num_sms = 0;
   int64_t launches = 0;
-  bool overlap_launches = true;  // programmatic dependent launch for the kernels that support it (QDIT_PDL=0 turns it off)
+  // Kernel-selection options (qdit_set_option).  Set once at creation from the QDIT_* environment variables of the
+  // same names, afterwards only through the call; no kernel launch reads the environment.
+  int opt[QDIT_OPT_COUNT] = {};
+  bool overlap_launches = true;  // = opt[QDIT_OPT_PDL]: programmatic dependent launch for the kernels that support it
+  std::unordered_set<const void*> attr_done;  // kernels whose dynamic shared-memory limit has been raised for this context
   std::string last_error;
   void* encode_fn = nullptr;  // cuTensorMapEncodeTiled
   std::unordered_map<TmapKey, CUtensorMap, TmapKeyHash> tmaps;
@@ -49,6 +54,9 @@ struct qdit_ctx {
   std::vector<ProfRec> prof;
   std::vector<cudaEvent_t> event_pool;
 };
+
+// Records a formatted message on the context and returns `code`.
+int32_t qdit_fail(qdit_ctx* ctx, int32_t code, const char* fmt, ...);
 
 // Brackets one kernel launch with events while profiling is enabled.
 struct ProfScope {
@@ -78,8 +86,18 @@ cudaError_t qdit_launch_overlapped(qdit_ctx* ctx, void (*kernel)(KArgs...), dim3
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-// Records a formatted message on the context and returns `code`.
-int32_t qdit_fail(qdit_ctx* ctx, int32_t code, const char* fmt, ...);
+// Raises a kernel's dynamic shared-memory limit once per context (the attribute is per device and function; a context
+// belongs to one device and is used by one thread at a time, so no process-wide state is involved).
+template <typename K>
+int32_t qdit_allow_smem(qdit_ctx* ctx, K kernel, int bytes) {
+  const void* key = reinterpret_cast<const void*>(kernel);
+  if (ctx->attr_done.count(key)) return QDIT_OK;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return qdit_fail(ctx, QDIT_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+  ctx->attr_done.insert(key);
+  return QDIT_OK;
+}
+
 // Checks the last launch; counts it.
 int32_t qdit_after_launch(qdit_ctx* ctx, const char* what);
 

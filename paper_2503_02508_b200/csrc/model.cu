@@ -484,11 +484,9 @@ int32_t qdit_sampler_create(qdit_ctx* ctx, qdit_model* m, const qdit_sampler_des
     const int64_t per_step = B * sh.depth * 6 * D * static_cast<int64_t>(sizeof(float));
     int64_t chunk = (int64_t(4) << 30) / per_step;
     if (chunk > d->num_steps) chunk = d->num_steps;
-    if (getenv("QDIT_STEPWISE_CONDITIONING")) chunk = 0;
-    if (const char* env = getenv("QDIT_CONDITIONING_CHUNK")) {  // smaller chunks on request (memory, tests)
-      const int64_t v = atoll(env);
-      if (v > 0 && v < chunk) chunk = v;
-    }
+    const int want = ctx->opt[QDIT_OPT_CONDITIONING_CHUNK];  // -1: per step; n > 0: at most n steps at once (memory, tests)
+    if (want < 0) chunk = 0;
+    if (want > 0 && want < chunk) chunk = want;
     s->traj_chunk = static_cast<int>(chunk);
     s->traj_c = s->traj_sc = s->traj_hidden = s->traj_feat = s->traj_mod = s->traj_modf = nullptr;
     s->traj_ca = nullptr;

@@ -7,6 +7,8 @@
 // tensors, in a process whose memory budget is fixed up front).  For them the partial maxima live in a
 // fixed array in the library's own device image.  Nothing here calls cudaMalloc, cudaFree or any routine
 // that allocates.
+#include <mutex>
+
 #include "common.cuh"
 #include "internal.h"
 
@@ -22,8 +24,28 @@ constexpr int kMaxPartials = 65536;            // => at most 65536 * 2048 = 134,
 static __device__ __align__(256) float g_partial_absmax[kMaxPartials];
 
 // In host code `g_partial_absmax` is only a handle; the device address comes from cudaGetSymbolAddress,
-// looked up once per device and kept here.
+// looked up once per device (under a lock: first calls from two threads may coincide) and kept here.
 float* g_scratch_ptr[64] = {};
+std::mutex g_scratch_lock;
+
+// Device address of the array on `device`.  The lookup needs that device to be current; the caller's current
+// device is put back afterwards.
+cudaError_t scratch_address(int device, float** out) {
+  std::lock_guard<std::mutex> guard(g_scratch_lock);
+  if (!g_scratch_ptr[device]) {
+    int prev = -1;
+    cudaError_t e = cudaGetDevice(&prev);
+    if (e != cudaSuccess) return e;
+    if (prev != device && (e = cudaSetDevice(device)) != cudaSuccess) return e;
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_partial_absmax);
+    if (prev != device) cudaSetDevice(prev);
+    if (e != cudaSuccess) return e;
+    g_scratch_ptr[device] = static_cast<float*>(p);
+  }
+  *out = g_scratch_ptr[device];
+  return cudaSuccess;
+}
 
 template <typename T>
 __global__ void __launch_bounds__(256) partial_absmax_kernel(const T* __restrict__ x, int64_t M, int64_t K, int64_t ldx,
@@ -94,19 +116,15 @@ extern "C" int32_t qdit_quantize_act_dynamic_static(qdit_ctx* ctx, const void* x
   const int64_t esz = x_dtype == QDIT_BF16 ? 2 : 4;
   if (!aligned16(x) || (ldx * esz) % 16 != 0) return qdit_fail(ctx, QDIT_ERR_ALIGN, "x must be 16-byte aligned (base and row pitch)");
   if ((reinterpret_cast<uintptr_t>(q) & 7u) || ldq % 8 != 0) return qdit_fail(ctx, QDIT_ERR_ALIGN, "q must be 8-byte aligned (base and row pitch)");
+  constexpr int64_t kMaxElems = static_cast<int64_t>(kMaxPartials) * kElemsPerCta;
+  // each factor is bounded before the product is formed, so M * K cannot overflow
+  if (M > kMaxElems || K > kMaxElems || M * K > kMaxElems)
+    return qdit_fail(ctx, QDIT_ERR_SHAPE, "M = %lld, K = %lld exceed the built-in scratch (at most %lld elements per call)",
+                     static_cast<long long>(M), static_cast<long long>(K), static_cast<long long>(kMaxElems));
   const int64_t ctas = (M * K + kElemsPerCta - 1) / kElemsPerCta;
-  if (ctas > kMaxPartials)
-    return qdit_fail(ctx, QDIT_ERR_SHAPE, "M*K = %lld exceeds the built-in scratch (at most %lld elements per call)",
-                     static_cast<long long>(M * K), static_cast<long long>(kMaxPartials) * kElemsPerCta);
   if (ctx->device < 0 || ctx->device >= 64) return qdit_fail(ctx, QDIT_ERR_UNSUPPORTED, "device index out of range");
-  float* scratch = g_scratch_ptr[ctx->device];
-  if (!scratch) {
-    // one-time set-up for this device (it must be the current device for the symbol lookup)
-    QDIT_CUDA_CHECK(ctx, cudaSetDevice(ctx->device));
-    void* p = nullptr;
-    QDIT_CUDA_CHECK(ctx, cudaGetSymbolAddress(&p, g_partial_absmax));
-    scratch = g_scratch_ptr[ctx->device] = static_cast<float*>(p);
-  }
+  float* scratch = nullptr;
+  QDIT_CUDA_CHECK(ctx, scratch_address(ctx->device, &scratch));  // first call on a device: the one-time lookup
   const unsigned grid = static_cast<unsigned>(ctas);
   if (x_dtype == QDIT_BF16)
     partial_absmax_kernel<__nv_bfloat16><<<grid, 256, 0, ctx->stream>>>(static_cast<const __nv_bfloat16*>(x), M, K, ldx, scratch);

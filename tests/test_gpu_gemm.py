@@ -9,7 +9,7 @@ import synth
 from oracle import dit, linear, quant
 from oracle.quant import QParams
 
-from gpu_util import bf16_to_f64, code_mismatch_report, dev, dev_i8, host_codes, max_rel_err
+from gpu_util import bf16_steps_err, bf16_to_f64, code_mismatch_report, dev, dev_i8, host_codes, max_rel_err
 
 pytestmark = pytest.mark.gpu
 
@@ -46,27 +46,26 @@ SHAPES = [(1, 8, 16), (128, 192, 128), (130, 200, 272), (256, 384, 1152), (517, 
           (1000, 3456, 1152), (64, 6912, 1152), (2048, 64, 64), (129, 1536, 384)]
 
 
+def _select_kernel(q, ctx, variant):
+    """"NNN": token-major kernel with 128 x NNN tiles; "tNNN": channel-major kernel with 128 x NNN tiles; else automatic."""
+    q.qdit_set_option(ctx, q.QDIT_OPT_GEMM_BN, 0)
+    q.qdit_set_option(ctx, q.QDIT_OPT_GEMM_T, 0)
+    if variant.startswith("t"):
+        q.qdit_set_option(ctx, q.QDIT_OPT_GEMM_T, int(variant[1:]))
+    elif variant.isdigit():
+        q.qdit_set_option(ctx, q.QDIT_OPT_GEMM_BN, int(variant))
+
+
 @pytest.mark.parametrize("M,N,K", SHAPES)
-@pytest.mark.parametrize("bn", ["auto", "64", "128", "192", "pair128", "pair192", "pair256", "t128", "t256"])
+@pytest.mark.parametrize("bn", ["auto", "64", "128", "192", "t128", "t256"])
 def test_accumulators_bit_exact(q, ctx, M, N, K, bn):
-    # "pairNNN": the CTA-pair kernel (256 x NNN tiles); plain numbers: the single-CTA kernel (128 x NNN)
-    os.environ.pop("QDIT_GEMM_BN", None)
-    os.environ.pop("QDIT_GEMM_PAIR", None)
-    os.environ.pop("QDIT_GEMM_T", None)
-    if bn.startswith("pair"):
-        os.environ["QDIT_GEMM_PAIR"] = bn[4:]
-    elif bn.startswith("t"):
-        os.environ["QDIT_GEMM_T"] = bn[1:]          # channel-major accumulator kernel, 128 x NNN tiles
-    elif bn != "auto":
-        os.environ["QDIT_GEMM_BN"] = bn
+    _select_kernel(q, ctx, bn)
     try:
         qa = _codes(31, f"a{M}.{K}", (M, K), -128, 127)
         qw = _codes(31, f"w{N}.{K}", (N, K), -127, 127)
         got = _run_i32(q, ctx, qa, qw)
     finally:
-        os.environ.pop("QDIT_GEMM_BN", None)
-        os.environ.pop("QDIT_GEMM_PAIR", None)
-        os.environ.pop("QDIT_GEMM_T", None)
+        _select_kernel(q, ctx, "auto")
     np.testing.assert_array_equal(got, linear.gemm_i8(qa, qw))
 
 
@@ -106,7 +105,7 @@ def _layer(seed, M, N, K, T, a_qp):
     x = synth.outlier_activations(seed, "x", M, K, gain=6.0)
     Wf = synth.normal(seed, "W", (N, K), 0.02)
     bias = synth.normal(seed, "b", (N,), 0.02)
-    gate = synth.normal(seed, "g", (M // T, N), 0.35)
+    gate = synth.normal(seed, "g", (-(-M // T), N), 0.35)
     resid = synth.normal(seed, "r", (M, N), 1.0)
     qw, s_w, cs = quant.quantize_weight_per_channel(Wf)
     qa = quant.quantize(x, a_qp)
@@ -131,17 +130,11 @@ def test_dequant_bias_f32(q, ctx, M, N, K, T, a_qp):
     assert max_rel_err(out.cpu().numpy(), ref) < 1e-5      # ... and what f32 arithmetic actually gives
 
 
-@pytest.fixture(params=["single", "pair192", "pair256", "t128", "t256"])
-def kernel_variant(request):
-    os.environ.pop("QDIT_GEMM_PAIR", None)
-    os.environ.pop("QDIT_GEMM_T", None)
-    if request.param.startswith("pair"):
-        os.environ["QDIT_GEMM_PAIR"] = request.param[4:]
-    elif request.param.startswith("t"):
-        os.environ["QDIT_GEMM_T"] = request.param[1:]
+@pytest.fixture(params=["single", "192", "t128", "t256"])
+def kernel_variant(request, q, ctx):
+    _select_kernel(q, ctx, request.param)
     yield request.param
-    os.environ.pop("QDIT_GEMM_PAIR", None)
-    os.environ.pop("QDIT_GEMM_T", None)
+    _select_kernel(q, ctx, "auto")
 
 
 def test_gate_residual_cache_epilogue(q, ctx, kernel_variant):
@@ -273,3 +266,111 @@ def test_rejects_bad_arguments(q, ctx):
     assert f(ctx, A.data_ptr(), W.data_ptr(), 128, 64, 64, qp, None, q.QDIT_EPI_OUT_F32, None, o.data_ptr(), 64) == q.QDIT_ERR_INVALID_ARG
     assert f(ctx, A.data_ptr(), W.data_ptr(), 0, 64, 64, qp, None, q.QDIT_EPI_OUT_I32, None, o.data_ptr(), 64) == q.QDIT_OK
     q.qdit_sync(ctx)
+
+
+@pytest.mark.parametrize("M,T", [(192, 64), (300, 100), (1184, 32)])
+def test_gated_epilogue_on_ragged_rows_with_an_exactly_sized_gate(q, ctx, kernel_variant, M, T):
+    """The last tile is ragged (M % 128 != 0) and the gate tensor has exactly ceil(M / T) rows: no row past it may
+    be read (the warps of a tile whose rows lie wholly past M have no sample)."""
+    N, K = 1152, 384
+    a_qp = QParams(0.05, 0, -127, 127)
+    L = _layer(46, M, N, K, T, a_qp)
+    B = -(-M // T)
+    gate_h = synth.normal(46, "g2", (B, N), 0.35)
+    A, W = dev_i8(L["qa"]), dev_i8(L["qw"])
+    ws, bi = dev(L["s_w"]), dev(L["bias"])
+    # the gate sits at the very end of its allocation, followed by a canary region that must stay untouched (reads
+    # past the end cannot be seen directly; the exact size is what the kernels are given)
+    g = dev(gate_h)
+    x = dev(L["resid"]).to(torch.bfloat16)
+    xh = bf16_to_f64(x)
+    cache = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    epi = q.epilogue(w_scale=ws, bias=bi, gate=g, ld_gate=N, tokens_per_sample=T, residual=x, cache_out=cache)
+    flags = q.QDIT_EPI_BIAS | q.QDIT_EPI_GATE | q.QDIT_EPI_RESIDUAL | q.QDIT_EPI_CACHE_STORE | q.QDIT_EPI_OUT_BF16
+    q.qdit_w8a8_linear(ctx, A, W, M, N, K, q.qparams(a_qp.scale), None, flags, epi, x, N)
+    q.qdit_sync(ctx)
+    f = linear.w8a8_linear(L["qa"], a_qp, L["qw"], L["s_w"], L["cs"], L["bias"])
+    rows = np.arange(M) // T
+    want_x = xh + gate_h.astype(np.float64)[rows] * f
+    got_c, got_x = bf16_to_f64(cache), bf16_to_f64(x)
+    assert (got_c != dit.round_bf16(f)).mean() < 1e-3
+    assert (got_x != dit.round_bf16(want_x)).mean() < 1e-3
+    assert max_rel_err(got_x, want_x) < 2.0 ** -8
+
+
+FULL_M = 8192   # tokens of the 50-step workload: network batch 32 x 256 tokens
+
+
+@pytest.mark.parametrize("K,N,name", [(1152, 3456, "qkv"), (1152, 1152, "proj"), (1152, 4608, "fc1"), (4608, 1152, "fc2")])
+def test_full_size_layers_element_by_element(q, ctx, K, N, name):
+    """The four block-level layers at the full workload's size, in the kernels the model path selects: raw int32
+    accumulators bit-exact, f32 outputs within 1e-3 (measured 1e-5), and each layer's own fused epilogue against the
+    oracle on every element."""
+    M, T = FULL_M, 256
+    a_qp = QParams(0.05, 0, -127, 127)
+    L = _layer(47, M, N, K, T, a_qp)
+    A, W = dev_i8(L["qa"]), dev_i8(L["qw"])
+    ws, bi, g = dev(L["s_w"]), dev(L["bias"]), dev(L["gate"])
+    acc = linear.gemm_i8(L["qa"], L["qw"])
+    f = linear.w8a8_linear(L["qa"], a_qp, L["qw"], L["s_w"], L["cs"], L["bias"])
+    for variant in ("auto", "t256"):
+        _select_kernel(q, ctx, variant)
+        try:
+            np.testing.assert_array_equal(_run_i32(q, ctx, L["qa"], L["qw"]), acc)
+            outf = torch.empty((M, N), dtype=torch.float32, device="cuda")
+            q.qdit_w8a8_linear(ctx, A, W, M, N, K, q.qparams(a_qp.scale), None, q.QDIT_EPI_BIAS | q.QDIT_EPI_OUT_F32,
+                               q.epilogue(w_scale=ws, bias=bi), outf, N)
+            q.qdit_sync(ctx)
+            assert max_rel_err(outf.cpu().numpy(), f) < 1e-5
+        finally:
+            _select_kernel(q, ctx, "auto")
+    if name == "qkv":
+        out = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        q.qdit_w8a8_linear(ctx, A, W, M, N, K, q.qparams(a_qp.scale), None, q.QDIT_EPI_BIAS | q.QDIT_EPI_OUT_BF16,
+                           q.epilogue(w_scale=ws, bias=bi), out, N)
+        q.qdit_sync(ctx)
+        got = bf16_to_f64(out)
+        assert (got != dit.round_bf16(f)).mean() < 1e-4 and bf16_steps_err(got, f) <= 1.0
+    elif name == "fc1":
+        u = dit.gelu_tanh(f)
+        o_qp = quant.qparams_symmetric(float(np.abs(u).max()) * 0.9)
+        out = torch.empty((M, N), dtype=torch.uint8, device="cuda")
+        q.qdit_w8a8_linear(ctx, A, W, M, N, K, q.qparams(a_qp.scale), None,
+                           q.QDIT_EPI_BIAS | q.QDIT_EPI_GELU | q.QDIT_EPI_QUANT_OUT,
+                           q.epilogue(w_scale=ws, bias=bi, out_qp=q.qparams(o_qp.scale)), out, N)
+        q.qdit_sync(ctx)
+        got, want = host_codes(out), quant.quantize(u, o_qp)
+        pre = u.astype(np.float32).astype(np.float64) * float(o_qp.inv_scale)
+        n_bad, ok = code_mismatch_report(got, want, pre, 2e-5 * np.abs(pre).max() + 1e-6)
+        assert ok and n_bad <= 1e-3 * got.size, (n_bad, got.size)
+    else:
+        x = dev(L["resid"]).to(torch.bfloat16)
+        xh = bf16_to_f64(x)
+        cache = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+        epi = q.epilogue(w_scale=ws, bias=bi, gate=g, ld_gate=N, tokens_per_sample=T, residual=x, cache_out=cache)
+        flags = q.QDIT_EPI_BIAS | q.QDIT_EPI_GATE | q.QDIT_EPI_RESIDUAL | q.QDIT_EPI_CACHE_STORE | q.QDIT_EPI_OUT_BF16
+        q.qdit_w8a8_linear(ctx, A, W, M, N, K, q.qparams(a_qp.scale), None, flags, epi, x, N)
+        q.qdit_sync(ctx)
+        want_x = xh + L["gate"].astype(np.float64)[np.arange(M) // T] * f
+        got_c, got_x = bf16_to_f64(cache), bf16_to_f64(x)
+        assert (got_c != dit.round_bf16(f)).mean() < 1e-4 and bf16_steps_err(got_c, f) <= 1.0
+        assert (got_x != dit.round_bf16(want_x)).mean() < 1e-3 and bf16_steps_err(got_x, want_x) <= 1.0
+
+
+def test_options_select_kernels_and_reject_bad_values(q, ctx):
+    assert q.qdit_get_option(ctx, q.QDIT_OPT_PDL) == 1
+    for opt, bad in ((q.QDIT_OPT_GEMM_BN, 96), (q.QDIT_OPT_GEMM_T, 64), (q.QDIT_OPT_ATTN, 3), (q.QDIT_OPT_PDL, 2), (99, 0)):
+        assert q.lib.qdit_set_option(ctx, opt, bad) == q.QDIT_ERR_INVALID_ARG
+    q.qdit_set_option(ctx, q.QDIT_OPT_GEMM_T, 128)
+    assert q.qdit_get_option(ctx, q.QDIT_OPT_GEMM_T) == 128
+    q.qdit_set_option(ctx, q.QDIT_OPT_GEMM_T, 0)
+    # with and without programmatic dependent launch: same bits
+    qa = _codes(35, "ap", (600, 384), -128, 127)
+    qw = _codes(35, "wp", (384, 384), -127, 127)
+    a = _run_i32(q, ctx, qa, qw)
+    q.qdit_set_option(ctx, q.QDIT_OPT_PDL, 0)
+    try:
+        b = _run_i32(q, ctx, qa, qw)
+    finally:
+        q.qdit_set_option(ctx, q.QDIT_OPT_PDL, 1)
+    np.testing.assert_array_equal(a, b)

@@ -395,7 +395,7 @@ def test_ddpm_sampler_tiny_matches_oracle(q, ctx, guidance):
         rig.close()
 
 
-def test_conditioning_chunks_give_the_same_trajectory(q, ctx, monkeypatch):
+def test_conditioning_chunks_give_the_same_trajectory(q, ctx):
     """The conditioning of a trajectory is evaluated for many steps at once; chunk size (all steps, 3 steps, one
     step at a time inside the network evaluation) must not change a bit of the result."""
     cfg = synth.DIT_TINY
@@ -404,20 +404,20 @@ def test_conditioning_chunks_give_the_same_trajectory(q, ctx, monkeypatch):
     try:
         kw = dict(num_steps=S, cache_interval=2, use_cfg=True, guidance=1.5)
         a, _ = _run_sampler(rig, latent, y, **kw)
-        monkeypatch.setenv("QDIT_CONDITIONING_CHUNK", "3")
+        q.qdit_set_option(ctx, q.QDIT_OPT_CONDITIONING_CHUNK, 3)
         l0 = q.qdit_launch_count(ctx)
         b, _ = _run_sampler(rig, latent, y, **kw)
         n_chunked = q.qdit_launch_count(ctx) - l0
-        monkeypatch.delenv("QDIT_CONDITIONING_CHUNK")
-        monkeypatch.setenv("QDIT_STEPWISE_CONDITIONING", "1")
+        q.qdit_set_option(ctx, q.QDIT_OPT_CONDITIONING_CHUNK, -1)
         c, _ = _run_sampler(rig, latent, y, **kw)
-        monkeypatch.delenv("QDIT_STEPWISE_CONDITIONING")
+        q.qdit_set_option(ctx, q.QDIT_OPT_CONDITIONING_CHUNK, 0)
         np.testing.assert_array_equal(a, b)
         assert rel_l2(c, a) < 5e-3          # the per-step path sums the small f32 linears in another order (code flips)
         # 4 chunks of conditioning (6 kernels each): steps 0, 3, 6, 9
         per_refresh, per_reuse = 1 + 7 * cfg.depth + 1 + 1, 1 + 1 + 1 + 1
         assert n_chunked == 4 * 6 + 5 * per_refresh + 5 * per_reuse
     finally:
+        q.qdit_set_option(ctx, q.QDIT_OPT_CONDITIONING_CHUNK, 0)
         rig.close()
 
 

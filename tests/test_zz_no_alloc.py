@@ -10,6 +10,7 @@ import pytest
 import torch
 
 import synth
+from oracle import quant
 
 pytestmark = pytest.mark.gpu
 
@@ -42,11 +43,21 @@ def test_static_scratch_quantizer_matches_regular_entry_point_twice_in_a_row():
             ref_q, ref_s, new_q, new_s = _both(q, ctx, x, dtype)
             assert new_s == ref_s                       # same scale, bit for bit (a maximum has no rounding order)
             np.testing.assert_array_equal(new_q, ref_q)  # same codes
+            # and both are the CPU oracle's dynamic quantizer (Eq. 1 with s = max|x| / 127) on the same input bits
+            xin = x if dtype == "f32" else torch.from_numpy(x).to(torch.bfloat16).float().numpy()
+            qp = quant.qparams_symmetric(float(np.abs(xin).max()))
+            assert new_s == np.float32(qp.scale)
+            np.testing.assert_array_equal(new_q.view(np.int8).astype(np.int32), quant.quantize(xin, qp))
         assert _both(q, ctx, np.zeros((8, 16), dtype=np.float32), "f32")[3] == 1.0
         # beyond the built-in scratch: refused with a clear message, nothing launched
         big_m = 65536 * 2048 // 1152 + 2
         st = q.lib.qdit_quantize_act_dynamic_static(ctx, 256, q.QDIT_F32, big_m, 1152, 1152, 256, 256, 1152)
         assert st == q.QDIT_ERR_SHAPE and b"built-in scratch" in q.lib.qdit_last_error(ctx)
+        # sizes whose product would wrap a 64-bit integer are refused the same way
+        st = q.lib.qdit_quantize_act_dynamic_static(ctx, 256, q.QDIT_F32, 2 ** 40, 2 ** 40, 2 ** 40, 256, 256, 2 ** 40)
+        assert st == q.QDIT_ERR_SHAPE and b"built-in scratch" in q.lib.qdit_last_error(ctx)
+        # the one-time set-up leaves the caller's current device as it was
+        assert torch.cuda.current_device() == 0
         q.qdit_sync(ctx)
     finally:
         q.qdit_destroy(ctx)
