@@ -334,12 +334,26 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
 // ---------------------------------------------------------------------------------------------------------
 // T = 256 (two key blocks): the whole score row fits the CTA's 256 tensor-memory columns, so the softmax is
-// taken in one piece instead of online.  Both K blocks and V_0 are requested at once (K_1 lands in the P tile,
-// which nobody needs before both S blocks are complete); S_0 and S_1 are issued back to back; V_1 is requested
-// into the Q tile as soon as the S products have finished reading Q.  One row maximum (one exchange between
-// the two threads of a row), no rescaling, both P.V products accumulate into the same columns (those of S_0),
-// which are read once at the end.  Same shared and tensor memory as the general kernel: two CTAs per SM.
-// Every barrier completes exactly once (phase 0).
+// taken in one piece instead of online, and the probabilities never leave tensor memory.
+//   * Q, both K blocks and V_0 are requested at once; S_0 and S_1 are issued back to back; V_1 is requested into
+//     Q's place as soon as the S products have finished reading Q.
+//   * One row maximum (one exchange between the two threads of a row), no rescaling.
+//   * P = exp2(..) is written back as bf16 pairs over the score columns the same thread has already read
+//     (tcgen05.st), and P.V takes its A operand from tensor memory: no shared-memory tile for P, no proxy fence,
+//     and P_1 does not wait for the first P.V product.
+// Tensor-memory columns of the CTA:  0..63 P_0 | 64..127 O (head dims 0..63) | 128..191 P_1 | 192..207 O (dims 64..79).
+// The two threads of a row split a key block into 32-key chunks 0, 2 (first thread) and 1, 3 (second): chunk c of
+// block j is read from columns 128 j + 32 c and its 16 packed columns go to 128 j + 32 (c & 1) + 16 (c >> 1), inside
+// columns that thread has read before.  P's key order along the columns is therefore chunk 0, 2, 1, 3, and the
+// k-steps of P.V pick their V rows in that order.  O's columns are free once both threads of every row have written
+// P_0 (main part) and P_1 (tail part): the barriers the MMA issuer waits for anyway.
+// 85 KB shared memory and 256 tensor-memory columns: two CTAs per SM.  Every barrier completes exactly once (phase 0).
+template <int DH>
+struct T256Cfg {
+  using B = TCfg<DH>;
+  static constexpr int SMEM_BYTES = 4 * B::OP_BYTES + 4096 + 1024;  // Q, K_0, K_1, V_0 (+ tails), barriers and row statistics, alignment
+};
+
 template <int DH>
 __global__ void __launch_bounds__(TC_THREADS, 2)
 attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -350,25 +364,24 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sQ = smem;                           // Q, later V_1
-  uint8_t* sK = sQ + C::MAIN_BYTES;             // K_0
-  uint8_t* sV = sK + C::MAIN_BYTES;             // V_0
-  uint8_t* sP = sV + C::MAIN_BYTES;             // K_1 (main tile, tail tile behind it), later P (two 64-key tiles)
-  uint8_t* sQt = sP + C::P_BYTES;               // tails (256-byte aligned: 32B-swizzle atoms); Q's, later V_1's
-  uint8_t* sKt = sQt + C::TAIL_BYTES;
-  uint8_t* sVt = sKt + C::TAIL_BYTES;
-  uint8_t* sK1 = sP;
-  uint8_t* sK1t = sP + C::MAIN_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sVt + C::TAIL_BYTES);
+  uint8_t* sK0 = sQ + C::MAIN_BYTES;
+  uint8_t* sK1 = sK0 + C::MAIN_BYTES;
+  uint8_t* sV0 = sK1 + C::MAIN_BYTES;
+  uint8_t* sQt = sV0 + C::MAIN_BYTES;           // tails (256-byte aligned: 32B-swizzle atoms); Q's, later V_1's
+  uint8_t* sK0t = sQt + C::TAIL_BYTES;
+  uint8_t* sK1t = sK0t + C::TAIL_BYTES;
+  uint8_t* sV0t = sK1t + C::TAIL_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sV0t + C::TAIL_BYTES);
   uint64_t* bar_q = bars + 0;      // Q tiles landed (tx)
   uint64_t* bar_qz = bars + 1;     // Q tail padding zeroed (256 arrivals)
   uint64_t* bar_k = bars + 2;      // [2] K block landed (tx)
   uint64_t* bar_v = bars + 4;      // [2] V block landed (tx)
   uint64_t* bar_s = bars + 6;      // [2] S block complete (commit); [1] also: Q and both K blocks have been read
-  uint64_t* bar_p = bars + 8;      // [2] P block written (256 arrivals)
-  uint64_t* bar_o = bars + 10;     // [2] P.V of block 0 / of both blocks complete (commit)
-  uint64_t* bar_l = bars + 12;     // row sums exchanged (256 arrivals)
-  uint64_t* bar_mx = bars + 13;    // [4] row maxima exchanged between the two warps of a lane quadrant (64 arrivals)
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 17);
+  uint64_t* bar_p = bars + 8;      // [2] P block written to tensor memory (256 arrivals)
+  uint64_t* bar_o = bars + 10;     // both P.V products complete (commit)
+  uint64_t* bar_l = bars + 11;     // row sums exchanged (256 arrivals)
+  uint64_t* bar_mx = bars + 12;    // [4] row maxima exchanged between the two warps of a lane quadrant (64 arrivals)
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 16);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
   float* s_l = reinterpret_cast<float*>(tmem_holder + 4);  // [2][128] partial row sums
   float* s_m = s_l + 256;                                  // [2][128] partial row maxima
@@ -376,6 +389,7 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q0 = blockIdx.x * TQ, h = blockIdx.y, b = blockIdx.z;
   const int row0 = b * p.T, col0 = h * DH;
+  constexpr uint32_t COL_O = 64, COL_OT = 192;   // accumulator columns: head dims 0..63, head dims 64..79
 
   if (threadIdx.x == 0) {
     mbar_init(bar_q, 1);
@@ -385,14 +399,20 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       mbar_init(&bar_v[i], 1);
       mbar_init(&bar_s[i], 1);
       mbar_init(&bar_p[i], SM_WARPS * 32);
-      mbar_init(&bar_o[i], 1);
     }
+    mbar_init(bar_o, 1);
     mbar_init(bar_l, SM_WARPS * 32);
     for (int i = 0; i < 4; ++i) mbar_init(&bar_mx[i], 64);
     *abort_flag = 0;
     mbar_fence_init();
   }
-  if (warp == SM_WARPS + 1) {
+  if (warp == SM_WARPS) {
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_q);
+      tma_prefetch_desc(&tm_k);
+      tma_prefetch_desc(&tm_v);
+    }
+  } else if (warp == SM_WARPS + 1) {
     tmem_alloc(tmem_holder, 256);
     tmem_relinquish();
   }
@@ -411,14 +431,14 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       tma_load_2d(sQ, &tm_q, col0, row0 + q0, bar_q);
       if (C::TAIL) tma_load_2d(sQt, &tm_qt, col0 + 64, row0 + q0, bar_q);
       mbar_expect_tx(&bar_k[0], C::OP_BYTES);
-      tma_load_2d(sK, &tm_k, col0, row0, &bar_k[0]);
-      if (C::TAIL) tma_load_2d(sKt, &tm_kt, col0 + 64, row0, &bar_k[0]);
+      tma_load_2d(sK0, &tm_k, col0, row0, &bar_k[0]);
+      if (C::TAIL) tma_load_2d(sK0t, &tm_kt, col0 + 64, row0, &bar_k[0]);
       mbar_expect_tx(&bar_k[1], C::OP_BYTES);
       tma_load_2d(sK1, &tm_k, col0, row0 + TK, &bar_k[1]);
       if (C::TAIL) tma_load_2d(sK1t, &tm_kt, col0 + 64, row0 + TK, &bar_k[1]);
       mbar_expect_tx(&bar_v[0], C::OP_BYTES);
-      tma_load_2d(sV, &tm_v, col0, row0, &bar_v[0]);
-      if (C::TAIL) tma_load_2d(sVt, &tm_vt, col0 + 64, row0, &bar_v[0]);
+      tma_load_2d(sV0, &tm_v, col0, row0, &bar_v[0]);
+      if (C::TAIL) tma_load_2d(sV0t, &tm_vt, col0 + 64, row0, &bar_v[0]);
       // V_1 takes Q's place once both S products have read Q
       if (mbar_wait(&bar_s[1], 0, abort_flag, p.status)) {
         mbar_expect_tx(&bar_v[1], C::OP_BYTES);
@@ -441,36 +461,46 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         if (C::TAIL) umma_bf16(d, umma_desc(smem_u32(sQt), 256, 6), umma_desc(smem_u32(k_tail), 256, 6), id_s, 1u);
         umma_commit(&bar_s[j]);
       };
-      // O += P_j V_j over columns 0..79: 8 k-steps of 16 keys; V's 8-key groups are 1024 (main) / 256 (tail) bytes apart
-      auto issue_pv = [&](int j, const uint8_t* v_main, const uint8_t* v_tail) {
+      // k-step s of a P.V product reads P columns 8 s .. 8 s + 7 of its block = 16 keys starting at key_of(s)
+      // (chunk order 0, 2, 1, 3); V's 8-key groups are 1024 (main tile) / 256 (tail tile) bytes apart
+      auto key16_of = [](int s) { return ((s & 4) ? 2 : 0) + ((s & 2) ? 4 : 0) + (s & 1); };  // in units of 16 keys
+      auto issue_pv_main = [&](int j, const uint8_t* v_main) {
 #pragma unroll
-        for (int k = 0; k < TK / 16; ++k) {
-          const uint64_t a = umma_desc(smem_u32(sP) + (k >> 2) * C::MAIN_BYTES + (k & 3) * 32, 1024, 2);
-          const uint32_t acc = (j | k) ? 1u : 0u;
-          umma_bf16(tmem, a, umma_desc(smem_u32(v_main) + k * 2048, 1024, 2), id_o, acc);
-          if (C::TAIL) umma_bf16(tmem + 64, a, umma_desc(smem_u32(v_tail) + k * 512, 256, 6), id_ot, acc);
-        }
-        umma_commit(&bar_o[j]);
+        for (int s = 0; s < 8; ++s)
+          umma_bf16_ta(tmem + COL_O, tmem + static_cast<uint32_t>(j * 128 + 8 * s),
+                       umma_desc(smem_u32(v_main) + key16_of(s) * 2048, 1024, 2), id_o, (j | s) ? 1u : 0u);
+      };
+      auto issue_pv_tail = [&](int j, const uint8_t* v_tail) {
+#pragma unroll
+        for (int s = 0; s < 8; ++s)
+          umma_bf16_ta(tmem + COL_OT, tmem + static_cast<uint32_t>(j * 128 + 8 * s),
+                       umma_desc(smem_u32(v_tail) + key16_of(s) * 512, 256, 6), id_ot, (j | s) ? 1u : 0u);
       };
       bool ok = mbar_wait(bar_qz, 0, abort_flag, p.status) && mbar_wait(&bar_k[0], 0, abort_flag, p.status);
       if (ok) {
         tc_fence_after();
-        issue_s(0, sK, sKt);
+        issue_s(0, sK0, sK0t);
       }
       ok = ok && mbar_wait(&bar_k[1], 0, abort_flag, p.status);
       if (ok) {
         tc_fence_after();
         issue_s(1, sK1, sK1t);
       }
+      // P_0 written: every thread has finished with the columns of S_0, which now hold P_0 and will hold O
       ok = ok && mbar_wait(&bar_p[0], 0, abort_flag, p.status) && mbar_wait(&bar_v[0], 0, abort_flag, p.status);
       if (ok) {
         tc_fence_after();
-        issue_pv(0, sV, sVt);
+        issue_pv_main(0, sV0);
       }
       ok = ok && mbar_wait(&bar_p[1], 0, abort_flag, p.status) && mbar_wait(&bar_v[1], 0, abort_flag, p.status);
       if (ok) {
         tc_fence_after();
-        issue_pv(1, sQ, sQt);
+        issue_pv_main(1, sQ);
+        if (C::TAIL) {
+          issue_pv_tail(0, sV0t);
+          issue_pv_tail(1, sQt);
+        }
+        umma_commit(bar_o);
       }
     }
   } else {
@@ -487,7 +517,8 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       }
       mbar_arrive(bar_qz);
     }
-    // row maximum over this thread's 64 keys of each block, then over the row with the other thread's value
+    // row maximum over this thread's 64 keys of each block (chunks half and half + 2), then over the row with the
+    // other thread's value
     float mx = -INFINITY;
 #pragma unroll 1
     for (int j = 0; j < 2 && ok; ++j) {
@@ -495,9 +526,9 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       __syncwarp();
       tc_fence_after();
       uint32_t v0[32], v1[32];  // both loads in flight, one wait
-      const uint32_t sbuf = trow + static_cast<uint32_t>(j * 128 + half * 64);
+      const uint32_t sbuf = trow + static_cast<uint32_t>(j * 128 + half * 32);
       tmem_ld_32x32(sbuf, v0);
-      tmem_ld_32x32(sbuf + 32, v1);
+      tmem_ld_32x32(sbuf + 64, v1);
       tmem_ld_wait();
       float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
@@ -515,40 +546,27 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     float rs = 0.0f;
     if (ok) {
       const float m_row = fmaxf(mx, s_m[(half ^ 1) * 128 + r]) * p.scale_log2;
-      const uint32_t tile = smem_u32(sP) + static_cast<uint32_t>(half * C::MAIN_BYTES + r * 128);
 #pragma unroll 1
-      for (int j = 0; j < 2 && ok; ++j) {
-        // P_j = exp2(s * scale - m) for this thread's 64 keys of block j: bf16, row sum in f32
-        const uint32_t sbuf = trow + static_cast<uint32_t>(j * 128 + half * 64);
-        uint32_t pk[32];
+      for (int j = 0; j < 2; ++j) {
+        // P_j = exp2(s * scale - m) for this thread's two chunks of block j: bf16 pairs back into tensor memory,
+        // over columns this thread has already read; row sum in f32
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
+        for (int w = 0; w < 2; ++w) {
           uint32_t v[32];
-          tmem_ld_32x32(sbuf + c * 32, v);
+          tmem_ld_32x32(trow + static_cast<uint32_t>(j * 128 + half * 32 + w * 64), v);
           tmem_ld_wait();
+          uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             const float p0 = ex2_approx(fmaf(__uint_as_float(v[2 * i]), p.scale_log2, -m_row));
             const float p1 = ex2_approx(fmaf(__uint_as_float(v[2 * i + 1]), p.scale_log2, -m_row));
             rs += p0 + p1;
-            pk[c * 16 + i] = pack_bf16x2(p0, p1);
+            pk[i] = pack_bf16x2(p0, p1);
           }
+          tmem_st_32x16(trow + static_cast<uint32_t>(j * 128 + half * 32 + w * 16), pk);
         }
-        // the P tile is free once the tensor core has read what it held: K_1 (both S complete: waited for above)
-        // for block 0, P_0 for block 1
-        if (j == 1) {
-          if (!mbar_wait(&bar_o[0], 0, abort_flag, p.status)) { ok = false; break; }
-          tc_fence_after();
-        }
-#pragma unroll
-        for (int g = 0; g < 8; ++g) {
-          const uint32_t addr = tile + ((static_cast<uint32_t>(g) ^ (static_cast<uint32_t>(r) & 7u)) << 4);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[4 * g]), "r"(pk[4 * g + 1]),
-                       "r"(pk[4 * g + 2]), "r"(pk[4 * g + 3])
-                       : "memory");
-        }
-        fence_async_smem();   // P is read by the tensor core through the async proxy
-        tc_fence_before();    // and (block 0) the S_0 columns are about to be overwritten by O
+        tmem_st_wait();
+        tc_fence_before();   // P_j is read, and the rest of S_j overwritten, by the tensor core
         mbar_arrive(&bar_p[j]);
       }
     }
@@ -558,33 +576,34 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       mbar_arrive(bar_l);
       ok = mbar_wait(bar_l, 0, abort_flag, p.status);
     }
-    if (ok && mbar_wait(&bar_o[1], 0, abort_flag, p.status)) {
+    if (ok && mbar_wait(bar_o, 0, abort_flag, p.status)) {
       __syncwarp();
       tc_fence_after();
-      float o[C::O_HALF];
-      const uint32_t src = trow + static_cast<uint32_t>(half * C::O_HALF);
+      // first thread of a row: head dims 0..31; second: head dims 32..63 and the tail 64..71
+      float o[40];
       {
         uint32_t v[32];
-        tmem_ld_32x32(src, v);
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(v[i]);
-        if (C::TAIL) {
+        tmem_ld_32x32(trow + COL_O + static_cast<uint32_t>(half * 32), v);
+        if (C::TAIL && half == 1) {
           uint32_t w[8];
-          tmem_ld_32x8(src + 32, w);
+          tmem_ld_32x8(trow + COL_OT, w);
           tmem_ld_wait();
 #pragma unroll
           for (int i = 0; i < 8; ++i) o[32 + i] = __uint_as_float(w[i]);
+        } else {
+          tmem_ld_wait();
         }
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(v[i]);
       }
       const float inv_l = 1.0f / (s_l[r] + s_l[128 + r]);
       const int64_t row = static_cast<int64_t>(row0) + q0 + r;
-      const int64_t base = row * (static_cast<int64_t>(p.H) * DH) + col0 + half * C::O_HALF;
-      const int ngroups = half == 0 ? C::O_HALF / 8 : (DH - C::O_HALF) / 8;  // output columns beyond DH are padding
+      const int64_t base = row * (static_cast<int64_t>(p.H) * DH) + col0 + half * 32;
+      const int ngroups = (C::TAIL && half == 1) ? 5 : 4;
       float q_inv = 0.0f;
       if (p.out_dtype == QDIT_I8) q_inv = __fdiv_rn(1.0f, p.qa.scale_dev ? __ldg(p.qa.scale_dev) : p.qa.scale);
 #pragma unroll
-      for (int g = 0; g < C::O_HALF / 8; ++g) {
+      for (int g = 0; g < 5; ++g) {
         if (g < ngroups) {
           float y[8];
 #pragma unroll
@@ -616,7 +635,7 @@ int32_t launch_tc(qdit_ctx* ctx, const void* q, const void* k, const void* v, in
                   const AttnTcParams& p) {
   using C = TCfg<DH>;
   QDIT_TRY(qdit_allow_smem(ctx, attention_tc_kernel<DH>, C::SMEM_BYTES));
-  QDIT_TRY(qdit_allow_smem(ctx, attention_tc256_kernel<DH>, C::SMEM_BYTES));
+  QDIT_TRY(qdit_allow_smem(ctx, attention_tc256_kernel<DH>, T256Cfg<DH>::SMEM_BYTES));
   const uint64_t rows = static_cast<uint64_t>(B) * T, cols = static_cast<uint64_t>(H) * DH;
   CUtensorMap tq, tk, tv, tqt, tkt, tvt;
   QDIT_TRY(qdit_get_tmap(ctx, q, rows, cols, ld, 128, 64, 1, 2, &tq));
@@ -633,7 +652,7 @@ int32_t launch_tc(qdit_ctx* ctx, const void* q, const void* k, const void* v, in
   dim3 grid(T / TQ, H, B);
   ProfScope prof(ctx, QDIT_PROF_ATTENTION, 4.0 * B * H * static_cast<double>(T) * T * DH);
   if (T == 2 * TK && ctx->opt[QDIT_OPT_ATTN] != 2) {  // the whole score row in tensor memory (option 2 forces the general kernel)
-    QDIT_CUDA_CHECK(ctx, qdit_launch_overlapped(ctx, attention_tc256_kernel<DH>, grid, dim3(TC_THREADS), C::SMEM_BYTES, tq, tk, tv, tqt, tkt, tvt, p));
+    QDIT_CUDA_CHECK(ctx, qdit_launch_overlapped(ctx, attention_tc256_kernel<DH>, grid, dim3(TC_THREADS), T256Cfg<DH>::SMEM_BYTES, tq, tk, tv, tqt, tkt, tvt, p));
     return qdit_after_launch(ctx, "attention_tc256_kernel");
   }
   QDIT_CUDA_CHECK(ctx, qdit_launch_overlapped(ctx, attention_tc_kernel<DH>, grid, dim3(TC_THREADS), C::SMEM_BYTES, tq, tk, tv, tqt, tkt, tvt, p));

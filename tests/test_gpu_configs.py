@@ -4,9 +4,12 @@ cache interval 2, VC) and the 100-step 512x512 sampler (batch 8, cache interval 
 The CPU oracle cannot run these workloads whole in test time, so it computes a sample of them: because
 activation scales are static and tensor-wise, VC statistics per sample and the cache per sample, every image's
 trajectory is independent of its batch-mates.  The oracle therefore follows ONE image (with its unconditional
-twin under guidance) for the first steps of the trajectory, and the full-batch CUDA run must match it on that
-image; the rest of the batch and of the trajectory is covered by properties that hold at any size (batch
-independence bit for bit, determinism, finiteness, the schedule's launch counts).
+twin under guidance): through ALL 50 steps of the 256x256 workload (about five minutes of CPU), so that the final
+latent of a full sampling run is compared, and through the first 7 of the 100 steps of the 512x512 workload (three
+cache refreshes; a refresh step at 1024 tokens costs the oracle close to a minute, all 34 would take half an hour).
+The full-batch CUDA run must match the oracle on that image; the rest of the batch and of the trajectory is
+covered by properties that hold at any size (batch independence bit for bit, determinism, finiteness, the
+schedule's launch counts).
 """
 import numpy as np
 import pytest
@@ -137,7 +140,7 @@ def _gpu_trajectory(q, ctx, rig, latent, labels, steps, interval, guidance, vc_t
 def test_ddim50_guided_cached_sampler_batch16(q, ctx, xl256):
     """50-step DDIM at 256x256, batch 16, guidance 1.5 (network batch 32), cache interval 2, VC every step."""
     cfg, seed = xl256.cfg, synth.CONFIG_SEEDS["ddim50_xl2"]
-    S, B, interval, guidance, n_prefix = 50, 16, 2, 1.5, 4
+    S, B, interval, guidance, n_prefix = 50, 16, 2, 1.5, 50     # the oracle follows image 0 through ALL steps
     latent = synth.normal(seed, "latent", (B, cfg.channels, cfg.latent_side, cfg.latent_side))
     labels = synth.uniform_int(seed, "labels", (B,), 0, cfg.num_classes)
     K = (1.0 + 0.02 * synth.normal(seed, "vc_table", (S, cfg.channels))).astype(np.float32)
@@ -146,10 +149,17 @@ def test_ddim50_guided_cached_sampler_batch16(q, ctx, xl256):
     xl256.set_scales(scales)
     ref = _oracle_prefix(xl256, scales, latent[:1], labels[:1], S, n_prefix, interval, guidance, K)
     snaps, final, launches = _gpu_trajectory(q, ctx, xl256, latent, labels, S, interval, guidance, K, set(range(n_prefix)))
-    for i in range(n_prefix):                      # steps 0..3 = refresh, reuse, refresh, reuse
+    worst = 0.0
+    for i in range(n_prefix):                      # steps 0, 1, 2, ... = refresh, reuse, refresh, ...
         err = rel_l2(snaps[i][:1], ref[i])
-        print(f"ddim50 step {i} latent rel-L2 vs oracle: {err:.3e}")
+        worst = max(worst, err)
+        if i < 4 or i % 10 == 9:
+            print(f"ddim50 step {i} latent rel-L2 vs oracle: {err:.3e}")
         assert err < 2e-2, (i, err)
+    # the benchmark spec's bound: the FINAL latent of the full 50-step run
+    err_final = rel_l2(final[:1], ref[S - 1])
+    print(f"ddim50 final latent (after step {S - 1}) rel-L2 vs oracle: {err_final:.3e}; worst step {worst:.3e}")
+    assert err_final < 2e-2, err_final
     assert np.isfinite(final).all()
     # launch accounting: the conditioning of all steps is evaluated once (6 kernels); refresh steps run 7 kernels
     # per block, reuse steps one kernel for all blocks
@@ -191,7 +201,7 @@ def test_forward_xl2_w4a8_matches_oracle(q, ctx):
 def test_ddim100_512_cached_sampler_batch8(q, ctx):
     """100-step DDIM at 512x512 (1024 tokens), batch 8, cache interval 3, VC every step, no guidance."""
     cfg, seed = synth.DIT_XL2_512, synth.CONFIG_SEEDS["ddim100_xl2_512"]
-    S, B, interval, n_prefix = 100, 8, 3, 3
+    S, B, interval, n_prefix = 100, 8, 3, 7      # steps 0..6: three refreshes (0, 3, 6) and the reuse steps between them
     rig = XLRig(q, ctx, cfg, seed)
     try:
         latent = synth.normal(seed, "latent", (B, cfg.channels, cfg.latent_side, cfg.latent_side))
@@ -201,7 +211,7 @@ def test_ddim100_512_cached_sampler_batch8(q, ctx):
         rig.set_scales(scales)
         ref = _oracle_prefix(rig, scales, latent[:1], labels[:1], S, n_prefix, interval, None, K)
         snaps, final, launches = _gpu_trajectory(q, ctx, rig, latent, labels, S, interval, None, K, set(range(n_prefix)))
-        for i in range(n_prefix):                  # refresh, reuse, reuse
+        for i in range(n_prefix):                  # refresh, reuse, reuse, refresh, ...
             err = rel_l2(snaps[i][:1], ref[i])
             print(f"ddim100_512 step {i} latent rel-L2 vs oracle: {err:.3e}")
             assert err < 2e-2, (i, err)

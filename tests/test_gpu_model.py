@@ -297,6 +297,44 @@ def test_sampler_tiny_matches_oracle(q, ctx, interval, guidance, use_vc):
         rig.close()
 
 
+@pytest.mark.parametrize("which", ["tiny", "xl_width_two_blocks"])
+def test_distance_to_the_oracle_without_storage_rounding(q, ctx, which):
+    """The default oracle rounds the residual stream, Q/K/V and the cache to bfloat16 where the CUDA path stores them
+    in bfloat16, and accumulates a fully skipped step once.  This test measures the CUDA path against the oracle with
+    neither: float64 storage throughout (Storage.exact) and the skipped step walked block by block.  Both distances
+    are printed; the stated end-to-end bound (relative L2 2e-2) is asserted against the un-rounded oracle."""
+    if which == "tiny":
+        cfg, seed, B, S = synth.DIT_TINY, 77, 3, 10
+    else:
+        cfg, seed, B, S = synth.DiTConfig(hidden=1152, heads=16, mlp=4608, depth=2, grid=16), 78, 2, 6
+    rig = Rig(q, ctx, cfg, seed)
+    try:
+        latent, t, y = _inputs(cfg, seed, B)
+        # activation ranges from the un-rounded network, so that the yardstick owes nothing to the storage formats
+        scales = calib.calibrate_model(rig.om, [(latent, t, y)], storage=dit.Storage.exact())
+        rig.set_scales(scales)
+        mirrored = dit.Context(quant="static", scales=scales)
+        plain = dit.Context(quant="static", scales=scales, storage=dit.Storage.exact(), reuse_walk=True)
+        # one network evaluation
+        got = rig.forward(rig.sampler(batch=B, num_steps=2), latent, t, y)
+        d_m = rel_l2(got, dit.forward(rig.om, mirrored, latent, t, y))
+        d_p = rel_l2(got, dit.forward(rig.om, plain, latent, t, y))
+        print(f"{which}: forward rel-L2 vs bf16-storage oracle {d_m:.3e}, vs float64-storage oracle {d_p:.3e}")
+        assert d_p < 2e-2 and d_m < 2e-2
+        # a cached, guided trajectory with VC
+        K = (1.0 + 0.03 * synth.normal(seed, "K", (S, cfg.channels))).astype(np.float32)
+        kw = dict(num_steps=S, cache_interval=2, use_cfg=True, guidance=1.5, vc_mode=q.QDIT_VC_K_TABLE, vc_table=K)
+        got_s, _ = _run_sampler(rig, latent, y, **kw)
+        scfg = sampler.SamplerConfig(S, cache_interval=2, guidance=1.5, vc_table=K)
+        s_m = rel_l2(got_s, sampler.sample(rig.om, mirrored, scfg, latent, y))
+        s_p = rel_l2(got_s, sampler.sample(rig.om, plain, scfg, latent, y))
+        print(f"{which}: {S}-step cached guided trajectory rel-L2 vs bf16-storage oracle {s_m:.3e}, "
+              f"vs float64-storage, block-by-block oracle {s_p:.3e}")
+        assert s_p < 2e-2 and s_m < 2e-2
+    finally:
+        rig.close()
+
+
 def test_sampler_per_branch_schedule_matches_oracle(q, ctx):
     """Per-block, per-branch reuse schedule ([steps, blocks, 2]) against the oracle, and its two reductions."""
     cfg = synth.DIT_TINY
