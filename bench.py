@@ -250,6 +250,7 @@ def run_ours(args):
     q.qdit_model_begin_calibration(ctx, model)
     for tval in (980.0, 500.0, 20.0):
         t_d = torch.full((beff,), tval, dtype=torch.float32, device="cuda")
+        torch.cuda.synchronize()     # t_d is filled on torch's stream, the library reads it on its own
         q.qdit_forward(ctx, sampler, lat_eff, t_d, y_eff, beff, net, q.QDIT_FWD_CALIBRATE)
         q.qdit_sync(ctx)
     q.qdit_model_finish_calibration(ctx, model)
@@ -260,6 +261,7 @@ def run_ours(args):
         gen.manual_seed(seed + rank)
         noise_d = torch.randn((steps, batch, cfg.channels, cfg.latent_side, cfg.latent_side), generator=gen,
                               dtype=torch.float32, device="cuda")
+        torch.cuda.synchronize()     # the noise is drawn on torch's stream, the library reads it on its own
         q.qdit_sampler_set_ddpm(ctx, sampler, noise_d)
 
     def trajectory_device():
@@ -319,7 +321,7 @@ def run_ours(args):
     int8_peak = 2.0 * peaks["bf16_sustained"]          # dense int8 : bf16 nominal ratio 4.5 : 2.25
     achieved = g_ops / (g_ms * 1e-3) / 1e12 if g_ms > 0 else 0.0
     roofline = {"bound": "tensor", "kernel": "int8 GEMMs (gemm_i8_t_kernel, gemm_i8_kernel)", "achieved": achieved,
-                "peak": int8_peak, "unit": "TOP/s", "frac": achieved / int8_peak,
+                "peak": int8_peak, "unit": "TOP/s", "frac": achieved / int8_peak, "frac_of_nominal_4500": achieved / 4500.0,
                 "traffic": NCU_GEMM_DRAM_BYTES_PER_LAUNCH if args.workload == "ddim50" else None,
                 "traffic_note": "launch-weighted mean of the four block-level layers at M = 8192 (ncu, L2-warm sweep)",
                 "peak_source": f"2 x {peaks['source']} sustained bf16 ({peaks['bf16_sustained']} TFLOP/s)",
@@ -337,6 +339,19 @@ def run_ours(args):
                                "rate": round(rate / 1e12, 2) if k < 2 else round(rate / 1e9, 1),
                                "unit": "TOP/s" if k == 0 else "TFLOP/s" if k == 1 else "GB/s",
                                "avg_us": round(1e3 * t / n, 2)}
+
+    # the metric's second half: the GEMM layers and the memory-bound kernels alone, at the workload's row count and at
+    # one larger than L2 (rank 0 of a single-GPU run only; a few seconds)
+    sweep = None
+    if rank == 0 and world == 1 and not args.no_sweep:
+        sclk = ClockSampler(local)
+        sclk.start()
+        srows = sweep_rows(q, ctx, [8192, 65536], 10, peaks, stream)
+        sweep = compact_sweep(srows, sclk.stop(), peaks)
+        for name, b in breakdown.items():
+            if name == "cache_reuse":
+                sweep["memory_bound"].append({"kernel": "cache_reuse_all (inside the trajectory, 1.06 GB per launch)",
+                                              "gbs": b["rate"], "frac_of_hbm": round(b["rate"] / peaks["hbm_gbs"], 3)})
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -360,6 +375,7 @@ def run_ours(args):
             "gpu_launches": int(launches),
             "roofline": roofline,
             "kernels": breakdown,
+            "sweep": sweep,
             "cpu_baseline": cpu,
         }
         print(json.dumps(line))
@@ -374,17 +390,16 @@ def run_ours(args):
 GEMM_SHAPES = [(1152, 3456, "qkv"), (1152, 1152, "proj"), (1152, 4608, "fc1"), (4608, 1152, "fc2")]
 
 
-def run_gemm_sweep(args):
-    """int8 GEMM + fused activation-quantizer sweep over the DiT-XL/2 linear shapes (K -> N) and M.
-    Activations: bf16 N(0,1) with 1 % of the channels scaled x20; weights: int8 with channel-wise scales.
-    Reports TOP/s of the GEMM alone (epilogue of that layer in the model) and of act-quant + GEMM."""
+def sweep_rows(q, ctx, ms_list, steps, peaks, stream=None):
+    """Times the block's four linear layers (with the epilogue each has in the model), the activation quantizer,
+    LayerNorm-modulate-quantize and attention at the given row counts.  Activations: bf16 N(0,1) with 1 % of the
+    channels scaled x20; weights: int8 with channel-wise scales.  Launches are repeated back to back on the same
+    operands (L2-warm below about 100 MB of operands, streaming from HBM above).  `stream`: the torch stream the
+    context launches on (None: the default stream); the timing events are recorded there."""
     import torch
-    import paper_2503_02508_b200 as q
     seed = synth.CONFIG_SEEDS["gemm_sweep"]
-    peaks = measured_peaks()
-    ctx = q.qdit_create(0, None)
     rows = []
-    for M in args.m:
+    for M in ms_list:
         for K, N, name in GEMM_SHAPES:
             x = torch.from_numpy(synth.outlier_activations(seed, f"x{M}.{K}", M, K)).cuda().to(torch.bfloat16)
             wq = torch.from_numpy(synth.uniform_int(seed, f"w{N}.{K}", (N, K), -127, 128).astype(np.int8)).cuda()
@@ -420,13 +435,14 @@ def run_gemm_sweep(args):
                     fn()
                 torch.cuda.synchronize()
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record()
-                for _ in range(args.steps):
+                e0.record(stream)
+                for _ in range(steps):
                     fn()
-                e1.record()
+                e1.record(stream)
                 torch.cuda.synchronize()
-                return e0.elapsed_time(e1) / args.steps
+                return e0.elapsed_time(e1) / steps
 
+            torch.cuda.synchronize()   # the operands were made on torch's stream
             quant()
             ops = 2.0 * M * N * K
             ms_g, ms_b, ms_q = t(gemm), t(both), t(quant)
@@ -443,6 +459,7 @@ def run_gemm_sweep(args):
                     q.qdit_adaln_modulate(ctx, x, M, K, 256, 1e-6, mod, mod[:, K:], 6 * K, a8, q.QDIT_I8, a_qp)
 
                 ms_l = t(ln)
+                row["ln_modulate_us"] = ms_l * 1e3
                 row["ln_modulate_gbs"] = 3.0 * M * K / ms_l / 1e6
                 row["ln_modulate_frac_of_hbm"] = row["ln_modulate_gbs"] / peaks["hbm_gbs"]
                 # and the block's attention on the layer's output shape (16 heads of 72, 256 tokens per image)
@@ -457,15 +474,53 @@ def run_gemm_sweep(args):
                 row["attention_us"] = ms_a * 1e3
                 row["attention_tflops"] = 4.0 * (M // 256) * 16 * 256 * 256 * (K // 16) / ms_a / 1e9
             rows.append(row)
+            del x, wq, resid, cache, a8, out
+    return rows
+
+
+def run_gemm_sweep(args):
+    """int8 GEMM + fused activation-quantizer sweep over the DiT-XL/2 linear shapes (K -> N) and M.
+    Reports TOP/s of the GEMM alone (epilogue of that layer in the model) and of act-quant + GEMM."""
+    import paper_2503_02508_b200 as q
+    peaks = measured_peaks()
+    ctx = q.qdit_create(0, None)
+    clocks = ClockSampler(0)
+    clocks.start()
+    rows = sweep_rows(q, ctx, args.m, args.steps, peaks)
+    clock_info = clocks.stop()
     q.qdit_sync(ctx)
     q.qdit_destroy(ctx)
     best = max(r["gemm_tops"] for r in rows)
     print(json.dumps({"metric": "int8 GEMM TOP/s (DiT-XL/2 linear shapes)", "value": best, "unit": "TOP/s", "n_gpus": 1,
                       "steps": args.steps, "warmup": 3, "higher_is_better": True, "dtype": "int8", "data": "synthetic",
                       "config": {"workload": "gemm_sweep", "l2": "repeated launches on the same operands (L2-warm)"},
+                      "clocks": clock_info,
                       "peaks": {"int8_2x_bf16_burst": 2 * peaks["bf16_burst"], "int8_nominal": 4500.0,
                                 "hbm_gbs": peaks["hbm_gbs"], "source": peaks["source"]},
                       "rows": rows}))
+
+
+def compact_sweep(rows, clock_info, peaks):
+    """The second half of the metric for the default bench line: per layer and M the GEMM rate and its fractions of
+    2 x burst bf16 (measured) and of the nominal 4500 TOP/s; the memory-bound kernels as fractions of the measured HBM
+    copy bandwidth."""
+    out = {"clocks": clock_info, "int8_peak_2x_bf16_burst": 2 * peaks["bf16_burst"], "int8_nominal": 4500.0,
+           "hbm_gbs": peaks["hbm_gbs"], "gemm": [], "memory_bound": [],
+           "note": "launches repeated back to back on the same operands: L2-warm at M = 8192, streaming from HBM at M = 65536"}
+    for r in rows:
+        out["gemm"].append({"layer": r["layer"], "M": r["M"], "us": round(r["gemm_us"], 1), "tops": round(r["gemm_tops"], 0),
+                            "frac_2x_bf16_burst": round(r["frac_of_2x_bf16_burst"], 3),
+                            "frac_nominal": round(r["frac_of_nominal_4500"], 3),
+                            "with_act_quant_tops": round(r["quant_gemm_tops"], 0)})
+        if r["layer"] in ("qkv", "fc2"):
+            out["memory_bound"].append({"kernel": "act_quant", "M": r["M"], "K": r["K"], "gbs": round(r["act_quant_gbs"], 0),
+                                        "frac_of_hbm": round(r["act_quant_frac_of_hbm"], 3)})
+        if "ln_modulate_gbs" in r:
+            out["memory_bound"].append({"kernel": "ln_modulate_q8", "M": r["M"], "K": r["K"], "us": round(r["ln_modulate_us"], 1),
+                                        "gbs": round(r["ln_modulate_gbs"], 0), "frac_of_hbm": round(r["ln_modulate_frac_of_hbm"], 3)})
+            out.setdefault("attention", []).append({"M": r["M"], "us": round(r["attention_us"], 1),
+                                                    "tflops": round(r["attention_tflops"], 0)})
+    return out
 
 
 def main():
@@ -476,6 +531,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="ddim50", choices=sorted(WORKLOADS) + ["gemm_sweep"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the per-layer sweep that follows the timed region")
     ap.add_argument("--weight-bits", type=int, default=8, help="code width of the quantized weights (4 = the paper's W4A8 setting)")
     ap.add_argument("--m", type=lambda v: [int(x) for x in v.split(",")], default=[256, 1024, 4096, 8192, 16384, 65536],
                     help="row counts of the GEMM sweep")

@@ -508,6 +508,10 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const int quad = warp & 3, half = warp >> 2;
     const int r = quad * 32 + lane;
     const uint32_t trow = tmem + (static_cast<uint32_t>(quad * 32) << 16);
+    // the output quantizer's scale is fetched now, long before it is needed (a load from global memory at the end
+    // of the chain would add its whole latency to the CTA's life)
+    float q_inv = 0.0f;
+    if (p.out_dtype == QDIT_I8) q_inv = __fdiv_rn(1.0f, p.qa.scale_dev ? __ldg(p.qa.scale_dev) : p.qa.scale);
     bool ok = mbar_wait(bar_q, 0, abort_flag, p.status);
     if (ok) {
       if (C::TAIL && half == 0) {  // zero columns 72..79 of this row of the Q tail (second 16-byte slot, 32B swizzle)
@@ -600,8 +604,6 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       const int64_t row = static_cast<int64_t>(row0) + q0 + r;
       const int64_t base = row * (static_cast<int64_t>(p.H) * DH) + col0 + half * 32;
       const int ngroups = (C::TAIL && half == 1) ? 5 : 4;
-      float q_inv = 0.0f;
-      if (p.out_dtype == QDIT_I8) q_inv = __fdiv_rn(1.0f, p.qa.scale_dev ? __ldg(p.qa.scale_dev) : p.qa.scale);
 #pragma unroll
       for (int g = 0; g < 5; ++g) {
         if (g < ngroups) {
