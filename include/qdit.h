@@ -192,12 +192,28 @@ int32_t qdit_w8a8_linear(qdit_ctx* ctx, const void* A, const void* W, int64_t M,
                          qdit_qparams a_qp, const float* a_scale_dev, uint32_t flags,
                          const qdit_epilogue* epi, void* out, int64_t ldo);
 
+/* W4A8 linear layer (Table 2, the 512 x 512 setting): the same operation on 4-bit channel-wise weight codes stored
+ * two per byte.  W_packed: [N, K/2] bytes, row n holds codes W[n, 2j] in the low nibble and W[n, 2j+1] in the high
+ * nibble of byte j, each a 4-bit two's-complement number in [-8, 7] (the byte layout is this library's; the paper
+ * fixes only the code width).  K % 32 == 0; QDIT_EPI_ROW_SCALE is not available; everything else as
+ * qdit_w8a8_linear, with identical results for identical codes.  The weights cross HBM at half the bytes: with
+ * few rows (M < 1024, or no scratch given) they are widened to int8 inside the GEMM kernel in front of the tensor
+ * core; with many rows and w8_scratch != NULL (device, N*K bytes, 16-byte aligned, overwritten) they are widened
+ * into the scratch first and the W8A8 kernels run on it.
+ * qdit_pack_weight_int4 / qdit_unpack_weight_int4 convert between [N, K] int8 codes and the packed form
+ * (K % 16 == 0; packing refuses codes outside [-8, 7] with QDIT_ERR_INVALID_ARG and synchronises the stream). */
+int32_t qdit_w4a8_linear(qdit_ctx* ctx, const void* A, const void* W_packed, int64_t M, int64_t N, int64_t K,
+                         qdit_qparams a_qp, const float* a_scale_dev, uint32_t flags,
+                         const qdit_epilogue* epi, void* out, int64_t ldo, void* w8_scratch);
+int32_t qdit_pack_weight_int4(qdit_ctx* ctx, const void* w8, int64_t N, int64_t K, void* packed);
+int32_t qdit_unpack_weight_int4(qdit_ctx* ctx, const void* packed, int64_t N, int64_t K, void* w8);
+
 /* Channel-wise symmetric weight quantizer (the weight side of Eq. 1): for each output row n of
  * w[N,K] (f32, device), s[n] = max_k|w| / 127 (1 if the row is zero), q = clip(round(w * (1/s)),-127,127),
  * colsum[n] = sum_k q[n,k].  q: [N,K] bytes, w_scale: [N] f32, w_colsum: [N] int32.  K % 4 == 0.
  * qdit_quantize_weight_bits is the same with b-bit codes (2 <= bits <= 8): top = 2^(bits-1) - 1 replaces 127.
- * With bits = 4 this is the weight side of the paper's W4A8 setting (Table 2); the codes are still stored one
- * per byte, so every kernel that takes 8-bit weights takes them unchanged. */
+ * With bits = 4 this is the weight side of the paper's W4A8 setting (Table 2); this call leaves the codes one per
+ * byte (qdit_pack_weight_int4 packs them two per byte for qdit_w4a8_linear). */
 int32_t qdit_quantize_weight(qdit_ctx* ctx, const float* w, int64_t N, int64_t K, void* q, float* w_scale,
                              int32_t* w_colsum);
 int32_t qdit_quantize_weight_bits(qdit_ctx* ctx, const float* w, int64_t N, int64_t K, int bits, void* q,
@@ -292,7 +308,8 @@ int32_t qdit_tap_laplacian(qdit_ctx* ctx, const float* x, const float* t, int n,
  * modulation linear, QKV, projection, fc1 and fc2; embedders and the final layer stay in f32. */
 typedef struct {
   int32_t hidden, heads, mlp, depth, grid, patch, channels, num_classes, freq_dim;
-  int32_t weight_bits; /* code width of the quantized linears' weights: 0 or 8 = W8A8, 4 = W4A8 (Table 2) */
+  int32_t weight_bits; /* code width of the quantized linears' weights: 0 or 8 = W8A8; 4 = W4A8 (Table 2), stored two
+                          codes per byte (half the weight memory); 2..7 other widths, stored one code per byte */
 } qdit_model_shape;
 
 typedef struct { /* HOST f32 arrays, each linear [out_features, in_features] row-major */
@@ -328,9 +345,14 @@ int32_t qdit_model_set_act_scales(qdit_ctx* ctx, qdit_model* model, const float*
 int32_t qdit_model_get_act_scales(qdit_ctx* ctx, qdit_model* model, float* ada_scale, float* block_scales);
 /* Device views of a quantized linear, for tests and for driving the primitives by hand.
  * which: 0 ada (of `block`; all blocks are stacked block-major in one [depth*6D, D] matrix),
- * 1 qkv, 2 proj, 3 fc1, 4 fc2.  Any out pointer may be NULL. */
+ * 1 qkv, 2 proj, 3 fc1, 4 fc2.  Any out pointer may be NULL.  w_q is [N, K] bytes, or the packed form [N, K/2] of
+ * qdit_w4a8_linear when the model stores 4-bit weights two per byte (weight_bits = 4 with hidden and mlp multiples
+ * of 32; qdit_model_weights_packed tells). */
 int32_t qdit_model_linear(qdit_model* model, int block, int which, const void** w_q, const float** w_scale,
                           const int32_t** w_colsum, const float** bias, int64_t* N, int64_t* K);
+
+/* 1 if the model keeps its quantized weights as two 4-bit codes per byte, else 0. */
+int32_t qdit_model_weights_packed(const qdit_model* model);
 
 typedef struct {
   int32_t batch;          /* images per trajectory batch */

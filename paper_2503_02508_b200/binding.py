@@ -101,6 +101,10 @@ _SIGNATURES = {
     "qdit_model_destroy": (_i32, [_vp]),
     "qdit_model_set_act_scales": (_i32, [_vp, _vp, _vp, _vp]),
     "qdit_model_get_act_scales": (_i32, [_vp, _vp, _vp, _vp]),
+    "qdit_model_weights_packed": (_i32, [_vp]),
+    "qdit_w4a8_linear": (_i32, [_vp, _vp, _vp, _i64, _i64, _i64, qdit_qparams, _vp, _u32, C.POINTER(qdit_epilogue), _vp, _i64, _vp]),
+    "qdit_pack_weight_int4": (_i32, [_vp, _vp, _i64, _i64, _vp]),
+    "qdit_unpack_weight_int4": (_i32, [_vp, _vp, _i64, _i64, _vp]),
     "qdit_model_linear": (_i32, [_vp, _int, _int, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp),
                                  C.POINTER(_i64), C.POINTER(_i64)]),
     "qdit_sampler_create": (_i32, [_vp, _vp, C.POINTER(qdit_sampler_desc), C.POINTER(_vp)]),
@@ -222,6 +226,23 @@ def epilogue(w_scale=None, w_colsum=None, bias=None, gate=None, ld_gate=0, token
 def qdit_w8a8_linear(ctx, A, W, M, N, K, a_qp, a_scale_dev, flags, epi, out, ldo):
     return check(ctx, lib.qdit_w8a8_linear(ctx, ptr(A), ptr(W), M, N, K, a_qp, ptr(a_scale_dev), flags,
                                            C.byref(epi) if epi is not None else None, ptr(out), ldo))
+
+
+def qdit_w4a8_linear(ctx, A, W_packed, M, N, K, a_qp, a_scale_dev, flags, epi, out, ldo, w8_scratch=None):
+    return check(ctx, lib.qdit_w4a8_linear(ctx, ptr(A), ptr(W_packed), M, N, K, a_qp, ptr(a_scale_dev), flags,
+                                           C.byref(epi) if epi is not None else None, ptr(out), ldo, ptr(w8_scratch)))
+
+
+def qdit_pack_weight_int4(ctx, w8, N, K, packed):
+    return check(ctx, lib.qdit_pack_weight_int4(ctx, ptr(w8), N, K, ptr(packed)))
+
+
+def qdit_unpack_weight_int4(ctx, packed, N, K, w8):
+    return check(ctx, lib.qdit_unpack_weight_int4(ctx, ptr(packed), N, K, ptr(w8)))
+
+
+def qdit_model_weights_packed(model):
+    return lib.qdit_model_weights_packed(model)
 
 
 def qdit_quantize_weight(ctx, w, N, K, q, w_scale, w_colsum):

@@ -249,3 +249,6 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t tacc
 
 // Channel-major accumulator kernel (gemm_i8_t.cu): tiles of 128 channels x bt tokens, bt in {128, 256}.
 int32_t qdit_launch_gemm_t(qdit_ctx* ctx, const void* A, const void* W, qgemm::GemmParams& p, bool a_unsigned, int bt);
+
+// Packed 4-bit weights widened inside the kernel (gemm_w4.cu): token-major tiles of 128 x 128.
+int32_t qdit_launch_gemm_w4(qdit_ctx* ctx, const void* A, const void* W_packed, qgemm::GemmParams& p, bool a_unsigned);

@@ -217,14 +217,19 @@ int pick_bn(int M, int N, int num_sms, int forced) {
 
 }  // namespace
 
-extern "C" int32_t qdit_w8a8_linear(qdit_ctx* ctx, const void* A, const void* W, int64_t M, int64_t N, int64_t K,
-                                    qdit_qparams a_qp, const float* a_scale_dev, uint32_t flags,
-                                    const qdit_epilogue* epi, void* out, int64_t ldo) {
+// Both linear layers: `packed4` = W holds 4-bit codes two per byte ([N, K/2]); `w8_scratch` = optional [N, K] int8
+// matrix the packed weights of a many-row layer are widened into first.
+static int32_t linear_impl(qdit_ctx* ctx, const void* A, const void* W, int64_t M, int64_t N, int64_t K, qdit_qparams a_qp,
+                           const float* a_scale_dev, uint32_t flags, const qdit_epilogue* epi, void* out, int64_t ldo,
+                           bool packed4, void* w8_scratch) {
   if (!ctx) return QDIT_ERR_INVALID_ARG;
   if (M < 0 || N < 0 || K < 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "negative size");
   if (M == 0 || N == 0) return QDIT_OK;
   if (!A || !W || !out) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "A, W or out is NULL");
   if (K == 0 || K % 16 != 0 || K > 32768) return qdit_fail(ctx, QDIT_ERR_SHAPE, "K = %lld must be a positive multiple of 16, at most 32768", static_cast<long long>(K));
+  if (packed4 && K % 32 != 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "K = %lld must be a multiple of 32 for packed 4-bit weights", static_cast<long long>(K));
+  if (packed4 && (flags & QDIT_EPI_ROW_SCALE)) return qdit_fail(ctx, QDIT_ERR_UNSUPPORTED, "per-token scales are not available with packed 4-bit weights");
+  if (w8_scratch && !aligned16(w8_scratch)) return qdit_fail(ctx, QDIT_ERR_ALIGN, "the weight scratch must be 16-byte aligned");
   if (N % 8 != 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "N = %lld must be a multiple of 8", static_cast<long long>(N));
   if (M > (1 << 30) || N > (1 << 30)) return qdit_fail(ctx, QDIT_ERR_SHAPE, "M or N too large");
   const uint32_t out_modes = flags & (QDIT_EPI_OUT_BF16 | QDIT_EPI_OUT_F32 | QDIT_EPI_OUT_I32 | QDIT_EPI_QUANT_OUT);
@@ -299,6 +304,17 @@ extern "C" int32_t qdit_w8a8_linear(qdit_ctx* ctx, const void* A, const void* W,
       p.o_qmax = static_cast<float>(epi->out_qp.qmax);
     }
   }
+  if (packed4) {
+    // many rows: the layer is bound by the tensor core and its epilogue, so the weights are widened once into the
+    // scratch matrix and the W8A8 kernels run on it; few rows (or no scratch): the weight bytes bound the layer and
+    // the kernel that widens them in front of the tensor core reads half of them
+    if (w8_scratch && M >= 1024) {
+      QDIT_TRY(qdit_unpack_weight_int4(ctx, W, N, K, w8_scratch));
+      W = w8_scratch;
+    } else {
+      return qdit_launch_gemm_w4(ctx, A, W, p, a_unsigned);
+    }
+  }
   // QDIT_OPT_GEMM_T forces the channel-major kernel with 128 x bt tiles (per-token scales exist only in the
   // token-major kernel's generic epilogue)
   const bool row_scale = (flags & QDIT_EPI_ROW_SCALE) != 0;
@@ -317,4 +333,16 @@ extern "C" int32_t qdit_w8a8_linear(qdit_ctx* ctx, const void* A, const void* W,
     case 128: return launch_gemm<128>(ctx, A, W, p, a_unsigned);
     default: return launch_gemm<192>(ctx, A, W, p, a_unsigned);
   }
+}
+
+extern "C" int32_t qdit_w8a8_linear(qdit_ctx* ctx, const void* A, const void* W, int64_t M, int64_t N, int64_t K,
+                                    qdit_qparams a_qp, const float* a_scale_dev, uint32_t flags,
+                                    const qdit_epilogue* epi, void* out, int64_t ldo) {
+  return linear_impl(ctx, A, W, M, N, K, a_qp, a_scale_dev, flags, epi, out, ldo, false, nullptr);
+}
+
+extern "C" int32_t qdit_w4a8_linear(qdit_ctx* ctx, const void* A, const void* W_packed, int64_t M, int64_t N, int64_t K,
+                                    qdit_qparams a_qp, const float* a_scale_dev, uint32_t flags,
+                                    const qdit_epilogue* epi, void* out, int64_t ldo, void* w8_scratch) {
+  return linear_impl(ctx, A, W_packed, M, N, K, a_qp, a_scale_dev, flags, epi, out, ldo, true, w8_scratch);
 }

@@ -32,11 +32,12 @@ struct DeviceArena {  // owns cudaMalloc'd blocks
 };
 
 struct QLinearDev {
-  int8_t* q = nullptr;
+  int8_t* q = nullptr;   // codes: [N, K] one per byte, or [N, K/2] two 4-bit codes per byte when `packed4`
   float* scale = nullptr;
   int32_t* colsum = nullptr;
   float* bias = nullptr;
   int64_t N = 0, K = 0;
+  bool packed4 = false;
 };
 
 }  // namespace
@@ -51,6 +52,8 @@ struct qdit_model {
   float* d_scales;      // [1 + 4*depth] static activation scales: [0] ada input, then per block qkv, proj, fc1, fc2
   float* d_absmax_run;  // [1 + 4*depth] widest range seen during calibration
   bool scales_set;
+  bool packed4;         // 4-bit weights stored two codes per byte (weight_bits == 4 and every K a multiple of 32)
+  int64_t max_block_weight;  // largest N*K among the block-level linears (size of the widening scratch)
   int n_scales() const { return 1 + 4 * s.depth; }
 };
 
@@ -66,6 +69,7 @@ struct qdit_sampler {
   int32_t *y, *labels;
   float* dyn_absmax;             // [1 + 4*depth] this pass's ranges (calibration)
   float* dyn_scale;              // [1 + 4*depth] and the scales derived from them
+  int8_t* w8_scratch;            // [max N*K] int8: a packed block-level weight matrix widened for the many-row kernels
   float* vc_table;               // device [S, C] or null
   // Conditioning of the whole trajectory, evaluated at step 0: the conditioning vector, and with it every block's
   // modulation, depends on the timestep and the label only, never on the latent.  Rows are (step, sample).
@@ -92,10 +96,11 @@ int32_t upload(qdit_ctx* ctx, DeviceArena& mem, const float* host, size_t n, flo
   return QDIT_OK;
 }
 
-int32_t alloc_qlinear(qdit_ctx* ctx, DeviceArena& mem, int64_t N, int64_t K, QLinearDev* l) {
+int32_t alloc_qlinear(qdit_ctx* ctx, DeviceArena& mem, int64_t N, int64_t K, bool packed4, QLinearDev* l) {
   l->N = N;
   l->K = K;
-  l->q = mem.alloc<int8_t>(static_cast<size_t>(N) * K);
+  l->packed4 = packed4;
+  l->q = mem.alloc<int8_t>(static_cast<size_t>(N) * K / (packed4 ? 2 : 1));
   l->scale = mem.alloc<float>(N);
   l->colsum = mem.alloc<int32_t>(N);
   l->bias = mem.alloc<float>(N);
@@ -103,12 +108,18 @@ int32_t alloc_qlinear(qdit_ctx* ctx, DeviceArena& mem, int64_t N, int64_t K, QLi
   return QDIT_OK;
 }
 
-// Uploads one f32 linear through the staging buffer and quantizes rows [row0, row0+N) of `l` on the device.
-int32_t quantize_into(qdit_ctx* ctx, float* staging, const float* w, const float* b, int64_t N, int64_t K,
+// Uploads one f32 linear through the staging buffer and quantizes rows [row0, row0+N) of `l` on the device
+// (`codes8`: N*K bytes of scratch for the one-per-byte codes of a layer that is stored packed).
+int32_t quantize_into(qdit_ctx* ctx, float* staging, int8_t* codes8, const float* w, const float* b, int64_t N, int64_t K,
                       QLinearDev* l, int64_t row0, int bits) {
   if (!w || !b) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "a block weight pointer is NULL");
   QDIT_CUDA_CHECK(ctx, cudaMemcpyAsync(staging, w, static_cast<size_t>(N) * K * sizeof(float), cudaMemcpyHostToDevice, ctx->stream));
-  QDIT_TRY(qdit_quantize_weight_bits(ctx, staging, N, K, bits, l->q + row0 * K, l->scale + row0, l->colsum + row0));
+  if (l->packed4) {
+    QDIT_TRY(qdit_quantize_weight_bits(ctx, staging, N, K, bits, codes8, l->scale + row0, l->colsum + row0));
+    QDIT_TRY(qdit_pack_weight_int4(ctx, codes8, N, K, l->q + row0 * K / 2));
+  } else {
+    QDIT_TRY(qdit_quantize_weight_bits(ctx, staging, N, K, bits, l->q + row0 * K, l->scale + row0, l->colsum + row0));
+  }
   QDIT_CUDA_CHECK(ctx, cudaMemcpyAsync(l->bias + row0, b, static_cast<size_t>(N) * sizeof(float), cudaMemcpyHostToDevice, ctx->stream));
   return QDIT_OK;
 }
@@ -139,28 +150,33 @@ int32_t build_model(qdit_ctx* ctx, const qdit_model_desc* desc, qdit_model* m) {
   QDIT_TRY(upload(ctx, m->mem, desc->b_out, od, &m->b_out));
 
   const int wbits = s.weight_bits == 0 ? 8 : s.weight_bits;
+  // 4-bit codes are stored two per byte when every reduction length allows it (packed rows must be multiples of 16 bytes)
+  const bool packed4 = wbits == 4 && D % 32 == 0 && F % 32 == 0;
+  m->packed4 = packed4;
+  m->max_block_weight = (3 * D > F ? 3 * D : F) * D;
   const int64_t big = 6 * D > F ? 6 * D : F;
   float* staging = nullptr;
-  if (cudaMalloc(&staging, static_cast<size_t>(big) * (D > F ? D : F) * sizeof(float)) != cudaSuccess) {
+  if (cudaMalloc(&staging, static_cast<size_t>(big) * (D > F ? D : F) * (sizeof(float) + (packed4 ? 1 : 0))) != cudaSuccess) {
     cudaGetLastError();
     return qdit_fail(ctx, QDIT_ERR_NOMEM, "out of device memory (staging)");
   }
-  int32_t st = alloc_qlinear(ctx, m->mem, static_cast<int64_t>(s.depth) * 6 * D, D, &m->ada_all);
+  int8_t* codes8 = reinterpret_cast<int8_t*>(staging + static_cast<size_t>(big) * (D > F ? D : F));
+  int32_t st = alloc_qlinear(ctx, m->mem, static_cast<int64_t>(s.depth) * 6 * D, D, packed4, &m->ada_all);
   m->qkv.resize(s.depth);
   m->proj.resize(s.depth);
   m->fc1.resize(s.depth);
   m->fc2.resize(s.depth);
   for (int i = 0; i < s.depth && st == QDIT_OK; ++i) {
     const qdit_block_weights& b = desc->blocks[i];
-    if ((st = alloc_qlinear(ctx, m->mem, 3 * D, D, &m->qkv[i])) != QDIT_OK) break;
-    if ((st = alloc_qlinear(ctx, m->mem, D, D, &m->proj[i])) != QDIT_OK) break;
-    if ((st = alloc_qlinear(ctx, m->mem, F, D, &m->fc1[i])) != QDIT_OK) break;
-    if ((st = alloc_qlinear(ctx, m->mem, D, F, &m->fc2[i])) != QDIT_OK) break;
-    if ((st = quantize_into(ctx, staging, b.w_ada, b.b_ada, 6 * D, D, &m->ada_all, static_cast<int64_t>(i) * 6 * D, wbits)) != QDIT_OK) break;
-    if ((st = quantize_into(ctx, staging, b.w_qkv, b.b_qkv, 3 * D, D, &m->qkv[i], 0, wbits)) != QDIT_OK) break;
-    if ((st = quantize_into(ctx, staging, b.w_proj, b.b_proj, D, D, &m->proj[i], 0, wbits)) != QDIT_OK) break;
-    if ((st = quantize_into(ctx, staging, b.w_fc1, b.b_fc1, F, D, &m->fc1[i], 0, wbits)) != QDIT_OK) break;
-    if ((st = quantize_into(ctx, staging, b.w_fc2, b.b_fc2, D, F, &m->fc2[i], 0, wbits)) != QDIT_OK) break;
+    if ((st = alloc_qlinear(ctx, m->mem, 3 * D, D, packed4, &m->qkv[i])) != QDIT_OK) break;
+    if ((st = alloc_qlinear(ctx, m->mem, D, D, packed4, &m->proj[i])) != QDIT_OK) break;
+    if ((st = alloc_qlinear(ctx, m->mem, F, D, packed4, &m->fc1[i])) != QDIT_OK) break;
+    if ((st = alloc_qlinear(ctx, m->mem, D, F, packed4, &m->fc2[i])) != QDIT_OK) break;
+    if ((st = quantize_into(ctx, staging, codes8, b.w_ada, b.b_ada, 6 * D, D, &m->ada_all, static_cast<int64_t>(i) * 6 * D, wbits)) != QDIT_OK) break;
+    if ((st = quantize_into(ctx, staging, codes8, b.w_qkv, b.b_qkv, 3 * D, D, &m->qkv[i], 0, wbits)) != QDIT_OK) break;
+    if ((st = quantize_into(ctx, staging, codes8, b.w_proj, b.b_proj, D, D, &m->proj[i], 0, wbits)) != QDIT_OK) break;
+    if ((st = quantize_into(ctx, staging, codes8, b.w_fc1, b.b_fc1, F, D, &m->fc1[i], 0, wbits)) != QDIT_OK) break;
+    if ((st = quantize_into(ctx, staging, codes8, b.w_fc2, b.b_fc2, D, F, &m->fc2[i], 0, wbits)) != QDIT_OK) break;
   }
   if (st == QDIT_OK) {
     m->d_scales = m->mem.alloc<float>(m->n_scales());
@@ -178,11 +194,15 @@ int32_t build_model(qdit_ctx* ctx, const qdit_model_desc* desc, qdit_model* m) {
 qdit_qparams sym_qp() { return qdit_qparams{1.0f, 0, -127, 127}; }
 
 // One quantized linear of the fused (static-scale) path.
+// `w8_scratch`: for a layer stored packed, the matrix its weights are widened into when the layer has many rows
+// (NULL: always widened inside the GEMM kernel, which is the form for the weight-streaming modulation GEMM).
 int32_t run_linear(qdit_ctx* ctx, const void* A, const QLinearDev& l, int64_t M, const float* a_scale_dev, uint32_t flags,
-                   qdit_epilogue epi, void* out) {
+                   qdit_epilogue epi, void* out, void* w8_scratch = nullptr) {
   epi.w_scale = l.scale;
   epi.w_colsum = l.colsum;
   epi.bias = l.bias;
+  if (l.packed4)
+    return qdit_w4a8_linear(ctx, A, l.q, M, l.N, l.K, sym_qp(), a_scale_dev, flags | QDIT_EPI_BIAS, &epi, out, l.N, w8_scratch);
   return qdit_w8a8_linear(ctx, A, l.q, M, l.N, l.K, sym_qp(), a_scale_dev, flags | QDIT_EPI_BIAS, &epi, out, l.N);
 }
 
@@ -257,13 +277,13 @@ static int32_t forward_impl(qdit_ctx* ctx, qdit_sampler* s, const float* latent,
         } else {
           QDIT_TRY(qdit_adaln_modulate(ctx, s->x, M, D, T, 1e-6f, mod, mod + D, ld_mod, s->h, QDIT_I8, &qp, sc_qkv));
           qdit_epilogue e0{};
-          QDIT_TRY(run_linear(ctx, s->h, m->qkv[i], M, sc_qkv, QDIT_EPI_OUT_BF16, e0, s->qkv));
+          QDIT_TRY(run_linear(ctx, s->h, m->qkv[i], M, sc_qkv, QDIT_EPI_OUT_BF16, e0, s->qkv, s->w8_scratch));
           const __nv_bfloat16* qkv = static_cast<const __nv_bfloat16*>(s->qkv);
           QDIT_TRY(qdit_attention(ctx, qkv, qkv + D, qkv + 2 * D, 3 * D, B, sh.heads, T, D / sh.heads, att_scale, s->a,
                                   QDIT_I8, &qp, sc_proj));
           gated.gate = mod + 2 * D;
           gated.cache_out = store ? qdit_cache_slot(s->cache, i, QDIT_BRANCH_ATTN, 1) : nullptr;
-          QDIT_TRY(run_linear(ctx, s->a, m->proj[i], M, sc_proj, gflags, gated, s->x));
+          QDIT_TRY(run_linear(ctx, s->a, m->proj[i], M, sc_proj, gflags, gated, s->x, s->w8_scratch));
         }
         // ---- MLP branch
         if (mask && mask[2 * i + 1]) {
@@ -273,32 +293,32 @@ static int32_t forward_impl(qdit_ctx* ctx, qdit_sampler* s, const float* latent,
           qdit_epilogue e1{};
           e1.out_qp = qp;
           e1.out_scale_dev = sc_fc2;
-          QDIT_TRY(run_linear(ctx, s->h, m->fc1[i], M, sc_fc1, QDIT_EPI_GELU | QDIT_EPI_QUANT_OUT, e1, s->u));
+          QDIT_TRY(run_linear(ctx, s->h, m->fc1[i], M, sc_fc1, QDIT_EPI_GELU | QDIT_EPI_QUANT_OUT, e1, s->u, s->w8_scratch));
           gated.gate = mod + 5 * D;
           gated.cache_out = store ? qdit_cache_slot(s->cache, i, QDIT_BRANCH_MLP, 1) : nullptr;
-          QDIT_TRY(run_linear(ctx, s->u, m->fc2[i], M, sc_fc2, gflags, gated, s->x));
+          QDIT_TRY(run_linear(ctx, s->u, m->fc2[i], M, sc_fc2, gflags, gated, s->x, s->w8_scratch));
         }
       } else {
         // ---- calibration: every quantizer input is materialised in f32, its range reduced, then quantized
         QDIT_TRY(qdit_adaln_modulate(ctx, s->x, M, D, T, 1e-6f, mod, mod + D, ld_mod, s->tmpf, QDIT_F32, nullptr, nullptr));
         QDIT_TRY(dyn_quant(ctx, s, 1 + 4 * i, s->tmpf, M, D, s->h));
         qdit_epilogue e0{};
-        QDIT_TRY(run_linear(ctx, s->h, m->qkv[i], M, sc_qkv, QDIT_EPI_OUT_BF16, e0, s->qkv));
+        QDIT_TRY(run_linear(ctx, s->h, m->qkv[i], M, sc_qkv, QDIT_EPI_OUT_BF16, e0, s->qkv, s->w8_scratch));
         const __nv_bfloat16* qkv = static_cast<const __nv_bfloat16*>(s->qkv);
         QDIT_TRY(qdit_attention(ctx, qkv, qkv + D, qkv + 2 * D, 3 * D, B, sh.heads, T, D / sh.heads, att_scale, s->tmpf,
                                 QDIT_F32, nullptr, nullptr));
         QDIT_TRY(dyn_quant(ctx, s, 2 + 4 * i, s->tmpf, M, D, s->a));
         gated.gate = mod + 2 * D;
         gated.cache_out = store ? qdit_cache_slot(s->cache, i, QDIT_BRANCH_ATTN, 1) : nullptr;
-        QDIT_TRY(run_linear(ctx, s->a, m->proj[i], M, sc_proj, gflags, gated, s->x));
+        QDIT_TRY(run_linear(ctx, s->a, m->proj[i], M, sc_proj, gflags, gated, s->x, s->w8_scratch));
         QDIT_TRY(qdit_adaln_modulate(ctx, s->x, M, D, T, 1e-6f, mod + 3 * D, mod + 4 * D, ld_mod, s->tmpf, QDIT_F32, nullptr, nullptr));
         QDIT_TRY(dyn_quant(ctx, s, 3 + 4 * i, s->tmpf, M, D, s->h));
         qdit_epilogue e1{};
-        QDIT_TRY(run_linear(ctx, s->h, m->fc1[i], M, sc_fc1, QDIT_EPI_GELU | QDIT_EPI_OUT_F32, e1, s->tmpf));
+        QDIT_TRY(run_linear(ctx, s->h, m->fc1[i], M, sc_fc1, QDIT_EPI_GELU | QDIT_EPI_OUT_F32, e1, s->tmpf, s->w8_scratch));
         QDIT_TRY(dyn_quant(ctx, s, 4 + 4 * i, s->tmpf, M, F, s->u));
         gated.gate = mod + 5 * D;
         gated.cache_out = store ? qdit_cache_slot(s->cache, i, QDIT_BRANCH_MLP, 1) : nullptr;
-        QDIT_TRY(run_linear(ctx, s->u, m->fc2[i], M, sc_fc2, gflags, gated, s->x));
+        QDIT_TRY(run_linear(ctx, s->u, m->fc2[i], M, sc_fc2, gflags, gated, s->x, s->w8_scratch));
       }
     }
   }
@@ -408,6 +428,8 @@ int32_t qdit_model_finish_calibration(qdit_ctx* ctx, qdit_model* m) {
   return QDIT_OK;
 }
 
+int32_t qdit_model_weights_packed(const qdit_model* m) { return m && m->packed4 ? 1 : 0; }
+
 int32_t qdit_model_linear(qdit_model* m, int block, int which, const void** w_q, const float** w_scale,
                           const int32_t** w_colsum, const float** bias, int64_t* N, int64_t* K) {
   if (!m || block < 0 || block >= m->s.depth || which < 0 || which > 4) return QDIT_ERR_INVALID_ARG;
@@ -415,7 +437,7 @@ int32_t qdit_model_linear(qdit_model* m, int block, int which, const void** w_q,
   if (which == 0) {
     const int64_t D = m->s.hidden, r0 = static_cast<int64_t>(block) * 6 * D;
     l = m->ada_all;
-    l.q += r0 * D;
+    l.q += r0 * D / (l.packed4 ? 2 : 1);
     l.scale += r0;
     l.colsum += r0;
     l.bias += r0;
@@ -475,6 +497,7 @@ int32_t qdit_sampler_create(qdit_ctx* ctx, qdit_model* m, const qdit_sampler_des
   s->y = a.alloc<int32_t>(B);
   s->labels = a.alloc<int32_t>(d->batch);
   s->tmpf = a.alloc<float>(M * F);
+  s->w8_scratch = m->packed4 ? a.alloc<int8_t>(m->max_block_weight) : nullptr;
   s->dyn_absmax = a.alloc<float>(m->n_scales());
   s->dyn_scale = a.alloc<float>(m->n_scales());
   // conditioning of as many steps at once as a 4 GB modulation table holds (all of them for the paper's 50- and
@@ -503,7 +526,7 @@ int32_t qdit_sampler_create(qdit_ctx* ctx, qdit_model* m, const qdit_sampler_des
     }
   }
   bool ok = traj_ok && s->x && s->qkv && s->h && s->a && s->u && s->ca && s->c && s->sc && s->hidden && s->feat && s->mod && s->modf && s->net &&
-            s->latent && s->t_all && s->y && s->labels && s->tmpf && s->dyn_absmax && s->dyn_scale;
+            s->latent && s->t_all && s->y && s->labels && s->tmpf && s->dyn_absmax && s->dyn_scale && (!m->packed4 || s->w8_scratch);
   if (ok && d->vc_mode != QDIT_VC_NONE) {
     s->vc_table = a.alloc<float>(static_cast<int64_t>(d->num_steps) * C);
     ok = s->vc_table && cudaMemcpy(s->vc_table, d->vc_table, sizeof(float) * d->num_steps * C, cudaMemcpyHostToDevice) == cudaSuccess;

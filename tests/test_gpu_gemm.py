@@ -374,3 +374,85 @@ def test_options_select_kernels_and_reject_bad_values(q, ctx):
     finally:
         q.qdit_set_option(ctx, q.QDIT_OPT_PDL, 1)
     np.testing.assert_array_equal(a, b)
+
+
+# ----------------------------------------------------------------------------- packed 4-bit weights (W4A8, Table 2)
+def _w4_codes(seed, name, N, K):
+    return synth.uniform_int(seed, name, (N, K), -8, 8).astype(np.int64)
+
+
+def test_w4_pack_unpack_match_the_oracle_bytes(q, ctx):
+    N, K = 200, 1152
+    codes = _w4_codes(51, "w4", N, K)
+    codes[0, :4] = [-8, 7, -1, 0]
+    w8 = dev_i8(codes)
+    packed = torch.zeros((N, K // 2), dtype=torch.uint8, device="cuda")
+    q.qdit_pack_weight_int4(ctx, w8, N, K, packed)
+    q.qdit_sync(ctx)
+    np.testing.assert_array_equal(packed.cpu().numpy(), quant.pack_int4(codes))
+    back = torch.zeros((N, K), dtype=torch.uint8, device="cuda")
+    q.qdit_unpack_weight_int4(ctx, packed, N, K, back)
+    q.qdit_sync(ctx)
+    np.testing.assert_array_equal(host_codes(back), codes)
+    np.testing.assert_array_equal(host_codes(back), quant.unpack_int4(quant.pack_int4(codes)))
+    # a code outside [-8, 7] cannot be stored
+    bad = codes.copy()
+    bad[3, 5] = 9
+    assert q.lib.qdit_pack_weight_int4(ctx, dev_i8(bad).data_ptr(), N, K, packed.data_ptr()) == q.QDIT_ERR_INVALID_ARG
+    assert q.lib.qdit_pack_weight_int4(ctx, w8.data_ptr(), N, 24, packed.data_ptr()) == q.QDIT_ERR_SHAPE
+
+
+@pytest.mark.parametrize("M,N,K", [(64, 392, 1152), (1152, 1152, 1152), (300, 6912, 384), (2048, 256, 4608)])
+@pytest.mark.parametrize("scratch", [False, True])
+def test_w4a8_accumulators_bit_exact_and_stage_equals_the_codes(q, ctx, M, N, K, scratch):
+    """The weight tile the tensor core reads must be the oracle's codes exactly: raw int32 accumulators on random
+    activations equal the oracle's integer product, and one-hot activations (row m selects column m of W) return the
+    widened codes themselves.  Both forms: widened inside the GEMM kernel, and widened into a scratch matrix first."""
+    codes = _w4_codes(52, f"w4.{N}.{K}", N, K)
+    packed = torch.from_numpy(quant.pack_int4(codes)).cuda()
+    w8s = torch.empty((N, K), dtype=torch.uint8, device="cuda") if scratch else None
+    qa = _codes(52, f"a4.{M}.{K}", (M, K), -128, 127)
+    out = torch.empty((M, N), dtype=torch.int32, device="cuda")
+    q.qdit_w4a8_linear(ctx, dev_i8(qa), packed, M, N, K, q.qparams(1.0), None, q.QDIT_EPI_OUT_I32, None, out, N, w8s)
+    q.qdit_sync(ctx)
+    np.testing.assert_array_equal(out.cpu().numpy().astype(np.int64), linear.gemm_i8(qa, codes))
+    Ms = min(M, K)
+    onehot = np.zeros((Ms, K), dtype=np.int64)
+    ks = synth.uniform_int(52, f"ks{K}", (Ms,), 0, K)
+    onehot[np.arange(Ms), ks] = 1
+    out1 = torch.empty((Ms, N), dtype=torch.int32, device="cuda")
+    q.qdit_w4a8_linear(ctx, dev_i8(onehot), packed, Ms, N, K, q.qparams(1.0), None, q.QDIT_EPI_OUT_I32, None, out1, N, w8s)
+    q.qdit_sync(ctx)
+    np.testing.assert_array_equal(out1.cpu().numpy(), quant.unpack_int4(quant.pack_int4(codes))[:, ks].T)
+
+
+@pytest.mark.parametrize("M,T", [(512, 256), (96, 32)])
+def test_w4a8_epilogues_equal_w8a8_on_the_same_codes(q, ctx, M, T):
+    """Same codes, same arithmetic after the accumulator: the packed layer and the one-code-per-byte layer give the
+    same bits for the f32, the GELU + re-quantised and the gated epilogue; and the f32 output matches the oracle."""
+    N, K = 1152, 1152
+    a_qp = QParams(0.05, 0, -127, 127)
+    L = _layer(53, M, N, K, T, a_qp)
+    Wf = synth.normal(53, "W", (N, K), 0.02)
+    codes, s_w, cs = quant.quantize_weight_per_channel(Wf, bits=4)
+    A = dev_i8(L["qa"])
+    W8, W4 = dev_i8(codes), torch.from_numpy(quant.pack_int4(codes)).cuda()
+    ws, bi, g = dev(s_w), dev(L["bias"]), dev(L["gate"])
+    ref = linear.w8a8_linear(L["qa"], a_qp, codes, s_w, cs, L["bias"])
+    outs = {}
+    for name, fn, W in (("w8", q.qdit_w8a8_linear, W8), ("w4", q.qdit_w4a8_linear, W4)):
+        of = torch.empty((M, N), dtype=torch.float32, device="cuda")
+        fn(ctx, A, W, M, N, K, q.qparams(a_qp.scale), None, q.QDIT_EPI_BIAS | q.QDIT_EPI_OUT_F32, q.epilogue(w_scale=ws, bias=bi), of, N)
+        oq = torch.empty((M, N), dtype=torch.uint8, device="cuda")
+        fn(ctx, A, W, M, N, K, q.qparams(a_qp.scale), None, q.QDIT_EPI_BIAS | q.QDIT_EPI_GELU | q.QDIT_EPI_QUANT_OUT,
+           q.epilogue(w_scale=ws, bias=bi, out_qp=q.qparams(0.01)), oq, N)
+        x = dev(L["resid"]).to(torch.bfloat16)
+        cache = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+        fn(ctx, A, W, M, N, K, q.qparams(a_qp.scale), None,
+           q.QDIT_EPI_BIAS | q.QDIT_EPI_GATE | q.QDIT_EPI_RESIDUAL | q.QDIT_EPI_CACHE_STORE | q.QDIT_EPI_OUT_BF16,
+           q.epilogue(w_scale=ws, bias=bi, gate=g, ld_gate=N, tokens_per_sample=T, residual=x, cache_out=cache), x, N)
+        q.qdit_sync(ctx)
+        outs[name] = (of.cpu().numpy(), oq.cpu().numpy(), x.float().cpu().numpy(), cache.float().cpu().numpy())
+    assert max_rel_err(outs["w4"][0], ref) < 1e-5
+    for a, b in zip(outs["w4"], outs["w8"]):
+        np.testing.assert_array_equal(a, b)

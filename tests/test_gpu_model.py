@@ -209,10 +209,44 @@ def test_forward_tiny_w4a8_matches_oracle(q, ctx):
             rig8.close()
         d = rel_l2(got, got8)
         assert 1e-3 < d < 0.5, d
-        # ... whose weight codes stay inside the 4-bit range
+        # ... whose weight codes stay inside the 4-bit range (this width, 144, is not a multiple of 32: one code per byte)
+        assert q.qdit_model_weights_packed(rig.gm) == 0
         lin = q.qdit_model_linear(rig.gm, 0, LINEAR_IDS["fc1"])
         codes = host_codes(view(lin["w_q"], (lin["N"], lin["K"]), "|i1"))
         assert codes.min() >= -7 and codes.max() <= 7 and np.abs(codes).max() == 7
+    finally:
+        rig.close()
+
+
+def test_forward_w4a8_packed_weights_match_oracle(q, ctx):
+    """W4A8 with the weights stored two codes per byte (widths that are multiples of 32): the stored bytes are the
+    oracle's packed codes, and the network evaluation on them matches the oracle (few rows: widened inside the GEMM
+    kernel; 512 rows per block layer here)."""
+    cfg = synth.DiTConfig(hidden=384, heads=6, mlp=1536, depth=2, grid=16)
+    rig = Rig(q, ctx, cfg, 75, weight_bits=4)
+    try:
+        assert q.qdit_model_weights_packed(rig.gm) == 1
+        for i, blk in enumerate(rig.om.blocks):
+            for name, wid in LINEAR_IDS.items():
+                L = q.qdit_model_linear(rig.gm, i, wid)
+                lin = getattr(blk, name)
+                got = view(L["w_q"], (L["N"], L["K"] // 2), "|u1").cpu().numpy()
+                np.testing.assert_array_equal(got, quant.pack_int4(lin.q.astype(np.int32)))
+        latent, t, y = _inputs(cfg, 75, 2)
+        scales = calib.calibrate_model(rig.om, [(latent, t, y)])
+        rig.set_scales(scales)
+        got = rig.forward(rig.sampler(batch=2, num_steps=2), latent, t, y)
+        ref = dit.forward(rig.om, dit.Context(quant="static", scales=scales), latent, t, y)
+        assert rel_l2(got, ref) < 5e-3, rel_l2(got, ref)
+        # many rows (8 images x 256 tokens = 2048 per block layer): the weights are widened into the scratch matrix
+        # and the W8A8 kernels run; each image's result is what the few-row path gives for it alone
+        lat8, t8, y8 = _inputs(cfg, 79, 8)
+        s8 = rig.sampler(batch=8, num_steps=2)
+        got8 = rig.forward(s8, lat8, t8, y8)
+        got1 = rig.forward(s8, lat8[3:4], t8[3:4], y8[3:4])
+        assert rel_l2(got8[3:4], got1) < 1e-6
+        ref8 = dit.forward(rig.om, dit.Context(quant="static", scales=scales), lat8[3:4], t8[3:4], y8[3:4])
+        assert rel_l2(got8[3:4], ref8) < 5e-3
     finally:
         rig.close()
 
