@@ -500,6 +500,56 @@ def run_gemm_sweep(args):
                       "rows": rows}))
 
 
+def run_w4_sweep(args):
+    """Packed 4-bit weights against one code per byte on the weight-streaming shapes: the stacked modulation GEMM of a
+    50-step trajectory (M = 1600, N = 28 x 6912, K = 1152) and the four block layers at M = 256 and 1024.  The W4A8
+    rows widen the weights inside the GEMM kernel (no scratch matrix)."""
+    import torch
+    import paper_2503_02508_b200 as q
+    seed = synth.CONFIG_SEEDS["gemm_sweep"]
+    peaks = measured_peaks()
+    ctx = q.qdit_create(0, None)
+    shapes = [(1600, 28 * 6912, 1152, "modulation (all blocks, 50 steps)")]
+    for M in (256, 1024):
+        shapes += [(M, N, K, name) for K, N, name in GEMM_SHAPES]
+    rows = []
+    for M, N, K, name in shapes:
+        codes = synth.uniform_int(seed, f"w4.{N}.{K}", (N, K), -7, 8).astype(np.int8)
+        w8 = torch.from_numpy(codes).cuda()
+        w4 = torch.empty((N, K // 2), dtype=torch.uint8, device="cuda")
+        q.qdit_pack_weight_int4(ctx, w8, N, K, w4)
+        a8 = torch.from_numpy(synth.uniform_int(seed, f"a.{M}.{K}", (M, K), -127, 128).astype(np.int8)).cuda()
+        ws = torch.from_numpy(np.abs(synth.normal(seed, f"ws{N}", (N,), 1e-3)) + 1e-4).cuda()
+        bias = torch.from_numpy(synth.normal(seed, f"b{N}", (N,), 0.02)).cuda()
+        out = torch.empty((M, N), dtype=torch.float32, device="cuda")
+        epi = q.epilogue(w_scale=ws, bias=bias)
+        flags = q.QDIT_EPI_BIAS | q.QDIT_EPI_OUT_F32
+        qp = q.qparams(0.03)
+
+        def t(fn):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(args.steps):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / args.steps
+
+        ms8 = t(lambda: q.qdit_w8a8_linear(ctx, a8, w8, M, N, K, qp, None, flags, epi, out, N))
+        ms4 = t(lambda: q.qdit_w4a8_linear(ctx, a8, w4, M, N, K, qp, None, flags, epi, out, N, None))
+        rows.append({"layer": name, "M": M, "N": N, "K": K, "w8a8_us": round(ms8 * 1e3, 1), "w4a8_us": round(ms4 * 1e3, 1),
+                     "speedup": round(ms8 / ms4, 3), "weight_mb_w8": round(N * K / 1e6, 1), "weight_mb_w4": round(N * K / 2e6, 1),
+                     "w4_weight_gbs": round(N * K / 2 / ms4 / 1e6, 0)})
+    q.qdit_destroy(ctx)
+    print(json.dumps({"metric": "W4A8 (packed) vs W8A8 linear layer time on weight-streaming shapes", "value": rows[0]["speedup"],
+                      "unit": "x (modulation GEMM)", "n_gpus": 1, "steps": args.steps, "warmup": 3, "higher_is_better": True,
+                      "dtype": "int8", "data": "synthetic", "config": {"workload": "w4_sweep", "output": "f32 + bias"},
+                      "hbm_gbs": peaks["hbm_gbs"], "rows": rows}))
+
+
 def compact_sweep(rows, clock_info, peaks):
     """The second half of the metric for the default bench line: per layer and M the GEMM rate and its fractions of
     2 x burst bf16 (measured) and of the nominal 4500 TOP/s; the memory-bound kernels as fractions of the measured HBM
@@ -529,7 +579,7 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="ddim50", choices=sorted(WORKLOADS) + ["gemm_sweep"])
+    ap.add_argument("--workload", default="ddim50", choices=sorted(WORKLOADS) + ["gemm_sweep", "w4_sweep"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-layer sweep that follows the timed region")
     ap.add_argument("--weight-bits", type=int, default=8, help="code width of the quantized weights (4 = the paper's W4A8 setting)")
@@ -540,6 +590,8 @@ def main():
     args = ap.parse_args()
     if args.workload == "gemm_sweep":
         run_gemm_sweep(args)
+    elif args.workload == "w4_sweep":
+        run_w4_sweep(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

@@ -180,7 +180,7 @@ __device__ __forceinline__ void prefetch_chunk(const GemmParams& p, int n, int r
 // stage back to the MMA issuer once this warp has read its share.  `stg` = this warp's 4 KB staging patch.
 // The epilogue is bound by the latency chain of one chunk (global loads, TMEM load, transpose, stores), so
 // the tile's chunks are spread over as many warps as the register file allows.
-template <int BN, int EPI, typename Release>
+template <int BN, int EPI, int SPLIT = EPI_SPLIT, typename Release>
 __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t tacc, int m0, int n0, int quad, int half,
                                               uint32_t stg, int lane, float a_scale, float o_inv, Release release) {
   const int cg = lane & 3;     // after the transpose: column group (8 columns) ...
@@ -188,8 +188,8 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t tacc
   const uint32_t flags = epi_flags<EPI>(p);
   const bool gate_uniform = (p.tokens % 32) == 0;  // the warp's 32 rows then belong to one sample
   constexpr int CHUNKS = BN / 32;
-  // this warp takes chunks half, half + EPI_SPLIT, ...; c_last = the last of them (-1: none)
-  const int c_last = half < CHUNKS ? half + ((CHUNKS - 1 - half) / EPI_SPLIT) * EPI_SPLIT : -1;
+  // this warp takes chunks half, half + SPLIT, ... (SPLIT = epilogue warps per lane quadrant); c_last = the last of them (-1: none)
+  const int c_last = half < CHUNKS ? half + ((CHUNKS - 1 - half) / SPLIT) * SPLIT : -1;
   if (c_last < 0) {  // nothing to read: hand the accumulator stage back untouched
     tc_fence_before();
     __syncwarp();
@@ -201,7 +201,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmParams& p, uint32_t tacc
 
   // plain order per chunk: global loads -> TMEM load -> transpose -> math and stores
 #pragma unroll 1
-  for (int c = half; c < CHUNKS; c += EPI_SPLIT) {
+  for (int c = half; c < CHUNKS; c += SPLIT) {
     const int n = n0 + c * 32 + cg * 8;
     const bool col_ok = n < p.N;
     const uint32_t patch = stg;

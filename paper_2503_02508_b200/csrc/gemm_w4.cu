@@ -5,10 +5,10 @@
 // right in front of the tensor core: the same tcgen05 kind::i8 main loop, TMEM accumulators and fused epilogue as
 // gemm_i8.cu (token-major, 128 x 128 tiles), with one more role.
 //   warp 0 lane 0   TMA producer: activation tile (128 x 128 B, 128B swizzle) and PACKED weight tile (128 x 64 B)
-//   warps 2..3      unpackers: nibbles -> sign-extended bytes, written into the weight stage in the 128B-swizzled
+//   warps 2..5      unpackers: nibbles -> sign-extended bytes, written into the weight stage in the 128B-swizzled
 //                   K-major layout the MMA descriptor expects; fence.proxy.async; arrive on ready[stage]
 //   warp 1 lane 0   MMA issuer: waits for ready[stage] instead of the TMA barrier
-//   warps 4..15     epilogue (shared with gemm_i8.cu)
+//   warps 6..13     epilogue (the fused epilogue of gemm_i8.cu, two warps per lane quadrant)
 // This is the form for weight-streaming shapes (few rows: the stacked modulation GEMM, small batches), where the
 // weight bytes are what bounds the layer.  Layers with thousands of rows are bound by the tensor core and their
 // epilogue instead; for them qdit_w4a8_linear widens the weights into a caller-provided scratch matrix first
@@ -20,8 +20,10 @@ namespace {
 using namespace qgemm;
 
 constexpr int W4_BN = 128;
-constexpr int W4_UNPACK_WARPS = 2;
-constexpr int W4_THREADS = 64 + W4_UNPACK_WARPS * 32 + NUM_EPI_WARPS * 32;
+constexpr int W4_UNPACK_WARPS = 4;   // measured: two warps take 0.36 us per 128 x 128 weight stage, more than the loads and the MMAs
+constexpr int W4_EPI_WARPS = 8;
+constexpr int W4_THREADS = 64 + W4_UNPACK_WARPS * 32 + W4_EPI_WARPS * 32;
+constexpr int W4_STAGING_BYTES = W4_EPI_WARPS * 32 * 128;
 
 struct W4Cfg {
   static constexpr int A_BYTES = BM * BK;
@@ -30,18 +32,20 @@ struct W4Cfg {
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + P_BYTES;
   static constexpr int BAR_BYTES = 512;
   static constexpr int SMEM_LIMIT = 232448;
-  static constexpr int STAGES_FIT = (SMEM_LIMIT - 1024 - BAR_BYTES - STAGING_BYTES) / STAGE_BYTES;
+  static constexpr int STAGES_FIT = (SMEM_LIMIT - 1024 - BAR_BYTES - W4_STAGING_BYTES) / STAGE_BYTES;
   static constexpr int STAGES = STAGES_FIT > 6 ? 6 : STAGES_FIT;
   static constexpr int TMEM_COLS = 256;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + BAR_BYTES + 1024;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + W4_STAGING_BYTES + BAR_BYTES + 1024;
 };
 
 // 8 packed bytes (16 codes) -> 16 sign-extended bytes.
 __device__ __forceinline__ uint4 widen16(uint2 pk) {
   auto widen = [](uint32_t w, uint32_t& lo4, uint32_t& hi4) {
-    // even codes sit in the low nibbles, odd codes in the high nibbles; (x ^ 8) - 8 sign-extends a nibble in its byte
-    const uint32_t e = __vsub4((w & 0x0F0F0F0Fu) ^ 0x08080808u, 0x08080808u);
-    const uint32_t o = __vsub4(((w >> 4) & 0x0F0F0F0Fu) ^ 0x08080808u, 0x08080808u);
+    // even codes sit in the low nibbles, odd codes in the high nibbles.  Sign extension of a nibble x inside its byte:
+    // x + 0x1E * (x & 8) sets bits 4..7 exactly when bit 3 is set (8 * 0x1E = 0xF0, no carry into the next byte)
+    uint32_t e = w & 0x0F0F0F0Fu, o = (w >> 4) & 0x0F0F0F0Fu;
+    e = (e & 0x08080808u) * 0x1Eu + e;
+    o = (o & 0x08080808u) * 0x1Eu + o;
     lo4 = __byte_perm(e, o, 0x5140);  // codes 0, 1, 2, 3 of the word
     hi4 = __byte_perm(e, o, 0x7362);  // codes 4, 5, 6, 7
   };
@@ -64,7 +68,7 @@ gemm_w4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   uint8_t* sB = sA + STAGES * C::A_BYTES;
   uint8_t* sP = sB + STAGES * C::B_BYTES;
   uint8_t* staging = sP + STAGES * C::P_BYTES;
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(staging + STAGING_BYTES);   // activation + packed weight tiles landed (tx)
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(staging + W4_STAGING_BYTES);   // activation + packed weight tiles landed (tx)
   uint64_t* ready_bar = full_bar + STAGES;                                      // weight tile widened (one arrival per unpack warp)
   uint64_t* empty_bar = ready_bar + STAGES;                                     // the MMAs have read the stage (commit)
   uint64_t* tfull_bar = empty_bar + STAGES;
@@ -83,7 +87,7 @@ gemm_w4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&tfull_bar[s], 1);
-      mbar_init(&tempty_bar[s], NUM_EPI_WARPS);
+      mbar_init(&tempty_bar[s], W4_EPI_WARPS);
     }
     *abort_flag = 0;
     mbar_fence_init();
@@ -168,12 +172,18 @@ gemm_w4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         if (!mbar_wait(&full_bar[stage], phase, abort_flag, p.status)) { ok = false; break; }
         const uint8_t* src = sP + stage * C::P_BYTES;
         uint8_t* dst = sB + stage * C::B_BYTES;
-#pragma unroll 4
-        for (int i = ut; i < BN * 8; i += W4_UNPACK_WARPS * 32) {
-          const int n = i >> 3, c = i & 7;
-          const uint2 pk = *reinterpret_cast<const uint2*>(src + n * 64 + c * 8);
-          *reinterpret_cast<uint4*>(dst + n * 128 + ((c ^ (n & 7)) << 4)) = widen16(pk);
-        }
+        // a thread's pieces: i = ut + 64 j, j = 0..15: row (ut >> 3) + 8 j, piece ut & 7 (the row's low three bits, and
+        // with them the swizzle term, do not depend on j).  All loads are issued before the first store.
+        constexpr int PER_THREAD = BN * 8 / (W4_UNPACK_WARPS * 32);
+        const int n_first = ut >> 3, c = ut & 7;
+        const uint8_t* s0 = src + n_first * 64 + c * 8;
+        uint8_t* d0 = dst + n_first * 128 + ((c ^ (n_first & 7)) << 4);
+        constexpr int ROW_STEP = W4_UNPACK_WARPS * 32 / 8;   // rows between a thread's consecutive pieces (a multiple of 8)
+        uint2 pk[PER_THREAD];
+#pragma unroll
+        for (int j = 0; j < PER_THREAD; ++j) pk[j] = *reinterpret_cast<const uint2*>(s0 + j * ROW_STEP * 64);
+#pragma unroll
+        for (int j = 0; j < PER_THREAD; ++j) *reinterpret_cast<uint4*>(d0 + j * ROW_STEP * 128) = widen16(pk[j]);
         fence_async_smem();   // the tensor core reads the stage through the async proxy
         __syncwarp();
         if (lane == 0) mbar_arrive(&ready_bar[stage]);
@@ -199,7 +209,7 @@ gemm_w4_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       __syncwarp();
       tc_fence_after();
       uint64_t* release_bar = &tempty_bar[as];
-      epilogue_tile<BN, EPI>(p, tmem_base + static_cast<uint32_t>(as * BN), m0, n0, quad, half, stg, lane, a_scale, o_inv,
+      epilogue_tile<BN, EPI, W4_EPI_WARPS / 4>(p, tmem_base + static_cast<uint32_t>(as * BN), m0, n0, quad, half, stg, lane, a_scale, o_inv,
                              [release_bar]() { mbar_arrive_relaxed(release_bar); });
     }
   }

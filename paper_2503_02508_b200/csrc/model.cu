@@ -153,7 +153,7 @@ int32_t build_model(qdit_ctx* ctx, const qdit_model_desc* desc, qdit_model* m) {
   // 4-bit codes are stored two per byte when every reduction length allows it (packed rows must be multiples of 16 bytes)
   const bool packed4 = wbits == 4 && D % 32 == 0 && F % 32 == 0;
   m->packed4 = packed4;
-  m->max_block_weight = (3 * D > F ? 3 * D : F) * D;
+  m->max_block_weight = (6 * D > F ? 6 * D : F) * D;   // the modulation linear of one block is the largest (6D x D) unless mlp > 6D
   const int64_t big = 6 * D > F ? 6 * D : F;
   float* staging = nullptr;
   if (cudaMalloc(&staging, static_cast<size_t>(big) * (D > F ? D : F) * (sizeof(float) + (packed4 ? 1 : 0))) != cudaSuccess) {
@@ -206,6 +206,25 @@ int32_t run_linear(qdit_ctx* ctx, const void* A, const QLinearDev& l, int64_t M,
   return qdit_w8a8_linear(ctx, A, l.q, M, l.N, l.K, sym_qp(), a_scale_dev, flags | QDIT_EPI_BIAS, &epi, out, l.N);
 }
 
+// The modulation linears of all blocks on `rows` conditioning rows: out[rows, depth * 6D].  One stacked GEMM; with
+// packed 4-bit weights and many rows (the whole trajectory's conditioning) block by block instead, each block's
+// 6D x D weights widened into the scratch matrix first (the stacked matrix would need a scratch of its own size).
+int32_t run_modulation(qdit_ctx* ctx, const qdit_model* m, const void* A, int64_t rows, const float* a_scale_dev, float* out,
+                       void* w8_scratch) {
+  qdit_epilogue epi{};
+  if (!(m->ada_all.packed4 && w8_scratch && rows >= 1024)) return run_linear(ctx, A, m->ada_all, rows, a_scale_dev, QDIT_EPI_OUT_F32, epi, out);
+  const int64_t D = m->s.hidden, n6 = 6 * D, ld = static_cast<int64_t>(m->s.depth) * n6;
+  for (int i = 0; i < m->s.depth; ++i) {
+    const int64_t r0 = i * n6;
+    epi.w_scale = m->ada_all.scale + r0;
+    epi.w_colsum = m->ada_all.colsum + r0;
+    epi.bias = m->ada_all.bias + r0;
+    QDIT_TRY(qdit_w4a8_linear(ctx, A, m->ada_all.q + r0 * D / 2, rows, n6, D, sym_qp(), a_scale_dev, QDIT_EPI_BIAS | QDIT_EPI_OUT_F32,
+                              &epi, out + r0, ld, w8_scratch));
+  }
+  return QDIT_OK;
+}
+
 // Calibration helper: range of an f32 tensor -> this pass's scale slot (and the running range), then codes.
 int32_t dyn_quant(qdit_ctx* ctx, qdit_sampler* s, int slot, const float* x, int64_t M, int64_t K, uint8_t* q) {
   QDIT_CUDA_CHECK(ctx, cudaMemsetAsync(s->dyn_absmax + slot, 0, sizeof(float), ctx->stream));
@@ -249,8 +268,7 @@ static int32_t forward_impl(qdit_ctx* ctx, qdit_sampler* s, const float* latent,
     } else {
       QDIT_TRY(qdit_quantize_act_dev(ctx, s->sc, B, D, sym_qp(), scales + 0, s->ca));
     }
-    qdit_epilogue epi{};
-    QDIT_TRY(run_linear(ctx, s->ca, m->ada_all, B, scales + 0, QDIT_EPI_OUT_F32, epi, s->mod));
+    QDIT_TRY(run_modulation(ctx, m, s->ca, B, scales + 0, s->mod, s->w8_scratch));
     mod_all = s->mod;
   }
 
@@ -343,8 +361,7 @@ static int32_t trajectory_conditioning(qdit_ctx* ctx, qdit_sampler* s, int first
   QDIT_TRY(launch_batched_linear(ctx, s->traj_hidden, m->w_t2, m->b_t2, m->y_table, s->y, s->traj_c, s->traj_sc, rows, D, D, 0, 0,
                                  s->Beff));
   QDIT_TRY(qdit_quantize_act_dev(ctx, s->traj_sc, rows, D, sym_qp(), m->d_scales + 0, s->traj_ca));
-  qdit_epilogue epi{};
-  QDIT_TRY(run_linear(ctx, s->traj_ca, m->ada_all, rows, m->d_scales + 0, QDIT_EPI_OUT_F32, epi, s->traj_mod));
+  QDIT_TRY(run_modulation(ctx, m, s->traj_ca, rows, m->d_scales + 0, s->traj_mod, s->w8_scratch));
   return launch_batched_linear(ctx, s->traj_c, m->w_ada_f, m->b_ada_f, nullptr, nullptr, s->traj_modf, nullptr, rows, 2 * D, D, 1, 0, 0);
 }
 
