@@ -297,10 +297,38 @@ int32_t qdit_vc_fit(qdit_ctx* ctx, const float* x_hat, const float* x_target, in
  *   A = alpha A_spatial + (1 - alpha) A_temporal,   L = D^e A D^e,  D = diag(row sums of A)
  * (A is symmetric, so the paper's row and column degree matrices coincide; the paper prints e = +1/2, the usual
  * normalised adjacency is e = -1/2: `exponent` selects).  L: device f32 [n,n].  workspace: device f32, n*d + 2n
- * floats, overwritten.  n % 4 == 0, d % 16 == 0.  Eigenvectors, k-means and the aggregation over subsamples are
- * left to the host. */
+ * floats, overwritten.  n % 4 == 0, d % 16 == 0. */
 int32_t qdit_tap_laplacian(qdit_ctx* ctx, const float* x, const float* t, int n, int d, float alpha, float exponent,
                            float* workspace, float* L);
+/* Spectral step of Algorithm 1 for the m subsamples as one batch: for each subsample the matrix L above, its top k
+ * eigenvectors (largest eigenvalues; L is symmetric positive semi-definite when the degrees are positive) and
+ * k-means on the rows of the n x k eigenvector matrix.  x [m, n, d], t [m, n] (device f32).
+ *   eigvals [m, k] descending, eigvecs [m, n, k] (column j = eigenvector j, unit length; its sign and, inside a
+ *   repeated eigenvalue, its rotation are arbitrary), labels [m, n] int32 in [0, k).
+ * Eigenvectors by orthogonal iteration on a block of k + 8 vectors (power_iters multiplications by L, each followed by
+ * re-orthonormalisation) and a Rayleigh-Ritz step; the gap between eigenvalue k and k + 9 sets how many iterations
+ * are needed.  k-means: Lloyd's iterations (at most kmeans_iters, stops when no label changes) from the
+ * farthest-point start: centre 0 = row 0, each further centre = the row farthest from the centres so far (ties to
+ * the lowest index); nearest centre with ties to the lowest centre; an emptied cluster keeps its centre.  (The
+ * paper fixes none of these details.)  n % 16 == 0, d % 16 == 0, k + 8 <= min(n, 128), n <= 8192.
+ * workspace: device f32, qdit_tap_cluster_workspace(m, n, d, k) floats, overwritten. */
+int64_t qdit_tap_cluster_workspace(int m, int n, int d, int k);
+int32_t qdit_tap_cluster(qdit_ctx* ctx, const float* x, const float* t, int m, int n, int d, float alpha, float exponent,
+                         int k, int power_iters, int kmeans_iters, float* workspace, float* eigvals, float* eigvecs,
+                         int32_t* labels);
+/* Last step of Algorithm 1, "aggregate cluster assignments from all subsamples" (the paper does not say how; this is
+ * the reading taken): every cluster of a subsample is summarised by the mean of its members' unit-length features
+ * and the mean of their timestamps; the clusters of subsamples 2..m are matched one-to-one to those of subsample 1,
+ * greedily by the similarity alpha cos + (1 - alpha) exp(-|dt|) of the summaries (largest remaining entry first);
+ * matched summaries are averaged with the cluster sizes as weights; every sample of the whole dataset
+ * (x_all [N, d], t_all [N]) is assigned to the aggregated cluster it is most similar to (ties to the lowest).
+ * labels [m, n] as written by qdit_tap_cluster.  Outputs: labels_all [N] int32, centroids [k, d], tau [k] (device).
+ * The matching of the m k summaries runs on the host inside this call (it synchronises the stream twice).
+ * d % 16 == 0, k % 4 == 0.  workspace: device f32, qdit_tap_aggregate_workspace(m, n, d, k, N) floats. */
+int64_t qdit_tap_aggregate_workspace(int m, int n, int d, int k, int64_t N);
+int32_t qdit_tap_aggregate(qdit_ctx* ctx, const float* x, const float* t, const int32_t* labels, int m, int n, int d, int k,
+                           float alpha, const float* x_all, const float* t_all, int64_t N, float* workspace,
+                           int32_t* labels_all, float* centroids, float* tau);
 
 /* ------------------------------------------------------------------------------------------------
  * Whole model and sampler.  The DiT architecture (adaLN-Zero blocks, patch 2, learned-sigma output)

@@ -96,6 +96,10 @@ _SIGNATURES = {
     "qdit_selftest_wait_timeout": (_i32, [_vp, C.c_uint32, _vp]),
     "qdit_vc_correct": (_i32, [_vp, _vp, _int, _int, _int, _int, _int, _vp, _f32]),
     "qdit_tap_laplacian": (_i32, [_vp, _vp, _vp, _int, _int, _f32, _f32, _vp, _vp]),
+    "qdit_tap_cluster_workspace": (_i64, [_int, _int, _int, _int]),
+    "qdit_tap_cluster": (_i32, [_vp, _vp, _vp, _int, _int, _int, _f32, _f32, _int, _int, _int, _vp, _vp, _vp, _vp]),
+    "qdit_tap_aggregate_workspace": (_i64, [_int, _int, _int, _int, _i64]),
+    "qdit_tap_aggregate": (_i32, [_vp, _vp, _vp, _vp, _int, _int, _int, _int, _f32, _vp, _vp, _i64, _vp, _vp, _vp, _vp]),
     "qdit_vc_fit": (_i32, [_vp, _vp, _vp, _int, _int, _int, _f32, _int, _vp, _vp]),
     "qdit_model_create": (_i32, [_vp, C.POINTER(qdit_model_desc), C.POINTER(_vp)]),
     "qdit_model_destroy": (_i32, [_vp]),
@@ -305,6 +309,24 @@ def qdit_selftest_wait_timeout(ctx, polls, observed):
 
 def qdit_vc_correct(ctx, latent, B, Cc, HW, step_index, mode, table, eps):
     return check(ctx, lib.qdit_vc_correct(ctx, ptr(latent), B, Cc, HW, step_index, mode, ptr(table), eps))
+
+
+def qdit_tap_cluster_workspace(m, n, d, k):
+    return lib.qdit_tap_cluster_workspace(m, n, d, k)
+
+
+def qdit_tap_cluster(ctx, x, t, m, n, d, alpha, exponent, k, power_iters, kmeans_iters, workspace, eigvals, eigvecs, labels):
+    return check(ctx, lib.qdit_tap_cluster(ctx, ptr(x), ptr(t), m, n, d, alpha, exponent, k, power_iters, kmeans_iters,
+                                           ptr(workspace), ptr(eigvals), ptr(eigvecs), ptr(labels)))
+
+
+def qdit_tap_aggregate_workspace(m, n, d, k, N):
+    return lib.qdit_tap_aggregate_workspace(m, n, d, k, N)
+
+
+def qdit_tap_aggregate(ctx, x, t, labels, m, n, d, k, alpha, x_all, t_all, N, workspace, labels_all, centroids, tau):
+    return check(ctx, lib.qdit_tap_aggregate(ctx, ptr(x), ptr(t), ptr(labels), m, n, d, k, alpha, ptr(x_all), ptr(t_all), N,
+                                             ptr(workspace), ptr(labels_all), ptr(centroids), ptr(tau)))
 
 
 def qdit_tap_laplacian(ctx, x, t, n, d, alpha, exponent, workspace, L):
