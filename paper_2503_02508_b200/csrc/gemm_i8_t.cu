@@ -24,6 +24,11 @@
 // stores (warp-level stores of 64-byte row pieces reach 4.2 TB/s on this chip, TMA stores of the same tiles
 // 6.7 TB/s, and they do not hold the issuing warp), and the residual of the gated epilogue arrives the same way
 // in reverse (TMA load one chunk ahead, ldmatrix.trans).
+// The epilogue that writes 8-bit codes (bias + GELU -> codes, class 2) keeps a channel per thread (per-channel
+// scalars, tcgen05.ld 32x32b) and writes each code with a one-byte shared-memory store into a tile of 32 tokens x 128
+// channels that the four quadrant warps of a token chunk fill together; one thread hands it to a TMA store (full
+// 128-byte rows; per-thread global stores of this layout are 32-byte pieces of 8 rows, which held that layer at the
+// speed of its stores).
 #include "gemm_common.cuh"
 
 
@@ -51,7 +56,11 @@ struct TWarps {
   // tile plus one tile shared by the cache copy and the output (2) or one tile each (3)
   static constexpr int TILES = EPI == 3 ? QDIT_T_GATED_TILES : 2;
   static constexpr int STAGING_PER_WARP = STAGED ? TILES * 2048 : 0;
-  static constexpr int STAGING_BYTES = EPI_WARPS * STAGING_PER_WARP;
+  // class 2 (8-bit codes): the four quadrant warps that work on the same token chunk share a tile of 32 tokens x 128
+  // channels (4 KB), two tiles used in turn per group of four
+  static constexpr bool GROUPED = EPI == 2;
+  static constexpr int GROUP_TILE_BYTES = 32 * BC;
+  static constexpr int STAGING_BYTES = STAGED ? EPI_WARPS * STAGING_PER_WARP : GROUPED ? SPLIT * 2 * GROUP_TILE_BYTES : 0;
 };
 
 template <int BT, int EPI>
@@ -122,35 +131,13 @@ __device__ __forceinline__ void epilogue_chunk_t(const GemmParams& p, const uint
   }
 }
 
-// 8 x 8 transpose of 32-bit words across the 8 lanes of a lane group (xor 4, 2, 1): afterwards x[c] on lane i
-// is what lane c held in x[i].
-__device__ __forceinline__ void transpose8(uint32_t (&x)[8], int lane) {
-#pragma unroll
-  for (int d = 4; d >= 1; d >>= 1) {
-    const bool up = (lane & d) != 0;
-#pragma unroll
-    for (int a = 0; a < 8; ++a) {
-      if ((a & d) == 0) {
-        const int b = a | d;
-        const uint32_t send = up ? x[a] : x[b];
-        const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, d);
-        if (up) x[a] = recv; else x[b] = recv;
-      }
-    }
-  }
-}
-
-// GELU layer (bias + GELU -> 8-bit codes): the math runs channel-major with scalar parameters; the finished codes
-// are then transposed inside each group of 8 lanes with shuffles, so that a lane stores 8 consecutive channels of a
-// token at once (8 bytes) and a warp instruction covers 8 tokens x 32 channels, without touching shared memory.
-// Lane (g, i) = (lane >> 3, lane & 7) ends up with channels 8g..8g+7 of tokens i, 8 + i, 16 + i, 24 + i.
+// GELU layer (bias + GELU -> 8-bit codes): the math runs channel-major with scalar parameters; the code of token j
+// goes to byte (j, col) of the group's tile with a one-byte store (a warp instruction writes 32 consecutive bytes).
 template <int EPI>
-__device__ __forceinline__ void epilogue_chunk_t_packed(const GemmParams& p, const uint32_t (&v)[32], int n, int lane,
-                                                        int m_base, float sc, float bias, int zcs, float o_inv) {
+__device__ __forceinline__ void epilogue_chunk_t_codes(const GemmParams& p, const uint32_t (&v)[32], float sc, float bias, int zcs,
+                                                       float o_inv, uint32_t tile_col_addr) {
   const uint32_t flags = epi_flags<EPI>(p);
-  const int i8 = lane & 7;
-  const int n8 = n - i8;  // first channel of this lane group
-  // The epilogue of the GELU layer is bound by instruction issue, so work that a symmetric quantizer does not
+  // The epilogue of the GELU layer has the most arithmetic per element, so work that a symmetric quantizer does not
   // need (zero-point terms) is skipped through branches that are uniform over the whole grid.
   float f[32];
   if (p.a_zp == 0) {
@@ -160,39 +147,18 @@ __device__ __forceinline__ void epilogue_chunk_t_packed(const GemmParams& p, con
 #pragma unroll
     for (int j = 0; j < 32; ++j) f[j] = static_cast<float>(static_cast<int>(v[j]) - zcs);
   }
+  const float lo_f = p.o_qmin - p.o_zp, hi_f = p.o_qmax - p.o_zp;
+  const uint32_t zp = static_cast<uint32_t>(static_cast<int>(p.o_zp));
 #pragma unroll
   for (int j = 0; j < 32; ++j) {
-    f[j] = (flags & QDIT_EPI_BIAS) ? __fmaf_rn(f[j], sc, bias) : __fmul_rn(f[j], sc);
-    if (flags & QDIT_EPI_GELU) f[j] = gelu_tanh_f(f[j]);
-  }
-  // one byte per token: word t = codes of tokens t, 8 + t, 16 + t, 24 + t
-  const float lo_f = p.o_qmin - p.o_zp, hi_f = p.o_qmax - p.o_zp;
-  const int zp = static_cast<int>(p.o_zp);
-  uint32_t w[8];
-#pragma unroll
-  for (int t = 0; t < 8; ++t) {
-    uint32_t m4[4];
-#pragma unroll
-    for (int s4 = 0; s4 < 4; ++s4) {
-      const float q = fminf(fmaxf(__fmul_rn(f[8 * s4 + t], o_inv), lo_f), hi_f);
-      m4[s4] = static_cast<uint32_t>(__float_as_int(__fadd_rn(q, 12582912.0f)));
-    }
-    w[t] = __byte_perm(__byte_perm(m4[0], m4[1], 0x0040), __byte_perm(m4[2], m4[3], 0x0040), 0x5410);
-    if (zp != 0) w[t] = __vadd4(w[t], static_cast<uint32_t>(zp & 0xFF) * 0x01010101u);  // code + z stays inside a byte
-  }
-  transpose8(w, lane);  // w[c] = codes of channel n8 + c for tokens i8, 8 + i8, 16 + i8, 24 + i8
-  if (n8 < p.N) {
-#pragma unroll
-    for (int s4 = 0; s4 < 4; ++s4) {
-      const int64_t m = m_base + 8 * s4 + i8;
-      if (m < p.M) {
-        // byte s4 of each of the 8 words
-        const uint32_t sel = 0x0000 | (s4) | ((4 + s4) << 4);  // (w_a byte s4, w_b byte s4) -> low two bytes
-        const uint32_t lo = __byte_perm(__byte_perm(w[0], w[1], sel), __byte_perm(w[2], w[3], sel), 0x5410);
-        const uint32_t hi = __byte_perm(__byte_perm(w[4], w[5], sel), __byte_perm(w[6], w[7], sel), 0x5410);
-        *reinterpret_cast<uint2*>(static_cast<uint8_t*>(p.out) + m * p.ldo + n8) = make_uint2(lo, hi);
-      }
-    }
+    float x = (flags & QDIT_EPI_BIAS) ? __fmaf_rn(f[j], sc, bias) : __fmul_rn(f[j], sc);
+    if (flags & QDIT_EPI_GELU) x = gelu_tanh_f(x);
+    // clip(rne(t) + z, qmin, qmax) == rne(clamp(t, qmin - z, qmax - z)) + z; adding 1.5 * 2^23 rounds to nearest-even and
+    // leaves the integer in the low mantissa bits; the low byte is the stored code
+    const float q = fminf(fmaxf(__fmul_rn(x, o_inv), lo_f), hi_f);
+    uint32_t m = static_cast<uint32_t>(__float_as_int(__fadd_rn(q, 12582912.0f)));
+    if (zp != 0u) m += zp;
+    asm volatile("st.shared.u8 [%0], %1;" ::"r"(tile_col_addr + static_cast<uint32_t>(j * BC)), "r"(m) : "memory");
   }
 }
 
@@ -249,7 +215,7 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sW = smem;
   uint8_t* sX = smem + STAGES * C::W_BYTES;
-  uint8_t* staging = smem + STAGES * C::STAGE_BYTES;  // [EPI_WARPS][2][2 KB] (staged epilogues only; 1024-byte aligned)
+  uint8_t* staging = smem + STAGES * C::STAGE_BYTES;  // classes 1, 3: [EPI_WARPS][tiles][2 KB]; class 2: [SPLIT][2][4 KB]; 1024-byte aligned
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(staging + TW::STAGING_BYTES);
   uint64_t* empty_bar = full_bar + STAGES;
   uint64_t* tfull_bar = empty_bar + STAGES;
@@ -517,6 +483,11 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
       if (r_inflight) mbar_wait(rbar, r_phase, abort_flag, p.status);
       if (lane == 0) tma_store_wait_all();
     } else {
+      // class 2: the tile pair of this warp's group (the four quadrant warps with the same `part`), used in turn
+      uint8_t* const gtile = staging + part * (2 * TW::GROUP_TILE_BYTES);
+      const bool issuer = quad == 0 && lane == 0;   // one thread per group hands the tiles to TMA
+      int turn = 0;
+      if (TW::GROUPED && issuer) tma_prefetch_desc(&tmap_out);
       int it = 0;
       for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
         const int as = it & 1;
@@ -554,12 +525,27 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
             if (lane == 0) mbar_arrive_relaxed(&tempty_bar[as]);
           }
           const int m_base = t0 + c * 32;
-          if (m_base < p.M) {
-            if (EPI == 2) epilogue_chunk_t_packed<EPI>(p, v, n, lane, m_base, sc, bias, zcs, o_inv);
-            else if (n_ok) epilogue_chunk_t<EPI>(p, v, n, m_base, sc, bias, zcs, o_inv);
+          if (m_base < p.M) {   // uniform over the four warps of a group: they work on the same token chunk
+            if (TW::GROUPED) {
+              uint8_t* const buf = gtile + turn * TW::GROUP_TILE_BYTES;
+              epilogue_chunk_t_codes<EPI>(p, v, sc, bias, zcs, o_inv, smem_u32(buf) + static_cast<uint32_t>(quad * 32 + lane));
+              fence_async_smem();
+              // the store that used the other tile (issued one chunk ago) has read it before anybody passes the barrier,
+              // so the next chunk may overwrite it
+              if (issuer) tma_store_wait_read<0>();
+              asm volatile("bar.sync %0, %1;" ::"r"(1 + part), "r"(128) : "memory");
+              if (issuer) {
+                tma_store_2d(&tmap_out, buf, (tile % num_c_tiles) * BC, m_base);
+                tma_store_commit();
+              }
+              turn ^= 1;
+            } else if (n_ok) {
+              epilogue_chunk_t<EPI>(p, v, n, m_base, sc, bias, zcs, o_inv);
+            }
           }
         }
       }
+      if (TW::GROUPED && issuer) tma_store_wait_all();
     }
   }
 
@@ -580,6 +566,7 @@ int32_t launch_t_epi(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p,
   QDIT_TRY(qdit_get_tmap(ctx, A, p.M, p.K, p.K, BT, BK, 1, 1, &tx));
   // staged epilogues: 32 tokens x 32 channels bf16 tiles (64-byte rows, 64B swizzle) of the output, the cache slot and the residual
   CUtensorMap to = tx, tc = tx, tr = tx;
+  if (TWarps<EPI>::GROUPED) QDIT_TRY(qdit_get_tmap(ctx, p.out, p.M, p.N, p.ldo, 32, BC, 0, 1, &to));   // 32 tokens x 128 channels of bytes
   if (TWarps<EPI>::STAGED) {
     QDIT_TRY(qdit_get_tmap(ctx, p.out, p.M, p.N, p.ldo, 32, 32, 2, 2, &to));
     tc = tr = to;
