@@ -598,15 +598,341 @@ __global__ void __launch_bounds__(512, 1) final_kernel(const __nv_bfloat16* __re
   }
 }
 
+// ----------------------------------------------------------------------------- final layer on the tensor cores
+// The same operation for the widths the DiT blocks use (D a multiple of 128, 64 rows of one sample per CTA), with the
+// D -> 32 linear on mma.sync (bf16 operands, f32 accumulation).  The row statistics are taken out of the product,
+//   out[o] = rstd (S[o] - mean c1[o]) + c2[o] + bias[o],   S[o] = sum_k x_k W'[o,k],   W'[o,k] = (1 + scale_k) W[o,k],
+//   c1[o] = sum_k W'[o,k],   c2[o] = sum_k shift_k W[o,k],
+// so the bf16 activations go to the tensor cores as they are (exactly), and are read once.  W' is specific to the
+// sample: the CTA forms it chunk by chunk in f32 and splits it into a bf16 head and a bf16 remainder (|lo| <= 2^-9 |W'|;
+// both products are accumulated, what is dropped is below 2^-17 relative).  The statistics (sum x, sum x^2 in f32) are
+// accumulated from the same fragments on the ordinary pipes: mma.sync issues one m16n8k16 per 16 cycles and scheduler
+// here, which is the kernel's limit, so nothing that the other pipes can do goes to it.  The CTA's 64 rows are one contiguous piece of memory; they are fetched whole, one bulk copy per
+// row (whole rows keep DRAM pages streaming; column chunks of 256 bytes per row ran at a third of the bandwidth), into
+// rows padded by 16 bytes.  Thirty-two warps: (row tile 0..3) x (k-step 0..7 of a 128-column chunk), so that each
+// scheduler has eight warps to hide the mma and ldmatrix latencies; W' chunks are double-buffered; the partial sums of
+// the eight k-step groups meet in shared memory at the end.
+constexpr int FT_ROWS = 64, FT_KC = 128, FT_THREADS = 1024, FT_KG = 8, FT_PITCH = FT_KC * 2 + 16, FT_DMAX = 1408, FT_RED_PITCH = 68;
+constexpr int FT_WBUF_BYTES = 2 * FIN_OUT * FT_PITCH;   // weight heads, weight remainders of one chunk
+constexpr int ft_smem_bytes(int D) {
+  return (2 * D + FT_KG * FT_ROWS * 2 + 2 * FIN_OUT) * 4 + 16 + 2 * FT_WBUF_BYTES + FT_ROWS * (2 * D + 16);
+}
+static_assert(ft_smem_bytes(FT_DMAX) <= 227 * 1024, "final layer: shared memory");
+constexpr int FT_DMIN = 5 * FT_KC;
+static_assert(FT_ROWS * (2 * FT_DMIN + 16) >= FT_KG * FIN_OUT * FT_RED_PITCH * 4, "the partial products reuse the activation tile");
+
+__device__ __forceinline__ void bulk_load_row(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(smem_dst)),
+               "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr)
+               : "memory");
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// (z0, z1) -> packed bf16 heads and packed bf16 remainders
+__device__ __forceinline__ void split_pair(float z0, float z1, uint32_t& hi, uint32_t& lo) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(z0, z1);
+  const __nv_bfloat162 l = __floats2bfloat162_rn(z0 - __low2float(h), z1 - __high2float(h));
+  hi = *reinterpret_cast<const uint32_t*>(&h);
+  lo = *reinterpret_cast<const uint32_t*>(&l);
+}
+
+__global__ void __launch_bounds__(FT_THREADS) final_tc_kernel(const __nv_bfloat16* __restrict__ x, int64_t M, int D, int T, float eps,
+                                                              const float* __restrict__ modf, const float* __restrict__ w,
+                                                              const float* __restrict__ bias, float* __restrict__ net, int grid, int patch,
+                                                              int* status) {
+  extern __shared__ __align__(16) uint8_t ft_smem[];
+  float* s_mul = reinterpret_cast<float*>(ft_smem);   // [D] 1 + scale
+  float* s_add = s_mul + D;                             // [D] shift
+  float* s_stat = s_add + D;                            // [8 k-step groups][64 rows][2] sum x, sum x^2; then [64][2] mean, rstd
+  float* s_c = s_stat + FT_KG * FT_ROWS * 2;                // [2][32] c1, c2
+  uint64_t* bar = reinterpret_cast<uint64_t*>(s_c + 2 * FIN_OUT);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar + 1);
+  uint8_t* wring = reinterpret_cast<uint8_t*>(bar + 2);   // [2] W' chunks
+  uint8_t* xt = wring + 2 * FT_WBUF_BYTES;                // [64][2 D + 16] activations; the partial products afterwards
+  const int xp = 2 * D + 16;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int kg = warp & 7, rt = warp >> 3;             // k-step (group), row tile
+  const int g = lane >> 2, t4 = lane & 3;
+  const int64_t row0 = static_cast<int64_t>(blockIdx.x) * FT_ROWS;   // the CTA's rows lie inside one sample (T % 64 == 0)
+  const int nc = D / FT_KC;
+  const float* sh = modf + (row0 / T) * 2 * D;
+  float2 mod_pre[2] = {make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f)};   // (shift, scale) of columns tid, tid + 1024: in flight during set-up
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+    if (tid + i * FT_THREADS < D) mod_pre[i] = make_float2(sh[tid + i * FT_THREADS], sh[D + tid + i * FT_THREADS]);
+  if (tid == 0) {
+    mbar_init(bar, FT_ROWS);
+    *abort_flag = 0;
+    mbar_fence_init();
+  }
+  __syncthreads();
+  if (tid < FT_ROWS) {
+    const int64_t row = row0 + tid < M ? row0 + tid : M - 1;   // rows past M repeat the last row (never stored)
+    mbar_expect_tx(bar, static_cast<uint32_t>(2 * D));
+    bulk_load_row(xt + tid * xp, x + row * D, static_cast<uint32_t>(2 * D), bar);
+  }
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+    if (tid + i * FT_THREADS < D) s_add[tid + i * FT_THREADS] = mod_pre[i].x, s_mul[tid + i * FT_THREADS] = 1.0f + mod_pre[i].y;
+  // W' of a chunk: thread -> output wo (= its warp), four consecutive columns from wk
+  const int wo = warp, wk = lane * 4;
+  const float* wrow = w + static_cast<int64_t>(wo) * D + wk;
+  float4 wa = *reinterpret_cast<const float4*>(wrow);
+  float c1 = 0.0f, c2 = 0.0f;
+  auto store_w = [&](int c) {   // wa holds W[wo, c * 128 + wk ..]
+    const float4 ma = *reinterpret_cast<const float4*>(s_mul + c * FT_KC + wk), da = *reinterpret_cast<const float4*>(s_add + c * FT_KC + wk);
+    const float z0 = wa.x * ma.x, z1 = wa.y * ma.y, z2 = wa.z * ma.z, z3 = wa.w * ma.w;
+    c1 += (z0 + z1) + (z2 + z3);
+    c2 = fmaf(wa.x, da.x, fmaf(wa.y, da.y, fmaf(wa.z, da.z, fmaf(wa.w, da.w, c2))));
+    uint32_t h0, h1, l0, l1;
+    split_pair(z0, z1, h0, l0);
+    split_pair(z2, z3, h1, l1);
+    uint8_t* dst = wring + (c & 1) * FT_WBUF_BYTES + wo * FT_PITCH + wk * 2;
+    *reinterpret_cast<uint2*>(dst) = make_uint2(h0, h1);
+    *reinterpret_cast<uint2*>(dst + FIN_OUT * FT_PITCH) = make_uint2(l0, l1);
+  };
+  __syncthreads();   // the modulation table is complete
+  store_w(0);
+  if (nc > 1) wa = *reinterpret_cast<const float4*>(wrow + FT_KC);
+  float acc[4][4], s1a = 0.0f, s2a = 0.0f, s1b = 0.0f, s2b = 0.0f;
+#pragma unroll
+  for (int n = 0; n < 4; ++n)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[n][i] = 0.0f;
+  const bool landed = mbar_wait(bar, 0, abort_flag, status);
+  if (!__syncthreads_and(landed)) return;   // bounded wait ran out: the status word is set, the whole CTA leaves together
+  const uint32_t xs = smem_u32(xt);
+  for (int c = 0; c < nc; ++c) {
+    if (c > 0) __syncthreads();   // W' of chunk c is there for everybody, and everybody is done with chunk c - 1
+    const uint32_t whs = smem_u32(wring + (c & 1) * FT_WBUF_BYTES), wls = whs + FIN_OUT * FT_PITCH;
+    {
+      const int ks = kg;
+      uint32_t a[4];   // a[0] row g, a[1] row g + 8 (columns 2 t4, + 1 of the k-step); a[2], a[3] the same rows, columns + 8
+      ldmatrix_x4(xs + (16 * rt + (lane & 15)) * xp + (c * FT_KC + ks * 16 + (lane >> 4) * 8) * 2, a);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {   // statistics of rows g (even i) and g + 8 (odd i)
+        float v0, v1;
+        unpack_bf16x2(a[i], v0, v1);
+        if (i & 1) {
+          s1b += v0 + v1;
+          s2b = fmaf(v0, v0, fmaf(v1, v1, s2b));
+        } else {
+          s1a += v0 + v1;
+          s2a = fmaf(v0, v0, fmaf(v1, v1, s2a));
+        }
+      }
+#pragma unroll
+      for (int n2 = 0; n2 < 2; ++n2) {   // two output tiles of 8 per ldmatrix
+        const uint32_t off = (n2 * 16 + (lane & 7) + ((lane >> 4) << 3)) * FT_PITCH + (ks * 16 + ((lane >> 3) & 1) * 8) * 2;
+        uint32_t bh[4], bl[4];
+        ldmatrix_x4(whs + off, bh);
+        ldmatrix_x4(wls + off, bl);
+        mma_bf16_16816(acc[2 * n2], a, bh[0], bh[1]);
+        mma_bf16_16816(acc[2 * n2], a, bl[0], bl[1]);
+        mma_bf16_16816(acc[2 * n2 + 1], a, bh[2], bh[3]);
+        mma_bf16_16816(acc[2 * n2 + 1], a, bl[2], bl[3]);
+      }
+    }
+    if (c + 1 < nc) {   // while the tensor pipe works through this chunk: W' of the next one, into the buffer of chunk c - 1
+      store_w(c + 1);
+      if (c + 2 < nc) wa = *reinterpret_cast<const float4*>(wrow + (c + 2) * FT_KC);
+    }
+  }
+  __syncthreads();   // the activation tile is free: it now holds the partial products [8 k-step groups][32 outputs][64 rows, padded]
+  float* red = reinterpret_cast<float*>(xt);
+  {
+    float* mine = red + (static_cast<size_t>(kg) * FIN_OUT + 2 * t4) * FT_RED_PITCH + 16 * rt + g;
+#pragma unroll
+    for (int n = 0; n < 4; ++n) {   // acc[n][0..1]: row g, outputs 8 n + 2 t4, + 1; acc[n][2..3]: row g + 8
+      mine[(8 * n) * FT_RED_PITCH] = acc[n][0];
+      mine[(8 * n + 1) * FT_RED_PITCH] = acc[n][1];
+      mine[(8 * n) * FT_RED_PITCH + 8] = acc[n][2];
+      mine[(8 * n + 1) * FT_RED_PITCH + 8] = acc[n][3];
+    }
+    float* st = s_stat + (kg * FT_ROWS + 16 * rt + g) * 2;
+#pragma unroll
+    for (int o = 1; o < 4; o <<= 1) {   // the four lanes of a row
+      s1a += __shfl_xor_sync(0xffffffffu, s1a, o);
+      s2a += __shfl_xor_sync(0xffffffffu, s2a, o);
+      s1b += __shfl_xor_sync(0xffffffffu, s1b, o);
+      s2b += __shfl_xor_sync(0xffffffffu, s2b, o);
+    }
+    if (t4 == 0) st[0] = s1a, st[1] = s2a, st[16] = s1b, st[17] = s2b;
+    c1 = warp_sum(c1);
+    c2 = warp_sum(c2);
+    if (lane == 0) s_c[wo] = c1, s_c[FIN_OUT + wo] = c2;
+  }
+  __syncthreads();
+  float mean = 0.0f, rstd = 0.0f;
+  if (tid < FT_ROWS) {
+    float s1 = 0.0f, s2 = 0.0f;
+#pragma unroll
+    for (int k = 0; k < FT_KG; ++k) s1 += s_stat[(k * FT_ROWS + tid) * 2], s2 += s_stat[(k * FT_ROWS + tid) * 2 + 1];
+    mean = s1 / static_cast<float>(D);
+    rstd = 1.0f / sqrtf(fmaxf(s2 / static_cast<float>(D) - mean * mean, 0.0f) + eps);
+  }
+  __syncthreads();   // every partial sum of the statistics has been read
+  if (tid < FT_ROWS) s_stat[2 * tid] = mean, s_stat[2 * tid + 1] = rstd;
+  __syncthreads();
+  // un-patchify: output o = (py, px, c); consecutive threads take consecutive tokens of one output
+  const int side = grid * patch, co = FIN_OUT / (patch * patch);
+  const int b = static_cast<int>(row0 / T), tok0 = static_cast<int>(row0 % T);
+  for (int i = tid; i < FT_ROWS * FIN_OUT; i += FT_THREADS) {
+    const int o = i / FT_ROWS, r = i % FT_ROWS;
+    if (row0 + r >= M) continue;
+    float sum = 0.0f;
+#pragma unroll
+    for (int k = 0; k < FT_KG; ++k) sum += red[(k * FIN_OUT + o) * FT_RED_PITCH + r];
+    const float v = fmaf(s_stat[2 * r + 1], sum - s_stat[2 * r] * s_c[o], s_c[FIN_OUT + o]) + bias[o];
+    const int t = tok0 + r, gy = t / grid, gx = t % grid;
+    const int cc = o % co, px = (o / co) % patch, py = o / (co * patch);
+    net[((static_cast<int64_t>(b) * co + cc) * side + gy * patch + py) * side + gx * patch + px] = v;
+  }
+}
+
+// ----------------------------------------------------------------------------- patch embedding on the tensor cores
+// The same operation for a patch vector of 16 values (4 latent channels, 2 x 2 patches): the reduction is exactly one
+// k-step of mma.sync m16n8k16.  f32 operands are split into a bf16 head and remainder and three products are
+// accumulated (hi.hi + lo.hi + hi.lo; what is dropped is below 2^-17 relative).  The weights are split and laid out in
+// fragment order once, when the model is built: one 16-byte load per lane and column tile.  A CTA owns the same 16
+// token positions of four samples (four 16-row tiles) and half of the columns, so a position row and a weight fragment
+// are fetched once for four tiles (position rows in f32 are twice the bytes of the output).  Every thread builds the
+// A fragments straight from the latent (a fragment pair is two horizontally adjacent latent values); a warp walks its
+// column tiles three at a time, with all of a batch's loads (weights, bias, position rows) issued before the first
+// use, adds bias and position, and stages bf16 pairs in shared memory; the rows then leave by bulk copies.
+constexpr int ET_TOK = 16, ET_SAMPLES = 4, ET_ROWS = ET_TOK * ET_SAMPLES, ET_THREADS = 256, ET_SPLIT = 2, ET_BATCH = 3;
+
+__device__ __forceinline__ void bulk_store_row(void* gdst, const void* smem_src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(reinterpret_cast<uint64_t>(gdst)),
+               "r"(smem_u32(smem_src)), "r"(bytes)
+               : "memory");
+}
+
+// frag[n][lane] = (head(j, j+1), remainder(j, j+1), head(j+8, j+9), remainder(j+8, j+9)) of W[d = 8 n + lane / 4][.],
+// j = 2 (lane % 4): the B fragment of column tile n, from the transposed weights wT[j][d].
+__global__ void embed_fragments_kernel(const float* __restrict__ wT, int D, uint4* __restrict__ frag) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (D >> 3) * 32) return;
+  const int n = i >> 5, lane = i & 31, g = lane >> 2, t4 = lane & 3;
+  const float* wc = wT + 8 * n + g;
+  uint4 f;
+  split_pair(wc[static_cast<int64_t>(2 * t4) * D], wc[static_cast<int64_t>(2 * t4 + 1) * D], f.x, f.y);
+  split_pair(wc[static_cast<int64_t>(2 * t4 + 8) * D], wc[static_cast<int64_t>(2 * t4 + 9) * D], f.z, f.w);
+  frag[i] = f;
+}
+
+__global__ void __launch_bounds__(ET_THREADS, 2) embed_tc_kernel(const float* __restrict__ latent, int latent_batch,
+                                                                 const uint4* __restrict__ frag, const float* __restrict__ bias,
+                                                                 const float* __restrict__ pos, __nv_bfloat16* __restrict__ x, int B,
+                                                                 int D, int grid, int C) {
+  extern __shared__ __align__(16) uint8_t et_smem[];   // [4 samples][16 tokens][D + 16 bytes]: the CTA's half of the bf16 rows, padded
+  const int dh = D / ET_SPLIT, xp = 2 * dh + 16;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t4 = lane & 3;
+  const int T = grid * grid, side = 2 * grid;
+  const int t0 = blockIdx.x * ET_TOK, b0 = blockIdx.y * ET_SAMPLES, d0 = blockIdx.z * dh;
+  // A fragments: value pair (j, j + 1) of a token with j = 2 t4 (+ 8) is latent[b, c, 2 gy + py, 2 gx .. 2 gx + 1],
+  // c = t4 / 2 (+ 2), py = t4 % 2.  Fragment registers of a 16-row tile: 0 row g, 1 row g + 8 (columns 2 t4, + 1);
+  // 2, 3 the same rows, columns + 8.
+  uint32_t ah[ET_SAMPLES][4], al[ET_SAMPLES][4];
+  {
+    const int64_t plane = static_cast<int64_t>(side) * side;
+    int off[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int t = t0 + g + 8 * i, gy = t / grid, gx = t % grid;
+      off[i] = (2 * gy + (t4 & 1)) * side + 2 * gx;
+    }
+    float2 pv[ET_SAMPLES][4];
+#pragma unroll
+    for (int sidx = 0; sidx < ET_SAMPLES; ++sidx) {
+      const float* base = latent + (static_cast<int64_t>((b0 + sidx) % latent_batch) * C + (t4 >> 1)) * plane;
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        pv[sidx][i] = *reinterpret_cast<const float2*>(base + off[i]);
+        pv[sidx][2 + i] = *reinterpret_cast<const float2*>(base + 2 * plane + off[i]);
+      }
+    }
+#pragma unroll
+    for (int sidx = 0; sidx < ET_SAMPLES; ++sidx)
+#pragma unroll
+      for (int r = 0; r < 4; ++r) split_pair(pv[sidx][r].x, pv[sidx][r].y, ah[sidx][r], al[sidx][r]);
+  }
+  const float* prow0 = pos + static_cast<int64_t>(t0 + g) * D + 2 * t4;   // position rows of tokens g and g + 8, at column 2 t4
+  const float* prow1 = prow0 + static_cast<int64_t>(8) * D;
+  const int n_end = (d0 + dh) >> 3;
+  for (int nb = (d0 >> 3) + warp; nb < n_end; nb += ET_BATCH * (ET_THREADS / 32)) {
+    uint4 f[ET_BATCH];
+    float2 bv[ET_BATCH], pa[ET_BATCH], pb[ET_BATCH];
+#pragma unroll
+    for (int u = 0; u < ET_BATCH; ++u) {
+      const int n = nb + u * (ET_THREADS / 32);
+      if (n < n_end) {
+        f[u] = frag[n * 32 + lane];
+        bv[u] = *reinterpret_cast<const float2*>(bias + 8 * n + 2 * t4);
+        pa[u] = *reinterpret_cast<const float2*>(prow0 + 8 * n);
+        pb[u] = *reinterpret_cast<const float2*>(prow1 + 8 * n);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < ET_BATCH; ++u) {
+      const int n = nb + u * (ET_THREADS / 32);
+      if (n < n_end) {
+        const int col = (8 * n - d0 + 2 * t4) * 2;   // byte offset inside a staged row
+#pragma unroll
+        for (int sidx = 0; sidx < ET_SAMPLES; ++sidx) {
+          float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+          mma_bf16_16816(acc, ah[sidx], f[u].x, f[u].z);
+          mma_bf16_16816(acc, al[sidx], f[u].x, f[u].z);
+          mma_bf16_16816(acc, ah[sidx], f[u].y, f[u].w);
+          *reinterpret_cast<uint32_t*>(et_smem + (ET_TOK * sidx + g) * xp + col) = pack_bf16x2((acc[0] + bv[u].x) + pa[u].x, (acc[1] + bv[u].y) + pa[u].y);
+          *reinterpret_cast<uint32_t*>(et_smem + (ET_TOK * sidx + g + 8) * xp + col) = pack_bf16x2((acc[2] + bv[u].x) + pb[u].x, (acc[3] + bv[u].y) + pb[u].y);
+        }
+      }
+    }
+  }
+  fence_async_smem();   // the staged rows are read by the bulk copies
+  __syncthreads();
+  if (tid < ET_ROWS && b0 + tid / ET_TOK < B) {   // the last group of samples may be short (its extra tiles repeat valid latents)
+    const int64_t m = static_cast<int64_t>(b0 + tid / ET_TOK) * T + t0 + tid % ET_TOK;
+    bulk_store_row(x + m * D + d0, et_smem + tid * xp, static_cast<uint32_t>(2 * dh));
+    tma_store_commit();
+    tma_store_wait_all();   // shared memory must outlive the copy
+  }
+}
+
 }  // namespace
 
 // ================================================================================ launchers
-int32_t launch_embed(qdit_ctx* ctx, const float* latent, int latent_batch, const float* wT, const float* bias,
+int32_t launch_embed_fragments(qdit_ctx* ctx, const float* wT, int D, void* frag) {
+  embed_fragments_kernel<<<(D / 8 * 32 + 255) / 256, 256, 0, ctx->stream>>>(wT, D, static_cast<uint4*>(frag));
+  return qdit_after_launch(ctx, "embed_fragments_kernel");
+}
+
+int32_t launch_embed(qdit_ctx* ctx, const float* latent, int latent_batch, const float* wT, const void* frag, const float* bias,
                      const float* pos, void* x, int64_t M, int D, int grid, int patch, int C) {
   const int pd = C * patch * patch;
   dim3 g(static_cast<unsigned>((M + EMB_ROWS - 1) / EMB_ROWS), static_cast<unsigned>((D / 2 + 255) / 256));
   __nv_bfloat16* xb = static_cast<__nv_bfloat16*>(x);
   ProfScope prof(ctx, QDIT_PROF_OTHER, static_cast<double>(M) * D * 2.0);
+  const int64_t T = static_cast<int64_t>(grid) * grid;
+  if (frag && pd == 16 && patch == 2 && D % (16 * ET_SPLIT) == 0 && D <= 2048 && T % ET_TOK == 0 && M % T == 0 &&
+      reinterpret_cast<uintptr_t>(x) % 16 == 0 && reinterpret_cast<uintptr_t>(latent) % 8 == 0) {   // the tensor-core form
+    const int smem = ET_ROWS * (D + 16);
+    QDIT_TRY(qdit_allow_smem(ctx, embed_tc_kernel, ET_ROWS * (2048 + 16)));
+    const int B = static_cast<int>(M / T);
+    embed_tc_kernel<<<dim3(static_cast<unsigned>(T / ET_TOK), static_cast<unsigned>((B + ET_SAMPLES - 1) / ET_SAMPLES), ET_SPLIT), ET_THREADS, smem,
+                      ctx->stream>>>(latent, latent_batch, static_cast<const uint4*>(frag), bias, pos, xb, B, D, grid, C);
+    return qdit_after_launch(ctx, "embed_tc_kernel");
+  }
   switch (pd) {
     case 16: embed_kernel<16><<<g, 256, 0, ctx->stream>>>(latent, latent_batch, wT, bias, pos, xb, M, D, grid, patch, C); break;
     case 4: embed_kernel<4><<<g, 256, 0, ctx->stream>>>(latent, latent_batch, wT, bias, pos, xb, M, D, grid, patch, C); break;
@@ -665,6 +991,13 @@ int32_t launch_final(qdit_ctx* ctx, const void* x, int64_t M, int D, int T, floa
                      const float* w, const float* bias, float* net, int grid, int patch, int OUT) {
   if (OUT != FIN_OUT) return qdit_fail(ctx, QDIT_ERR_SHAPE, "final layer width %d not supported (needs patch*patch*2*channels = %d)", OUT, FIN_OUT);
   const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(x);
+  if (D % FT_KC == 0 && D >= FT_DMIN && D <= FT_DMAX && T % FT_ROWS == 0 && reinterpret_cast<uintptr_t>(x) % 16 == 0) {   // the tensor-core form
+    QDIT_TRY(qdit_allow_smem(ctx, final_tc_kernel, ft_smem_bytes(FT_DMAX)));
+    ProfScope prof(ctx, QDIT_PROF_OTHER, static_cast<double>(M) * D * 2.0);
+    final_tc_kernel<<<static_cast<unsigned>((M + FT_ROWS - 1) / FT_ROWS), FT_THREADS, ft_smem_bytes(D), ctx->stream>>>(
+        xb, M, D, T, eps, modf, w, bias, net, grid, patch, ctx->d_status);
+    return qdit_after_launch(ctx, "final_tc_kernel");
+  }
   const int nv = (D / 8 + 31) / 32;
   const size_t smem = static_cast<size_t>(FIN_OUT) * nv * 2 * 32 * sizeof(float4);
   int64_t want = (M + 31) / 32;

@@ -13,8 +13,11 @@ struct DdpmCoef {
 };
 
 // x[m,:] = bf16(W_patch . patch(m) + b + pos); sample b reads latent[b % latent_batch]; wT = W_patch transposed [pd][D].
-int32_t launch_embed(qdit_ctx* ctx, const float* latent, int latent_batch, const float* wT, const float* bias,
+// frag (optional, for pd = 16): the weights in tensor-core fragment order, (D / 8) * 512 bytes written by
+// launch_embed_fragments; with it the product runs on the tensor cores.
+int32_t launch_embed(qdit_ctx* ctx, const float* latent, int latent_batch, const float* wT, const void* frag, const float* bias,
                      const float* pos, void* x, int64_t M, int D, int grid, int patch, int C);
+int32_t launch_embed_fragments(qdit_ctx* ctx, const float* wT, int D, void* frag);
 // feat[b, :] = (cos(t_b w_j), sin(t_b w_j)), w_j = 10000^(-j / (F/2))
 int32_t launch_timestep_features(qdit_ctx* ctx, const float* t, float* feat, int B, int F);
 // h[b,:] = SiLU(W1 . sinusoid(t_b) + b1); feat is scratch [B, F]

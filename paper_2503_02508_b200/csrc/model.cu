@@ -49,6 +49,7 @@ struct qdit_model {
   QLinearDev ada_all;                     // [depth*6D, D], block-major
   std::vector<QLinearDev> qkv, proj, fc1, fc2;
   float *w_patch, *b_patch, *pos, *w_t1, *b_t1, *w_t2, *b_t2, *y_table, *w_ada_f, *b_ada_f, *w_out, *b_out;
+  uint8_t* w_patch_frag = nullptr;   // patch-embedding weights in tensor-core fragment order (patch vectors of 16 values)
   float* d_scales;      // [1 + 4*depth] static activation scales: [0] ada input, then per block qkv, proj, fc1, fc2
   float* d_absmax_run;  // [1 + 4*depth] widest range seen during calibration
   bool scales_set;
@@ -135,6 +136,11 @@ int32_t build_model(qdit_ctx* ctx, const qdit_model_desc* desc, qdit_model* m) {
     for (int64_t d = 0; d < D; ++d)
       for (int j = 0; j < pd; ++j) wt[static_cast<size_t>(j) * D + d] = desc->w_patch[d * pd + j];
     QDIT_TRY(upload(ctx, m->mem, wt.data(), D * pd, &m->w_patch));
+    if (pd == 16 && D % 8 == 0) {
+      m->w_patch_frag = m->mem.alloc<uint8_t>(static_cast<size_t>(D / 8) * 512);
+      if (!m->w_patch_frag) return qdit_fail(ctx, QDIT_ERR_NOMEM, "out of device memory");
+      QDIT_TRY(launch_embed_fragments(ctx, m->w_patch, D, m->w_patch_frag));
+    }
     QDIT_CUDA_CHECK(ctx, cudaStreamSynchronize(ctx->stream));  // `wt` is a host temporary
   }
   QDIT_TRY(upload(ctx, m->mem, desc->b_patch, D, &m->b_patch));
@@ -257,7 +263,7 @@ static int32_t forward_impl(qdit_ctx* ctx, qdit_sampler* s, const float* latent,
   if (reuse && (store || calib)) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "REUSE cannot be combined with STORE_CACHE or CALIBRATE");
   const float* scales = calib ? s->dyn_scale : m->d_scales;
 
-  QDIT_TRY(launch_embed(ctx, latent, latent_batch, m->w_patch, m->b_patch, m->pos, s->x, M, D, sh.grid, sh.patch, sh.channels));
+  QDIT_TRY(launch_embed(ctx, latent, latent_batch, m->w_patch, m->w_patch_frag, m->b_patch, m->pos, s->x, M, D, sh.grid, sh.patch, sh.channels));
   const float* mod_all = pre_mod;
   if (!pre_mod) {
     QDIT_TRY(launch_cond1(ctx, t, m->w_t1, m->b_t1, s->feat, s->hidden, B, D, sh.freq_dim));
