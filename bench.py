@@ -550,6 +550,42 @@ def run_w4_sweep(args):
                       "hbm_gbs": peaks["hbm_gbs"], "rows": rows}))
 
 
+def run_mma_probe(args):
+    """What the tensor pipe gives the int8 GEMM kernels at most: tcgen05.mma kind::i8 (M 128, K 32) issued by one thread
+    per SM, with the operands resident in shared memory (the instruction path alone) and with a TMA producer refilling
+    a four-stage ring from an L2-resident matrix as the GEMM kernels' main loop does, no epilogue."""
+    import torch
+    import paper_2503_02508_b200 as q
+    peaks = measured_peaks()
+    ctx = q.qdit_create(0, None)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    rows_op = 4096
+    operands = torch.randint(-127, 128, (rows_op, 1024), dtype=torch.int8, device="cuda")
+    torch.cuda.synchronize()
+    iters = 8192
+    clocks = ClockSampler(0)
+    clocks.start()
+    rows = []
+    for mode, name in ((0, "operands resident in shared memory"), (1, "TMA-fed four-stage ring, no epilogue")):
+        for n in (128, 192, 256):
+            for _ in range(3):
+                q.qdit_probe_mma_rate(ctx, mode, n, iters, operands, rows_op)
+            ms = min(q.qdit_probe_mma_rate(ctx, mode, n, iters, operands, rows_op) for _ in range(max(args.steps, 3)))
+            ops = sms * iters * 4 * 2.0 * 128 * n * 32
+            us_per_group = ms * 1e3 / iters
+            rows.append({"mode": name, "n": n, "ms": round(ms, 3), "tops": round(ops / ms / 1e9, 0),
+                         "us_per_128_byte_k_block": round(us_per_group, 3),
+                         "frac_of_2x_bf16_burst": round(ops / ms / 1e9 / (2 * peaks["bf16_burst"]), 3),
+                         "frac_of_nominal_4500": round(ops / ms / 1e9 / 4500.0, 3)})
+    clock_info = clocks.stop()
+    q.qdit_destroy(ctx)
+    best = max(r["tops"] for r in rows if r["n"] == 256)
+    print(json.dumps({"metric": "tcgen05.mma kind::i8 rate, all SMs (probe)", "value": best, "unit": "TOP/s", "n_gpus": 1,
+                      "steps": max(args.steps, 3), "warmup": 3, "higher_is_better": True, "dtype": "int8", "data": "synthetic",
+                      "config": {"workload": "mma_probe", "iters": iters, "timing": "CUDA events around one launch, best of steps"},
+                      "clocks": clock_info, "int8_peak_2x_bf16_burst": 2 * peaks["bf16_burst"], "rows": rows}))
+
+
 def compact_sweep(rows, clock_info, peaks):
     """The second half of the metric for the default bench line: per layer and M the GEMM rate and its fractions of
     2 x burst bf16 (measured) and of the nominal 4500 TOP/s; the memory-bound kernels as fractions of the measured HBM
@@ -579,7 +615,7 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="ddim50", choices=sorted(WORKLOADS) + ["gemm_sweep", "w4_sweep"])
+    ap.add_argument("--workload", default="ddim50", choices=sorted(WORKLOADS) + ["gemm_sweep", "w4_sweep", "mma_probe"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-layer sweep that follows the timed region")
     ap.add_argument("--weight-bits", type=int, default=8, help="code width of the quantized weights (4 = the paper's W4A8 setting)")
@@ -592,6 +628,8 @@ def main():
         run_gemm_sweep(args)
     elif args.workload == "w4_sweep":
         run_w4_sweep(args)
+    elif args.workload == "mma_probe":
+        run_mma_probe(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

@@ -57,6 +57,14 @@ int32_t qdit_sync(qdit_ctx* ctx);
  * normally; the next qdit_sync returns QDIT_ERR_TIMEOUT once and the context stays usable.
  * observed_dev: device int[2], set to {1, 1} when both threads left their wait the intended way. */
 int32_t qdit_selftest_wait_timeout(qdit_ctx* ctx, uint32_t polls, int* observed_dev);
+/* Tensor-pipe probe (the paper has no counterpart; bench.py --workload mma_probe reports it): every SM runs
+ * `iters` groups of four tcgen05.mma kind::i8 instructions (M 128, N = n in {64, 128, 192, 256}, K 32 each), the
+ * products are discarded.  mode 0: the operands stay in shared memory (the instruction path's own rate); mode 1: a TMA
+ * producer refills a four-stage ring of 128 + n rows of 128 bytes per group from `operands` and the issuer frees each
+ * stage with a commit, as the GEMM kernels' main loop does, with no epilogue.  operands: int8 [rows][1024], rows a
+ * multiple of 256, values arbitrary.  Synchronous: returns the kernel's duration in milliseconds in *ms_host (host
+ * pointer); int-ops performed = SMs x iters x 4 x 2 x 128 x n x 32.  iters in 1..65536. */
+int32_t qdit_probe_mma_rate(qdit_ctx* ctx, int mode, int n, int iters, const void* operands, int64_t rows, float* ms_host);
 const char* qdit_status_string(int32_t status);
 const char* qdit_last_error(const qdit_ctx* ctx);
 /* Number of kernels this context has launched since creation (for launch accounting). */

@@ -94,6 +94,7 @@ _SIGNATURES = {
     "qdit_cache_reuse": (_i32, [_vp, _vp, _int, _int, _vp, _i64, _i64, _vp]),
     "qdit_cache_reuse_all": (_i32, [_vp, _vp, _vp, _i64, _i64, _vp]),
     "qdit_selftest_wait_timeout": (_i32, [_vp, C.c_uint32, _vp]),
+    "qdit_probe_mma_rate": (_i32, [_vp, _int, _int, _int, _vp, _i64, C.POINTER(C.c_float)]),
     "qdit_vc_correct": (_i32, [_vp, _vp, _int, _int, _int, _int, _int, _vp, _f32]),
     "qdit_tap_laplacian": (_i32, [_vp, _vp, _vp, _int, _int, _f32, _f32, _vp, _vp]),
     "qdit_tap_cluster_workspace": (_i64, [_int, _int, _int, _int]),
@@ -305,6 +306,13 @@ def qdit_cache_reuse_all(ctx, cache, mod_all, ld_mod, T, x):
 
 def qdit_selftest_wait_timeout(ctx, polls, observed):
     return check(ctx, lib.qdit_selftest_wait_timeout(ctx, polls, ptr(observed)))
+
+
+def qdit_probe_mma_rate(ctx, mode, n, iters, operands, rows):
+    """Kernel duration in milliseconds."""
+    ms = C.c_float(0.0)
+    check(ctx, lib.qdit_probe_mma_rate(ctx, mode, n, iters, ptr(operands), rows, C.byref(ms)))
+    return ms.value
 
 
 def qdit_vc_correct(ctx, latent, B, Cc, HW, step_index, mode, table, eps):

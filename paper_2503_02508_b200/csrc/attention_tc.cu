@@ -347,6 +347,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 // columns that thread has read before.  P's key order along the columns is therefore chunk 0, 2, 1, 3, and the
 // k-steps of P.V pick their V rows in that order.  O's columns are free once both threads of every row have written
 // P_0 (main part) and P_1 (tail part): the barriers the MMA issuer waits for anyway.
+//   * Head dim 72: the row sum comes out of the tensor core.  Columns 72..79 of a V tail tile are padding (whatever
+//     follows the head in memory); the loader warp sets column 72 of every key row to one once the tile has landed, so
+//     accumulator column 200 is sum_k P[q,k] over the same bf16 probabilities that multiply V, and the softmax threads
+//     neither add the probabilities up nor exchange partial sums.
+//   * 8-bit output: the codes of a CTA (128 rows x 72 bytes) are staged in shared memory (K_0's place) and leave with
+//     row-contiguous 8-byte stores, 9 per row, instead of every thread writing pieces of its own row.
 // 85 KB shared memory and 256 tensor-memory columns: two CTAs per SM.  Every barrier completes exactly once (phase 0).
 template <int DH>
 struct T256Cfg {
@@ -381,7 +387,8 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   uint64_t* bar_o = bars + 10;     // both P.V products complete (commit)
   uint64_t* bar_l = bars + 11;     // row sums exchanged (256 arrivals)
   uint64_t* bar_mx = bars + 12;    // [4] row maxima exchanged between the two warps of a lane quadrant (64 arrivals)
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 16);
+  uint64_t* bar_vp = bars + 16;    // [2] V tail block patched: column 72 set to one (32 arrivals)
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 18);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
   float* s_l = reinterpret_cast<float*>(tmem_holder + 4);  // [2][128] partial row sums
   float* s_m = s_l + 256;                                  // [2][128] partial row maxima
@@ -403,6 +410,7 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     mbar_init(bar_o, 1);
     mbar_init(bar_l, SM_WARPS * 32);
     for (int i = 0; i < 4; ++i) mbar_init(&bar_mx[i], 64);
+    for (int i = 0; i < 2; ++i) mbar_init(&bar_vp[i], 32);
     *abort_flag = 0;
     mbar_fence_init();
   }
@@ -444,6 +452,21 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         mbar_expect_tx(&bar_v[1], C::OP_BYTES);
         tma_load_2d(sQ, &tm_v, col0, row0 + TK, &bar_v[1]);
         if (C::TAIL) tma_load_2d(sQt, &tm_vt, col0 + 64, row0 + TK, &bar_v[1]);
+      }
+    }
+    if (C::TAIL) {
+      // the whole warp: column 72 of the landed V tail tiles := 1 (second 16-byte slot of the 32-byte row, 32B swizzle)
+#pragma unroll 1
+      for (int j = 0; j < 2; ++j) {
+        if (!mbar_wait(&bar_v[j], 0, abort_flag, p.status)) break;
+        const uint32_t tile = smem_u32(j == 0 ? sV0t : sQt);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t kr = static_cast<uint32_t>(lane + 32 * i);
+          asm volatile("st.shared.u16 [%0], %1;" ::"r"(tile + kr * 32u + ((1u ^ ((kr >> 2) & 1u)) << 4)), "h"(static_cast<uint16_t>(0x3F80)) : "memory");
+        }
+        fence_async_smem();
+        mbar_arrive(&bar_vp[j]);
       }
     }
   } else if (warp == SM_WARPS + 1) {
@@ -493,6 +516,7 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         issue_pv_main(0, sV0);
       }
       ok = ok && mbar_wait(&bar_p[1], 0, abort_flag, p.status) && mbar_wait(&bar_v[1], 0, abort_flag, p.status);
+      if (C::TAIL) ok = ok && mbar_wait(&bar_vp[0], 0, abort_flag, p.status) && mbar_wait(&bar_vp[1], 0, abort_flag, p.status);
       if (ok) {
         tc_fence_after();
         issue_pv_main(1, sQ);
@@ -548,23 +572,26 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       ok = mbar_wait(&bar_mx[quad], 0, abort_flag, p.status);
     }
     float rs = 0.0f;
+    bool staged = false;
     if (ok) {
       const float m_row = fmaxf(mx, s_m[(half ^ 1) * 128 + r]) * p.scale_log2;
+      const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(-m_row, -m_row);
 #pragma unroll 1
       for (int j = 0; j < 2; ++j) {
         // P_j = exp2(s * scale - m) for this thread's two chunks of block j: bf16 pairs back into tensor memory,
         // over columns this thread has already read; row sum in f32
+        uint32_t va[32], vb[32];   // both chunks in flight, one wait
+        tmem_ld_32x32(trow + static_cast<uint32_t>(j * 128 + half * 32), va);
+        tmem_ld_32x32(trow + static_cast<uint32_t>(j * 128 + half * 32 + 64), vb);
+        tmem_ld_wait();
 #pragma unroll
         for (int w = 0; w < 2; ++w) {
-          uint32_t v[32];
-          tmem_ld_32x32(trow + static_cast<uint32_t>(j * 128 + half * 32 + w * 64), v);
-          tmem_ld_wait();
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const float p0 = ex2_approx(fmaf(__uint_as_float(v[2 * i]), p.scale_log2, -m_row));
-            const float p1 = ex2_approx(fmaf(__uint_as_float(v[2 * i + 1]), p.scale_log2, -m_row));
-            rs += p0 + p1;
+            const float2 a = __ffma2_rn(make_float2(__uint_as_float(w ? vb[2 * i] : va[2 * i]), __uint_as_float(w ? vb[2 * i + 1] : va[2 * i + 1])), sc2, nm2);
+            const float p0 = ex2_approx(a.x), p1 = ex2_approx(a.y);
+            if (!C::TAIL) rs += p0 + p1;
             pk[i] = pack_bf16x2(p0, p1);
           }
           tmem_st_32x16(trow + static_cast<uint32_t>(j * 128 + half * 32 + w * 16), pk);
@@ -574,8 +601,8 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         mbar_arrive(&bar_p[j]);
       }
     }
-    // the two threads of a row exchange their partial sums
-    if (ok) {
+    // the two threads of a row exchange their partial sums (with a tail, the sum is accumulator column 200)
+    if (ok && !C::TAIL) {
       s_l[half * 128 + r] = rs;
       mbar_arrive(bar_l);
       ok = mbar_wait(bar_l, 0, abort_flag, p.status);
@@ -585,40 +612,73 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
       tc_fence_after();
       // first thread of a row: head dims 0..31; second: head dims 32..63 and the tail 64..71
       float o[40];
+      float l_row = 0.0f;
       {
         uint32_t v[32];
         tmem_ld_32x32(trow + COL_O + static_cast<uint32_t>(half * 32), v);
-        if (C::TAIL && half == 1) {
-          uint32_t w[8];
-          tmem_ld_32x8(trow + COL_OT, w);
+        if (C::TAIL) {
+          uint32_t w[8], wl[8];
+          if (half == 1) tmem_ld_32x8(trow + COL_OT, w);
+          tmem_ld_32x8(trow + COL_OT + 8, wl);   // column 200: the row sum
           tmem_ld_wait();
+          if (half == 1) {
 #pragma unroll
-          for (int i = 0; i < 8; ++i) o[32 + i] = __uint_as_float(w[i]);
+            for (int i = 0; i < 8; ++i) o[32 + i] = __uint_as_float(w[i]);
+          }
+          l_row = __uint_as_float(wl[0]);
         } else {
           tmem_ld_wait();
+          l_row = s_l[r] + s_l[128 + r];
         }
 #pragma unroll
         for (int i = 0; i < 32; ++i) o[i] = __uint_as_float(v[i]);
       }
-      const float inv_l = 1.0f / (s_l[r] + s_l[128 + r]);
+      const float inv_l = 1.0f / l_row;
       const int64_t row = static_cast<int64_t>(row0) + q0 + r;
       const int64_t base = row * (static_cast<int64_t>(p.H) * DH) + col0 + half * 32;
       const int ngroups = (C::TAIL && half == 1) ? 5 : 4;
+      if (p.out_dtype == QDIT_I8) {
+        // codes into the staging tile (K_0's place: both S products are long done): rows of DH bytes, pitch DH + 8
+        uint8_t* srow = sK0 + r * (DH + 8) + half * 32;
 #pragma unroll
-      for (int g = 0; g < 5; ++g) {
-        if (g < ngroups) {
-          float y[8];
+        for (int g = 0; g < 5; ++g) {
+          if (g < ngroups) {
+            float y[8];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) y[i] = o[8 * g + i] * inv_l;
-          if (p.out_dtype == QDIT_I8) {
-            *reinterpret_cast<uint2*>(static_cast<uint8_t*>(p.out) + base + 8 * g) = quantize_pack8(y, q_inv, p.qa.zp, p.qa.qmin, p.qa.qmax);
-          } else if (p.out_dtype == QDIT_BF16) {
-            *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + base + 8 * g) = pack_bf16x8(y);
-          } else {
-            float* of = static_cast<float*>(p.out) + base + 8 * g;
-            *reinterpret_cast<float4*>(of) = make_float4(y[0], y[1], y[2], y[3]);
-            *reinterpret_cast<float4*>(of + 4) = make_float4(y[4], y[5], y[6], y[7]);
+            for (int i = 0; i < 8; ++i) y[i] = o[8 * g + i] * inv_l;
+            *reinterpret_cast<uint2*>(srow + 8 * g) = quantize_pack8(y, q_inv, p.qa.zp, p.qa.qmin, p.qa.qmax);
           }
+        }
+        staged = true;
+      } else {
+#pragma unroll
+        for (int g = 0; g < 5; ++g) {
+          if (g < ngroups) {
+            float y[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) y[i] = o[8 * g + i] * inv_l;
+            if (p.out_dtype == QDIT_BF16) {
+              *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.out) + base + 8 * g) = pack_bf16x8(y);
+            } else {
+              float* of = static_cast<float*>(p.out) + base + 8 * g;
+              *reinterpret_cast<float4*>(of) = make_float4(y[0], y[1], y[2], y[3]);
+              *reinterpret_cast<float4*>(of + 4) = make_float4(y[4], y[5], y[6], y[7]);
+            }
+          }
+        }
+      }
+    }
+    // 8-bit output: the staged codes leave row by row, 8 bytes per thread and piece.  Every softmax thread comes here
+    // (also after a failed wait), so the named barrier is complete.
+    if (p.out_dtype == QDIT_I8) {
+      asm volatile("bar.sync 1, %0;" ::"n"(SM_WARPS * 32) : "memory");
+      if (staged && !*abort_flag) {
+        constexpr int PIECES = DH / 8;
+        uint8_t* gout = static_cast<uint8_t*>(p.out) + (static_cast<int64_t>(row0) + q0) * (static_cast<int64_t>(p.H) * DH) + col0;
+        for (int i = threadIdx.x; i < 128 * PIECES; i += SM_WARPS * 32) {
+          const int rr = i / PIECES, pc = i % PIECES;
+          *reinterpret_cast<uint2*>(gout + static_cast<int64_t>(rr) * (static_cast<int64_t>(p.H) * DH) + 8 * pc) =
+              *reinterpret_cast<const uint2*>(sK0 + rr * (DH + 8) + 8 * pc);
         }
       }
     }

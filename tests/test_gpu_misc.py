@@ -201,3 +201,23 @@ def test_vc_correct(q, ctx, B, C, HW):
     q.qdit_vc_correct(ctx, xd, B, C, HW, 0, q.QDIT_VC_K_TABLE, dev(np.ones((S, C), dtype=np.float32)), 1e-6)
     q.qdit_sync(ctx)
     np.testing.assert_allclose(xd.cpu().numpy(), x, rtol=0, atol=1e-6)
+
+
+def test_mma_probe_runs_and_scales_with_the_work(q, ctx):
+    """The tensor-pipe probe: both modes end by themselves with a clean status, the time grows with the number of
+    instruction groups, and bad arguments are refused before any launch."""
+    operands = torch.randint(-127, 128, (1024, 1024), dtype=torch.int8, device="cuda")
+    torch.cuda.synchronize()
+    for mode in (0, 1):
+        for n in (64, 256):
+            q.qdit_probe_mma_rate(ctx, mode, n, 256, operands, 1024)       # warm-up
+            short = min(q.qdit_probe_mma_rate(ctx, mode, n, 512, operands, 1024) for _ in range(3))
+            long_ = min(q.qdit_probe_mma_rate(ctx, mode, n, 4096, operands, 1024) for _ in range(3))
+            assert 0.0 < short < long_ < 50.0, (mode, n, short, long_)
+            assert long_ > 3.0 * short - 0.05, (mode, n, short, long_)      # 8 x the groups, minus the fixed launch cost
+    q.qdit_sync(ctx)                                                       # no wait ran out
+    import ctypes as C
+    ms = C.c_float()
+    for bad in ((2, 128, 16, 1024), (0, 100, 16, 1024), (0, 128, 0, 1024), (0, 128, 1 << 17, 1024), (0, 128, 16, 100)):
+        mode, n, iters, rows = bad
+        assert q.lib.qdit_probe_mma_rate(ctx, mode, n, iters, operands.data_ptr(), rows, C.byref(ms)) < 0, bad

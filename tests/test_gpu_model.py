@@ -140,9 +140,11 @@ def test_block_s2_from_primitives(q, ctx):
         # modulation: a de-quantized layer output -> max relative error 1e-3
         assert max_rel_err(mod.cpu().numpy(), taps["blk0.mod"]) < 1e-3
         np.testing.assert_array_equal(host_codes(ca), taps["blk0.ada.qa"])
-        # fused LN quantizer: codes equal the oracle's except within f32 reach of a rounding boundary
+        # fused LN quantizer: codes equal the oracle's except where the oracle's pre-rounding value lies within 2e-3 code
+        # units of a rounding boundary (f32 statistics and products against f64: a few 1e-7 of |pre| <= 127, plus the
+        # 1e-5 relative difference of the modulation the kernel was given)
         pre = taps["blk0.qkv.in"].astype(np.float32).astype(np.float64) * float(scales.blocks[0]["qkv"].inv_scale)
-        n_bad, ok = code_mismatch_report(host_codes(h), taps["blk0.qkv.qa"], pre, 1e-3 * np.abs(pre).max())
+        n_bad, ok = code_mismatch_report(host_codes(h), taps["blk0.qkv.qa"], pre, 2e-3)
         assert ok and n_bad < 2e-3 * h.numel(), n_bad
         # QKV in bf16: oracle value rounded to bf16, up to one step at ties
         got_qkv = bf16_to_f64(qkv)
