@@ -437,6 +437,18 @@ int32_t qdit_sampler_set_ddpm(qdit_ctx* ctx, qdit_sampler* s, const float* noise
 int32_t qdit_sample(qdit_ctx* ctx, qdit_sampler* s, const float* latent_host, const int32_t* labels_host,
                     float* out_host);
 
+/* The un-quantized layers around the blocks (the paper takes them from the DiT architecture it cites and leaves them
+ * in floating point), as calls of their own:
+ *   qdit_patch_embed: x[m,:] = bf16(W_patch . patch(m) + b_patch + pos[m mod T,:]) for the B*T tokens of B samples;
+ *     a patch vector holds the p x p x C latent values of a token in (channel, row, column) order.
+ *     latent f32 [B,C,Hl,Wl], x bf16 [B*T, D] (both DEVICE, 16-byte aligned).
+ *   qdit_final_layer: out = unpatchify(W_out . (LN(x[m,:]) * (1 + scale_b) + shift_b) + b_out): LayerNorm without
+ *     affine (eps 1e-6, biased variance), the sample's modulation mod[b] = (shift | scale), a D -> p*p*2C linear in f32
+ *     accuracy, output vector ordered (row, column, channel).  x bf16 [B*T, D], mod f32 [B, 2D], out f32 [B,2C,Hl,Wl].
+ * Both return QDIT_ERR_ALIGN for a misaligned pointer and launch nothing then. */
+int32_t qdit_patch_embed(qdit_ctx* ctx, qdit_model* model, const float* latent, int B, void* x);
+int32_t qdit_final_layer(qdit_ctx* ctx, qdit_model* model, const void* x, const float* mod, int B, float* out);
+
 /* One network evaluation on B <= (use_cfg ? 2 : 1) * batch samples, no sampler update:
  * latent [B,C,Hl,Wl] f32, t [B] f32 timesteps, y [B] int32 labels, out [B,2C,Hl,Wl] f32 (all DEVICE).
  * flags: QDIT_FWD_STORE_CACHE writes the cache, QDIT_FWD_REUSE serves all blocks from it,

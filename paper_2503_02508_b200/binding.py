@@ -94,6 +94,8 @@ _SIGNATURES = {
     "qdit_cache_reuse": (_i32, [_vp, _vp, _int, _int, _vp, _i64, _i64, _vp]),
     "qdit_cache_reuse_all": (_i32, [_vp, _vp, _vp, _i64, _i64, _vp]),
     "qdit_selftest_wait_timeout": (_i32, [_vp, C.c_uint32, _vp]),
+    "qdit_patch_embed": (_i32, [_vp, _vp, _vp, _int, _vp]),
+    "qdit_final_layer": (_i32, [_vp, _vp, _vp, _vp, _int, _vp]),
     "qdit_probe_mma_rate": (_i32, [_vp, _int, _int, _int, _vp, _i64, C.POINTER(C.c_float)]),
     "qdit_vc_correct": (_i32, [_vp, _vp, _int, _int, _int, _int, _int, _vp, _f32]),
     "qdit_tap_laplacian": (_i32, [_vp, _vp, _vp, _int, _int, _f32, _f32, _vp, _vp]),
@@ -306,6 +308,14 @@ def qdit_cache_reuse_all(ctx, cache, mod_all, ld_mod, T, x):
 
 def qdit_selftest_wait_timeout(ctx, polls, observed):
     return check(ctx, lib.qdit_selftest_wait_timeout(ctx, polls, ptr(observed)))
+
+
+def qdit_patch_embed(ctx, model, latent, B, x):
+    return check(ctx, lib.qdit_patch_embed(ctx, model, ptr(latent), B, ptr(x)))
+
+
+def qdit_final_layer(ctx, model, x, mod, B, out):
+    return check(ctx, lib.qdit_final_layer(ctx, model, ptr(x), ptr(mod), B, ptr(out)))
 
 
 def qdit_probe_mma_rate(ctx, mode, n, iters, operands, rows):

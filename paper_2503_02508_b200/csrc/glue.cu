@@ -604,16 +604,18 @@ __global__ void __launch_bounds__(512, 1) final_kernel(const __nv_bfloat16* __re
 //   out[o] = rstd (S[o] - mean c1[o]) + c2[o] + bias[o],   S[o] = sum_k x_k W'[o,k],   W'[o,k] = (1 + scale_k) W[o,k],
 //   c1[o] = sum_k W'[o,k],   c2[o] = sum_k shift_k W[o,k],
 // so the bf16 activations go to the tensor cores as they are (exactly), and are read once.  W' is specific to the
-// sample: the CTA forms it chunk by chunk in f32 and splits it into a bf16 head and a bf16 remainder (|lo| <= 2^-9 |W'|;
-// both products are accumulated, what is dropped is below 2^-17 relative).  The statistics (sum x, sum x^2 in f32) are
+// sample: the CTA forms it chunk by chunk in f32 and splits it into three bf16 parts, head + remainder + second
+// remainder, which together hold all 24 bits of the f32 value; the three products are accumulated in f32, so the
+// result has the accuracy of an f32 dot product (with two parts the 2^-18 truncation per term showed as 7e-6 of the
+// output's rms).  The statistics (sum x, sum x^2 in f32) are
 // accumulated from the same fragments on the ordinary pipes: mma.sync issues one m16n8k16 per 16 cycles and scheduler
 // here, which is the kernel's limit, so nothing that the other pipes can do goes to it.  The CTA's 64 rows are one contiguous piece of memory; they are fetched whole, one bulk copy per
 // row (whole rows keep DRAM pages streaming; column chunks of 256 bytes per row ran at a third of the bandwidth), into
 // rows padded by 16 bytes.  Thirty-two warps: (row tile 0..3) x (k-step 0..7 of a 128-column chunk), so that each
 // scheduler has eight warps to hide the mma and ldmatrix latencies; W' chunks are double-buffered; the partial sums of
 // the eight k-step groups meet in shared memory at the end.
-constexpr int FT_ROWS = 64, FT_KC = 128, FT_THREADS = 1024, FT_KG = 8, FT_PITCH = FT_KC * 2 + 16, FT_DMAX = 1408, FT_RED_PITCH = 68;
-constexpr int FT_WBUF_BYTES = 2 * FIN_OUT * FT_PITCH;   // weight heads, weight remainders of one chunk
+constexpr int FT_ROWS = 64, FT_KC = 128, FT_THREADS = 1024, FT_KG = 8, FT_PITCH = FT_KC * 2 + 16, FT_DMAX = 1152, FT_RED_PITCH = 68;
+constexpr int FT_WBUF_BYTES = 3 * FIN_OUT * FT_PITCH;   // weight heads, remainders, second remainders of one chunk
 constexpr int ft_smem_bytes(int D) {
   return (2 * D + FT_KG * FT_ROWS * 2 + 2 * FIN_OUT) * 4 + 16 + 2 * FT_WBUF_BYTES + FT_ROWS * (2 * D + 16);
 }
@@ -643,6 +645,16 @@ __device__ __forceinline__ void split_pair(float z0, float z1, uint32_t& hi, uin
   const __nv_bfloat162 l = __floats2bfloat162_rn(z0 - __low2float(h), z1 - __high2float(h));
   hi = *reinterpret_cast<const uint32_t*>(&h);
   lo = *reinterpret_cast<const uint32_t*>(&l);
+}
+// (z0, z1) -> three packed bf16 pairs with hi + lo + lo2 == z (8 + 8 + 8 mantissa bits: all of an f32 value)
+__device__ __forceinline__ void split_triple(float z0, float z1, uint32_t& hi, uint32_t& lo, uint32_t& lo2) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(z0, z1);
+  const float r0 = z0 - __low2float(h), r1 = z1 - __high2float(h);
+  const __nv_bfloat162 l = __floats2bfloat162_rn(r0, r1);
+  const __nv_bfloat162 m = __floats2bfloat162_rn(r0 - __low2float(l), r1 - __high2float(l));
+  hi = *reinterpret_cast<const uint32_t*>(&h);
+  lo = *reinterpret_cast<const uint32_t*>(&l);
+  lo2 = *reinterpret_cast<const uint32_t*>(&m);
 }
 
 __global__ void __launch_bounds__(FT_THREADS) final_tc_kernel(const __nv_bfloat16* __restrict__ x, int64_t M, int D, int T, float eps,
@@ -693,12 +705,13 @@ __global__ void __launch_bounds__(FT_THREADS) final_tc_kernel(const __nv_bfloat1
     const float z0 = wa.x * ma.x, z1 = wa.y * ma.y, z2 = wa.z * ma.z, z3 = wa.w * ma.w;
     c1 += (z0 + z1) + (z2 + z3);
     c2 = fmaf(wa.x, da.x, fmaf(wa.y, da.y, fmaf(wa.z, da.z, fmaf(wa.w, da.w, c2))));
-    uint32_t h0, h1, l0, l1;
-    split_pair(z0, z1, h0, l0);
-    split_pair(z2, z3, h1, l1);
+    uint32_t h0, h1, l0, l1, m0, m1;
+    split_triple(z0, z1, h0, l0, m0);
+    split_triple(z2, z3, h1, l1, m1);
     uint8_t* dst = wring + (c & 1) * FT_WBUF_BYTES + wo * FT_PITCH + wk * 2;
     *reinterpret_cast<uint2*>(dst) = make_uint2(h0, h1);
     *reinterpret_cast<uint2*>(dst + FIN_OUT * FT_PITCH) = make_uint2(l0, l1);
+    *reinterpret_cast<uint2*>(dst + 2 * FIN_OUT * FT_PITCH) = make_uint2(m0, m1);
   };
   __syncthreads();   // the modulation table is complete
   store_w(0);
@@ -713,7 +726,7 @@ __global__ void __launch_bounds__(FT_THREADS) final_tc_kernel(const __nv_bfloat1
   const uint32_t xs = smem_u32(xt);
   for (int c = 0; c < nc; ++c) {
     if (c > 0) __syncthreads();   // W' of chunk c is there for everybody, and everybody is done with chunk c - 1
-    const uint32_t whs = smem_u32(wring + (c & 1) * FT_WBUF_BYTES), wls = whs + FIN_OUT * FT_PITCH;
+    const uint32_t whs = smem_u32(wring + (c & 1) * FT_WBUF_BYTES), wls = whs + FIN_OUT * FT_PITCH, wms = wls + FIN_OUT * FT_PITCH;
     {
       const int ks = kg;
       uint32_t a[4];   // a[0] row g, a[1] row g + 8 (columns 2 t4, + 1 of the k-step); a[2], a[3] the same rows, columns + 8
@@ -733,13 +746,16 @@ __global__ void __launch_bounds__(FT_THREADS) final_tc_kernel(const __nv_bfloat1
 #pragma unroll
       for (int n2 = 0; n2 < 2; ++n2) {   // two output tiles of 8 per ldmatrix
         const uint32_t off = (n2 * 16 + (lane & 7) + ((lane >> 4) << 3)) * FT_PITCH + (ks * 16 + ((lane >> 3) & 1) * 8) * 2;
-        uint32_t bh[4], bl[4];
+        uint32_t bh[4], bl[4], bm[4];
         ldmatrix_x4(whs + off, bh);
         ldmatrix_x4(wls + off, bl);
-        mma_bf16_16816(acc[2 * n2], a, bh[0], bh[1]);
+        ldmatrix_x4(wms + off, bm);
+        mma_bf16_16816(acc[2 * n2], a, bm[0], bm[1]);   // smallest parts first
+        mma_bf16_16816(acc[2 * n2 + 1], a, bm[2], bm[3]);
         mma_bf16_16816(acc[2 * n2], a, bl[0], bl[1]);
-        mma_bf16_16816(acc[2 * n2 + 1], a, bh[2], bh[3]);
         mma_bf16_16816(acc[2 * n2 + 1], a, bl[2], bl[3]);
+        mma_bf16_16816(acc[2 * n2], a, bh[0], bh[1]);
+        mma_bf16_16816(acc[2 * n2 + 1], a, bh[2], bh[3]);
       }
     }
     if (c + 1 < nc) {   // while the tensor pipe works through this chunk: W' of the next one, into the buffer of chunk c - 1

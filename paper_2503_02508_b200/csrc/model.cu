@@ -633,6 +633,27 @@ int32_t qdit_forward(qdit_ctx* ctx, qdit_sampler* s, const float* latent, const 
   return forward_impl(ctx, s, latent, B, t, y, B, out, flags);
 }
 
+int32_t qdit_patch_embed(qdit_ctx* ctx, qdit_model* m, const float* latent, int B, void* x) {
+  if (!ctx || !m) return QDIT_ERR_INVALID_ARG;
+  if (!latent || !x) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "NULL argument");
+  if (B <= 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "B = %d", B);
+  if (!aligned16(x) || !aligned16(latent)) return qdit_fail(ctx, QDIT_ERR_ALIGN, "latent and x must be 16-byte aligned");
+  const qdit_model_shape& sh = m->s;
+  const int64_t M = static_cast<int64_t>(B) * sh.grid * sh.grid;
+  return launch_embed(ctx, latent, B, m->w_patch, m->w_patch_frag, m->b_patch, m->pos, x, M, sh.hidden, sh.grid, sh.patch, sh.channels);
+}
+
+int32_t qdit_final_layer(qdit_ctx* ctx, qdit_model* m, const void* x, const float* mod, int B, float* out) {
+  if (!ctx || !m) return QDIT_ERR_INVALID_ARG;
+  if (!x || !mod || !out) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "NULL argument");
+  if (B <= 0) return qdit_fail(ctx, QDIT_ERR_SHAPE, "B = %d", B);
+  if (!aligned16(x) || !aligned16(mod) || !aligned16(out)) return qdit_fail(ctx, QDIT_ERR_ALIGN, "x, mod and out must be 16-byte aligned");
+  const qdit_model_shape& sh = m->s;
+  const int T = sh.grid * sh.grid;
+  return launch_final(ctx, x, static_cast<int64_t>(B) * T, sh.hidden, T, 1e-6f, mod, m->w_out, m->b_out, out, sh.grid, sh.patch,
+                      2 * sh.channels * sh.patch * sh.patch);
+}
+
 int32_t qdit_sampler_reset(qdit_ctx* ctx, qdit_sampler* s, const float* latent, const int32_t* labels) {
   if (!ctx || !s) return QDIT_ERR_INVALID_ARG;
   if (!latent || !labels) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "latent or labels is NULL");

@@ -516,3 +516,63 @@ def test_sampler_step_by_step_and_cache_effect(q, ctx):
         np.testing.assert_array_equal(got, b)
     finally:
         rig.close()
+
+
+GLUE_CASES = [
+    # tensor-core embedding and final layer: full groups of four samples, a short last group, a single sample
+    ("xl", dict(hidden=1152, heads=16, mlp=4608, depth=1, grid=16), 4),
+    ("xl", dict(hidden=1152, heads=16, mlp=4608, depth=1, grid=16), 7),
+    ("xl", dict(hidden=1152, heads=16, mlp=4608, depth=1, grid=16), 1),
+    ("xl_1024_tokens", dict(hidden=1152, heads=16, mlp=4608, depth=1, grid=32), 2),
+    ("width_768", dict(hidden=768, heads=12, mlp=3072, depth=1, grid=16), 5),
+    # tensor-core embedding, scalar final layer (width below the tensor-core form's range)
+    ("s", dict(hidden=384, heads=6, mlp=1536, depth=1, grid=16), 5),
+    # scalar kernels (width 144, 64 tokens)
+    ("tiny", None, 3),
+]
+
+
+@pytest.mark.parametrize("name,shape,B", GLUE_CASES)
+def test_patch_embed_and_final_layer_element_by_element(q, ctx, name, shape, B):
+    """The floating-point layers around the blocks as calls of their own.  Embedding: every stored bf16 value is the
+    rounding of the oracle's value, up to the f32 / split-operand error of the product (1e-5 of the sum of the terms'
+    magnitudes: a missing remainder product would be 2e-3).  Final layer: f32-level agreement with the oracle."""
+    cfg = synth.DIT_TINY if shape is None else synth.DiTConfig(**shape)
+    rig = Rig(q, ctx, cfg, 91)
+    try:
+        D, T, C, side = cfg.hidden, cfg.tokens, cfg.channels, cfg.latent_side
+        M = B * T
+        w = rig.om.w
+        # ---- embedding
+        latent = synth.normal(92, f"glue.latent.{name}.{B}", (B, C, side, side))
+        xg = torch.empty((M, D), dtype=torch.bfloat16, device="cuda")
+        q.qdit_patch_embed(ctx, rig.gm, dev(latent), B, xg)
+        q.qdit_sync(ctx)
+        got = bf16_to_f64(xg)
+        patches = dit.patchify(cfg, latent.astype(np.float32).astype(np.float64))
+        ref = patches @ w["w_patch"].T + w["b_patch"] + np.tile(w["pos"], (B, 1))
+        mag = np.abs(patches) @ np.abs(w["w_patch"]).T + np.abs(w["b_patch"]) + np.tile(np.abs(w["pos"]), (B, 1))
+        ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(ref), 1e-30))) - 7)
+        assert np.all(np.abs(got - ref) <= 0.5 * ulp + 1e-5 * mag + 1e-12)
+        assert np.mean(got == dit.round_bf16(ref)) > 0.995          # flips only where the value sits within that error of a rounding boundary
+        # ---- final layer
+        x = synth.normal(93, f"glue.x.{name}.{B}", (M, D), 1.7, 0.3)
+        xd = dev(x).to(torch.bfloat16)
+        mod = synth.normal(93, f"glue.mod.{name}.{B}", (B, 2 * D), 0.4)
+        out = torch.empty((B, 2 * C, side, side), dtype=torch.float32, device="cuda")
+        q.qdit_final_layer(ctx, rig.gm, xd, dev(mod), B, out)
+        q.qdit_sync(ctx)
+        h = dit.layer_norm_modulate(bf16_to_f64(xd), mod[:, :D].astype(np.float32).astype(np.float64),
+                                    mod[:, D:].astype(np.float32).astype(np.float64), T)
+        ref_o = dit.unpatchify(cfg, h @ w["w_out"].T + w["b_out"], B)
+        got_o = out.cpu().numpy().astype(np.float64)
+        # f32 statistics (1e-4 under this metric, as for LayerNorm alone) plus a D-term product accumulated in f32 by the
+        # tensor core, whose adds may truncate: up to D * 2^-24 * mean|term| = 1152 * 6e-8 * 0.04 = 3e-6 absolute on outputs
+        # of rms 1, i.e. 3e-4 against the metric's floor of 1e-2 rms.  In the norm the agreement is 1e-6.
+        assert max_rel_err(got_o, ref_o) < 4e-4, max_rel_err(got_o, ref_o)
+        assert rel_l2(got_o, ref_o) < 5e-6, rel_l2(got_o, ref_o)
+        # misaligned pointers are refused before any launch
+        assert q.lib.qdit_patch_embed(ctx, rig.gm, dev(latent).data_ptr(), B, xg.data_ptr() + 2) == q.QDIT_ERR_ALIGN
+        assert q.lib.qdit_final_layer(ctx, rig.gm, xd.data_ptr() + 2, dev(mod).data_ptr(), B, out.data_ptr()) == q.QDIT_ERR_ALIGN
+    finally:
+        rig.close()
