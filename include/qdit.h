@@ -83,10 +83,13 @@ int64_t qdit_launch_count(const qdit_ctx* ctx);
  *                                   2: the online-softmax tcgen05 kernel also at 256 tokens
  *   QDIT_OPT_CONDITIONING_CHUNK     sampling steps whose conditioning a sampler evaluates at once: 0 (default) as many
  *                                   as fit a 4 GB modulation table, -1 step by step, n > 0 at most n (read by
- *                                   qdit_sampler_create) */
+ *                                   qdit_sampler_create)
+ *   QDIT_OPT_ATTN_STAGGER_NS        256-token attention: the CTAs that become the second resident of an SM in the first
+ *                                   wave start this many nanoseconds late (default 2000; 0 = together), so that the two
+ *                                   CTAs of an SM do not run their phases in lockstep; 0..20000 */
 enum {
   QDIT_OPT_PDL = 0, QDIT_OPT_GEMM_BN = 1, QDIT_OPT_GEMM_T = 2, QDIT_OPT_GEMM_GENERIC_EPILOGUE = 3, QDIT_OPT_ATTN = 4,
-  QDIT_OPT_CONDITIONING_CHUNK = 5, QDIT_OPT_COUNT = 6
+  QDIT_OPT_CONDITIONING_CHUNK = 5, QDIT_OPT_ATTN_STAGGER_NS = 6, QDIT_OPT_COUNT = 7
 };
 int32_t qdit_set_option(qdit_ctx* ctx, int option, int value);
 int32_t qdit_get_option(const qdit_ctx* ctx, int option, int* value);

@@ -27,7 +27,7 @@ QDIT_VC_NONE, QDIT_VC_K_TABLE, QDIT_VC_VAR_RATIO = 0, 1, 2
 QDIT_VC_FIT_DERIVED, QDIT_VC_FIT_PRINTED = 0, 1
 QDIT_FWD_STORE_CACHE, QDIT_FWD_REUSE, QDIT_FWD_CALIBRATE = 1, 2, 4
 (QDIT_OPT_PDL, QDIT_OPT_GEMM_BN, QDIT_OPT_GEMM_T, QDIT_OPT_GEMM_GENERIC_EPILOGUE, QDIT_OPT_ATTN,
- QDIT_OPT_CONDITIONING_CHUNK) = range(6)
+ QDIT_OPT_CONDITIONING_CHUNK, QDIT_OPT_ATTN_STAGGER_NS) = range(7)
 
 _vp, _i32, _i64, _u32, _f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_float
 _int = C.c_int

@@ -37,6 +37,8 @@ struct AttnTcParams {
   int out_dtype;
   QuantArgs qa;
   int* status;
+  int stagger_ns;      // 256-token kernel: start delay of an SM's second CTA in the first wave
+  unsigned num_sms;
 };
 
 template <int DH>
@@ -431,6 +433,17 @@ attention_tc256_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
   // shared and tensor memory only so far; Q, K and V come from the previous kernel of the stream
   grid_dependency_wait();
   grid_dependency_release();
+  // The CTAs of the first wave that share an SM would run their phases (loads, products, exponentials, output) in
+  // lockstep, each phase's unit busy in bursts and idle in between.  The second CTA of every SM starts `stagger_ns`
+  // late, once: after that the CTAs of an SM stay out of phase, since every later CTA starts when another one ends.
+  if (p.stagger_ns > 0) {
+    const unsigned linear = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+    if (linear >= p.num_sms && linear < 2u * p.num_sms) {
+      const long long t0 = clock64();
+      const long long span = static_cast<long long>(p.stagger_ns) * 2;   // clocks at <= 2 GHz: an upper bound, not a timer
+      for (int i = 0; i < 4096 && clock64() - t0 < span; ++i) __nanosleep(200);
+    }
+  }
 
   if (warp == SM_WARPS) {
     if (lane == 0) {
@@ -734,6 +747,8 @@ int32_t qdit_launch_attention_tc(qdit_ctx* ctx, const void* q, const void* k, co
   p.out_dtype = out_dtype;
   p.qa = qa;
   p.status = ctx->d_status;
+  p.stagger_ns = ctx->opt[QDIT_OPT_ATTN_STAGGER_NS];
+  p.num_sms = static_cast<unsigned>(ctx->num_sms);
   if (dh == 64) return launch_tc<64>(ctx, q, k, v, ld, B, H, T, p);
   return launch_tc<72>(ctx, q, k, v, ld, B, H, T, p);
 }

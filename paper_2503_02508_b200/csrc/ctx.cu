@@ -150,11 +150,12 @@ int32_t qdit_create(qdit_ctx** out, int device, void* cuda_stream) {
   ctx->stream = static_cast<cudaStream_t>(cuda_stream);
   ctx->num_sms = prop.multiProcessorCount;
   ctx->opt[QDIT_OPT_PDL] = 1;
+  ctx->opt[QDIT_OPT_ATTN_STAGGER_NS] = 2000;
   {  // initial option values from the environment, read here once and nowhere else
     static const struct { const char* name; int opt; } kEnv[] = {
         {"QDIT_PDL", QDIT_OPT_PDL}, {"QDIT_GEMM_BN", QDIT_OPT_GEMM_BN}, {"QDIT_GEMM_T", QDIT_OPT_GEMM_T},
         {"QDIT_GEMM_GENERIC_EPILOGUE", QDIT_OPT_GEMM_GENERIC_EPILOGUE}, {"QDIT_ATTN", QDIT_OPT_ATTN},
-        {"QDIT_CONDITIONING_CHUNK", QDIT_OPT_CONDITIONING_CHUNK}};
+        {"QDIT_CONDITIONING_CHUNK", QDIT_OPT_CONDITIONING_CHUNK}, {"QDIT_ATTN_STAGGER_NS", QDIT_OPT_ATTN_STAGGER_NS}};
     for (const auto& e : kEnv)
       if (const char* v = getenv(e.name)) qdit_set_option(ctx, e.opt, atoi(v));
   }
@@ -190,6 +191,7 @@ int32_t qdit_set_option(qdit_ctx* ctx, int option, int value) {
     case QDIT_OPT_GEMM_GENERIC_EPILOGUE: ok = value == 0 || value == 1; break;
     case QDIT_OPT_ATTN: ok = value >= 0 && value <= 2; break;
     case QDIT_OPT_CONDITIONING_CHUNK: ok = value >= -1; break;
+    case QDIT_OPT_ATTN_STAGGER_NS: ok = value >= 0 && value <= 20000; break;
     default: return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "unknown option %d", option);
   }
   if (!ok) return qdit_fail(ctx, QDIT_ERR_INVALID_ARG, "value %d not valid for option %d", value, option);

@@ -108,6 +108,25 @@ def test_attention_fused_quantizer(q, ctx):
     assert n_bad < 0.2 * got.size
 
 
+def test_attention_start_stagger_changes_no_value(q, ctx):
+    """The start delay of an SM's second CTA (a scheduling option) must not change a single output byte: 12 samples x
+    16 heads x 2 query blocks = 384 CTAs, so the delayed group (CTAs 148..295) exists."""
+    B, T, H, dh = 12, 256, 16, 72
+    D = H * dh
+    xd = dev(synth.normal(54, "qkvs", (B * T, 3 * D), 1.0)).to(torch.bfloat16)
+    qp = q.qparams(0.01)
+    assert q.qdit_get_option(ctx, q.QDIT_OPT_ATTN_STAGGER_NS) == 2000
+    a = host_codes(_run(q, ctx, xd, B, T, H, dh, q.QDIT_I8, qp))
+    try:
+        for ns in (0, 20000):
+            q.qdit_set_option(ctx, q.QDIT_OPT_ATTN_STAGGER_NS, ns)
+            np.testing.assert_array_equal(host_codes(_run(q, ctx, xd, B, T, H, dh, q.QDIT_I8, qp)), a)
+        assert q.lib.qdit_set_option(ctx, q.QDIT_OPT_ATTN_STAGGER_NS, 20001) == q.QDIT_ERR_INVALID_ARG
+        assert q.lib.qdit_set_option(ctx, q.QDIT_OPT_ATTN_STAGGER_NS, -1) == q.QDIT_ERR_INVALID_ARG
+    finally:
+        q.qdit_set_option(ctx, q.QDIT_OPT_ATTN_STAGGER_NS, 2000)
+
+
 def test_attention_rejects_bad_arguments(q, ctx):
     t = torch.zeros((64, 3 * 64), dtype=torch.bfloat16, device="cuda")
     o = torch.zeros((64, 64), dtype=torch.float32, device="cuda")
