@@ -73,7 +73,8 @@ int64_t qdit_launch_count(const qdit_ctx* ctx);
 /* Kernel-selection options of a context (tuning and test aid; the paper has no counterpart).  Every option chooses
  * among kernels that compute the same values.  A new context takes its initial values from the environment
  * variables of the same names (QDIT_PDL, QDIT_GEMM_BN, QDIT_GEMM_T, QDIT_GEMM_GENERIC_EPILOGUE, QDIT_ATTN,
- * QDIT_CONDITIONING_CHUNK), read once inside qdit_create; afterwards only qdit_set_option changes them.
+ * QDIT_CONDITIONING_CHUNK, QDIT_ATTN_STAGGER_NS), read once inside qdit_create; afterwards only qdit_set_option changes
+ * them.
  *   QDIT_OPT_PDL                    1 (default): kernels are launched with programmatic stream serialization, so that
  *                                   a kernel's preamble overlaps the tail of the kernel before it; 0: plain launches
  *   QDIT_OPT_GEMM_BN                0 (default): automatic; 64 | 128 | 192: token-major GEMM kernel with 128 x BN tiles

@@ -125,8 +125,11 @@ extern "C" int32_t qdit_probe_mma_rate(qdit_ctx* ctx, int mode, int n, int iters
   QDIT_TRY(qdit_allow_smem(ctx, mma_probe_kernel, PROBE_STAGES * (128 * 128 + 256 * 128) + 256 + 1024));
   cudaEvent_t e0, e1;
   QDIT_CUDA_CHECK(ctx, cudaEventCreate(&e0));
-  QDIT_CUDA_CHECK(ctx, cudaEventCreate(&e1));
-  QDIT_CUDA_CHECK(ctx, cudaEventRecord(e0, ctx->stream));
+  if (cudaEventCreate(&e1) != cudaSuccess) {
+    cudaEventDestroy(e0);
+    return qdit_fail(ctx, QDIT_ERR_CUDA, "probe timing: event creation failed");
+  }
+  cudaEventRecord(e0, ctx->stream);
   mma_probe_kernel<<<ctx->num_sms, PROBE_THREADS, smem, ctx->stream>>>(tw, ta, p);
   int32_t st = qdit_after_launch(ctx, "mma_probe_kernel");
   cudaEventRecord(e1, ctx->stream);
