@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(256, 2) cache_reuse_all_kernel(__nv_bfloat16* 
   float acc[R][8];
 #pragma unroll
   for (int r = 0; r < R; ++r) Load8<__nv_bfloat16>::load(x + off + static_cast<int64_t>(r) * D, acc[r]);
-#pragma unroll 2
+#pragma unroll(R >= 4 ? 1 : 2)
   for (int b = 0; b < blocks; ++b) {
     float ga[8], gm[8];
     Load8<float>::load(mrow + static_cast<int64_t>(b) * 6 * D + 2 * D, ga);
@@ -1136,10 +1136,17 @@ int32_t qdit_cache_reuse_all(qdit_ctx* ctx, qdit_cache* c, const float* mod_all,
     if (!c->filled[i]) return qdit_fail(ctx, QDIT_ERR_STATE, "cache slot (block %zu, branch %zu) reused before any store", i / 2, i % 2);
   if (!aligned16(mod_all) || !aligned16(x) || ld_mod % 4 != 0) return qdit_fail(ctx, QDIT_ERR_ALIGN, "mod_all and x must be 16-byte aligned, ld_mod a multiple of 4");
   ProfScope prof(ctx, QDIT_PROF_CACHE_REUSE, static_cast<double>(c->M) * c->D * 2.0 * (2.0 * c->blocks + 2.0));
-  // rows per thread: 2 when samples are made of whole groups of 2 rows and there is work for every SM, else 1
+  // rows per thread: 4 (else 2) when samples are made of whole groups of that many rows and there is work for every SM,
+  // else 1: the gate vectors, as many bytes from L2 as the cache is from HBM with one row per thread, are then read
+  // once per group of rows (0.71 / 0.81 / 0.95 of the measured copy bandwidth with 1 / 2 / 4 rows)
   constexpr int R = 2;
   const bool wide = c->M % R == 0 && T % R == 0 && c->M * (c->D / 8) >= static_cast<int64_t>(R) * 256 * 4 * ctx->num_sms;
-  if (wide) {
+  const bool wide4 = c->M % 4 == 0 && T % 4 == 0 && c->M * (c->D / 8) >= static_cast<int64_t>(4) * 256 * 4 * ctx->num_sms;
+  if (wide4) {
+    const int64_t n = (c->M / 4) * (c->D / 8);
+    cache_reuse_all_kernel<4><<<static_cast<unsigned>((n + 255) / 256), 256, 0, ctx->stream>>>(
+        static_cast<__nv_bfloat16*>(x), c->data, mod_all, ld_mod, c->M, static_cast<int>(c->D), T, c->blocks);
+  } else if (wide) {
     const int64_t n = (c->M / R) * (c->D / 8);
     cache_reuse_all_kernel<R><<<static_cast<unsigned>((n + 255) / 256), 256, 0, ctx->stream>>>(
         static_cast<__nv_bfloat16*>(x), c->data, mod_all, ld_mod, c->M, static_cast<int>(c->D), T, c->blocks);
