@@ -70,7 +70,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return mbar_wait_limited(bar, parity, abort_flag, status, kSpinLimit);
 }
 
-// ----------------------------------------------------------------------------- TMA (no multicast anywhere)
+// ----------------------------------------------------------------------------- TMA (every copy serves the issuing CTA alone)
 __device__ __forceinline__ void tma_prefetch_desc(const void* tmap) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
 }
