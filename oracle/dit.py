@@ -71,7 +71,7 @@ def silu(x):
 
 
 def gelu_tanh(x):
-    return 0.5 * x * (1.0 + np.tanh(np.sqrt(2.0 / np.pi) * (x + 0.044715 * x ** 3)))
+    return 0.5 * x * (1.0 + np.tanh(np.sqrt(2.0 / np.pi) * (x + 0.044715 * (x * x * x))))
 
 
 def layer_norm_modulate(x, shift, scale, tokens: int, eps: float = LN_EPS):
@@ -89,11 +89,12 @@ def attention(q, k, v, scale: Optional[float] = None):
     q, k, v = (np.asarray(a, dtype=np.float64) for a in (q, k, v))
     if scale is None:
         scale = 1.0 / np.sqrt(q.shape[-1])
-    s = np.einsum("bthd,bshd->bhts", q, k) * scale
+    qh, kh, vh = (a.transpose(0, 2, 1, 3) for a in (q, k, v))    # [B,H,T,dh]
+    s = (qh @ kh.transpose(0, 1, 3, 2)) * scale                  # [B,H,T,T] scores (library matrix product per head)
     s = s - s.max(axis=-1, keepdims=True)
     p = np.exp(s)
     p = p / p.sum(axis=-1, keepdims=True)
-    return np.einsum("bhts,bshd->bthd", p, v)
+    return (p @ vh).transpose(0, 2, 1, 3)
 
 
 # ----------------------------------------------------------------------------- quantized model
@@ -162,7 +163,17 @@ def _qlinear_apply(ctx: Context, lin: QLinear, x, qp: Optional[QParams], name: s
         ctx.emit(name + ".absmax", np.float64(qp.scale) * qp.qmax)
     qa = quantize(x, qp)
     ctx.emit(name + ".qa", qa)
-    return w8a8_linear(qa, qp, lin.q, lin.scale, lin.colsum, lin.bias)
+    return w8a8_linear(qa, qp, _codes_f64(lin), lin.scale, lin.colsum, lin.bias)
+
+
+def _codes_f64(lin: QLinear) -> np.ndarray:
+    """The weight codes as the float64 array the integer product takes (same integers; converted once per layer
+    instead of once per call)."""
+    c = getattr(lin, "_q64", None)
+    if c is None:
+        c = np.asarray(lin.q, dtype=np.float64)
+        lin._q64 = c
+    return c
 
 
 def modulation(ctx: Context, blk: QBlock, c, index: int):
