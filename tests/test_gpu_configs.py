@@ -201,7 +201,7 @@ def test_forward_xl2_w4a8_matches_oracle(q, ctx):
 def test_ddim100_512_cached_sampler_batch8(q, ctx):
     """100-step DDIM at 512x512 (1024 tokens), batch 8, cache interval 3, VC every step, no guidance."""
     cfg, seed = synth.DIT_XL2_512, synth.CONFIG_SEEDS["ddim100_xl2_512"]
-    S, B, interval, n_prefix = 100, 8, 3, 7      # steps 0..6: three refreshes (0, 3, 6) and the reuse steps between them
+    S, B, interval, n_prefix = 100, 8, 3, 25     # steps 0..24: nine refreshes (0, 3, .., 24) and the reuse steps between them
     rig = XLRig(q, ctx, cfg, seed)
     try:
         latent = synth.normal(seed, "latent", (B, cfg.channels, cfg.latent_side, cfg.latent_side))
