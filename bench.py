@@ -142,9 +142,9 @@ def images_per_second(world, batch, n_traj, ms):
 
 
 # ------------------------------------------------------------------------------------------ CPU oracle leg
-def oracle_sample_rate(name, n_images=1, n_steps=4):
-    """Times the oracle on `n_images` images for the first `n_steps` sampling steps (two refreshes and the reuse
-    steps after them when n_steps = 4 and the interval is 2 or 3: about 10 s of CPU work) and scales the mean refresh
+def oracle_sample_rate(name, n_images=1, n_steps=6):
+    """Times the oracle on `n_images` images for the first `n_steps` sampling steps (with n_steps = 6: three refreshes
+    and three reuse steps at interval 2, two and four at interval 3: 10-15 s of CPU work) and scales the mean refresh
     and reuse times to the whole trajectory.  Returns (images/s, info)."""
     from oracle import calib, dit, sampler as osampler
     cfg, seed, steps, batch, guidance, interval, latent, labels, vc_table = workload_inputs(name)
