@@ -52,7 +52,7 @@ constexpr uint32_t EPI_FLAGS_FC1 = QDIT_EPI_BIAS | QDIT_EPI_GELU | QDIT_EPI_QUAN
 constexpr uint32_t EPI_FLAGS_GATED = QDIT_EPI_BIAS | QDIT_EPI_GATE | QDIT_EPI_RESIDUAL | QDIT_EPI_CACHE_STORE | QDIT_EPI_OUT_BF16;
 template <int EPI>
 __device__ __forceinline__ uint32_t epi_flags(const GemmParams& p) {
-  return EPI == 1 ? EPI_FLAGS_QKV : EPI == 2 ? EPI_FLAGS_FC1 : EPI == 3 ? EPI_FLAGS_GATED : p.flags;
+  return EPI == 1 ? EPI_FLAGS_QKV : EPI == 2 ? EPI_FLAGS_FC1 : (EPI == 3 || EPI == 4) ? EPI_FLAGS_GATED : p.flags;
 }
 inline int epi_class(uint32_t flags) {
   return flags == EPI_FLAGS_QKV ? 1 : flags == EPI_FLAGS_FC1 ? 2 : flags == EPI_FLAGS_GATED ? 3 : 0;

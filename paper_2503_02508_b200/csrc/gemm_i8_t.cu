@@ -45,8 +45,9 @@ constexpr int BC = 128;  // channels per tile = TMEM lanes
 #endif
 template <int EPI>
 struct TWarps {
-  static constexpr bool STAGED = EPI == 1 || EPI == 3;
-  static constexpr int EPI_WARPS = STAGED ? QDIT_T_STAGED_WARPS : 12;
+  static constexpr bool GATED = EPI == 3 || EPI == 4;   // 4: the gated class for short reductions (see launch_t)
+  static constexpr bool STAGED = EPI == 1 || GATED;
+  static constexpr int EPI_WARPS = EPI == 4 ? 12 : (STAGED ? QDIT_T_STAGED_WARPS : 12);
   static constexpr int SPLIT = EPI_WARPS / 4;
   static constexpr int THREADS = 64 + EPI_WARPS * 32;
 #ifndef QDIT_T_GATED_TILES
@@ -54,7 +55,7 @@ struct TWarps {
 #endif
   // 2 KB tiles of 32 tokens x 32 channels bf16 per warp: class 1 two output tiles used in turn; class 3 the residual
   // tile plus one tile shared by the cache copy and the output (2) or one tile each (3)
-  static constexpr int TILES = EPI == 3 ? QDIT_T_GATED_TILES : 2;
+  static constexpr int TILES = GATED ? QDIT_T_GATED_TILES : 2;
   static constexpr int STAGING_PER_WARP = STAGED ? TILES * 2048 : 0;
   // class 2 (8-bit codes): the four quadrant warps that work on the same token chunk share a tile of 32 tokens x 128
   // channels (4 KB), two tiles used in turn per group of four
@@ -344,7 +345,7 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
       };
       if (lane == 0) {
         tma_prefetch_desc(&tmap_out);
-        if (EPI == 3) {
+        if (TW::GATED) {
           tma_prefetch_desc(&tmap_cache);
           tma_prefetch_desc(&tmap_res);
         }
@@ -353,7 +354,7 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
         // the residual of the tile's first chunk, unless the previous tile's last chunk has already asked for it
-        if (EPI == 3 && !r_inflight && chunk_live(tile, part)) {
+        if (TW::GATED && !r_inflight && chunk_live(tile, part)) {
           if (lane == 0) issue_residual(tile, part);
           r_inflight = true;
         }
@@ -388,7 +389,7 @@ gemm_i8_t_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
           const bool live = m_base < p.M && c0q < p.N;   // uniform over the warp
           uint32_t a[16], b[16];
           float gate[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-          if (EPI == 3 && live) {
+          if (TW::GATED && live) {
             const float* grow = p.gate + static_cast<int64_t>(m_base / p.tokens) * p.ld_gate;
 #pragma unroll
             for (int k = 0; k < 4; ++k)
@@ -570,7 +571,7 @@ int32_t launch_t_epi(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p,
   if (TWarps<EPI>::STAGED) {
     QDIT_TRY(qdit_get_tmap(ctx, p.out, p.M, p.N, p.ldo, 32, 32, 2, 2, &to));
     tc = tr = to;
-    if (EPI == 3) {
+    if (TWarps<EPI>::GATED) {
       QDIT_TRY(qdit_get_tmap(ctx, p.cache_out, p.M, p.N, p.N, 32, 32, 2, 2, &tc));
       QDIT_TRY(qdit_get_tmap(ctx, p.residual, p.M, p.N, p.ldo, 32, 32, 2, 2, &tr));
     }
@@ -592,7 +593,13 @@ int32_t launch_t(qdit_ctx* ctx, const void* A, const void* W, GemmParams& p, boo
   switch (ctx->opt[QDIT_OPT_GEMM_GENERIC_EPILOGUE] ? 0 : epi_class(p.flags)) {
     case 1: return launch_t_epi<BT, 1>(ctx, A, W, p, a_unsigned);
     case 2: return launch_t_epi<BT, 2>(ctx, A, W, p, a_unsigned);
-    case 3: return launch_t_epi<BT, 3>(ctx, A, W, p, a_unsigned);
+    case 3:
+      // A short reduction leaves the gated epilogue (residual in, two tiles out per chunk) as the longer part of a tile,
+      // and with few tiles per CTA the last one is exposed: three warps per lane quadrant instead of two shorten it,
+      // at the price of one pipeline stage (48 KB of staging instead of 32), which only a long reduction would miss
+      // (K = 1152: 17.5 -> 16.6 us at 8192 rows, 129 -> 120 us at 65536; K = 4608: 37.0 -> 41.3 us).
+      if (p.K < 2048) return launch_t_epi<BT, 4>(ctx, A, W, p, a_unsigned);
+      return launch_t_epi<BT, 3>(ctx, A, W, p, a_unsigned);
     default: return launch_t_epi<BT, 0>(ctx, A, W, p, a_unsigned);
   }
 }
