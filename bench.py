@@ -42,9 +42,9 @@ STOCHASTIC = {"ddpm250"}
 
 
 # DRAM bytes (read + written) per GEMM launch, from the ncu capture summarised in
-# profiles/gemm_i8_layers_m8192_sections.txt: QKV 18.1 MB, proj 30.0 MB, fc1 14.9 MB, fc2 66.0 MB per launch at
+# profiles/gemm_i8_layers_m8192_sections.txt: QKV 18.3 MB, proj 30.0 MB, fc1 14.9 MB, fc2 65.5 MB per launch at
 # M = 8192 (the shapes of the 50-step workload); each layer is 700 of the trajectory's 2801 GEMM launches.
-NCU_GEMM_DRAM_BYTES_PER_LAUNCH = 700 * (18.1e6 + 30.0e6 + 14.9e6 + 66.0e6) / 2801
+NCU_GEMM_DRAM_BYTES_PER_LAUNCH = 700 * (18.3e6 + 30.0e6 + 14.9e6 + 65.5e6) / 2801
 
 
 def measured_peaks():
