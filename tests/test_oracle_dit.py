@@ -175,3 +175,24 @@ def test_block_samples_are_independent(tiny):
     one = dit.forward(model, ctx, latent[1:2], t[1:2], y[1:2])
     np.testing.assert_allclose(full[1:2], one, rtol=0, atol=1e-6)   # up to summation order and rare code flips
     assert np.abs(full[1:2] - one).mean() < 1e-9
+
+
+def test_quantized_linear_with_cached_codes_is_the_integer_definition(tiny):
+    """The layer evaluation keeps a float64 copy of the weight codes (made once): its output must be, bit for bit, the
+    definition on the integer codes - brute-force int64 products, then the affine de-quantisation."""
+    from oracle import linear, quant
+    cfg, w, *_ = tiny
+    lin = dit.make_qlinear(w["blocks"][0]["w_fc1"], w["blocks"][0]["b_fc1"])
+    x = synth.normal(12, "cached.x", (7, lin.q.shape[1]), 1.3)
+    qp = quant.qparams_symmetric(float(np.abs(x.astype(np.float32)).max()))
+    ctx = dit.Context(quant="static")
+    got1 = dit._qlinear_apply(ctx, lin, x, qp, "t")
+    got2 = dit._qlinear_apply(ctx, lin, x, qp, "t")            # second call: the cached copy
+    qa = quant.quantize(x, qp).astype(np.int64)
+    acc = np.zeros((7, lin.q.shape[0]), dtype=np.int64)
+    for k in range(qa.shape[1]):                                # integer accumulation, no floating point involved
+        acc += qa[:, k:k + 1] * lin.q[:, k].astype(np.int64)[None, :]
+    want = linear.dequant_affine(acc, qp, lin.scale, lin.colsum, lin.bias)
+    np.testing.assert_array_equal(got1, want)
+    np.testing.assert_array_equal(got2, want)
+    assert lin.q.dtype == np.int8                               # the stored codes themselves are untouched
